@@ -1,0 +1,108 @@
+"""ctypes front end of the fp64 CPU oracle (`fspad_oracle.c`).
+
+TEST INFRASTRUCTURE ONLY: the tests, the smoke check and the benchmark's
+CPU-baseline leg use it; the CUDA library and its Python binding never
+import this package, and this package imports nothing of theirs.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from typing import Optional
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "fspad_oracle.c")
+_LIB = os.path.join(_HERE, "libfspad_oracle.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (plain C, -O2, OpenMP over independent units)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + ".tmp.%d" % os.getpid()
+        subprocess.check_call(["gcc", "-O2", "-std=c11", "-fopenmp", "-fPIC", "-shared", "-o", tmp,
+                               _SRC, "-lm"])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        _lib = ctypes.CDLL(build())
+    return _lib
+
+
+def _p(a: Optional[np.ndarray], dtype):
+    if a is None:
+        return None
+    assert a.dtype == dtype and a.flags["C_CONTIGUOUS"], (a.dtype, dtype)
+    return a.ctypes.data_as(ctypes.c_void_p)
+
+
+def set_threads(n: int) -> None:
+    os.environ["OMP_NUM_THREADS"] = str(n)
+
+
+def tree_attn(q, k_cache, v_cache, tree_k, tree_v, parent, prefix_len, scale: Optional[float] = None):
+    """fp64 tree-masked attention; bf16 inputs as uint16 bit arrays. Returns [B][N][Hq][d] float64."""
+    B, N, Hq, d = q.shape
+    _, Hkv, max_len, _ = k_cache.shape
+    scale = 1.0 / np.sqrt(d) if scale is None else scale
+    out = np.empty((B, N, Hq, d), dtype=np.float64)
+    rc = lib().oracle_tree_attn(_p(q, np.uint16), _p(k_cache, np.uint16), _p(v_cache, np.uint16),
+                                _p(tree_k, np.uint16), _p(tree_v, np.uint16), _p(parent, np.int32),
+                                _p(prefix_len, np.int32), B, N, Hq, Hkv, d, max_len,
+                                ctypes.c_double(scale), _p(out, np.float64))
+    if rc != 0:
+        raise RuntimeError("oracle_tree_attn failed: %d" % rc)
+    return out
+
+
+def row_stats(logits: np.ndarray, T: float = 1.0):
+    R, V = logits.shape
+    m = np.empty(R, np.float64)
+    s = np.empty(R, np.float64)
+    a = np.empty(R, np.int32)
+    lib().oracle_row_stats(_p(logits, np.float32), R, V, ctypes.c_double(T), _p(m, np.float64),
+                           _p(s, np.float64), _p(a, np.int32))
+    return m, s, a
+
+
+def tree_accept(target_logits, draft_probs, draft_tokens, parent, temperature, uniforms,
+                force: Optional[np.ndarray] = None):
+    """Lossless tree acceptance. Returns a dict with accepted_path [B][N] (-1 padded),
+    n_accepted [B], bonus_token [B] and the fp64 decision trace."""
+    B, N, V = target_logits.shape
+    path = np.empty((B, N), np.int32)
+    n_acc = np.empty(B, np.int32)
+    bonus = np.empty(B, np.int32)
+    trq = np.empty((B, N), np.float64)
+    tp = np.empty((B, N), np.float64)
+    binfo = np.empty((B, 6), np.float64)
+    rc = lib().oracle_tree_accept(_p(target_logits, np.float32), _p(draft_probs, np.float32),
+                                  _p(draft_tokens, np.int32), _p(parent, np.int32),
+                                  _p(temperature, np.float32), _p(uniforms, np.float32),
+                                  _p(force, np.int32), B, N, V, _p(path, np.int32),
+                                  _p(n_acc, np.int32), _p(bonus, np.int32), _p(trq, np.float64),
+                                  _p(tp, np.float64), _p(binfo, np.float64))
+    if rc != 0:
+        raise RuntimeError("oracle_tree_accept failed: %d" % rc)
+    return {"accepted_path": path, "n_accepted": n_acc, "bonus_token": bonus,
+            "trace_rq": trq, "trace_p": tp, "bonus_info": binfo}
+
+
+def kv_compact(cache: np.ndarray, accepted_path, n_accepted, prefix_len):
+    """In-place accepted-path compaction of cache [layers][2][B][Hkv][max_len][d] (uint16)."""
+    n_layers, two, B, Hkv, max_len, d = cache.shape
+    assert two == 2
+    new_len = np.empty(B, np.int32)
+    rc = lib().oracle_kv_compact(_p(cache, np.uint16), _p(accepted_path, np.int32),
+                                 _p(n_accepted, np.int32), _p(prefix_len, np.int32), n_layers, B,
+                                 Hkv, max_len, d, accepted_path.shape[1], _p(new_len, np.int32))
+    if rc != 0:
+        raise RuntimeError("oracle_kv_compact failed: %d" % rc)
+    return new_len

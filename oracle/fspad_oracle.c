@@ -1,0 +1,322 @@
+/*
+ * fp64 CPU oracle for the tree-verification step of lossless speculative
+ * decoding (paper Section "Preliminaries": flattened token tree + attention
+ * mask -> one target forward -> strict comparison, mismatching tokens and
+ * their descendants discarded; Section "Experiments": temperature 0 and 1,
+ * acceptance conditions never relaxed).
+ *
+ * TEST INFRASTRUCTURE ONLY. This file defines what the CUDA library must
+ * compute and is deliberately slow and plain: scalar loops in double
+ * precision, no blocking, no fusion. It shares no code with the CUDA path.
+ * Only the tests, the smoke check and the benchmark's CPU-baseline leg may
+ * call it; the product never does.
+ *
+ * Parity pins (tests/test_oracle_*.py): chain tree == dense causal
+ * attention, per-path brute force, greedy == naive per-path comparison,
+ * exact emitted-token distribution of the rejection sampler at vocab 8,
+ * hand-worked decision traces, brute-force compaction.
+ *
+ * The only parallelism is an OpenMP loop over independent units (heads,
+ * node rows, cache slices); each unit runs the plain definition.
+ *
+ * Conventions (the paper is silent on them; they are the library's stated
+ * reading): node 0 is the root (last emitted token, always accepted,
+ * parent[0] = -1); nodes are in topological order (parent[i] < i); children
+ * are visited in increasing node index; kv head of query head h is
+ * h / (Hq / Hkv); softmax scale is passed in; bf16 inputs are converted to
+ * double exactly.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+static double bf16_to_f64(uint16_t h)
+{
+    uint32_t u = (uint32_t)h << 16;
+    float f;
+    memcpy(&f, &u, sizeof f);
+    return (double)f;
+}
+
+/* ------------------------------------------------------------------------
+ * Tree-masked verify attention ("Preliminaries": the mask built from the
+ * token tree makes every token see only what it depends on).
+ * Query node i sees the L cached prefix keys and tree key j iff j == i or j
+ * is an ancestor of i.  out = softmax(q.k * scale) . v over that set.
+ *
+ *   q        [B][N][Hq][d]        bf16 bits
+ *   k_cache  [B][Hkv][max_len][d] bf16 bits (v_cache alike)
+ *   tree_k   [B][Hkv][N][d]       bf16 bits, or NULL: tree rows are cache
+ *                                 rows prefix_len[b] .. prefix_len[b]+N-1
+ *   out      [B][N][Hq][d]        double
+ * ---------------------------------------------------------------------- */
+int oracle_tree_attn(const uint16_t *q, const uint16_t *k_cache, const uint16_t *v_cache,
+                     const uint16_t *tree_k, const uint16_t *tree_v, const int32_t *parent,
+                     const int32_t *prefix_len, int B, int N, int Hq, int Hkv, int d, int max_len,
+                     double scale, double *out)
+{
+    if (Hkv <= 0 || Hq % Hkv != 0) return -1;
+    const int G = Hq / Hkv;
+    int bad = 0;
+#pragma omp parallel for collapse(2) schedule(dynamic)
+    for (int b = 0; b < B; ++b) {
+        for (int h = 0; h < Hq; ++h) {
+            const int g = h / G;
+            const int L = prefix_len[b];
+            const int32_t *par = parent + (size_t)b * N;
+            double *s = (double *)malloc(sizeof(double) * (size_t)(L + N));
+            char *vis = (char *)malloc((size_t)N);
+            if (!s || !vis) { bad = 1; free(s); free(vis); continue; }
+            const uint16_t *kc = k_cache + ((size_t)b * Hkv + g) * (size_t)max_len * d;
+            const uint16_t *vc = v_cache + ((size_t)b * Hkv + g) * (size_t)max_len * d;
+            const uint16_t *tk = tree_k ? tree_k + ((size_t)b * Hkv + g) * (size_t)N * d
+                                        : kc + (size_t)L * d;
+            const uint16_t *tv = tree_v ? tree_v + ((size_t)b * Hkv + g) * (size_t)N * d
+                                        : vc + (size_t)L * d;
+            for (int i = 0; i < N; ++i) {
+                const uint16_t *qi = q + (((size_t)b * N + i) * Hq + h) * d;
+                memset(vis, 0, (size_t)N);
+                for (int a = i; a >= 0; a = par[a]) vis[a] = 1;
+                double m = -INFINITY;
+                for (int t = 0; t < L + N; ++t) {
+                    if (t >= L && !vis[t - L]) { s[t] = -INFINITY; continue; }
+                    const uint16_t *kr = t < L ? kc + (size_t)t * d : tk + (size_t)(t - L) * d;
+                    double acc = 0.0;
+                    for (int c = 0; c < d; ++c) acc += bf16_to_f64(qi[c]) * bf16_to_f64(kr[c]);
+                    s[t] = acc * scale;
+                    if (s[t] > m) m = s[t];
+                }
+                double denom = 0.0;
+                for (int t = 0; t < L + N; ++t) {
+                    s[t] = (s[t] == -INFINITY) ? 0.0 : exp(s[t] - m);
+                    denom += s[t];
+                }
+                double *o = out + (((size_t)b * N + i) * Hq + h) * d;
+                for (int c = 0; c < d; ++c) o[c] = 0.0;
+                for (int t = 0; t < L + N; ++t) {
+                    if (s[t] == 0.0) continue;
+                    const uint16_t *vr = t < L ? vc + (size_t)t * d : tv + (size_t)(t - L) * d;
+                    for (int c = 0; c < d; ++c) o[c] += s[t] * bf16_to_f64(vr[c]);
+                }
+                for (int c = 0; c < d; ++c) o[c] /= denom;
+            }
+            free(s);
+            free(vis);
+        }
+    }
+    return bad ? -2 : 0;
+}
+
+/* ------------------------------------------------------------------------
+ * Per-node vocabulary scan: m = max logit, a = its lowest index,
+ * S = sum_j exp((x_j - m) / T)   (T <= 0 is treated as 1 for S).
+ *   logits [R][V] fp32 ; row_max, row_sum double [R] ; row_arg int32 [R]
+ * ---------------------------------------------------------------------- */
+int oracle_row_stats(const float *logits, int R, int V, double T, double *row_max, double *row_sum,
+                     int32_t *row_arg)
+{
+    const double Td = T > 0.0 ? T : 1.0;
+#pragma omp parallel for schedule(static)
+    for (int r = 0; r < R; ++r) {
+        const float *x = logits + (size_t)r * V;
+        double m = -INFINITY;
+        int a = 0;
+        for (int j = 0; j < V; ++j)
+            if ((double)x[j] > m) { m = (double)x[j]; a = j; }
+        double S = 0.0;
+        for (int j = 0; j < V; ++j) S += exp(((double)x[j] - m) / Td);
+        row_max[r] = m;
+        row_sum[r] = S;
+        row_arg[r] = a;
+    }
+    return 0;
+}
+
+/* Inverse-CDF draw: weights w_j >= 0 summed in index order to Z; the token is
+ * the smallest j whose running sum exceeds u*Z; if rounding leaves none, the
+ * largest j with w_j > 0.  info (may be NULL) receives
+ * {u*Z, lower edge, upper edge, Z, previous positive token, next positive token}. */
+static int inverse_cdf(const double *w, int V, double u, double *info)
+{
+    double Z = 0.0;
+    for (int j = 0; j < V; ++j) Z += w[j];
+    const double target = u * Z;
+    double run = 0.0, lo = 0.0;
+    int tok = -1;
+    for (int j = 0; j < V; ++j) {
+        lo = run;
+        run += w[j];
+        if (run > target) { tok = j; break; }
+    }
+    if (tok < 0) {
+        for (int j = V - 1; j >= 0; --j)
+            if (w[j] > 0.0) { tok = j; break; }
+        if (tok < 0) tok = 0;
+        lo = run - w[tok];
+    }
+    if (info) {
+        int prev = -1, next = -1;
+        for (int j = tok - 1; j >= 0; --j) if (w[j] > 0.0) { prev = j; break; }
+        for (int j = tok + 1; j < V; ++j) if (w[j] > 0.0) { next = j; break; }
+        info[0] = target; info[1] = lo; info[2] = lo + w[tok]; info[3] = Z;
+        info[4] = (double)prev; info[5] = (double)next;
+    }
+    return tok;
+}
+
+/* ------------------------------------------------------------------------
+ * Lossless tree acceptance ("Preliminaries": strict comparison, differing
+ * tokens and their descendants discarded; "Experiments": T = 0 greedy,
+ * T = 1 sampling with unrelaxed acceptance).
+ *
+ * Per sequence b:
+ *   T == 0: from cur = root, accept the first child (index order) whose
+ *           token equals argmax of cur's target row (lowest index on ties);
+ *           stop when none matches; bonus = argmax of the last node's row.
+ *   T  > 0: recursive speculative rejection sampling.  At node cur,
+ *           p = softmax(logits[cur] / T), q = draft_probs[cur].  For each
+ *           child c in index order with token x and uniform r = uniforms[c]:
+ *           accept iff r * q[x] < p[x]; on reject, p <- normalise(max(p - q, 0))
+ *           (p kept if that sum is 0), q[x] <- 0, q <- q / sum(q) (kept if 0).
+ *           When no child is accepted (or cur is a leaf) the bonus token is
+ *           the inverse-CDF draw from the current p with uniforms[N].
+ *
+ *   target_logits [B][N][V] fp32 ; draft_probs [B][N][V] fp32 (NULL if every T is 0)
+ *   draft_tokens, parent [B][N] int32 ; temperature [B] fp32 ; uniforms [B][N+1] fp32
+ *   force [B][N] int32 or NULL: 0 reject / 1 accept overrides the test at that child, -1 natural
+ *   accepted_path [B][N] int32 (-1 padded) ; n_accepted [B] ; bonus_token [B]
+ *   trace_rq, trace_p [B][N] double or NULL: r*q[x] and p[x] at each tested child (NaN if untested)
+ *   bonus_info [B][6] double or NULL: see inverse_cdf (greedy: all zero)
+ * ---------------------------------------------------------------------- */
+int oracle_tree_accept(const float *target_logits, const float *draft_probs,
+                       const int32_t *draft_tokens, const int32_t *parent, const float *temperature,
+                       const float *uniforms, const int32_t *force, int B, int N, int V,
+                       int32_t *accepted_path, int32_t *n_accepted, int32_t *bonus_token,
+                       double *trace_rq, double *trace_p, double *bonus_info)
+{
+    int bad = 0;
+    for (int b = 0; b < B; ++b) {
+        const float *lg = target_logits + (size_t)b * N * V;
+        const int32_t *par = parent + (size_t)b * N;
+        const int32_t *tok = draft_tokens + (size_t)b * N;
+        const int32_t *frc = force ? force + (size_t)b * N : NULL;
+        int32_t *path = accepted_path + (size_t)b * N;
+        const double T = (double)temperature[b];
+        for (int i = 0; i < N; ++i) path[i] = -1;
+        if (trace_rq) for (int i = 0; i < N; ++i) trace_rq[(size_t)b * N + i] = NAN;
+        if (trace_p) for (int i = 0; i < N; ++i) trace_p[(size_t)b * N + i] = NAN;
+        if (bonus_info) for (int i = 0; i < 6; ++i) bonus_info[(size_t)b * 6 + i] = 0.0;
+
+        /* step: per-node vocabulary scan over all N rows */
+        double *rmax = (double *)malloc(sizeof(double) * N);
+        double *rsum = (double *)malloc(sizeof(double) * N);
+        int32_t *rarg = (int32_t *)malloc(sizeof(int32_t) * N);
+        if (!rmax || !rsum || !rarg) { free(rmax); free(rsum); free(rarg); return -2; }
+        oracle_row_stats(lg, N, V, T, rmax, rsum, rarg);
+
+        int cur = 0, len = 1;
+        path[0] = 0;
+        if (!(T > 0.0)) {
+            for (;;) {
+                int next = -1;
+                for (int c = cur + 1; c < N; ++c) {
+                    if (par[c] != cur) continue;
+                    int take = tok[c] == rarg[cur];
+                    if (frc && frc[c] >= 0) take = frc[c];
+                    if (take) { next = c; break; }
+                }
+                if (next < 0) break;
+                path[len++] = next;
+                cur = next;
+            }
+            bonus_token[b] = rarg[cur];
+        } else {
+            if (!draft_probs || !uniforms) { free(rmax); free(rsum); free(rarg); return -3; }
+            const float *dp = draft_probs + (size_t)b * N * V;
+            const float *un = uniforms + (size_t)b * (N + 1);
+            double *p = (double *)malloc(sizeof(double) * V);
+            double *qd = (double *)malloc(sizeof(double) * V);
+            if (!p || !qd) { bad = 1; free(p); free(qd); free(rmax); free(rsum); free(rarg); break; }
+            for (;;) {
+                const float *x = lg + (size_t)cur * V;
+                for (int j = 0; j < V; ++j) p[j] = exp(((double)x[j] - rmax[cur]) / T) / rsum[cur];
+                for (int j = 0; j < V; ++j) qd[j] = (double)dp[(size_t)cur * V + j];
+                int next = -1;
+                for (int c = cur + 1; c < N; ++c) {
+                    if (par[c] != cur) continue;
+                    const int xt = tok[c];
+                    const double rq = (double)un[c] * qd[xt];
+                    if (trace_rq) trace_rq[(size_t)b * N + c] = rq;
+                    if (trace_p) trace_p[(size_t)b * N + c] = p[xt];
+                    int take = rq < p[xt];
+                    if (frc && frc[c] >= 0) take = frc[c];
+                    if (take) { next = c; break; }
+                    /* residual target distribution */
+                    double Z = 0.0;
+                    for (int j = 0; j < V; ++j) {
+                        double wj = p[j] - qd[j];
+                        Z += wj > 0.0 ? wj : 0.0;
+                    }
+                    if (Z > 0.0)
+                        for (int j = 0; j < V; ++j) {
+                            double wj = p[j] - qd[j];
+                            p[j] = (wj > 0.0 ? wj : 0.0) / Z;
+                        }
+                    /* draft distribution without the rejected token */
+                    qd[xt] = 0.0;
+                    double s = 0.0;
+                    for (int j = 0; j < V; ++j) s += qd[j];
+                    if (s > 0.0)
+                        for (int j = 0; j < V; ++j) qd[j] /= s;
+                }
+                if (next < 0) break;
+                path[len++] = next;
+                cur = next;
+            }
+            bonus_token[b] = inverse_cdf(p, V, (double)un[N], bonus_info ? bonus_info + (size_t)b * 6 : NULL);
+            free(p);
+            free(qd);
+        }
+        n_accepted[b] = len;
+        free(rmax); free(rsum); free(rarg);
+    }
+    return bad ? -2 : 0;
+}
+
+/* ------------------------------------------------------------------------
+ * Accepted-path KV compaction ("Preliminaries": rejected tokens are
+ * discarded, so only the accepted path's rows stay in the cache).
+ * For every layer, K and V, sequence, kv head: row L + path[j] moves to row
+ * L + j for j = 0 .. n-1, as if all moves happened at once.  Rows at or after
+ * L + n are left untouched.  new_len[b] = L + n.
+ *   cache [layers][2][B][Hkv][max_len][d] bf16 bits, in place
+ * ---------------------------------------------------------------------- */
+int oracle_kv_compact(uint16_t *cache, const int32_t *accepted_path, const int32_t *n_accepted,
+                      const int32_t *prefix_len, int n_layers, int B, int Hkv, int max_len, int d,
+                      int path_stride, int32_t *new_len)
+{
+    int bad = 0;
+#pragma omp parallel for collapse(2) schedule(static)
+    for (int l = 0; l < n_layers; ++l) {
+        for (int kv = 0; kv < 2; ++kv) {
+            for (int b = 0; b < B; ++b) {
+                const int L = prefix_len[b], n = n_accepted[b];
+                const int32_t *path = accepted_path + (size_t)b * path_stride;
+                uint16_t *tmp = (uint16_t *)malloc(sizeof(uint16_t) * (size_t)(n > 0 ? n : 1) * d);
+                if (!tmp) { bad = 1; continue; }
+                for (int h = 0; h < Hkv; ++h) {
+                    uint16_t *base = cache + ((((size_t)l * 2 + kv) * B + b) * Hkv + h) * (size_t)max_len * d;
+                    for (int j = 0; j < n; ++j)
+                        memcpy(tmp + (size_t)j * d, base + (size_t)(L + path[j]) * d, sizeof(uint16_t) * d);
+                    for (int j = 0; j < n; ++j)
+                        memcpy(base + (size_t)(L + j) * d, tmp + (size_t)j * d, sizeof(uint16_t) * d);
+                }
+                free(tmp);
+            }
+        }
+    }
+    if (new_len)
+        for (int b = 0; b < B; ++b) new_len[b] = prefix_len[b] + n_accepted[b];
+    return bad ? -2 : 0;
+}
