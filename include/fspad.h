@@ -1,0 +1,200 @@
+/*
+ * fspad.h - C ABI of the B200 (sm_100a) tree-verification library.
+ *
+ * One verify step of lossless speculative decoding, as the paper states it
+ * (Section "Preliminaries"): the target model runs once over the flattened
+ * draft tree under a mask that lets every token see only what it depends on,
+ * its results are compared strictly with the tree, and mismatching tokens and
+ * their descendants are discarded.  Three operations:
+ *
+ *   fspad_tree_attn    tree-masked verify attention of one layer
+ *   fspad_tree_accept  lossless acceptance (greedy, or recursive rejection
+ *                      sampling at temperature > 0; Section "Experiments"
+ *                      evaluates T = 0 and T = 1 with unrelaxed acceptance)
+ *   fspad_kv_compact   keep the accepted path's K/V rows, contiguous in the cache
+ *
+ * Conventions (shared by every call)
+ *   - A tree has N <= 64 nodes in topological order: parent[0] = -1 (node 0 is
+ *     the root = the last token already emitted; it is always accepted) and
+ *     0 <= parent[i] < i.  Children of a node are visited in increasing index.
+ *   - "bf16" is a 16-bit brain-float bit pattern (typedef below).
+ *   - Unless a parameter says "host", every pointer is a DEVICE pointer owned by
+ *     the caller, 16-byte aligned, valid until the work queued on `stream` has
+ *     finished.  The library never frees or reallocates caller memory.
+ *   - Calls are asynchronous on `stream` (a cudaStream_t passed as void*; NULL =
+ *     the default stream).  Calls that share a context must be queued on one
+ *     stream at a time (the context owns scratch buffers).
+ *   - Return value: 0 (FSPAD_OK) or a negative fspad_error.  Errors detectable
+ *     on the host are returned before anything is launched.  Errors only the
+ *     device can see (a malformed parent[] array, a prefix length that does not
+ *     fit) are recorded in the context's status word, read by fspad_status();
+ *     the outputs of that call are then unspecified but every access stays
+ *     inside the caller's buffers.  Nothing traps, asserts or exits.
+ */
+#ifndef FSPAD_H
+#define FSPAD_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef uint16_t fspad_bf16;
+typedef struct fspad_ctx fspad_ctx;
+
+typedef enum {
+    FSPAD_OK = 0,
+    FSPAD_ERR_NULL = -1,           /* a required pointer is NULL                       */
+    FSPAD_ERR_ALIGN = -2,          /* a pointer is not 16-byte aligned                 */
+    FSPAD_ERR_SHAPE = -3,          /* sizes inconsistent with the context              */
+    FSPAD_ERR_TREE_TOO_LARGE = -4, /* n_nodes > 64 or > max_nodes                      */
+    FSPAD_ERR_RANGE = -5,          /* prefix_len + n_nodes > max_len, T < 0 or NaN     */
+    FSPAD_ERR_CUDA = -6,           /* a CUDA runtime call or launch failed             */
+    FSPAD_ERR_TIMEOUT = -7,        /* a bounded device-side wait ran out               */
+    FSPAD_ERR_BAD_TREE = -8,       /* parent[0] != -1 or parent[i] outside [0, i)      */
+    FSPAD_ERR_NOMEM = -9           /* device or host allocation failed at create time  */
+} fspad_error;
+
+typedef struct {
+    int n_q_heads;        /* Hq                                                     */
+    int n_kv_heads;       /* Hkv, divides Hq; query head h uses kv head h/(Hq/Hkv)   */
+    int head_dim;         /* d, must be 128                                         */
+    int max_nodes;        /* largest N any call will pass, 1..64                    */
+    int vocab;            /* V                                                      */
+    int n_layers;         /* layers in the cache handed to fspad_kv_compact          */
+    int max_len;          /* rows per (sequence, kv head) of the cache               */
+    int max_batch;        /* largest batch any call will pass                       */
+    float softmax_scale;  /* 0 selects 1/sqrt(d)                                    */
+} fspad_config;
+
+/* Create a context on the CURRENT device: allocates the scratch buffers every
+ * call needs (split-KV partials, per-node statistics, staging for the host
+ * entry point), sized from `cfg`.  Synchronous.  *out is NULL on failure. */
+int fspad_create(const fspad_config *cfg, fspad_ctx **out);
+
+/* Free everything the context owns.  Synchronises the device first. */
+void fspad_destroy(fspad_ctx *ctx);
+
+/* Synchronise `stream`, return the first device-recorded error since the last
+ * call (FSPAD_OK if none) and clear it. */
+int fspad_status(fspad_ctx *ctx, void *stream);
+
+/* Static, human-readable name of an fspad_error. */
+const char *fspad_strerror(int err);
+
+/* Number of kernels the library has launched through this context so far
+ * (host counter; lets a caller verify that work ran on the device). */
+long long fspad_launch_count(const fspad_ctx *ctx);
+
+/*
+ * Tree-masked verify attention of one layer ("Preliminaries": the flattened
+ * token tree is the target's input and the attention mask built from the tree
+ * introduces the dependencies between its tokens).
+ *
+ * For sequence b, query node i and query head h (kv head g = h / (Hq/Hkv)):
+ *   keys   = cache rows 0 .. L_b-1 of kv head g   (L_b = prefix_len[b])
+ *          + tree row j for every j that is i itself or an ancestor of i
+ *   out[b][i][h] = softmax(q[b][i][h] . k * softmax_scale) . v     over those keys
+ * bf16 inputs, fp32 accumulation and softmax, bf16 output (round to nearest even).
+ * q/k are used as given: no positional encoding is applied here.
+ *
+ *   q        [batch][n_nodes][Hq][d]
+ *   k_cache, v_cache   [batch][Hkv][max_len][d]
+ *   tree_k, tree_v     [batch][Hkv][n_nodes][d]; both may be NULL, in which case
+ *            the tree rows are cache rows L_b .. L_b+n_nodes-1 of the same sequence
+ *   parent   [batch][n_nodes] int32      prefix_len [batch] int32
+ *   out      [batch][n_nodes][Hq][d]     (must not alias an input)
+ * Requires 0 <= L_b and L_b + n_nodes <= max_len (device-checked: FSPAD_ERR_RANGE).
+ */
+int fspad_tree_attn(fspad_ctx *ctx, const fspad_bf16 *q, const fspad_bf16 *k_cache,
+                    const fspad_bf16 *v_cache, const fspad_bf16 *tree_k, const fspad_bf16 *tree_v,
+                    const int32_t *parent, const int32_t *prefix_len, int n_nodes, int batch,
+                    fspad_bf16 *out, void *stream);
+
+/*
+ * Lossless tree acceptance ("Preliminaries": strict comparison of the tree with
+ * the target's results, differing tokens and their descendants discarded;
+ * "Experiments": greedy T = 0 and sampling T = 1, acceptance never relaxed).
+ *
+ * Per sequence b with T = temperature[b]:
+ *   T == 0  walk from the root; at node cur accept the first child (index order)
+ *           whose draft token equals argmax(target_logits[cur]) (lowest index on
+ *           ties); stop when no child matches; bonus = argmax of the last node.
+ *   T  > 0  recursive rejection sampling.  p = softmax(target_logits[cur]/T),
+ *           q = draft_probs[cur].  For each child c (index order) with token x:
+ *           accept iff uniforms[c] * q[x] < p[x]; on reject p <- normalise(
+ *           max(p - q, 0)) (unchanged if that sum is 0), q[x] <- 0, q <- q/sum(q).
+ *           When no child is accepted the bonus token is the inverse-CDF draw of
+ *           the current p with uniforms[n_nodes]: the smallest token whose running
+ *           sum (index order) exceeds u * sum; the largest positive-weight token
+ *           if rounding leaves none.  Decisive scalars are evaluated in fp64.
+ *   The rule at T > 0 is exactly lossless when the children of a node were drawn
+ *   one after another without replacement from draft_probs[node].
+ *
+ *   target_logits [batch][n_nodes][V] fp32 (finite or -inf; NaN is a precondition violation)
+ *   draft_probs   [batch][n_nodes][V] fp32 >= 0; may be NULL iff every temperature is 0
+ *   draft_tokens, parent  [batch][n_nodes] int32, tokens in [0, V)
+ *   temperature   [batch] fp32 >= 0
+ *   uniforms      [batch][n_nodes+1] fp32 in [0,1); may be NULL iff draft_probs is NULL
+ *   accepted_path [batch][max_nodes] int32: node ids from the root, -1 padded
+ *   n_accepted    [batch] int32: nodes on the path, root included
+ *   bonus_token   [batch] int32
+ * Outputs stay on the device so fspad_kv_compact can consume them without a host sync.
+ */
+int fspad_tree_accept(fspad_ctx *ctx, const float *target_logits, const float *draft_probs,
+                      const int32_t *draft_tokens, const int32_t *parent, const float *temperature,
+                      const float *uniforms, int n_nodes, int batch, int32_t *accepted_path,
+                      int32_t *n_accepted, int32_t *bonus_token, void *stream);
+
+/*
+ * The first stage of fspad_tree_accept on its own: one pass over every row of
+ * logits [rows][V] giving row_max (fp32 maximum), row_arg (its lowest index)
+ * and row_sum = sum_j exp((x_j - max)/T_row) accumulated from fp32 exponentials
+ * (relative accuracy about 1e-6; the acceptance walk re-derives exact sums
+ * where a decision is close).  temperature [rows / rows_per_seq] fp32, 0 -> 1.
+ */
+int fspad_accept_stats(fspad_ctx *ctx, const float *logits, const float *temperature, int rows,
+                       int rows_per_seq, float *row_max, double *row_sum, int32_t *row_arg,
+                       void *stream);
+
+/*
+ * Accepted-path KV compaction ("Preliminaries": the discarded tokens leave the
+ * sequence; only the accepted path continues it).  For every layer, K and V,
+ * sequence b and kv head: row L_b + accepted_path[b][j] moves to row L_b + j for
+ * j = 0 .. n_accepted[b]-1, as if all moves happened at once (a destination may
+ * be another move's source).  Rows >= L_b + n_accepted[b] keep their old
+ * contents and are dead.  new_len[b] = L_b + n_accepted[b] (may be NULL).
+ *
+ *   cache [n_layers][2][batch][Hkv][max_len][d] bf16, updated in place
+ *   accepted_path [batch][max_nodes], n_accepted [batch], prefix_len [batch], new_len [batch]: int32
+ */
+int fspad_kv_compact(fspad_ctx *ctx, fspad_bf16 *cache, const int32_t *accepted_path,
+                     const int32_t *n_accepted, const int32_t *prefix_len, int batch,
+                     int32_t *new_len, void *stream);
+
+/*
+ * One whole verify step from HOST buffers: copies the step's inputs to device
+ * staging owned by the context, writes the tree rows into cache rows L_b.. of
+ * layer 0, runs fspad_tree_attn, fspad_tree_accept and fspad_kv_compact on
+ * `stream`, copies the results back and synchronises the stream.  The KV cache
+ * is device-resident state that persists between steps (the caller's device
+ * pointer `cache`, layout as in fspad_kv_compact); everything else is host
+ * memory (pinned memory makes the copies asynchronous).  Host outputs:
+ * attn_out [batch][n_nodes][Hq][d] bf16, accepted_path [batch][max_nodes],
+ * n_accepted, bonus_token, new_len [batch].  draft_probs/uniforms may be NULL
+ * when every temperature is 0.  Returns the first host- or device-detected error.
+ */
+int fspad_verify_step_host(fspad_ctx *ctx, fspad_bf16 *cache /* device */,
+                           const fspad_bf16 *q, const fspad_bf16 *tree_k, const fspad_bf16 *tree_v,
+                           const int32_t *parent, const int32_t *prefix_len,
+                           const float *target_logits, const float *draft_probs,
+                           const int32_t *draft_tokens, const float *temperature,
+                           const float *uniforms, int n_nodes, int batch, fspad_bf16 *attn_out,
+                           int32_t *accepted_path, int32_t *n_accepted, int32_t *bonus_token,
+                           int32_t *new_len, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FSPAD_H */

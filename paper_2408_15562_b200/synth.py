@@ -313,7 +313,7 @@ def hashed_u16(shape, salt: int) -> np.ndarray:
     """Deterministic 16-bit filler (an integer hash of the flat index); used for
     the cache layers that only the byte-copy compaction touches."""
     n = int(np.prod(shape))
-    i = np.arange(n, dtype=np.uint64) + np.uint64(salt) * np.uint64(0x9E3779B97F4A7C15)
+    i = np.arange(n, dtype=np.uint64) + np.uint64((int(salt) * 0x9E3779B97F4A7C15) & 0xFFFFFFFFFFFFFFFF)
     i ^= i >> np.uint64(33)
     i *= np.uint64(0xFF51AFD7ED558CCD)
     i ^= i >> np.uint64(29)
