@@ -1,0 +1,208 @@
+"""Thin ctypes binding of libfspad.so: argument marshalling only.
+
+Every function takes torch tensors (device memory, streams), checks dtype,
+shape and contiguity, and forwards raw pointers to the C ABI declared in
+`include/fspad.h`.  No step of the verify path is computed here, and there is
+no fallback: if the library has not been built the first call raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libfspad.so")
+_lib = None
+
+EXPORTS = ["fspad_create", "fspad_destroy", "fspad_status", "fspad_strerror", "fspad_launch_count",
+           "fspad_tree_attn", "fspad_tree_accept", "fspad_accept_stats", "fspad_kv_compact",
+           "fspad_verify_step_host"]
+
+
+class FspadConfig(ctypes.Structure):
+    _fields_ = [("n_q_heads", ctypes.c_int), ("n_kv_heads", ctypes.c_int), ("head_dim", ctypes.c_int),
+                ("max_nodes", ctypes.c_int), ("vocab", ctypes.c_int), ("n_layers", ctypes.c_int),
+                ("max_len", ctypes.c_int), ("max_batch", ctypes.c_int), ("softmax_scale", ctypes.c_float)]
+
+
+class FspadError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__("%s: %s (%d)" % (where, strerror(code), code))
+
+
+def load():
+    """Open libfspad.so (built in-tree by `python -m paper_2408_15562_b200.build`)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError("libfspad.so is missing: build it with `python -m paper_2408_15562_b200.build` "
+                           "(there is no CPU or PyTorch fallback)")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, ci = ctypes.c_void_p, ctypes.c_int
+    lib.fspad_create.argtypes = [ctypes.POINTER(FspadConfig), ctypes.POINTER(vp)]
+    lib.fspad_destroy.argtypes = [vp]
+    lib.fspad_destroy.restype = None
+    lib.fspad_status.argtypes = [vp, vp]
+    lib.fspad_strerror.argtypes = [ci]
+    lib.fspad_strerror.restype = ctypes.c_char_p
+    lib.fspad_launch_count.argtypes = [vp]
+    lib.fspad_launch_count.restype = ctypes.c_longlong
+    lib.fspad_tree_attn.argtypes = [vp] * 8 + [ci, ci, vp, vp]
+    lib.fspad_tree_accept.argtypes = [vp] * 7 + [ci, ci, vp, vp, vp, vp]
+    lib.fspad_accept_stats.argtypes = [vp, vp, vp, ci, ci, vp, vp, vp, vp]
+    lib.fspad_kv_compact.argtypes = [vp, vp, vp, vp, vp, ci, vp, vp]
+    lib.fspad_verify_step_host.argtypes = [vp] * 12 + [ci, ci] + [vp] * 6
+    _lib = lib
+    return lib
+
+
+def strerror(code: int) -> str:
+    return load().fspad_strerror(code).decode()
+
+
+def _ptr(t: Optional[torch.Tensor], dtype, device_type: str = "cuda"):
+    if t is None:
+        return None
+    if t.dtype != dtype:
+        raise TypeError("expected %s, got %s" % (dtype, t.dtype))
+    if not t.is_contiguous():
+        raise ValueError("tensor must be contiguous")
+    if t.device.type != device_type:
+        raise ValueError("tensor must live on %s, not %s" % (device_type, t.device))
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream: Optional[torch.cuda.Stream]):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+class Context:
+    """Owns an `fspad_ctx` on the current CUDA device."""
+
+    def __init__(self, n_q_heads: int, n_kv_heads: int, vocab: int, max_len: int, max_nodes: int = 64,
+                 n_layers: int = 1, max_batch: int = 1, head_dim: int = 128, softmax_scale: float = 0.0):
+        if not torch.cuda.is_available():
+            raise RuntimeError("fspad needs a CUDA device (there is no CPU fallback)")
+        self.cfg = FspadConfig(n_q_heads, n_kv_heads, head_dim, max_nodes, vocab, n_layers, max_len,
+                               max_batch, softmax_scale)
+        self._h = ctypes.c_void_p()
+        rc = load().fspad_create(ctypes.byref(self.cfg), ctypes.byref(self._h))
+        if rc != 0:
+            raise FspadError(rc, "fspad_create")
+
+    def close(self):
+        if getattr(self, "_h", None) is not None and self._h.value:
+            load().fspad_destroy(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -- raw return-code forms (used by the boundary tests) -----------------
+    def status(self, stream=None) -> int:
+        return load().fspad_status(self._h, _stream(stream))
+
+    def launch_count(self) -> int:
+        return int(load().fspad_launch_count(self._h))
+
+    def check(self, stream=None):
+        rc = self.status(stream)
+        if rc != 0:
+            raise FspadError(rc, "device status")
+
+    # -- the three operations --------------------------------------------------
+    def tree_attn(self, q, k_cache, v_cache, tree_k, tree_v, parent, prefix_len, out=None, stream=None):
+        B, N = q.shape[0], q.shape[1]
+        if out is None:
+            out = torch.empty_like(q)
+        bf = torch.bfloat16
+        rc = load().fspad_tree_attn(self._h, _ptr(q, bf), _ptr(k_cache, bf), _ptr(v_cache, bf),
+                                    _ptr(tree_k, bf), _ptr(tree_v, bf), _ptr(parent, torch.int32),
+                                    _ptr(prefix_len, torch.int32), N, B, _ptr(out, bf), _stream(stream))
+        if rc != 0:
+            raise FspadError(rc, "fspad_tree_attn")
+        return out
+
+    def tree_accept(self, target_logits, draft_probs, draft_tokens, parent, temperature, uniforms,
+                    accepted_path=None, n_accepted=None, bonus_token=None, stream=None):
+        B, N = target_logits.shape[0], target_logits.shape[1]
+        dev = target_logits.device
+        if accepted_path is None:
+            accepted_path = torch.empty((B, self.cfg.max_nodes), dtype=torch.int32, device=dev)
+        if n_accepted is None:
+            n_accepted = torch.empty((B,), dtype=torch.int32, device=dev)
+        if bonus_token is None:
+            bonus_token = torch.empty((B,), dtype=torch.int32, device=dev)
+        f32, i32 = torch.float32, torch.int32
+        rc = load().fspad_tree_accept(self._h, _ptr(target_logits, f32), _ptr(draft_probs, f32),
+                                      _ptr(draft_tokens, i32), _ptr(parent, i32), _ptr(temperature, f32),
+                                      _ptr(uniforms, f32), N, B, _ptr(accepted_path, i32),
+                                      _ptr(n_accepted, i32), _ptr(bonus_token, i32), _stream(stream))
+        if rc != 0:
+            raise FspadError(rc, "fspad_tree_accept")
+        return accepted_path, n_accepted, bonus_token
+
+    def accept_stats(self, logits, temperature, rows_per_seq, stream=None):
+        rows = logits.shape[0]
+        dev = logits.device
+        row_max = torch.empty((rows,), dtype=torch.float32, device=dev)
+        row_sum = torch.empty((rows,), dtype=torch.float64, device=dev)
+        row_arg = torch.empty((rows,), dtype=torch.int32, device=dev)
+        rc = load().fspad_accept_stats(self._h, _ptr(logits, torch.float32), _ptr(temperature, torch.float32),
+                                       rows, rows_per_seq, _ptr(row_max, torch.float32),
+                                       _ptr(row_sum, torch.float64), _ptr(row_arg, torch.int32),
+                                       _stream(stream))
+        if rc != 0:
+            raise FspadError(rc, "fspad_accept_stats")
+        return row_max, row_sum, row_arg
+
+    def kv_compact(self, cache, accepted_path, n_accepted, prefix_len, new_len=None, stream=None):
+        B = prefix_len.shape[0]
+        if new_len is None:
+            new_len = torch.empty((B,), dtype=torch.int32, device=cache.device)
+        i32 = torch.int32
+        rc = load().fspad_kv_compact(self._h, _ptr(cache, torch.bfloat16), _ptr(accepted_path, i32),
+                                     _ptr(n_accepted, i32), _ptr(prefix_len, i32), B, _ptr(new_len, i32),
+                                     _stream(stream))
+        if rc != 0:
+            raise FspadError(rc, "fspad_kv_compact")
+        return new_len
+
+    def verify_step_host(self, cache, q, tree_k, tree_v, parent, prefix_len, target_logits, draft_probs,
+                         draft_tokens, temperature, uniforms, attn_out, accepted_path, n_accepted,
+                         bonus_token, new_len, stream=None):
+        """All tensors except `cache` are HOST tensors (pinned recommended); outputs are written in place."""
+        B, N = q.shape[0], q.shape[1]
+        bf, f32, i32 = torch.bfloat16, torch.float32, torch.int32
+        h = "cpu"
+        rc = load().fspad_verify_step_host(
+            self._h, _ptr(cache, bf), _ptr(q, bf, h), _ptr(tree_k, bf, h), _ptr(tree_v, bf, h),
+            _ptr(parent, i32, h), _ptr(prefix_len, i32, h), _ptr(target_logits, f32, h),
+            _ptr(draft_probs, f32, h), _ptr(draft_tokens, i32, h), _ptr(temperature, f32, h),
+            _ptr(uniforms, f32, h), N, B, _ptr(attn_out, bf, h), _ptr(accepted_path, i32, h),
+            _ptr(n_accepted, i32, h), _ptr(bonus_token, i32, h), _ptr(new_len, i32, h), _stream(stream))
+        if rc != 0:
+            raise FspadError(rc, "fspad_verify_step_host")
+        return attn_out, accepted_path, n_accepted, bonus_token, new_len
+
+
+def bf16_tensor(bits, device="cuda"):
+    """numpy uint16 bit patterns -> torch.bfloat16 tensor on `device` (no value conversion)."""
+    import numpy as np
+    t = torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).view(torch.bfloat16)
+    return t.to(device) if device != "cpu" else t
+
+
+def bf16_bits(t: torch.Tensor):
+    """torch.bfloat16 tensor -> numpy uint16 bit patterns."""
+    import numpy as np
+    return t.detach().cpu().contiguous().view(torch.int16).numpy().view(np.uint16)

@@ -1,0 +1,485 @@
+// Lossless tree acceptance, second stage: the walk from the root.
+//
+// Greedy (T = 0): strict comparison of each child's draft token with the
+// target's argmax at its parent (paper, Section "Preliminaries": differing
+// tokens and their descendants are discarded).  Sampling (T > 0, Section
+// "Experiments": T = 1 with unrelaxed acceptance): recursive rejection
+// sampling over the children of the current node with residual-distribution
+// resampling over the whole vocabulary.
+//
+// One thread-block cluster serves one sequence.  The walk itself is a short
+// serial chain of scalar decisions taken in fp64; whenever a decision needs a
+// whole-vocabulary quantity (an exact softmax denominator, the mass of a
+// residual distribution, the inverse CDF of the bonus draw) the cluster sweeps
+// the node's logits and draft rows once, every CTA reducing its contiguous
+// slice of the vocabulary and the CTAs exchanging partial sums through
+// distributed shared memory.  Only rows on the realised path are ever read.
+//
+// The residual after k rejections at a node is kept in closed form instead of
+// as a vector: for a token j that has not been rejected,
+//     u_j = max(p_j - c * q_j, 0),   p_j = softmax(logits/T)_j,  q_j = draft_j
+// with one scalar c that grows with every rejection; a rejected token keeps the
+// value it had when it was rejected.  The current target distribution is u / U
+// (U = sum of u) and the current draft distribution is q restricted to the
+// tokens not yet rejected, divided by its sum D.  A rejection of token x turns
+// c into c + U / D, which is exactly p <- norm(max(p - q, 0)), q <- norm(q
+// without x) written without materialising either vector.
+#include <cooperative_groups.h>
+
+#include "common.cuh"
+
+namespace cg = cooperative_groups;
+
+namespace {
+
+constexpr int kMaxCluster = 16;
+constexpr int kWalkThreads = 512;
+constexpr int kWarps = kWalkThreads / 32;
+constexpr double kAmbiguous = 1e-4;   // relative margin inside which the approximate denominator is not trusted
+
+struct WalkArgs {
+    const float *logits, *draft, *temperature, *uniforms;
+    const int *tokens, *parent;
+    const float *row_max;
+    const double *row_sum;
+    const int *row_arg;
+    int N, V, path_stride;
+    int *path, *n_acc, *bonus, *status;
+};
+
+enum { MODE_SUM = 0, MODE_RESID = 1, MODE_CDF = 2 };
+
+struct Shared {
+    int parent[FSPAD_MAX_NODES];
+    int tok[FSPAD_MAX_NODES];
+    int path[FSPAD_MAX_NODES];
+    // state of the current node (written by thread 0, read by all after a barrier)
+    double S, c, U, D, m, T;
+    int exact, nrem, decision, xnew, ridx, next, len, cur;
+    double cprime, ex, qx;
+    int sel;
+    int rem_tok[FSPAD_MAX_NODES];
+    double rem_frozen[FSPAD_MAX_NODES];
+    // reductions
+    double warp_a[kWarps], warp_b[kWarps];
+    double slot[2][2];              // this CTA's partial sums, by pass parity (read by peers)
+    double tot[2];                  // cluster totals, broadcast inside the CTA
+    double cta_total[kMaxCluster];  // CDF: every CTA's total
+    double warp_off[kWarps];
+};
+
+__device__ __forceinline__ double warp_sum(double v)
+{
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+    return v;
+}
+
+// Weight of token j in the current (unnormalised) residual target distribution.
+__device__ __forceinline__ double weight(double e, double q, double invS, double c)
+{
+    const double w = e * invS - c * q;
+    return w > 0.0 ? w : 0.0;
+}
+
+struct Sweep {
+    double a, b;
+};
+
+// One sweep of this thread's contiguous chunk [lo, hi) of the vocabulary.
+//   MODE_SUM  : a = sum exp((x - m)/T)
+//   MODE_RESID: a = sum of residual weights at coefficient c (tokens already
+//               rejected contribute their frozen value), b = sum of q over
+//               tokens neither rejected before nor equal to xnew
+//   MODE_CDF  : a = sum of residual weights at coefficient c
+// When `locate` is set (CDF owner thread) the sweep instead returns in a the
+// first token whose running sum pushes base + run above target (or -1).
+template <int MODE>
+__device__ Sweep sweep_chunk(const Shared &sh, const float *__restrict__ x, const float *__restrict__ q,
+                             int lo, int hi, bool vec, double c, int xnew, bool locate, double base,
+                             double run0, double target, int *found)
+{
+    const double m = sh.m, T = sh.T, invS = 1.0 / sh.S;
+    const int nrem = sh.nrem;
+    bool special = false;
+    if (MODE != MODE_SUM) {
+        for (int r = 0; r < nrem; ++r) special |= (sh.rem_tok[r] >= lo && sh.rem_tok[r] < hi);
+        if (MODE == MODE_RESID) special |= (xnew >= lo && xnew < hi);
+    }
+    double a = 0.0, b = 0.0, run = run0;
+    int last_pos = -1, hit = -1;
+    for (int j = lo; j < hi; j += 4) {
+        float xv[4], qv[4] = {0.f, 0.f, 0.f, 0.f};
+        const int n = min(4, hi - j);
+        const bool need_q = (MODE == MODE_RESID) || (MODE == MODE_CDF && c != 0.0);
+        if (vec && n == 4) {
+            const float4 t = *reinterpret_cast<const float4 *>(x + j);
+            xv[0] = t.x; xv[1] = t.y; xv[2] = t.z; xv[3] = t.w;
+            if (need_q) {
+                const float4 u = *reinterpret_cast<const float4 *>(q + j);
+                qv[0] = u.x; qv[1] = u.y; qv[2] = u.z; qv[3] = u.w;
+            }
+        } else {
+#pragma unroll
+            for (int t = 0; t < 4; ++t) {
+                xv[t] = (t < n) ? x[j + t] : -INFINITY;
+                if (need_q) qv[t] = (t < n) ? q[j + t] : 0.f;
+            }
+        }
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+            if (t >= n) break;
+            const double e = exp(((double)xv[t] - m) / T);
+            if (MODE == MODE_SUM) {
+                a += e;
+                continue;
+            }
+            double w = weight(e, (double)qv[t], invS, c);
+            bool q_counts = true;
+            if (special) {
+                const int id = j + t;
+                for (int r = 0; r < nrem; ++r)
+                    if (sh.rem_tok[r] == id) { w = sh.rem_frozen[r]; q_counts = false; }
+                if (id == xnew) q_counts = false;
+            }
+            if (MODE == MODE_RESID) {
+                a += w;
+                if (q_counts) b += (double)qv[t];
+            } else {
+                a += w;
+                if (locate) {
+                    run += w;
+                    if (w > 0.0) last_pos = j + t;
+                    if (hit < 0 && base + run > target) hit = j + t;
+                }
+            }
+        }
+    }
+    if (locate) *found = (hit >= 0) ? hit : last_pos;
+    return Sweep{a, b};
+}
+
+__global__ void __launch_bounds__(kWalkThreads)
+accept_walk_kernel(const WalkArgs args)
+{
+    cg::cluster_group cluster = cg::this_cluster();
+    const int C = (int)cluster.num_blocks();
+    const int rank = (int)cluster.block_rank();
+    const int b = blockIdx.x / C;
+    const int tid = threadIdx.x, nthr = blockDim.x;
+    const int N = args.N, V = args.V;
+
+    __shared__ Shared sh;
+
+    const int *par_g = args.parent + (size_t)b * N;
+    const int *tok_g = args.tokens + (size_t)b * N;
+    for (int i = tid; i < N; i += nthr) {
+        int p = par_g[i], t = tok_g[i];
+        if (i == 0) {
+            if (p != -1) fspad_report(args.status, FSPAD_ERR_BAD_TREE);
+            p = -1;
+        } else if (p < 0 || p >= i) {
+            fspad_report(args.status, FSPAD_ERR_BAD_TREE);
+            p = 0;
+        }
+        if (t < 0 || t >= V) {
+            fspad_report(args.status, FSPAD_ERR_RANGE);
+            t = 0;
+        }
+        sh.parent[i] = p;
+        sh.tok[i] = t;
+    }
+    float Tf = args.temperature[b];
+    if (!(Tf >= 0.0f)) {
+        if (tid == 0 && rank == 0) fspad_report(args.status, FSPAD_ERR_RANGE);
+        Tf = 0.0f;
+    }
+    const bool sampling = Tf > 0.0f && args.draft != nullptr && args.uniforms != nullptr;
+    if (Tf > 0.0f && !sampling && tid == 0 && rank == 0) fspad_report(args.status, FSPAD_ERR_NULL);
+    __syncthreads();
+
+    const float *lg = args.logits + (size_t)b * N * V;
+    const float *rmax = args.row_max + (size_t)b * N;
+    const double *rsum = args.row_sum + (size_t)b * N;
+    const int *rarg = args.row_arg + (size_t)b * N;
+    int *out_path = args.path + (size_t)b * args.path_stride;
+
+    if (!sampling) {
+        // ---- greedy: strict token comparison against the target argmax ----
+        if (rank == 0 && tid == 0) {
+            int cur = 0, len = 1;
+            sh.path[0] = 0;
+            for (;;) {
+                const int want = rarg[cur];
+                int next = -1;
+                for (int c = cur + 1; c < N; ++c)
+                    if (sh.parent[c] == cur && sh.tok[c] == want) { next = c; break; }
+                if (next < 0) break;
+                sh.path[len++] = next;
+                cur = next;
+            }
+            args.n_acc[b] = len;
+            args.bonus[b] = rarg[cur];
+            sh.len = len;
+        }
+        __syncthreads();
+        if (rank == 0)
+            for (int i = tid; i < args.path_stride; i += nthr) out_path[i] = (i < sh.len) ? sh.path[i] : -1;
+        return;   // the whole cluster takes this branch together; no peer memory is touched
+    }
+
+    // ---- sampling ----
+    const float *dp = args.draft + (size_t)b * N * V;
+    const float *un = args.uniforms + (size_t)b * (N + 1);
+    const bool vec = (V % 4 == 0) && ((reinterpret_cast<uintptr_t>(args.logits) & 15) == 0) &&
+                     ((reinterpret_cast<uintptr_t>(args.draft) & 15) == 0);
+    // contiguous slice per CTA, contiguous chunk per thread (multiples of 4 tokens)
+    const int per_cta = (((V + C - 1) / C) + 3) & ~3;
+    const int per_thr = (((per_cta + nthr - 1) / nthr) + 3) & ~3;
+    const int cta_lo = rank * per_cta, cta_hi = min(V, cta_lo + per_cta);
+    const int lo = min(cta_hi, cta_lo + tid * per_thr), hi = min(cta_hi, lo + per_thr);
+    int parity = 0;
+
+    // cluster-wide reduction of (a, b); result in sh.tot[] for every thread of every CTA
+    auto reduce_exchange = [&](double a, double bb) {
+        a = warp_sum(a);
+        bb = warp_sum(bb);
+        if ((tid & 31) == 0) { sh.warp_a[tid >> 5] = a; sh.warp_b[tid >> 5] = bb; }
+        __syncthreads();
+        if (tid == 0) {
+            double sa = 0.0, sb = 0.0;
+            for (int w = 0; w < nthr / 32; ++w) { sa += sh.warp_a[w]; sb += sh.warp_b[w]; }
+            sh.slot[parity][0] = sa;
+            sh.slot[parity][1] = sb;
+        }
+        cluster.sync();
+        if (tid == 0) {
+            double ta = 0.0, tb = 0.0;
+            for (int r = 0; r < C; ++r) {
+                const double *peer = cluster.map_shared_rank(&sh.slot[parity][0], r);
+                ta += peer[0];
+                tb += peer[1];
+            }
+            sh.tot[0] = ta;
+            sh.tot[1] = tb;
+        }
+        __syncthreads();
+        parity ^= 1;
+    };
+
+    if (tid == 0) { sh.cur = 0; sh.len = 1; sh.path[0] = 0; }
+    __syncthreads();
+
+    for (;;) {   // one iteration per node on the path
+        const int cur = sh.cur;
+        const float *x = lg + (size_t)cur * V;
+        const float *q = dp + (size_t)cur * V;
+        if (tid == 0) {
+            sh.m = (double)rmax[cur];
+            sh.S = rsum[cur];
+            sh.T = (double)Tf;
+            sh.exact = 0;
+            sh.c = 0.0; sh.U = 1.0; sh.D = 1.0;
+            sh.nrem = 0;
+            sh.next = -1;
+        }
+        __syncthreads();
+
+        for (int ch = cur + 1; ch < N; ++ch) {
+            if (sh.parent[ch] != cur) continue;          // uniform: shared data
+            const int xt = sh.tok[ch];
+            // -- evaluate the accept test (thread 0), possibly twice if the denominator must be refined
+            for (int attempt = 0; attempt < 2; ++attempt) {
+                if (tid == 0) {
+                    const double r = (double)un[ch];
+                    const double qx = (double)q[xt];
+                    const double ex = exp(((double)x[xt] - sh.m) / sh.T);
+                    int ridx = -1;
+                    for (int k = 0; k < sh.nrem; ++k) if (sh.rem_tok[k] == xt) ridx = k;
+                    double qk, pk;
+                    if (ridx >= 0) { qk = 0.0; pk = sh.rem_frozen[ridx] / sh.U; }
+                    else { qk = qx / sh.D; pk = weight(ex, qx, 1.0 / sh.S, sh.c) / sh.U; }
+                    const double lhs = r * qk;
+                    int dec = (lhs < pk) ? 1 : 0;
+                    if (!sh.exact) {
+                        const double big = fmax(lhs, pk);
+                        if (big > 0.0 && fabs(lhs - pk) <= kAmbiguous * big) dec = 2;
+                        else if (dec == 0) dec = 2;      // a rejection needs the exact denominator anyway
+                    }
+                    sh.decision = dec;
+                    sh.ex = ex; sh.qx = qx; sh.ridx = ridx; sh.xnew = xt;
+                }
+                __syncthreads();
+                if (sh.decision != 2) break;
+                // exact softmax denominator of this node
+                Sweep s = sweep_chunk<MODE_SUM>(sh, x, q, lo, hi, vec, 0.0, -1, false, 0, 0, 0, nullptr);
+                reduce_exchange(s.a, 0.0);
+                if (tid == 0) { sh.S = sh.tot[0]; sh.exact = 1; }
+                __syncthreads();
+            }
+            if (sh.decision == 1) {
+                if (tid == 0) sh.next = ch;
+                __syncthreads();
+                break;
+            }
+            // -- rejected: one sweep gives the new residual mass and the new draft mass
+            if (tid == 0) sh.cprime = sh.c + sh.U / sh.D;
+            __syncthreads();
+            {
+                Sweep s = sweep_chunk<MODE_RESID>(sh, x, q, lo, hi, vec, sh.cprime, xt, false, 0, 0, 0, nullptr);
+                reduce_exchange(s.a, s.b);
+            }
+            if (tid == 0) {
+                const double W = sh.tot[0], Dn = sh.tot[1];
+                double frozen;
+                if (W > 0.0) {
+                    frozen = weight(sh.ex, sh.qx, 1.0 / sh.S, sh.cprime);
+                    sh.c = sh.cprime;
+                    sh.U = W;
+                } else {
+                    frozen = weight(sh.ex, sh.qx, 1.0 / sh.S, sh.c);   // residual vanished: p is kept
+                }
+                if (sh.ridx < 0 && sh.nrem < FSPAD_MAX_NODES) {
+                    sh.rem_tok[sh.nrem] = xt;
+                    sh.rem_frozen[sh.nrem] = frozen;
+                    sh.nrem++;
+                }
+                if (Dn > 0.0) sh.D = Dn;
+            }
+            __syncthreads();
+        }
+
+        if (sh.next < 0) break;                           // uniform
+        if (tid == 0) {
+            sh.path[sh.len++] = sh.next;
+            sh.cur = sh.next;
+        }
+        __syncthreads();
+    }
+
+    // ---- bonus token: inverse CDF of the current residual at the last node ----
+    {
+        const int cur = sh.cur;
+        const float *x = lg + (size_t)cur * V;
+        const float *q = dp + (size_t)cur * V;
+        if (!sh.exact) {
+            Sweep s = sweep_chunk<MODE_SUM>(sh, x, q, lo, hi, vec, 0.0, -1, false, 0, 0, 0, nullptr);
+            reduce_exchange(s.a, 0.0);
+            if (tid == 0) { sh.S = sh.tot[0]; sh.exact = 1; }
+            __syncthreads();
+        }
+        const double c = sh.c;
+        Sweep s = sweep_chunk<MODE_CDF>(sh, x, q, lo, hi, vec, c, -1, false, 0, 0, 0, nullptr);
+        // block-wide inclusive scan of the per-thread sums (index order)
+        double incl = s.a;
+        const int lane = tid & 31, wid = tid >> 5;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const double t = __shfl_up_sync(0xffffffffu, incl, off);
+            if (lane >= off) incl += t;
+        }
+        double prev_incl = __shfl_up_sync(0xffffffffu, incl, 1);
+        if (lane == 31) sh.warp_a[wid] = incl;
+        __syncthreads();
+        if (tid == 0) {
+            double off = 0.0;
+            for (int w = 0; w < nthr / 32; ++w) { sh.warp_off[w] = off; off = off + sh.warp_a[w]; }
+            sh.slot[parity][0] = off;                     // CTA total = inclusive prefix of the last thread
+        }
+        __syncthreads();
+        const double woff = sh.warp_off[wid];
+        const double P = woff + incl;
+        const double E = (lane == 0) ? woff : woff + prev_incl;
+        cluster.sync();
+        if (tid == 0)
+            for (int r = 0; r < C; ++r) sh.cta_total[r] = *cluster.map_shared_rank(&sh.slot[parity][0], r);
+        __syncthreads();
+        double Z = 0.0, base = 0.0;
+        for (int r = 0; r < C; ++r) {
+            if (r == rank) base = Z;
+            Z = Z + sh.cta_total[r];
+        }
+        const double target = (double)un[N] * Z;
+        int owner = -1;
+        {
+            double cum = 0.0;
+            for (int r = 0; r < C; ++r) {
+                cum = cum + sh.cta_total[r];
+                if (cum > target) { owner = r; break; }
+            }
+        }
+        if (owner == rank) {
+            // the first thread (index order) whose inclusive prefix passes the target owns the draw
+            if (tid == 0) sh.sel = 0x7fffffff;
+            __syncthreads();
+            if (base + P > target) atomicMin(&sh.sel, tid);
+            __syncthreads();
+            if (tid == sh.sel) {
+                int found = -1;
+                sweep_chunk<MODE_CDF>(sh, x, q, lo, hi, vec, c, -1, true, base, E, target, &found);
+                if (found < 0) found = min(lo, V - 1);
+                args.bonus[b] = found;
+            }
+        }
+        if (owner < 0 && rank == 0 && tid == 0) args.bonus[b] = 0;   // no positive weight anywhere
+        if (rank == 0) {
+            if (tid == 0) args.n_acc[b] = sh.len;
+            for (int i = tid; i < args.path_stride; i += nthr) out_path[i] = (i < sh.len) ? sh.path[i] : -1;
+        }
+        cluster.sync();    // nobody leaves while a peer may still read its shared memory
+    }
+}
+
+}  // namespace
+
+cudaError_t fspad_launch_accept_walk(fspad_ctx *ctx, const float *logits, const float *draft,
+                                     const int *tokens, const int *parent, const float *temperature,
+                                     const float *uniforms, int N, int B, int V, int *path,
+                                     int *n_acc, int *bonus, cudaStream_t st)
+{
+    if (B == 0) return cudaSuccess;
+    WalkArgs a;
+    a.logits = logits; a.draft = draft; a.temperature = temperature; a.uniforms = uniforms;
+    a.tokens = tokens; a.parent = parent;
+    a.row_max = ctx->row_max; a.row_sum = ctx->row_sum; a.row_arg = ctx->row_arg;
+    a.N = N; a.V = V; a.path_stride = ctx->cfg.max_nodes;
+    a.path = path; a.n_acc = n_acc; a.bonus = bonus; a.status = ctx->d_status;
+
+    const bool sampling = draft != nullptr && uniforms != nullptr;
+    int cluster = 1, threads = 64;
+    if (sampling) {
+        threads = kWalkThreads;
+        if (ctx->walk_cluster == 0) {
+            // largest cluster the device can co-schedule for this kernel: 16 (opt-in), else 8
+            ctx->walk_cluster = 8;
+            if (cudaFuncSetAttribute(accept_walk_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) ==
+                cudaSuccess) {
+                cudaLaunchConfig_t probe = {};
+                probe.gridDim = dim3(kMaxCluster);
+                probe.blockDim = dim3(kWalkThreads);
+                cudaLaunchAttribute at[1];
+                at[0].id = cudaLaunchAttributeClusterDimension;
+                at[0].val.clusterDim.x = kMaxCluster; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+                probe.attrs = at; probe.numAttrs = 1;
+                int n = 0;
+                if (cudaOccupancyMaxActiveClusters(&n, accept_walk_kernel, &probe) == cudaSuccess && n >= 1)
+                    ctx->walk_cluster = kMaxCluster;
+            }
+            (void)cudaGetLastError();
+        }
+        cluster = ctx->walk_cluster;
+        // small vocabularies do not need the whole cluster
+        while (cluster > 1 && (V + cluster - 1) / cluster < 1024) cluster >>= 1;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(B * cluster));
+    cfg.blockDim = dim3(threads);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = cluster; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    ctx->launches++;
+    return cudaLaunchKernelEx(&cfg, accept_walk_kernel, a);
+}

@@ -1,0 +1,302 @@
+// C ABI of libfspad.so: context management, argument validation and the
+// host-buffer entry point.  All arithmetic of the verify step lives in the
+// kernel translation units; nothing here computes on the host.
+#include <cmath>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+
+#include "common.cuh"
+
+namespace {
+
+inline bool misaligned(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
+
+template <typename T>
+bool dev_alloc(T **p, size_t count)
+{
+    *p = nullptr;
+    if (count == 0) count = 1;
+    return cudaMalloc(reinterpret_cast<void **>(p), count * sizeof(T)) == cudaSuccess;
+}
+
+int check_common(const fspad_ctx *ctx, int n_nodes, int batch)
+{
+    if (!ctx) return FSPAD_ERR_NULL;
+    if (n_nodes > FSPAD_MAX_NODES || n_nodes > ctx->cfg.max_nodes) return FSPAD_ERR_TREE_TOO_LARGE;
+    if (n_nodes < 1 || batch < 0 || batch > ctx->cfg.max_batch) return FSPAD_ERR_SHAPE;
+    return FSPAD_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char *fspad_strerror(int err)
+{
+    switch (err) {
+    case FSPAD_OK: return "ok";
+    case FSPAD_ERR_NULL: return "required pointer is NULL";
+    case FSPAD_ERR_ALIGN: return "pointer is not 16-byte aligned";
+    case FSPAD_ERR_SHAPE: return "sizes inconsistent with the context";
+    case FSPAD_ERR_TREE_TOO_LARGE: return "tree has more nodes than supported";
+    case FSPAD_ERR_RANGE: return "value out of range (prefix length, token id, temperature or path)";
+    case FSPAD_ERR_CUDA: return "CUDA runtime call failed";
+    case FSPAD_ERR_TIMEOUT: return "bounded device-side wait ran out";
+    case FSPAD_ERR_BAD_TREE: return "parent[] is not a topologically ordered tree rooted at node 0";
+    case FSPAD_ERR_NOMEM: return "allocation failed";
+    default: return "unknown error";
+    }
+}
+
+int fspad_create(const fspad_config *cfg, fspad_ctx **out)
+{
+    if (!out) return FSPAD_ERR_NULL;
+    *out = nullptr;
+    if (!cfg) return FSPAD_ERR_NULL;
+    if (cfg->head_dim != FSPAD_HEAD_DIM || cfg->n_kv_heads < 1 || cfg->n_q_heads < 1 ||
+        cfg->n_q_heads % cfg->n_kv_heads != 0 || cfg->vocab < 1 || cfg->n_layers < 1 ||
+        cfg->max_len < 1 || cfg->max_batch < 1 || cfg->max_nodes < 1)
+        return FSPAD_ERR_SHAPE;
+    if (cfg->max_nodes > FSPAD_MAX_NODES) return FSPAD_ERR_TREE_TOO_LARGE;
+    if (cfg->max_nodes > cfg->max_len) return FSPAD_ERR_RANGE;
+    if (!(cfg->softmax_scale >= 0.0f)) return FSPAD_ERR_RANGE;
+
+    fspad_ctx *ctx = new (std::nothrow) fspad_ctx();
+    if (!ctx) return FSPAD_ERR_NOMEM;
+    std::memset(ctx, 0, sizeof(*ctx));
+    ctx->cfg = *cfg;
+    ctx->scale = cfg->softmax_scale > 0.0f ? cfg->softmax_scale : 1.0f / std::sqrt((float)cfg->head_dim);
+    if (cudaGetDevice(&ctx->device) != cudaSuccess ||
+        cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, ctx->device) != cudaSuccess) {
+        delete ctx;
+        return FSPAD_ERR_CUDA;
+    }
+
+    const int G = cfg->n_q_heads / cfg->n_kv_heads;
+    const size_t B = (size_t)cfg->max_batch, Nmax = (size_t)cfg->max_nodes;
+    // split-KV partials: worst case over every (n_nodes, batch) a call may pass
+    size_t part_rows = 0;
+    int max_splits = 1;
+    for (int n = 1; n <= cfg->max_nodes; ++n)
+        for (int b = 1; b <= cfg->max_batch; ++b) {
+            const int s = fspad_attn_splits(ctx, n, b);
+            const size_t rows = (size_t)b * cfg->n_kv_heads * s * n * G;
+            if (rows > part_rows) part_rows = rows;
+            if (s > max_splits) max_splits = s;
+        }
+    ctx->attn_max_splits = max_splits;
+    const size_t rows = B * Nmax;
+    ctx->stats_max_slices = 64;
+
+    bool ok = dev_alloc(&ctx->d_status, 1);
+    ok = ok && dev_alloc(&ctx->part_o, part_rows * FSPAD_HEAD_DIM);
+    ok = ok && dev_alloc(&ctx->part_ml, part_rows * 2);
+    ok = ok && dev_alloc(&ctx->st_pmax, rows * ctx->stats_max_slices);
+    ok = ok && dev_alloc(&ctx->st_psum, rows * ctx->stats_max_slices);
+    ok = ok && dev_alloc(&ctx->st_parg, rows * ctx->stats_max_slices);
+    ok = ok && dev_alloc(&ctx->st_counter, rows);
+    ok = ok && dev_alloc(&ctx->row_max, rows);
+    ok = ok && dev_alloc(&ctx->row_sum, rows);
+    ok = ok && dev_alloc(&ctx->row_arg, rows);
+    if (ok) {
+        ok = cudaMemset(ctx->d_status, 0, sizeof(int)) == cudaSuccess &&
+             cudaMemset(ctx->st_counter, 0, rows * sizeof(unsigned)) == cudaSuccess &&
+             cudaDeviceSynchronize() == cudaSuccess;
+    }
+    if (!ok) {
+        fspad_destroy(ctx);
+        return FSPAD_ERR_NOMEM;
+    }
+    *out = ctx;
+    return FSPAD_OK;
+}
+
+void fspad_destroy(fspad_ctx *ctx)
+{
+    if (!ctx) return;
+    cudaDeviceSynchronize();
+    void *ptrs[] = {ctx->d_status, ctx->part_o, ctx->part_ml, ctx->st_pmax, ctx->st_psum, ctx->st_parg,
+                    ctx->st_counter, ctx->row_max, ctx->row_sum, ctx->row_arg, ctx->h_q, ctx->h_tk,
+                    ctx->h_tv, ctx->h_out, ctx->h_parent, ctx->h_prefix, ctx->h_tokens, ctx->h_path,
+                    ctx->h_nacc, ctx->h_bonus, ctx->h_newlen, ctx->h_logits, ctx->h_draft, ctx->h_temp,
+                    ctx->h_unif};
+    for (void *p : ptrs)
+        if (p) cudaFree(p);
+    delete ctx;
+}
+
+int fspad_status(fspad_ctx *ctx, void *stream)
+{
+    if (!ctx) return FSPAD_ERR_NULL;
+    cudaStream_t st = fspad_stream(stream);
+    int h = 0;
+    if (cudaMemcpyAsync(&h, ctx->d_status, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaStreamSynchronize(st) != cudaSuccess)
+        return FSPAD_ERR_CUDA;
+    if (h != 0) {
+        if (cudaMemsetAsync(ctx->d_status, 0, sizeof(int), st) != cudaSuccess ||
+            cudaStreamSynchronize(st) != cudaSuccess)
+            return FSPAD_ERR_CUDA;
+    }
+    return h;
+}
+
+long long fspad_launch_count(const fspad_ctx *ctx) { return ctx ? ctx->launches : 0; }
+
+int fspad_tree_attn(fspad_ctx *ctx, const fspad_bf16 *q, const fspad_bf16 *k_cache,
+                    const fspad_bf16 *v_cache, const fspad_bf16 *tree_k, const fspad_bf16 *tree_v,
+                    const int32_t *parent, const int32_t *prefix_len, int n_nodes, int batch,
+                    fspad_bf16 *out, void *stream)
+{
+    int rc = check_common(ctx, n_nodes, batch);
+    if (rc) return rc;
+    if (!q || !k_cache || !v_cache || !parent || !prefix_len || !out) return FSPAD_ERR_NULL;
+    if ((tree_k == nullptr) != (tree_v == nullptr)) return FSPAD_ERR_NULL;
+    if (misaligned(q) || misaligned(k_cache) || misaligned(v_cache) || misaligned(tree_k) ||
+        misaligned(tree_v) || misaligned(out))
+        return FSPAD_ERR_ALIGN;
+    if (n_nodes > ctx->cfg.max_len) return FSPAD_ERR_RANGE;
+    if (batch == 0) return FSPAD_OK;
+    cudaError_t e = fspad_launch_tree_attn(ctx, q, k_cache, v_cache, tree_k, tree_v, parent, prefix_len,
+                                           n_nodes, batch, out, fspad_stream(stream));
+    return e == cudaSuccess ? FSPAD_OK : FSPAD_ERR_CUDA;
+}
+
+int fspad_accept_stats(fspad_ctx *ctx, const float *logits, const float *temperature, int rows,
+                       int rows_per_seq, float *row_max, double *row_sum, int32_t *row_arg,
+                       void *stream)
+{
+    if (!ctx) return FSPAD_ERR_NULL;
+    if (!logits || !row_max || !row_sum || !row_arg) return FSPAD_ERR_NULL;
+    if (rows < 0 || rows_per_seq < 1 || rows > ctx->cfg.max_batch * ctx->cfg.max_nodes)
+        return FSPAD_ERR_SHAPE;
+    if (rows == 0) return FSPAD_OK;
+    cudaError_t e = fspad_launch_accept_stats(ctx, logits, temperature, rows, rows_per_seq, ctx->cfg.vocab,
+                                              row_max, row_sum, row_arg, fspad_stream(stream));
+    return e == cudaSuccess ? FSPAD_OK : FSPAD_ERR_CUDA;
+}
+
+int fspad_tree_accept(fspad_ctx *ctx, const float *target_logits, const float *draft_probs,
+                      const int32_t *draft_tokens, const int32_t *parent, const float *temperature,
+                      const float *uniforms, int n_nodes, int batch, int32_t *accepted_path,
+                      int32_t *n_accepted, int32_t *bonus_token, void *stream)
+{
+    int rc = check_common(ctx, n_nodes, batch);
+    if (rc) return rc;
+    if (!target_logits || !draft_tokens || !parent || !temperature || !accepted_path || !n_accepted ||
+        !bonus_token)
+        return FSPAD_ERR_NULL;
+    if ((draft_probs == nullptr) != (uniforms == nullptr)) return FSPAD_ERR_NULL;
+    if (misaligned(target_logits) || misaligned(draft_probs)) return FSPAD_ERR_ALIGN;
+    if (batch == 0) return FSPAD_OK;
+    cudaStream_t st = fspad_stream(stream);
+    cudaError_t e = fspad_launch_accept_stats(ctx, target_logits, temperature, batch * n_nodes, n_nodes,
+                                              ctx->cfg.vocab, ctx->row_max, ctx->row_sum, ctx->row_arg, st);
+    if (e != cudaSuccess) return FSPAD_ERR_CUDA;
+    e = fspad_launch_accept_walk(ctx, target_logits, draft_probs, draft_tokens, parent, temperature,
+                                 uniforms, n_nodes, batch, ctx->cfg.vocab, accepted_path, n_accepted,
+                                 bonus_token, st);
+    return e == cudaSuccess ? FSPAD_OK : FSPAD_ERR_CUDA;
+}
+
+int fspad_kv_compact(fspad_ctx *ctx, fspad_bf16 *cache, const int32_t *accepted_path,
+                     const int32_t *n_accepted, const int32_t *prefix_len, int batch,
+                     int32_t *new_len, void *stream)
+{
+    if (!ctx) return FSPAD_ERR_NULL;
+    if (!cache || !accepted_path || !n_accepted || !prefix_len) return FSPAD_ERR_NULL;
+    if (misaligned(cache)) return FSPAD_ERR_ALIGN;
+    if (batch < 0 || batch > ctx->cfg.max_batch) return FSPAD_ERR_SHAPE;
+    if (batch == 0) return FSPAD_OK;
+    cudaError_t e = fspad_launch_kv_compact(ctx, cache, accepted_path, n_accepted, prefix_len, batch,
+                                            new_len, fspad_stream(stream));
+    return e == cudaSuccess ? FSPAD_OK : FSPAD_ERR_CUDA;
+}
+
+int fspad_verify_step_host(fspad_ctx *ctx, fspad_bf16 *cache, const fspad_bf16 *q,
+                           const fspad_bf16 *tree_k, const fspad_bf16 *tree_v, const int32_t *parent,
+                           const int32_t *prefix_len, const float *target_logits,
+                           const float *draft_probs, const int32_t *draft_tokens,
+                           const float *temperature, const float *uniforms, int n_nodes, int batch,
+                           fspad_bf16 *attn_out, int32_t *accepted_path, int32_t *n_accepted,
+                           int32_t *bonus_token, int32_t *new_len, void *stream)
+{
+    int rc = check_common(ctx, n_nodes, batch);
+    if (rc) return rc;
+    if (!cache || !q || !tree_k || !tree_v || !parent || !prefix_len || !target_logits || !draft_tokens ||
+        !temperature || !attn_out || !accepted_path || !n_accepted || !bonus_token || !new_len)
+        return FSPAD_ERR_NULL;
+    if ((draft_probs == nullptr) != (uniforms == nullptr)) return FSPAD_ERR_NULL;
+    if (misaligned(cache)) return FSPAD_ERR_ALIGN;
+    if (batch == 0) return FSPAD_OK;
+    const fspad_config &c = ctx->cfg;
+    cudaStream_t st = fspad_stream(stream);
+
+    // staging buffers are created on first use, sized for the context's maxima
+    if (!ctx->h_q) {
+        const size_t B = (size_t)c.max_batch, N = (size_t)c.max_nodes;
+        bool ok = dev_alloc(&ctx->h_q, B * N * c.n_q_heads * FSPAD_HEAD_DIM);
+        ok = ok && dev_alloc(&ctx->h_out, B * N * c.n_q_heads * FSPAD_HEAD_DIM);
+        ok = ok && dev_alloc(&ctx->h_tk, B * c.n_kv_heads * N * FSPAD_HEAD_DIM);
+        ok = ok && dev_alloc(&ctx->h_tv, B * c.n_kv_heads * N * FSPAD_HEAD_DIM);
+        ok = ok && dev_alloc(&ctx->h_parent, B * N) && dev_alloc(&ctx->h_tokens, B * N);
+        ok = ok && dev_alloc(&ctx->h_prefix, B) && dev_alloc(&ctx->h_nacc, B);
+        ok = ok && dev_alloc(&ctx->h_bonus, B) && dev_alloc(&ctx->h_newlen, B);
+        ok = ok && dev_alloc(&ctx->h_path, B * N) && dev_alloc(&ctx->h_temp, B);
+        ok = ok && dev_alloc(&ctx->h_unif, B * (N + 1));
+        ok = ok && dev_alloc(&ctx->h_logits, B * N * c.vocab);
+        ok = ok && dev_alloc(&ctx->h_draft, B * N * c.vocab);
+        if (!ok) return FSPAD_ERR_NOMEM;
+    }
+    const size_t B = (size_t)batch, N = (size_t)n_nodes;
+    const size_t q_bytes = B * N * c.n_q_heads * FSPAD_HEAD_DIM * sizeof(fspad_bf16);
+    const size_t t_bytes = B * c.n_kv_heads * N * FSPAD_HEAD_DIM * sizeof(fspad_bf16);
+    const size_t lg_bytes = B * N * c.vocab * sizeof(float);
+    bool ok = true;
+    auto h2d = [&](void *dst, const void *src, size_t bytes) {
+        ok = ok && cudaMemcpyAsync(dst, src, bytes, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    };
+    auto d2h = [&](void *dst, const void *src, size_t bytes) {
+        ok = ok && cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    };
+    h2d(ctx->h_q, q, q_bytes);
+    h2d(ctx->h_tk, tree_k, t_bytes);
+    h2d(ctx->h_tv, tree_v, t_bytes);
+    h2d(ctx->h_parent, parent, B * N * sizeof(int));
+    h2d(ctx->h_prefix, prefix_len, B * sizeof(int));
+    h2d(ctx->h_tokens, draft_tokens, B * N * sizeof(int));
+    h2d(ctx->h_temp, temperature, B * sizeof(float));
+    h2d(ctx->h_logits, target_logits, lg_bytes);
+    if (draft_probs) {
+        h2d(ctx->h_draft, draft_probs, lg_bytes);
+        h2d(ctx->h_unif, uniforms, B * (N + 1) * sizeof(float));
+    }
+    if (!ok) return FSPAD_ERR_CUDA;
+
+    // layer 0 of the cache: K at [0][0], V at [0][1]
+    const size_t plane = B * c.n_kv_heads * (size_t)c.max_len * FSPAD_HEAD_DIM;
+    if (fspad_launch_tree_scatter(ctx, cache, ctx->h_tk, ctx->h_tv, ctx->h_prefix, n_nodes, batch, st) !=
+        cudaSuccess)
+        return FSPAD_ERR_CUDA;
+    rc = fspad_tree_attn(ctx, ctx->h_q, cache, cache + plane, nullptr, nullptr, ctx->h_parent, ctx->h_prefix,
+                         n_nodes, batch, ctx->h_out, stream);
+    if (rc) return rc;
+    rc = fspad_tree_accept(ctx, ctx->h_logits, draft_probs ? ctx->h_draft : nullptr, ctx->h_tokens,
+                           ctx->h_parent, ctx->h_temp, draft_probs ? ctx->h_unif : nullptr, n_nodes, batch,
+                           ctx->h_path, ctx->h_nacc, ctx->h_bonus, stream);
+    if (rc) return rc;
+    rc = fspad_kv_compact(ctx, cache, ctx->h_path, ctx->h_nacc, ctx->h_prefix, batch, ctx->h_newlen, stream);
+    if (rc) return rc;
+
+    d2h(attn_out, ctx->h_out, q_bytes);
+    // the device path array has max_nodes entries per sequence, and so has the host one
+    d2h(accepted_path, ctx->h_path, B * (size_t)c.max_nodes * sizeof(int));
+    d2h(n_accepted, ctx->h_nacc, B * sizeof(int));
+    d2h(bonus_token, ctx->h_bonus, B * sizeof(int));
+    d2h(new_len, ctx->h_newlen, B * sizeof(int));
+    if (!ok) return FSPAD_ERR_CUDA;
+    return fspad_status(ctx, stream);
+}
+
+}  // extern "C"
