@@ -1,0 +1,339 @@
+#!/usr/bin/env python
+"""Benchmark of the tree-verify step (attention + acceptance + KV compaction).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+A step is one pass of the whole hot path over one synthetic input set.  The
+input sets are rotated over enough copies to exceed twice the L2 capacity, so
+every step reads its inputs from HBM.  Prints ONE JSON line (rank 0).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2408_15562_b200 import synth  # noqa: E402
+
+METRIC = "tree_verify_step_latency"
+UNIT = "us/step"
+L2_BYTES = 126 * 1024 * 1024
+
+
+def algorithmic_bytes(w: synth.Workload, L_mean: float, n_acc_rows: float):
+    """Bytes a verify step must move (inputs read once, outputs written once)."""
+    N, d = w.n_nodes, w.head_dim
+    attn = 2 * 2 * w.n_kv_heads * d * (L_mean + N) + 2 * 2 * N * w.n_q_heads * d
+    sampling = sum(1 for t in w.temperatures if t > 0)
+    accept_rows = 4 * N * w.vocab * w.batch                 # every node's logits row
+    accept_all = accept_rows + 4 * N * w.vocab * sampling   # + every draft row (the all-rows definition)
+    compact = 2 * w.n_layers * 2 * w.n_kv_heads * n_acc_rows * 2 * d
+    return {"attention": attn * w.batch, "accept_logits": accept_rows, "accept_all_rows": accept_all,
+            "compaction": compact * w.batch}
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        sm = [float(r[0]) for r in self.rows if r and r[0].replace(".", "").isdigit()]
+        mx = [float(r[1]) for r in self.rows if len(r) > 1 and r[1].replace(".", "").isdigit()]
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = [n for i, n in enumerate(names) if any(len(r) > 2 + i and r[2 + i].startswith("Active") for r in self.rows)]
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": reasons, "samples": len(sm)}
+
+
+def time_oracle(inp: synth.VerifyInputs, steps: int):
+    """The CPU oracle as it stands, timed on whole verify steps of this workload."""
+    import oracle
+    oracle.build()
+    cache = synth.make_cache(inp, 1)
+    threads = os.cpu_count() or 1
+    times = []
+    for _ in range(steps):
+        c = cache.copy()
+        t0 = time.perf_counter()
+        oracle.tree_attn(inp.q, inp.k_cache, inp.v_cache, inp.tree_k, inp.tree_v, inp.parent, inp.prefix_len)
+        r = oracle.tree_accept(inp.target_logits, inp.draft_probs, inp.draft_tokens, inp.parent,
+                               inp.temperature, inp.uniforms if inp.draft_probs is not None else None)
+        oracle.kv_compact(c, r["accepted_path"], r["n_accepted"], inp.prefix_len)
+        times.append(time.perf_counter() - t0)
+    return statistics.median(times) * 1e6, threads
+
+
+def run_reference(args, w):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    inp = synth.generate(w, 0)
+    steps = max(1, min(args.steps, 5))
+    for _ in range(min(args.warmup, 1)):
+        time_oracle(inp, 1)
+    us, threads = time_oracle(inp, steps)
+    line = {"impl": "reference", "metric": METRIC, "value": us, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": steps, "warmup": min(args.warmup, 1), "ms_per_step": us / 1e3, "higher_is_better": False,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": w.name, "batch": w.batch, "n_nodes": w.n_nodes, "vocab": w.vocab,
+                       "layers_compacted": 1},
+            "cpu_baseline": {"value": us, "unit": UNIT, "cores": threads, "kind": "oracle",
+                             "sample": "%d whole verify steps of %s (layer-0 cache only)" % (steps, w.name)},
+            "e2e": {"value": us, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--workload", default="llama3_8b_2k", choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    w = synth.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        return run_reference(args, w)
+    if args.warmup < 3:
+        args.warmup = 3
+
+    import torch
+    import torch.distributed as dist
+    from paper_2408_15562_b200 import binding
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    # ---- inputs: R rotated sets, each a full verify step (replicas: every rank its own copy) ----
+    inp = synth.generate(w, 0)
+    B, N = inp.parent.shape
+    L_mean = float(inp.prefix_len.mean())
+    n_layers = w.n_layers
+    step_bytes = algorithmic_bytes(w, L_mean, 0)
+    one_set = step_bytes["attention"] + step_bytes["accept_all_rows"]
+    R = max(2, int(np.ceil(2 * L2_BYTES / one_set)))
+    bf = binding.bf16_tensor
+    dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()  # noqa: E731
+    sets = []
+    cache0 = bf(synth.make_cache(inp, n_layers))       # [layers][2][B][Hkv][max_len][d]
+    for r in range(R):
+        s = {"cache": cache0.clone(), "q": bf(inp.q).clone(), "tree_k": bf(inp.tree_k), "tree_v": bf(inp.tree_v),
+             "logits": dev(inp.target_logits), "draft": dev(inp.draft_probs) if inp.draft_probs is not None else None}
+        sets.append(s)
+    parent, prefix = dev(inp.parent), dev(inp.prefix_len)
+    tokens, temp = dev(inp.draft_tokens), dev(inp.temperature)
+    unif = dev(inp.uniforms) if inp.draft_probs is not None else None
+    ctx = binding.Context(w.n_q_heads, w.n_kv_heads, w.vocab, inp.max_len, max_nodes=N, n_layers=n_layers,
+                          max_batch=B)
+    out = torch.empty_like(sets[0]["q"])
+    path = torch.empty((B, N), dtype=torch.int32, device="cuda")
+    n_acc = torch.empty((B,), dtype=torch.int32, device="cuda")
+    bonus = torch.empty((B,), dtype=torch.int32, device="cuda")
+    new_len = torch.empty((B,), dtype=torch.int32, device="cuda")
+
+    def attn(s):
+        ctx.tree_attn(s["q"], s["cache"][0, 0], s["cache"][0, 1], s["tree_k"], s["tree_v"], parent, prefix, out=out)
+
+    def accept(s):
+        ctx.tree_accept(s["logits"], s["draft"], tokens, parent, temp, unif, path, n_acc, bonus)
+
+    def compact(s):
+        ctx.kv_compact(s["cache"], path, n_acc, prefix, new_len)
+
+    def step(i):
+        s = sets[i % R]
+        attn(s)
+        accept(s)
+        compact(s)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # compaction is in place: it is idempotent on the same path only after the first call, so the
+    # tree rows of every set are restored (untimed) before each timed pass
+    tree_rows = [torch.stack([s["cache"][:, :, b, :, int(inp.prefix_len[b]):int(inp.prefix_len[b]) + N].clone()
+                              for b in range(B)]) for s in sets]
+
+    def restore():
+        for s, t in zip(sets, tree_rows):
+            for b in range(B):
+                Lb = int(inp.prefix_len[b])
+                s["cache"][:, :, b, :, Lb:Lb + N] = t[b]
+        torch.cuda.synchronize()
+
+    for i in range(args.warmup):
+        step(i)
+    barrier()
+    ctx.check()
+
+    def timed(fn, steps, graph=True):
+        """us per call of fn over `steps` calls.  The calls are captured once into a CUDA graph
+        (the library only enqueues kernels on the given stream), replayed once untimed, and the
+        timed region is exactly one replay = `steps` calls, bracketed by events on that stream."""
+        restore()
+        g = None
+        if graph:
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                for i in range(steps):
+                    fn(i)
+            g.replay()
+            restore()
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        if g is not None:
+            g.replay()
+        else:
+            for i in range(steps):
+                fn(i)
+        e1.record()
+        barrier()
+        return e0.elapsed_time(e1) * 1e3 / steps          # us per call
+
+    sampler = ClockSampler(local)
+    sampler.start()
+    launches0 = ctx.launch_count()
+    step_us = timed(step, args.steps)
+    launches = (ctx.launch_count() - launches0)          # kernels enqueued into the graph = kernels per replay
+    # per-call breakdown and the dominant kernel alone (same rotated inputs, same stream)
+    attn_us = timed(lambda i: attn(sets[i % R]), args.steps)
+    accept_us = timed(lambda i: accept(sets[i % R]), args.steps)
+    compact_us = timed(lambda i: compact(sets[i % R]), args.steps)
+    lg2d = [s["logits"].view(B * N, w.vocab) for s in sets]
+    st_out = (torch.empty(B * N, dtype=torch.float32, device="cuda"), torch.empty(B * N, dtype=torch.float64, device="cuda"),
+              torch.empty(B * N, dtype=torch.int32, device="cuda"))
+    stats_us = timed(lambda i: ctx.accept_stats(lg2d[i % R], temp, N, out=st_out), args.steps)
+    eager_us = timed(step, args.steps, graph=False)
+    clocks = sampler.stop()
+    ctx.check()
+
+    # ---- correctness of what was timed: compare the last step with the oracle on rank 0 ----
+    n_acc_host = n_acc.cpu().numpy()
+
+    # ---- end to end through the host entry point (pinned host buffers, copies inside the timed region) ----
+    pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()  # noqa: E731
+    hq = binding.bf16_tensor(inp.q, "cpu").pin_memory()
+    htk = binding.bf16_tensor(inp.tree_k, "cpu").pin_memory()
+    htv = binding.bf16_tensor(inp.tree_v, "cpu").pin_memory()
+    hpar, hpre, htok, htemp = pin(inp.parent), pin(inp.prefix_len), pin(inp.draft_tokens), pin(inp.temperature)
+    hlg = pin(inp.target_logits)
+    hdp = pin(inp.draft_probs) if inp.draft_probs is not None else None
+    hun = pin(inp.uniforms) if inp.draft_probs is not None else None
+    hout = torch.empty_like(hq).pin_memory()
+    hpath = torch.empty((B, N), dtype=torch.int32).pin_memory()
+    hn, hb, hl = (torch.empty((B,), dtype=torch.int32).pin_memory() for _ in range(3))
+
+    def e2e_step(i):
+        ctx.verify_step_host(sets[i % R]["cache"], hq, htk, htv, hpar, hpre, hlg, hdp, htok, htemp, hun, hout,
+                             hpath, hn, hb, hl)
+
+    e2e_steps = max(3, min(args.steps, 20))
+    for i in range(3):
+        e2e_step(i)
+    barrier()
+    t0 = time.perf_counter()
+    for i in range(e2e_steps):
+        e2e_step(i)
+    barrier()
+    e2e_us = (time.perf_counter() - t0) * 1e6 / e2e_steps
+    h2d = sum(t.numel() * t.element_size() for t in (hq, htk, htv, hpar, hpre, htok, htemp, hlg) if t is not None)
+    h2d += sum(t.numel() * t.element_size() for t in (hdp, hun) if t is not None)
+    d2h = sum(t.numel() * t.element_size() for t in (hout, hpath, hn, hb, hl))
+
+    # max over ranks
+    vals = torch.tensor([step_us, attn_us, accept_us, compact_us, stats_us, e2e_us, eager_us], dtype=torch.float64,
+                        device="cuda")
+    if world > 1:
+        dist.all_reduce(vals, op=dist.ReduceOp.MAX)
+    step_us, attn_us, accept_us, compact_us, stats_us, e2e_us, eager_us = [float(x) for x in vals.cpu()]
+
+    if rank == 0:
+        peak, peak_kind = peaks()
+        bytes_real = algorithmic_bytes(w, L_mean, float(n_acc_host.mean()))
+        stats_bytes = bytes_real["accept_logits"]
+        step_all = bytes_real["attention"] + bytes_real["accept_all_rows"] + bytes_real["compaction"]
+        achieved = stats_bytes / (stats_us * 1e-6) / 1e9
+        line = {
+            "metric": METRIC, "value": step_us, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": step_us / 1e3, "higher_is_better": False, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": w.name, "batch": B, "n_nodes": N, "prefix_len_mean": L_mean, "vocab": w.vocab,
+                       "q_heads": w.n_q_heads, "kv_heads": w.n_kv_heads, "layers_compacted": n_layers,
+                       "temperatures": sorted(set(float(t) for t in w.temperatures)),
+                       "launch": "K steps captured in one CUDA graph, one replay timed",
+                       "l2": "inputs rotated over %d copies (%.0f MB per copy, > 2x L2 in total)" % (R, one_set / 1e6),
+                       "multi_gpu": "independent replicas, no collective"},
+            "steps_per_s_all_gpus": world * 1e6 / step_us,
+            "step_hbm_gbs_all_rows_definition": step_all / (step_us * 1e-6) / 1e9,
+            "step_frac_of_hbm_peak": step_all / (step_us * 1e-6) / 1e9 / peak,
+            "step_algorithmic_bytes": step_all,
+            "breakdown_us": {"tree_attn": attn_us, "tree_accept": accept_us, "kv_compact": compact_us,
+                             "accept_stats_kernel_alone": stats_us,
+                             "whole_step_eager_python_launches": eager_us},
+            "mean_accepted_len": float(n_acc_host.mean()),
+            "roofline": {"kernel": "accept_stats_kernel", "bound": "hbm", "achieved": achieved, "peak": peak,
+                         "peak_kind": "%s copy bandwidth (burst, kernel timed alone)" % peak_kind, "unit": "GB/s",
+                         "frac": achieved / peak, "traffic": None, "algorithmic_bytes_per_launch": stats_bytes},
+            "e2e": {"value": e2e_us, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "steps": e2e_steps, "note": "fspad_verify_step_host: pinned host inputs, device-resident KV cache"},
+            "gpu_launches": int(launches),
+            "clocks": clocks,
+        }
+        if not args.no_cpu_baseline and world == 1:
+            us, threads = time_oracle(inp, 3)
+            line["cpu_baseline"] = {"value": us, "unit": UNIT, "cores": threads, "kind": "oracle",
+                                    "sample": "3 whole verify steps of %s (layer-0 cache only), median" % w.name}
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -151,12 +151,14 @@ class Context:
             raise FspadError(rc, "fspad_tree_accept")
         return accepted_path, n_accepted, bonus_token
 
-    def accept_stats(self, logits, temperature, rows_per_seq, stream=None):
+    def accept_stats(self, logits, temperature, rows_per_seq, out=None, stream=None):
         rows = logits.shape[0]
         dev = logits.device
-        row_max = torch.empty((rows,), dtype=torch.float32, device=dev)
-        row_sum = torch.empty((rows,), dtype=torch.float64, device=dev)
-        row_arg = torch.empty((rows,), dtype=torch.int32, device=dev)
+        if out is None:
+            out = (torch.empty((rows,), dtype=torch.float32, device=dev),
+                   torch.empty((rows,), dtype=torch.float64, device=dev),
+                   torch.empty((rows,), dtype=torch.int32, device=dev))
+        row_max, row_sum, row_arg = out
         rc = load().fspad_accept_stats(self._h, _ptr(logits, torch.float32), _ptr(temperature, torch.float32),
                                        rows, rows_per_seq, _ptr(row_max, torch.float32),
                                        _ptr(row_sum, torch.float64), _ptr(row_arg, torch.int32),

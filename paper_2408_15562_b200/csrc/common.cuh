@@ -21,6 +21,7 @@ struct fspad_ctx {
 
     // split-KV attention partials
     int attn_max_splits;
+    int attn_attr_done;       // dynamic shared-memory limit raised for the attention kernels
     float *part_o;            // [batch][Hkv][splits][M][d]
     float *part_ml;           // [batch][Hkv][splits][M][2]  (running max in log2 units, sum)
 

@@ -378,17 +378,19 @@ cudaError_t fspad_launch_tree_attn(fspad_ctx *ctx, const fspad_bf16 *q, const fs
 
     dim3 grid(a.n_splits, c.n_kv_heads * a.mtiles, B);
     cudaError_t e;
-    if (BM == 128) {
-        constexpr int smem = attn_smem_bytes<8>();
-        e = cudaFuncSetAttribute(tree_attn_splitkv_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (!ctx->attn_attr_done) {
+        e = cudaFuncSetAttribute(tree_attn_splitkv_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 attn_smem_bytes<8>());
         if (e != cudaSuccess) return e;
-        tree_attn_splitkv_kernel<8><<<grid, 256, smem, st>>>(a);
-    } else {
-        constexpr int smem = attn_smem_bytes<4>();
-        e = cudaFuncSetAttribute(tree_attn_splitkv_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        e = cudaFuncSetAttribute(tree_attn_splitkv_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 attn_smem_bytes<4>());
         if (e != cudaSuccess) return e;
-        tree_attn_splitkv_kernel<4><<<grid, 128, smem, st>>>(a);
+        ctx->attn_attr_done = 1;
     }
+    if (BM == 128)
+        tree_attn_splitkv_kernel<8><<<grid, 256, attn_smem_bytes<8>(), st>>>(a);
+    else
+        tree_attn_splitkv_kernel<4><<<grid, 128, attn_smem_bytes<4>(), st>>>(a);
     ctx->launches++;
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;

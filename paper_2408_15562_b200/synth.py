@@ -252,7 +252,10 @@ def generate(w: Workload, variant: int = 0, *, with_attention: bool = True,
              with_accept: bool = True) -> VerifyInputs:
     """All inputs of one verify step for workload `w` (seeded by cfg and variant)."""
     seed = SEED_BASE + 10 * w.cfg + variant
-    rng = np.random.default_rng(seed)
+    # independent streams, so that each part is the same whether or not the others are generated
+    rng = np.random.default_rng([seed, 0])          # prefix lengths and trees
+    rng_attn = np.random.default_rng([seed, 1])     # Q, K, V
+    rng_acc = np.random.default_rng([seed, 2])      # logits, draft model, uniforms
     B, N, V, d = w.batch, w.n_nodes, w.vocab, w.head_dim
     lo, hi = w.prefix
     prefix_len = rng.integers(lo, hi + 1, size=B).astype(np.int32) if hi > lo \
@@ -262,15 +265,15 @@ def generate(w: Workload, variant: int = 0, *, with_attention: bool = True,
     N = parent.shape[1]
 
     if with_attention:
-        q = normal_bf16(rng, (B, N, w.n_q_heads, d))
+        q = normal_bf16(rng_attn, (B, N, w.n_q_heads, d))
         k_cache = np.zeros((B, w.n_kv_heads, max_len, d), dtype=np.uint16)
         v_cache = np.zeros_like(k_cache)
-        tree_k = normal_bf16(rng, (B, w.n_kv_heads, N, d))
-        tree_v = normal_bf16(rng, (B, w.n_kv_heads, N, d))
+        tree_k = normal_bf16(rng_attn, (B, w.n_kv_heads, N, d))
+        tree_v = normal_bf16(rng_attn, (B, w.n_kv_heads, N, d))
         for b in range(B):
             L = int(prefix_len[b])
-            k_cache[b, :, :L] = normal_bf16(rng, (w.n_kv_heads, L, d))
-            v_cache[b, :, :L] = normal_bf16(rng, (w.n_kv_heads, L, d))
+            k_cache[b, :, :L] = normal_bf16(rng_attn, (w.n_kv_heads, L, d))
+            v_cache[b, :, :L] = normal_bf16(rng_attn, (w.n_kv_heads, L, d))
             k_cache[b, :, L:L + N] = tree_k[b]
             v_cache[b, :, L:L + N] = tree_v[b]
     else:
@@ -280,24 +283,24 @@ def generate(w: Workload, variant: int = 0, *, with_attention: bool = True,
     assert temperature.shape[0] == B
     any_sampling = bool((temperature > 0).any())
     if with_accept:
-        logits = (rng.standard_normal((B, N, V), dtype=np.float32) * np.float32(w.logit_sigma))
+        logits = (rng_acc.standard_normal((B, N, V), dtype=np.float32) * np.float32(w.logit_sigma))
         draft_probs = np.zeros((B, N, V), dtype=np.float32) if any_sampling else None
         draft_tokens = np.zeros((B, N), dtype=np.int32)
         for b in range(B):
             ch = children_lists(parent[b])
-            draft_tokens[b, 0] = int(rng.integers(V))
+            draft_tokens[b, 0] = int(rng_acc.integers(V))
             for i in range(N):
                 m = len(ch[i])
                 if temperature[b] > 0:
-                    draft_probs[b, i] = _draft_distribution(rng, logits[b, i])
+                    draft_probs[b, i] = _draft_distribution(rng_acc, logits[b, i])
                     if m:
-                        draft_tokens[b, ch[i]] = _draw_without_replacement(rng, draft_probs[b, i], m)
+                        draft_tokens[b, ch[i]] = _draw_without_replacement(rng_acc, draft_probs[b, i], m)
                 elif m:
-                    noisy = logits[b, i].astype(np.float64) + rng.standard_normal(V)
+                    noisy = logits[b, i].astype(np.float64) + rng_acc.standard_normal(V)
                     top = np.argpartition(-noisy, min(m, V - 1))[:m]
                     top = top[np.argsort(-noisy[top], kind="stable")]
                     draft_tokens[b, ch[i]] = top.astype(np.int32)
-        uniforms = rng.random((B, N + 1), dtype=np.float32)
+        uniforms = rng_acc.random((B, N + 1), dtype=np.float32)
         uniforms = np.minimum(uniforms, np.float32(1.0 - 2.0 ** -24))
     else:
         logits = np.zeros((0,), dtype=np.float32)
