@@ -53,7 +53,8 @@ typedef enum {
     FSPAD_ERR_CUDA = -6,           /* a CUDA runtime call or launch failed             */
     FSPAD_ERR_TIMEOUT = -7,        /* a bounded device-side wait ran out               */
     FSPAD_ERR_BAD_TREE = -8,       /* parent[0] != -1 or parent[i] outside [0, i)      */
-    FSPAD_ERR_NOMEM = -9           /* device or host allocation failed at create time  */
+    FSPAD_ERR_NOMEM = -9,          /* device or host allocation failed at create time  */
+    FSPAD_ERR_TOO_LARGE = -10      /* size beyond the fixed capacity of a no-allocation call */
 } fspad_error;
 
 typedef struct {
@@ -157,6 +158,35 @@ int fspad_tree_accept(fspad_ctx *ctx, const float *target_logits, const float *d
 int fspad_accept_stats(fspad_ctx *ctx, const float *logits, const float *temperature, int rows,
                        int rows_per_seq, float *row_max, double *row_sum, int32_t *row_arg,
                        void *stream);
+
+/*
+ * fspad_accept_stats without any allocation.  (The paper has no counterpart:
+ * this entry point exists for the sake of the hosting program, not the method.)
+ *
+ * Who needs it: a caller that is not allowed to allocate device memory - for
+ * instance a serving process whose own memory pool has claimed the whole GPU
+ * and treats any outside cudaMalloc as an error, or code on a latency-critical
+ * path where the implicit device synchronisation of an allocation is ruled out.
+ * Such a caller cannot use fspad_create (it allocates the context's scratch),
+ * so this call takes no context.  Its scratch (per-slice partial results and
+ * per-row arrival counters) is a fixed array inside the library's device image:
+ * about 0.5 MB that every GPU loading the library keeps until the process ends.
+ *
+ * Same inputs, outputs and results as fspad_accept_stats (vocab is passed
+ * explicitly since there is no context), all DEVICE pointers owned by the caller.
+ * Limits: rows <= 1024; larger calls return FSPAD_ERR_TOO_LARGE and launch nothing.
+ * The call allocates and frees nothing, on the device or through any library.
+ *
+ * The first call on each device looks up the scratch array's device address
+ * (a cudaGetSymbolAddress query, with that device current); make that first
+ * call outside any stream capture.  All calls on a device share the one array:
+ * the counters are cleared at the start of every call, but two calls whose GPU
+ * work overlaps (different streams, or different host threads) race on it and
+ * give undefined results - serialise them.
+ */
+int fspad_accept_stats_noalloc(const float *logits, const float *temperature, int rows,
+                               int rows_per_seq, int vocab, float *row_max, double *row_sum,
+                               int32_t *row_arg, void *stream);
 
 /*
  * Accepted-path KV compaction ("Preliminaries": the discarded tokens leave the

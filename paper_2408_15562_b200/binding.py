@@ -19,7 +19,7 @@ _lib = None
 
 EXPORTS = ["fspad_create", "fspad_destroy", "fspad_status", "fspad_strerror", "fspad_launch_count",
            "fspad_tree_attn", "fspad_tree_accept", "fspad_accept_stats", "fspad_kv_compact",
-           "fspad_verify_step_host"]
+           "fspad_verify_step_host", "fspad_accept_stats_noalloc"]
 
 
 class FspadConfig(ctypes.Structure):
@@ -56,6 +56,7 @@ def load():
     lib.fspad_tree_accept.argtypes = [vp] * 7 + [ci, ci, vp, vp, vp, vp]
     lib.fspad_accept_stats.argtypes = [vp, vp, vp, ci, ci, vp, vp, vp, vp]
     lib.fspad_kv_compact.argtypes = [vp, vp, vp, vp, vp, ci, vp, vp]
+    lib.fspad_accept_stats_noalloc.argtypes = [vp, vp, ci, ci, ci, vp, vp, vp, vp]
     lib.fspad_verify_step_host.argtypes = [vp] * 12 + [ci, ci] + [vp] * 6
     _lib = lib
     return lib
@@ -195,6 +196,17 @@ class Context:
         if rc != 0:
             raise FspadError(rc, "fspad_verify_step_host")
         return attn_out, accepted_path, n_accepted, bonus_token, new_len
+
+
+def accept_stats_noalloc(logits, temperature, rows_per_seq, out, stream=None) -> int:
+    """Context-free per-node scan for callers that may not allocate device memory; the
+    caller supplies the three output tensors.  Returns the library's status code."""
+    rows, vocab = logits.shape
+    row_max, row_sum, row_arg = out
+    return load().fspad_accept_stats_noalloc(_ptr(logits, torch.float32), _ptr(temperature, torch.float32), rows,
+                                             rows_per_seq, vocab, _ptr(row_max, torch.float32),
+                                             _ptr(row_sum, torch.float64), _ptr(row_arg, torch.int32),
+                                             _stream(stream))
 
 
 def bf16_tensor(bits, device="cuda"):

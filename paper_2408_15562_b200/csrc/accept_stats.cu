@@ -185,3 +185,80 @@ cudaError_t fspad_launch_accept_stats(fspad_ctx *ctx, const float *logits, const
     ctx->launches++;
     return cudaGetLastError();
 }
+
+// ---------------------------------------------------------------------------
+// The same scan for callers that must not allocate device memory.
+//
+// Some hosts of this library run where cudaMalloc is off limits: inside a
+// serving process whose memory pool owns the whole device and forbids outside
+// allocations, or in a start-up path where an allocation (which synchronises
+// the device) is not acceptable.  They cannot create an fspad_ctx, so this entry
+// point needs none: the slice partials and arrival counters live in the fixed
+// device array below, which every GPU that loads the library holds until the
+// process exits (about 0.5 MB).
+// ---------------------------------------------------------------------------
+namespace {
+
+constexpr int kNoAllocMaxRows = 1024;     // e.g. 16 sequences x 64 nodes
+constexpr int kNoAllocMaxSlices = 32;
+constexpr size_t kNaSlots = (size_t)kNoAllocMaxRows * kNoAllocMaxSlices;
+constexpr size_t kNaOffSum = 0;                                        // double[kNaSlots]
+constexpr size_t kNaOffMax = kNaOffSum + kNaSlots * sizeof(double);    // float [kNaSlots]
+constexpr size_t kNaOffArg = kNaOffMax + kNaSlots * sizeof(float);     // int   [kNaSlots]
+constexpr size_t kNaOffCnt = kNaOffArg + kNaSlots * sizeof(int);       // unsigned[kNoAllocMaxRows]
+constexpr size_t kNaBytes = kNaOffCnt + kNoAllocMaxRows * sizeof(unsigned);
+
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNaBytes];
+
+constexpr int kMaxDevices = 64;
+struct NoAllocDevice {
+    unsigned char *scratch;   // device address of g_noalloc_scratch on this device (NULL = not set up)
+    int sm_count;
+};
+NoAllocDevice g_na_dev[kMaxDevices];
+
+}  // namespace
+
+extern "C" int fspad_accept_stats_noalloc(const float *logits, const float *temperature, int rows,
+                                          int rows_per_seq, int vocab, float *row_max, double *row_sum,
+                                          int32_t *row_arg, void *stream)
+{
+    if (!logits || !row_max || !row_sum || !row_arg) return FSPAD_ERR_NULL;
+    if (rows < 0 || rows_per_seq < 1 || vocab < 1) return FSPAD_ERR_SHAPE;
+    if (rows > kNoAllocMaxRows) return FSPAD_ERR_TOO_LARGE;
+    if (rows == 0) return FSPAD_OK;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return FSPAD_ERR_CUDA;
+    NoAllocDevice &nd = g_na_dev[dev];
+    if (!nd.scratch) {
+        // First call on this device: g_noalloc_scratch is only a host-side handle here, the
+        // kernel needs the array's address in this device's memory.
+        void *p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_noalloc_scratch) != cudaSuccess || !p) return FSPAD_ERR_CUDA;
+        if (cudaDeviceGetAttribute(&nd.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+            return FSPAD_ERR_CUDA;
+        nd.scratch = static_cast<unsigned char *>(p);
+    }
+    int slices = (nd.sm_count * 4 + rows - 1) / rows;
+    const int max_by_size = (vocab + 4 * kThreads - 1) / (4 * kThreads);
+    if (slices > max_by_size) slices = max_by_size;
+    if (slices > kNoAllocMaxSlices) slices = kNoAllocMaxSlices;
+    if (slices < 1) slices = 1;
+
+    cudaStream_t st = fspad_stream(stream);
+    double *psum = reinterpret_cast<double *>(nd.scratch + kNaOffSum);
+    float *pmax = reinterpret_cast<float *>(nd.scratch + kNaOffMax);
+    int *parg = reinterpret_cast<int *>(nd.scratch + kNaOffArg);
+    unsigned *counter = reinterpret_cast<unsigned *>(nd.scratch + kNaOffCnt);
+    // the arrival counters must start at zero whatever an earlier call left behind
+    if (cudaMemsetAsync(counter, 0, (size_t)rows * sizeof(unsigned), st) != cudaSuccess) return FSPAD_ERR_CUDA;
+    dim3 grid((unsigned)slices * (unsigned)rows);
+    const bool vec = (vocab % 4 == 0) && ((reinterpret_cast<uintptr_t>(logits) & 15) == 0);
+    if (vec)
+        accept_stats_kernel<true><<<grid, kThreads, 0, st>>>(logits, temperature, vocab, rows_per_seq, slices, pmax,
+                                                             psum, parg, counter, row_max, row_sum, row_arg);
+    else
+        accept_stats_kernel<false><<<grid, kThreads, 0, st>>>(logits, temperature, vocab, rows_per_seq, slices, pmax,
+                                                              psum, parg, counter, row_max, row_sum, row_arg);
+    return cudaGetLastError() == cudaSuccess ? FSPAD_OK : FSPAD_ERR_CUDA;
+}

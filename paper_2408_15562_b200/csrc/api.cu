@@ -45,6 +45,7 @@ const char *fspad_strerror(int err)
     case FSPAD_ERR_TIMEOUT: return "bounded device-side wait ran out";
     case FSPAD_ERR_BAD_TREE: return "parent[] is not a topologically ordered tree rooted at node 0";
     case FSPAD_ERR_NOMEM: return "allocation failed";
+    case FSPAD_ERR_TOO_LARGE: return "size exceeds the fixed capacity of the no-allocation entry point";
     default: return "unknown error";
     }
 }
