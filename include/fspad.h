@@ -168,8 +168,8 @@ int fspad_accept_stats(fspad_ctx *ctx, const float *logits, const float *tempera
  * and treats any outside cudaMalloc as an error, or code on a latency-critical
  * path where the implicit device synchronisation of an allocation is ruled out.
  * Such a caller cannot use fspad_create (it allocates the context's scratch),
- * so this call takes no context.  Its scratch (per-slice partial results and
- * per-row arrival counters) is a fixed array inside the library's device image:
+ * so this call takes no context.  Its scratch (the per-CTA partial results of
+ * each row) is a fixed array inside the library's device image:
  * about 0.5 MB that every GPU loading the library keeps until the process ends.
  *
  * Same inputs, outputs and results as fspad_accept_stats (vocab is passed
@@ -180,7 +180,8 @@ int fspad_accept_stats(fspad_ctx *ctx, const float *logits, const float *tempera
  * The first call on each device looks up the scratch array's device address
  * (a cudaGetSymbolAddress query, with that device current); make that first
  * call outside any stream capture.  All calls on a device share the one array:
- * the counters are cleared at the start of every call, but two calls whose GPU
+ * a call rewrites every slot it later reads, so nothing needs clearing between
+ * calls, but two calls whose GPU
  * work overlaps (different streams, or different host threads) race on it and
  * give undefined results - serialise them.
  */

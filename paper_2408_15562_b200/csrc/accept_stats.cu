@@ -5,165 +5,202 @@
 // (Section "Preliminaries") needs the target's result for every tree node;
 // this kernel produces all of them in one HBM-bound sweep.
 //
-// Layout: logits [rows][V] fp32.  Grid rows*slices: a CTA owns one
-// contiguous slice of one row, issues all of its 128-bit loads up front,
-// reduces with warp shuffles, and the last CTA of a row to finish merges the
-// row's slice partials (a self-resetting arrival counter, no second launch).
+// Layout: logits [rows][V] fp32, viewed as one flat array that is cut into
+// equal contiguous ranges, one per CTA (four CTAs per SM, a single wave), so
+// the load is balanced whatever rows and V are.  A range may cross row
+// boundaries; each (row, CTA) piece yields one partial (max, argmax, sum).
+// A thread issues eight 128-bit loads before it touches the data, takes the
+// maximum of the 32 values in registers, rescales its running sum once and
+// adds the 32 exponentials: no per-element branch.  Partials are merged per
+// row by whoever needs them (the acceptance walk for the rows it visits, or
+// the small merge kernel behind fspad_accept_stats).
 #include "common.cuh"
 
 namespace {
 
 constexpr int kThreads = 256;
-constexpr int kBatch = 4;                 // float4 loads in flight per thread per round
+constexpr int kDeep = 8;                  // load units in flight per thread
 constexpr float kLog2e = 1.4426950408889634f;
 
-struct Part {
-    float m;     // running maximum
-    float s;     // sum of exp2((x - m) * k)
-    int a;       // lowest index of the maximum
-};
-
-__device__ __forceinline__ float safe_sub(float m_old, float m_new)
+__device__ __forceinline__ float ex2(float x)
 {
-    // (m_old - m_new) with -inf - -inf := -inf, so that an all -inf prefix scales to zero
-    return (m_old == -INFINITY) ? -INFINITY : m_old - m_new;
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
 }
 
-__device__ __forceinline__ void merge(Part &p, const Part &o, float k)
+struct Acc {
+    float m, s;
+    int a;
+};
+
+__device__ __forceinline__ void acc_merge(Acc &p, float om, float os, int oa, float k)
 {
-    const float mn = fmaxf(p.m, o.m);
-    const float sp = p.s * exp2f(safe_sub(p.m, mn) * k);
-    const float so = o.s * exp2f(safe_sub(o.m, mn) * k);
-    const bool take_o = (o.m > p.m) || (o.m == p.m && o.a < p.a);
-    p.a = take_o ? o.a : p.a;
+    const float mn = fmaxf(p.m, om);
+    const float sp = (p.m == -INFINITY) ? 0.f : p.s * ex2((p.m - mn) * k);
+    const float so = (om == -INFINITY) ? 0.f : os * ex2((om - mn) * k);
+    if (om > p.m || (om == p.m && oa < p.a)) p.a = oa;
     p.m = mn;
     p.s = sp + so;
 }
 
-__device__ __forceinline__ void absorb4(Part &p, const float4 v, int j, float k)
+template <int UNIT>
+__global__ void __launch_bounds__(kThreads, 4)
+accept_stats_kernel(const float *__restrict__ logits, const float *__restrict__ temperature,
+                    int rows_per_seq, const FspadStatsGeom g, FspadStatsPart *__restrict__ parts)
 {
-    float bm = fmaxf(fmaxf(v.x, v.y), fmaxf(v.z, v.w));
-    if (bm > p.m) {
-        p.s *= exp2f(safe_sub(p.m, bm) * k);
-        p.m = bm;
-        p.a = (v.x == bm) ? j : (v.y == bm) ? j + 1 : (v.z == bm) ? j + 2 : j + 3;
-    }
-    if (p.m != -INFINITY) {
-        const float m = p.m;
-        p.s += exp2f((v.x - m) * k) + exp2f((v.y - m) * k) + exp2f((v.z - m) * k) +
-               exp2f((v.w - m) * k);
+    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    const long long lo = (long long)blockIdx.x * g.chunk;
+    const long long hi = min(g.total, lo + g.chunk);
+    __shared__ Acc wacc[kThreads / 32];
+
+    long long seg_lo = lo;
+    while (seg_lo < hi) {
+        const int row = (int)(seg_lo / g.upr);
+        const long long row_lo = (long long)row * g.upr;
+        const long long seg_hi = min(hi, row_lo + g.upr);
+        float T = temperature ? temperature[row / rows_per_seq] : 1.0f;
+        if (!(T > 0.0f)) T = 1.0f;
+        const float k = kLog2e / T;
+
+        Acc p{-INFINITY, 0.f, 0x7fffffff};
+        for (long long base = seg_lo; base < seg_hi; base += (long long)kThreads * kDeep) {
+            if (UNIT == 4) {
+                float4 v[kDeep];
+                const float4 *x4 = reinterpret_cast<const float4 *>(logits);
+#pragma unroll
+                for (int u = 0; u < kDeep; ++u) {
+                    const long long i = base + u * kThreads + tid;
+                    v[u] = (i < seg_hi) ? __ldg(x4 + i) : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+                }
+                float bm = -INFINITY;
+#pragma unroll
+                for (int u = 0; u < kDeep; ++u) bm = fmaxf(bm, fmaxf(fmaxf(v[u].x, v[u].y), fmaxf(v[u].z, v[u].w)));
+                if (bm > p.m) {
+                    // lowest index attaining the new maximum: scan from the back so the first match wins
+                    int a = 0;
+#pragma unroll
+                    for (int u = kDeep - 1; u >= 0; --u) {
+                        const int j = (int)((base + u * kThreads + tid - row_lo) << 2);
+                        if (v[u].w == bm) a = j + 3;
+                        if (v[u].z == bm) a = j + 2;
+                        if (v[u].y == bm) a = j + 1;
+                        if (v[u].x == bm) a = j;
+                    }
+                    p.s = (p.m == -INFINITY) ? 0.f : p.s * ex2((p.m - bm) * k);
+                    p.m = bm;
+                    p.a = a;
+                }
+                if (p.m != -INFINITY) {
+                    const float m = p.m;
+                    float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+                    for (int u = 0; u < kDeep; ++u) {
+                        s0 += ex2((v[u].x - m) * k) + ex2((v[u].y - m) * k);
+                        s1 += ex2((v[u].z - m) * k) + ex2((v[u].w - m) * k);
+                    }
+                    p.s += s0 + s1;
+                }
+            } else {
+                float v[kDeep];
+#pragma unroll
+                for (int u = 0; u < kDeep; ++u) {
+                    const long long i = base + u * kThreads + tid;
+                    v[u] = (i < seg_hi) ? __ldg(logits + i) : -INFINITY;
+                }
+                float bm = -INFINITY;
+#pragma unroll
+                for (int u = 0; u < kDeep; ++u) bm = fmaxf(bm, v[u]);
+                if (bm > p.m) {
+                    int a = 0;
+#pragma unroll
+                    for (int u = kDeep - 1; u >= 0; --u)
+                        if (v[u] == bm) a = (int)(base + u * kThreads + tid - row_lo);
+                    p.s = (p.m == -INFINITY) ? 0.f : p.s * ex2((p.m - bm) * k);
+                    p.m = bm;
+                    p.a = a;
+                }
+                if (p.m != -INFINITY) {
+                    float s0 = 0.f;
+#pragma unroll
+                    for (int u = 0; u < kDeep; ++u) s0 += ex2((v[u] - p.m) * k);
+                    p.s += s0;
+                }
+            }
+        }
+        // block reduction of (m, s, a)
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+            const float om = __shfl_xor_sync(0xffffffffu, p.m, off);
+            const float os = __shfl_xor_sync(0xffffffffu, p.s, off);
+            const int oa = __shfl_xor_sync(0xffffffffu, p.a, off);
+            acc_merge(p, om, os, oa, k);
+        }
+        if (lane == 0) wacc[wid] = p;
+        __syncthreads();
+        if (wid == 0) {
+            Acc q = (lane < kThreads / 32) ? wacc[lane] : Acc{-INFINITY, 0.f, 0x7fffffff};
+#pragma unroll
+            for (int off = 4; off > 0; off >>= 1) {
+                const float om = __shfl_xor_sync(0xffffffffu, q.m, off);
+                const float os = __shfl_xor_sync(0xffffffffu, q.s, off);
+                const int oa = __shfl_xor_sync(0xffffffffu, q.a, off);
+                acc_merge(q, om, os, oa, k);
+            }
+            if (lane == 0) {
+                const int first = (int)(row_lo / g.chunk);
+                FspadStatsPart out;
+                out.m = q.m; out.s = q.s; out.a = q.a; out.pad = 0;
+                parts[(size_t)row * g.slots + (blockIdx.x - first)] = out;
+            }
+        }
+        __syncthreads();
+        seg_lo = seg_hi;
     }
 }
 
-__device__ __forceinline__ void absorb1(Part &p, float x, int j, float k)
+// rows -> (max, sum, argmax) from the partials; one warp per row
+__global__ void __launch_bounds__(128)
+accept_stats_merge_kernel(const FspadStatsPart *__restrict__ parts, const FspadStatsGeom g,
+                          const float *__restrict__ temperature, int rows, int rows_per_seq,
+                          float *__restrict__ row_max, double *__restrict__ row_sum, int *__restrict__ row_arg)
 {
-    if (x > p.m) {
-        p.s *= exp2f(safe_sub(p.m, x) * k);
-        p.m = x;
-        p.a = j;
-    }
-    if (p.m != -INFINITY) p.s += exp2f((x - p.m) * k);
-}
-
-template <bool VEC4>
-__global__ void __launch_bounds__(kThreads)
-accept_stats_kernel(const float *__restrict__ logits, const float *__restrict__ temperature, int V,
-                    int rows_per_seq, int slices, float *__restrict__ pmax, double *__restrict__ psum,
-                    int *__restrict__ parg, unsigned *__restrict__ counter, float *__restrict__ row_max,
-                    double *__restrict__ row_sum, int *__restrict__ row_arg)
-{
-    const int row = blockIdx.x / slices, slice = blockIdx.x % slices, tid = threadIdx.x;
+    const int lane = threadIdx.x & 31;
+    const int row = blockIdx.x * 4 + (threadIdx.x >> 5);
+    if (row >= rows) return;
     float T = temperature ? temperature[row / rows_per_seq] : 1.0f;
     if (!(T > 0.0f)) T = 1.0f;
-    const float k = kLog2e / T;
-    const float *x = logits + (size_t)row * V;
+    float M;
+    double S;
+    int A;
+    fspad_stats_merge_warp(parts, g, row, kLog2e / T, lane, M, S, A);
+    if (lane == 0) {
+        row_max[row] = M;
+        row_sum[row] = S;
+        row_arg[row] = A;
+    }
+}
 
-    Part p{-INFINITY, 0.0f, 0x7fffffff};
-    if (VEC4) {
-        const int n4 = V >> 2;
-        const int per = (n4 + slices - 1) / slices;
-        const int lo = slice * per, hi = min(n4, lo + per);
-        const float4 *x4 = reinterpret_cast<const float4 *>(x);
-        int i = lo + tid;
-        for (; i + (kBatch - 1) * kThreads < hi; i += kBatch * kThreads) {
-            float4 v[kBatch];
-#pragma unroll
-            for (int u = 0; u < kBatch; ++u) v[u] = __ldg(x4 + i + u * kThreads);
-#pragma unroll
-            for (int u = 0; u < kBatch; ++u) absorb4(p, v[u], (i + u * kThreads) << 2, k);
-        }
-        for (; i < hi; i += kThreads) absorb4(p, __ldg(x4 + i), i << 2, k);
-    } else {
-        const int per = (V + slices - 1) / slices;
-        const int lo = slice * per, hi = min(V, lo + per);
-        for (int i = lo + tid; i < hi; i += kThreads) absorb1(p, x[i], i, k);
-    }
-
-    // warp reduction
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) {
-        Part o;
-        o.m = __shfl_xor_sync(0xffffffffu, p.m, off);
-        o.s = __shfl_xor_sync(0xffffffffu, p.s, off);
-        o.a = __shfl_xor_sync(0xffffffffu, p.a, off);
-        merge(p, o, k);
-    }
-    __shared__ Part wp[kThreads / 32];
-    __shared__ bool is_last;
-    if ((tid & 31) == 0) wp[tid >> 5] = p;
-    __syncthreads();
-    if (tid == 0) {
-        // block merge in double for the sum
-        float m = wp[0].m;
-        int a = wp[0].a;
-        for (int w = 1; w < kThreads / 32; ++w) {
-            if (wp[w].m > m || (wp[w].m == m && wp[w].a < a)) { m = wp[w].m; a = wp[w].a; }
-        }
-        double s = 0.0;
-        for (int w = 0; w < kThreads / 32; ++w)
-            s += (double)wp[w].s * (double)exp2f(safe_sub(wp[w].m, m) * k);
-        const size_t slot = (size_t)row * slices + slice;
-        pmax[slot] = m;
-        psum[slot] = s;
-        parg[slot] = a;
-        __threadfence();
-        const unsigned prev = atomicAdd(counter + row, 1u);
-        is_last = (prev == (unsigned)slices - 1u);
-        if (is_last) {
-            __threadfence();
-            const size_t base = (size_t)row * slices;
-            float M = -INFINITY;
-            int A = 0x7fffffff;
-            for (int sl = 0; sl < slices; ++sl) {
-                const float ms = __ldcg(pmax + base + sl);
-                const int as = __ldcg(parg + base + sl);
-                if (ms > M || (ms == M && as < A)) { M = ms; A = as; }
-            }
-            double S = 0.0;
-            for (int sl = 0; sl < slices; ++sl) {
-                const float ms = __ldcg(pmax + base + sl);
-                S += __ldcg(psum + base + sl) * exp2((double)safe_sub(ms, M) * (double)k);
-            }
-            row_max[row] = M;
-            row_sum[row] = S;
-            row_arg[row] = (A == 0x7fffffff) ? 0 : A;
-            counter[row] = 0u;       // ready for the next call
-        }
-    }
+cudaError_t launch_partials(const float *logits, const float *temperature, int rows_per_seq,
+                            const FspadStatsGeom &g, FspadStatsPart *parts, cudaStream_t st)
+{
+    if (g.unit == 4)
+        accept_stats_kernel<4><<<g.n_cta, kThreads, 0, st>>>(logits, temperature, rows_per_seq, g, parts);
+    else
+        accept_stats_kernel<1><<<g.n_cta, kThreads, 0, st>>>(logits, temperature, rows_per_seq, g, parts);
+    return cudaGetLastError();
 }
 
 }  // namespace
 
-int fspad_stats_slices(const fspad_ctx *ctx, int rows, int V)
+cudaError_t fspad_launch_stats_partials(fspad_ctx *ctx, const float *logits, const float *temperature,
+                                        int rows, int rows_per_seq, int V, FspadStatsGeom *geom,
+                                        cudaStream_t st)
 {
-    // about four CTAs per SM in one wave, each with at least a few KB to read
-    const int target_ctas = ctx->sm_count * 4;
-    int s = (target_ctas + rows - 1) / rows;
-    const int max_by_size = (V + 4 * kThreads - 1) / (4 * kThreads);   // >= one float4 per thread
-    if (s > max_by_size) s = max_by_size;
-    if (s > ctx->stats_max_slices) s = ctx->stats_max_slices;
-    if (s < 1) s = 1;
-    return s;
+    const bool vec = (V % 4 == 0) && ((reinterpret_cast<uintptr_t>(logits) & 15) == 0);
+    *geom = fspad_stats_geom(ctx->sm_count, rows, V, vec, ctx->stats_slots);
+    ctx->launches++;
+    return launch_partials(logits, temperature, rows_per_seq, *geom, ctx->st_part, st);
 }
 
 cudaError_t fspad_launch_accept_stats(fspad_ctx *ctx, const float *logits, const float *temperature,
@@ -171,17 +208,11 @@ cudaError_t fspad_launch_accept_stats(fspad_ctx *ctx, const float *logits, const
                                       double *row_sum, int *row_arg, cudaStream_t st)
 {
     if (rows == 0) return cudaSuccess;
-    const int slices = fspad_stats_slices(ctx, rows, V);
-    dim3 grid((unsigned)slices * (unsigned)rows);
-    const bool vec = (V % 4 == 0) && ((reinterpret_cast<uintptr_t>(logits) & 15) == 0);
-    if (vec)
-        accept_stats_kernel<true><<<grid, kThreads, 0, st>>>(logits, temperature, V, rows_per_seq, slices,
-                                                             ctx->st_pmax, ctx->st_psum, ctx->st_parg,
-                                                             ctx->st_counter, row_max, row_sum, row_arg);
-    else
-        accept_stats_kernel<false><<<grid, kThreads, 0, st>>>(logits, temperature, V, rows_per_seq, slices,
-                                                              ctx->st_pmax, ctx->st_psum, ctx->st_parg,
-                                                              ctx->st_counter, row_max, row_sum, row_arg);
+    FspadStatsGeom g;
+    cudaError_t e = fspad_launch_stats_partials(ctx, logits, temperature, rows, rows_per_seq, V, &g, st);
+    if (e != cudaSuccess) return e;
+    accept_stats_merge_kernel<<<(rows + 3) / 4, 128, 0, st>>>(ctx->st_part, g, temperature, rows,
+                                                                 rows_per_seq, row_max, row_sum, row_arg);
     ctx->launches++;
     return cudaGetLastError();
 }
@@ -193,20 +224,14 @@ cudaError_t fspad_launch_accept_stats(fspad_ctx *ctx, const float *logits, const
 // serving process whose memory pool owns the whole device and forbids outside
 // allocations, or in a start-up path where an allocation (which synchronises
 // the device) is not acceptable.  They cannot create an fspad_ctx, so this entry
-// point needs none: the slice partials and arrival counters live in the fixed
-// device array below, which every GPU that loads the library holds until the
-// process exits (about 0.5 MB).
+// point needs none: the per-CTA partials live in the fixed device array below,
+// which every GPU that loads the library holds until the process exits (0.5 MB).
 // ---------------------------------------------------------------------------
 namespace {
 
 constexpr int kNoAllocMaxRows = 1024;     // e.g. 16 sequences x 64 nodes
-constexpr int kNoAllocMaxSlices = 32;
-constexpr size_t kNaSlots = (size_t)kNoAllocMaxRows * kNoAllocMaxSlices;
-constexpr size_t kNaOffSum = 0;                                        // double[kNaSlots]
-constexpr size_t kNaOffMax = kNaOffSum + kNaSlots * sizeof(double);    // float [kNaSlots]
-constexpr size_t kNaOffArg = kNaOffMax + kNaSlots * sizeof(float);     // int   [kNaSlots]
-constexpr size_t kNaOffCnt = kNaOffArg + kNaSlots * sizeof(int);       // unsigned[kNoAllocMaxRows]
-constexpr size_t kNaBytes = kNaOffCnt + kNoAllocMaxRows * sizeof(unsigned);
+constexpr int kNoAllocSlots = 32;         // partial slots per row
+constexpr size_t kNaBytes = (size_t)kNoAllocMaxRows * kNoAllocSlots * sizeof(FspadStatsPart);
 
 static __device__ __align__(256) unsigned char g_noalloc_scratch[kNaBytes];
 
@@ -232,33 +257,21 @@ extern "C" int fspad_accept_stats_noalloc(const float *logits, const float *temp
     NoAllocDevice &nd = g_na_dev[dev];
     if (!nd.scratch) {
         // First call on this device: g_noalloc_scratch is only a host-side handle here, the
-        // kernel needs the array's address in this device's memory.
+        // kernels need the array's address in this device's memory.
         void *p = nullptr;
         if (cudaGetSymbolAddress(&p, g_noalloc_scratch) != cudaSuccess || !p) return FSPAD_ERR_CUDA;
         if (cudaDeviceGetAttribute(&nd.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
             return FSPAD_ERR_CUDA;
         nd.scratch = static_cast<unsigned char *>(p);
     }
-    int slices = (nd.sm_count * 4 + rows - 1) / rows;
-    const int max_by_size = (vocab + 4 * kThreads - 1) / (4 * kThreads);
-    if (slices > max_by_size) slices = max_by_size;
-    if (slices > kNoAllocMaxSlices) slices = kNoAllocMaxSlices;
-    if (slices < 1) slices = 1;
-
     cudaStream_t st = fspad_stream(stream);
-    double *psum = reinterpret_cast<double *>(nd.scratch + kNaOffSum);
-    float *pmax = reinterpret_cast<float *>(nd.scratch + kNaOffMax);
-    int *parg = reinterpret_cast<int *>(nd.scratch + kNaOffArg);
-    unsigned *counter = reinterpret_cast<unsigned *>(nd.scratch + kNaOffCnt);
-    // the arrival counters must start at zero whatever an earlier call left behind
-    if (cudaMemsetAsync(counter, 0, (size_t)rows * sizeof(unsigned), st) != cudaSuccess) return FSPAD_ERR_CUDA;
-    dim3 grid((unsigned)slices * (unsigned)rows);
     const bool vec = (vocab % 4 == 0) && ((reinterpret_cast<uintptr_t>(logits) & 15) == 0);
-    if (vec)
-        accept_stats_kernel<true><<<grid, kThreads, 0, st>>>(logits, temperature, vocab, rows_per_seq, slices, pmax,
-                                                             psum, parg, counter, row_max, row_sum, row_arg);
-    else
-        accept_stats_kernel<false><<<grid, kThreads, 0, st>>>(logits, temperature, vocab, rows_per_seq, slices, pmax,
-                                                              psum, parg, counter, row_max, row_sum, row_arg);
+    const FspadStatsGeom g = fspad_stats_geom(nd.sm_count, rows, vocab, vec, kNoAllocSlots);
+    FspadStatsPart *parts = reinterpret_cast<FspadStatsPart *>(nd.scratch);
+    // every slot the merge reads is rewritten by this call's first kernel, so the contents an
+    // earlier call left in the shared array never need clearing
+    if (launch_partials(logits, temperature, rows_per_seq, g, parts, st) != cudaSuccess) return FSPAD_ERR_CUDA;
+    accept_stats_merge_kernel<<<(rows + 3) / 4, 128, 0, st>>>(parts, g, temperature, rows, rows_per_seq,
+                                                                 row_max, row_sum, row_arg);
     return cudaGetLastError() == cudaSuccess ? FSPAD_OK : FSPAD_ERR_CUDA;
 }

@@ -11,9 +11,11 @@
 // serial chain of scalar decisions taken in fp64; whenever a decision needs a
 // whole-vocabulary quantity (an exact softmax denominator, the mass of a
 // residual distribution, the inverse CDF of the bonus draw) the cluster sweeps
-// the node's logits and draft rows once, every CTA reducing its contiguous
-// slice of the vocabulary and the CTAs exchanging partial sums through
-// distributed shared memory.  Only rows on the realised path are ever read.
+// the node's rows, every CTA reducing its contiguous slice of the vocabulary
+// and the CTAs exchanging partial sums through distributed shared memory.
+// Only rows on the realised path are ever read.  The first sweep at a node
+// evaluates exp((x - max)/T) in fp64 once per token and parks the values (and
+// the draft row) in shared memory, so later sweeps at that node are cheap.
 //
 // The residual after k rejections at a node is kept in closed form instead of
 // as a vector: for a token j that has not been rejected,
@@ -24,6 +26,11 @@
 // tokens not yet rejected, divided by its sum D.  A rejection of token x turns
 // c into c + U / D, which is exactly p <- norm(max(p - q, 0)), q <- norm(q
 // without x) written without materialising either vector.
+//
+// The per-row maximum and argmax come exact from the vocabulary scan; its sum
+// of exponentials is fp32-accurate and is trusted only when a decision clears
+// a 1e-4 relative margin, otherwise (and before any residual) the exact sum is
+// swept here.
 #include <cooperative_groups.h>
 
 #include "common.cuh"
@@ -33,40 +40,65 @@ namespace cg = cooperative_groups;
 namespace {
 
 constexpr int kMaxCluster = 16;
-constexpr int kWalkThreads = 512;
+constexpr int kWalkThreads = 1024;
 constexpr int kWarps = kWalkThreads / 32;
-constexpr double kAmbiguous = 1e-4;   // relative margin inside which the approximate denominator is not trusted
+constexpr int kSmemBudget = 200 * 1024;   // dynamic shared memory for the per-node cache
+constexpr double kAmbiguous = 1e-4;
+constexpr float kLog2eF = 1.4426950408889634f;
 
 struct WalkArgs {
     const float *logits, *draft, *temperature, *uniforms;
     const int *tokens, *parent;
-    const float *row_max;
-    const double *row_sum;
-    const int *row_arg;
-    int N, V, path_stride;
+    const FspadStatsPart *parts;
+    FspadStatsGeom geom;
+    int N, V, path_stride, cache_ok;
     int *path, *n_acc, *bonus, *status;
 };
 
-enum { MODE_SUM = 0, MODE_RESID = 1, MODE_CDF = 2 };
-
 struct Shared {
+    double exp_tbl[64];             // 2^(i/64)
     int parent[FSPAD_MAX_NODES];
     int tok[FSPAD_MAX_NODES];
     int path[FSPAD_MAX_NODES];
     // state of the current node (written by thread 0, read by all after a barrier)
-    double S, c, U, D, m, T;
-    int exact, nrem, decision, xnew, ridx, next, len, cur;
+    double S, c, U, D, m, invT;
+    int exact, nrem, decision, xnew, ridx, next, len, cur, have_e, have_q, sel;
     double cprime, ex, qx;
-    int sel;
     int rem_tok[FSPAD_MAX_NODES];
     double rem_frozen[FSPAD_MAX_NODES];
+    // gathered once, in parallel, before the walk: the scan result of every row and, for
+    // every node, its parent's logit and draft probability at the node's token and its uniform
+    float rowM[FSPAD_MAX_NODES];
+    double rowS[FSPAD_MAX_NODES];
+    int rowA[FSPAD_MAX_NODES];
+    float cx[FSPAD_MAX_NODES], cq[FSPAD_MAX_NODES], cu[FSPAD_MAX_NODES];
+    float ubonus;
     // reductions
-    double warp_a[kWarps], warp_b[kWarps];
+    double warp_a[kWarps], warp_b[kWarps], warp_off[kWarps];
     double slot[2][2];              // this CTA's partial sums, by pass parity (read by peers)
-    double tot[2];                  // cluster totals, broadcast inside the CTA
-    double cta_total[kMaxCluster];  // CDF: every CTA's total
-    double warp_off[kWarps];
+    double tot[2];                  // cluster totals
+    double cta_total[kMaxCluster];
 };
+
+// exp(a) for a <= 0 in double precision: a = (64 n + i) ln2/64 + r, |r| <= ln2/128,
+// exp(a) = 2^n * 2^(i/64) * (1 + r + ... + r^5/120); relative error about 4e-16.
+__device__ __forceinline__ double exp_neg(double a, const double *tbl)
+{
+    if (!(a > -700.0)) return 0.0;                        // also -inf and NaN
+    const double t = a * 92.33248261689366;               // 64 / ln 2
+    const int k = __double2int_rn(t);
+    const double kd = (double)k;
+    double r = fma(-kd, 0.010830424696249145, a);         // ln2/64, high part
+    r = fma(-kd, 3.623510646634843e-19, r);               // low part
+    double p = fma(r, 1.0 / 120.0, 1.0 / 24.0);
+    p = fma(p, r, 1.0 / 6.0);
+    p = fma(p, r, 0.5);
+    p = fma(p, r, 1.0);
+    p = fma(p, r, 1.0);
+    const double y = tbl[k & 63] * p;
+    const int n = k >> 6;                                  // floor(k / 64), n in [-1010, 0]
+    return __hiloint2double(__double2hiint(y) + (n << 20), __double2loint(y));
+}
 
 __device__ __forceinline__ double warp_sum(double v)
 {
@@ -75,66 +107,93 @@ __device__ __forceinline__ double warp_sum(double v)
     return v;
 }
 
-// Weight of token j in the current (unnormalised) residual target distribution.
 __device__ __forceinline__ double weight(double e, double q, double invS, double c)
 {
     const double w = e * invS - c * q;
     return w > 0.0 ? w : 0.0;
 }
 
+enum { MODE_EXP = 0, MODE_RESID = 1, MODE_CDF = 2 };
+
 struct Sweep {
     double a, b;
 };
 
 // One sweep of this thread's contiguous chunk [lo, hi) of the vocabulary.
-//   MODE_SUM  : a = sum exp((x - m)/T)
+//   MODE_EXP  : a = sum of e_j = exp((x_j - m)/T); e_j parked in shared memory
 //   MODE_RESID: a = sum of residual weights at coefficient c (tokens already
 //               rejected contribute their frozen value), b = sum of q over
 //               tokens neither rejected before nor equal to xnew
-//   MODE_CDF  : a = sum of residual weights at coefficient c
-// When `locate` is set (CDF owner thread) the sweep instead returns in a the
-// first token whose running sum pushes base + run above target (or -1).
+//   MODE_CDF  : a = sum of the weights the bonus token is drawn from
+//               (nothing rejected at this node: the e_j themselves)
+// With `locate` the running sum starts at run0 and *found receives the first
+// token where base + run exceeds target (else the last positive-weight token).
 template <int MODE>
 __device__ Sweep sweep_chunk(const Shared &sh, const float *__restrict__ x, const float *__restrict__ q,
-                             int lo, int hi, bool vec, double c, int xnew, bool locate, double base,
-                             double run0, double target, int *found)
+                             double *__restrict__ se, float *__restrict__ sq, int cta_lo, int lo, int hi,
+                             bool vec, bool cache_ok, bool have_e, bool have_q, double c, int xnew,
+                             bool locate, double base, double run0, double target, int *found)
 {
-    const double m = sh.m, T = sh.T, invS = 1.0 / sh.S;
+    const double m = sh.m, invT = sh.invT;
     const int nrem = sh.nrem;
+    // bonus draw with nothing rejected at this node: the weights are the e_j themselves
+    const double invS = (MODE == MODE_CDF && c == 0.0 && nrem == 0) ? 1.0 : 1.0 / sh.S;
+    const bool need_q = (MODE == MODE_RESID) || (MODE == MODE_CDF && c != 0.0);
     bool special = false;
-    if (MODE != MODE_SUM) {
+    if (MODE != MODE_EXP) {
         for (int r = 0; r < nrem; ++r) special |= (sh.rem_tok[r] >= lo && sh.rem_tok[r] < hi);
         if (MODE == MODE_RESID) special |= (xnew >= lo && xnew < hi);
     }
     double a = 0.0, b = 0.0, run = run0;
     int last_pos = -1, hit = -1;
     for (int j = lo; j < hi; j += 4) {
-        float xv[4], qv[4] = {0.f, 0.f, 0.f, 0.f};
         const int n = min(4, hi - j);
-        const bool need_q = (MODE == MODE_RESID) || (MODE == MODE_CDF && c != 0.0);
-        if (vec && n == 4) {
-            const float4 t = *reinterpret_cast<const float4 *>(x + j);
-            xv[0] = t.x; xv[1] = t.y; xv[2] = t.z; xv[3] = t.w;
-            if (need_q) {
-                const float4 u = *reinterpret_cast<const float4 *>(q + j);
-                qv[0] = u.x; qv[1] = u.y; qv[2] = u.z; qv[3] = u.w;
-            }
+        double ev[4];
+        float qv[4] = {0.f, 0.f, 0.f, 0.f};
+        if (have_e) {
+#pragma unroll
+            for (int t = 0; t < 4; ++t) ev[t] = (t < n) ? se[j - cta_lo + t] : 0.0;
         } else {
+            float xv[4];
+            if (vec && n == 4) {
+                const float4 t4 = __ldg(reinterpret_cast<const float4 *>(x + j));
+                xv[0] = t4.x; xv[1] = t4.y; xv[2] = t4.z; xv[3] = t4.w;
+            } else {
+#pragma unroll
+                for (int t = 0; t < 4; ++t) xv[t] = (t < n) ? x[j + t] : -INFINITY;
+            }
 #pragma unroll
             for (int t = 0; t < 4; ++t) {
-                xv[t] = (t < n) ? x[j + t] : -INFINITY;
-                if (need_q) qv[t] = (t < n) ? q[j + t] : 0.f;
+                ev[t] = exp_neg(((double)xv[t] - m) * invT, sh.exp_tbl);
+                if (cache_ok && t < n) se[j - cta_lo + t] = ev[t];
+            }
+        }
+        if (need_q) {
+            if (have_q) {
+#pragma unroll
+                for (int t = 0; t < 4; ++t) qv[t] = (t < n) ? sq[j - cta_lo + t] : 0.f;
+            } else {
+                if (vec && n == 4) {
+                    const float4 u4 = __ldg(reinterpret_cast<const float4 *>(q + j));
+                    qv[0] = u4.x; qv[1] = u4.y; qv[2] = u4.z; qv[3] = u4.w;
+                } else {
+#pragma unroll
+                    for (int t = 0; t < 4; ++t) qv[t] = (t < n) ? q[j + t] : 0.f;
+                }
+                if (cache_ok) {
+#pragma unroll
+                    for (int t = 0; t < 4; ++t) if (t < n) sq[j - cta_lo + t] = qv[t];
+                }
             }
         }
 #pragma unroll
         for (int t = 0; t < 4; ++t) {
             if (t >= n) break;
-            const double e = exp(((double)xv[t] - m) / T);
-            if (MODE == MODE_SUM) {
-                a += e;
+            if (MODE == MODE_EXP) {
+                a += ev[t];
                 continue;
             }
-            double w = weight(e, (double)qv[t], invS, c);
+            double w = weight(ev[t], (double)qv[t], invS, c);
             bool q_counts = true;
             if (special) {
                 const int id = j + t;
@@ -142,16 +201,13 @@ __device__ Sweep sweep_chunk(const Shared &sh, const float *__restrict__ x, cons
                     if (sh.rem_tok[r] == id) { w = sh.rem_frozen[r]; q_counts = false; }
                 if (id == xnew) q_counts = false;
             }
+            a += w;
             if (MODE == MODE_RESID) {
-                a += w;
                 if (q_counts) b += (double)qv[t];
-            } else {
-                a += w;
-                if (locate) {
-                    run += w;
-                    if (w > 0.0) last_pos = j + t;
-                    if (hit < 0 && base + run > target) hit = j + t;
-                }
+            } else if (locate) {
+                run += w;
+                if (w > 0.0) last_pos = j + t;
+                if (hit < 0 && base + run > target) hit = j + t;
             }
         }
     }
@@ -159,7 +215,7 @@ __device__ Sweep sweep_chunk(const Shared &sh, const float *__restrict__ x, cons
     return Sweep{a, b};
 }
 
-__global__ void __launch_bounds__(kWalkThreads)
+__global__ void __launch_bounds__(kWalkThreads, 1)
 accept_walk_kernel(const WalkArgs args)
 {
     cg::cluster_group cluster = cg::this_cluster();
@@ -170,6 +226,7 @@ accept_walk_kernel(const WalkArgs args)
     const int N = args.N, V = args.V;
 
     __shared__ Shared sh;
+    extern __shared__ __align__(16) unsigned char dyn_smem[];
 
     const int *par_g = args.parent + (size_t)b * N;
     const int *tok_g = args.tokens + (size_t)b * N;
@@ -189,6 +246,7 @@ accept_walk_kernel(const WalkArgs args)
         sh.parent[i] = p;
         sh.tok[i] = t;
     }
+    if (tid < 64) sh.exp_tbl[tid] = exp2((double)tid * (1.0 / 64.0));
     float Tf = args.temperature[b];
     if (!(Tf >= 0.0f)) {
         if (tid == 0 && rank == 0) fspad_report(args.status, FSPAD_ERR_RANGE);
@@ -199,10 +257,31 @@ accept_walk_kernel(const WalkArgs args)
     __syncthreads();
 
     const float *lg = args.logits + (size_t)b * N * V;
-    const float *rmax = args.row_max + (size_t)b * N;
-    const double *rsum = args.row_sum + (size_t)b * N;
-    const int *rarg = args.row_arg + (size_t)b * N;
+    const float *dp = args.draft ? args.draft + (size_t)b * N * V : nullptr;
+    const float *un = args.uniforms ? args.uniforms + (size_t)b * (N + 1) : nullptr;
     int *out_path = args.path + (size_t)b * args.path_stride;
+    const float kT = kLog2eF / (Tf > 0.0f ? Tf : 1.0f);
+    {
+        // every row's (max, sum, argmax): one warp per row, all partial slots fetched at once
+        const int lane = tid & 31, nwarps = nthr >> 5;
+        for (int row = tid >> 5; row < N; row += nwarps) {
+            float M; double S; int A;
+            fspad_stats_merge_warp(args.parts, args.geom, b * N + row, kT, lane, M, S, A);
+            if (lane == 0) { sh.rowM[row] = M; sh.rowS[row] = S; sh.rowA[row] = A; }
+        }
+        if (sampling) {
+            for (int c = tid; c < N; c += nthr) {
+                if (c >= 1) {
+                    const size_t at = (size_t)sh.parent[c] * V + sh.tok[c];
+                    sh.cx[c] = lg[at];
+                    sh.cq[c] = dp[at];
+                    sh.cu[c] = un[c];
+                }
+            }
+            if (tid == 0) sh.ubonus = un[N];
+        }
+    }
+    __syncthreads();
 
     if (!sampling) {
         // ---- greedy: strict token comparison against the target argmax ----
@@ -210,16 +289,15 @@ accept_walk_kernel(const WalkArgs args)
             int cur = 0, len = 1;
             sh.path[0] = 0;
             for (;;) {
-                const int want = rarg[cur];
+                const int want = sh.rowA[cur];
                 int next = -1;
                 for (int c = cur + 1; c < N; ++c)
                     if (sh.parent[c] == cur && sh.tok[c] == want) { next = c; break; }
-                if (next < 0) break;
+                if (next < 0) { args.bonus[b] = want; break; }
                 sh.path[len++] = next;
                 cur = next;
             }
             args.n_acc[b] = len;
-            args.bonus[b] = rarg[cur];
             sh.len = len;
         }
         __syncthreads();
@@ -229,8 +307,6 @@ accept_walk_kernel(const WalkArgs args)
     }
 
     // ---- sampling ----
-    const float *dp = args.draft + (size_t)b * N * V;
-    const float *un = args.uniforms + (size_t)b * (N + 1);
     const bool vec = (V % 4 == 0) && ((reinterpret_cast<uintptr_t>(args.logits) & 15) == 0) &&
                      ((reinterpret_cast<uintptr_t>(args.draft) & 15) == 0);
     // contiguous slice per CTA, contiguous chunk per thread (multiples of 4 tokens)
@@ -238,9 +314,12 @@ accept_walk_kernel(const WalkArgs args)
     const int per_thr = (((per_cta + nthr - 1) / nthr) + 3) & ~3;
     const int cta_lo = rank * per_cta, cta_hi = min(V, cta_lo + per_cta);
     const int lo = min(cta_hi, cta_lo + tid * per_thr), hi = min(cta_hi, lo + per_thr);
+    const bool cache_ok = args.cache_ok != 0;
+    double *se = reinterpret_cast<double *>(dyn_smem);
+    float *sq = reinterpret_cast<float *>(dyn_smem + (size_t)per_cta * sizeof(double));
     int parity = 0;
 
-    // cluster-wide reduction of (a, b); result in sh.tot[] for every thread of every CTA
+    // cluster-wide reduction of (a, b); result in sh.tot[] (read by thread 0 only)
     auto reduce_exchange = [&](double a, double bb) {
         a = warp_sum(a);
         bb = warp_sum(bb);
@@ -275,10 +354,10 @@ accept_walk_kernel(const WalkArgs args)
         const float *x = lg + (size_t)cur * V;
         const float *q = dp + (size_t)cur * V;
         if (tid == 0) {
-            sh.m = (double)rmax[cur];
-            sh.S = rsum[cur];
-            sh.T = (double)Tf;
-            sh.exact = 0;
+            sh.m = (double)sh.rowM[cur];
+            sh.S = sh.rowS[cur];
+            sh.invT = 1.0 / (double)Tf;
+            sh.exact = 0; sh.have_e = 0; sh.have_q = 0;
             sh.c = 0.0; sh.U = 1.0; sh.D = 1.0;
             sh.nrem = 0;
             sh.next = -1;
@@ -288,12 +367,11 @@ accept_walk_kernel(const WalkArgs args)
         for (int ch = cur + 1; ch < N; ++ch) {
             if (sh.parent[ch] != cur) continue;          // uniform: shared data
             const int xt = sh.tok[ch];
-            // -- evaluate the accept test (thread 0), possibly twice if the denominator must be refined
             for (int attempt = 0; attempt < 2; ++attempt) {
                 if (tid == 0) {
-                    const double r = (double)un[ch];
-                    const double qx = (double)q[xt];
-                    const double ex = exp(((double)x[xt] - sh.m) / sh.T);
+                    const double r = (double)sh.cu[ch];
+                    const double qx = (double)sh.cq[ch];
+                    const double ex = exp_neg(((double)sh.cx[ch] - sh.m) * sh.invT, sh.exp_tbl);
                     int ridx = -1;
                     for (int k = 0; k < sh.nrem; ++k) if (sh.rem_tok[k] == xt) ridx = k;
                     double qk, pk;
@@ -311,10 +389,11 @@ accept_walk_kernel(const WalkArgs args)
                 }
                 __syncthreads();
                 if (sh.decision != 2) break;
-                // exact softmax denominator of this node
-                Sweep s = sweep_chunk<MODE_SUM>(sh, x, q, lo, hi, vec, 0.0, -1, false, 0, 0, 0, nullptr);
+                // exact softmax denominator of this node (parks e_j in shared memory)
+                Sweep s = sweep_chunk<MODE_EXP>(sh, x, q, se, sq, cta_lo, lo, hi, vec, cache_ok, false, false, 0.0,
+                                                -1, false, 0, 0, 0, nullptr);
                 reduce_exchange(s.a, 0.0);
-                if (tid == 0) { sh.S = sh.tot[0]; sh.exact = 1; }
+                if (tid == 0) { sh.S = sh.tot[0]; sh.exact = 1; sh.have_e = cache_ok; }
                 __syncthreads();
             }
             if (sh.decision == 1) {
@@ -326,7 +405,8 @@ accept_walk_kernel(const WalkArgs args)
             if (tid == 0) sh.cprime = sh.c + sh.U / sh.D;
             __syncthreads();
             {
-                Sweep s = sweep_chunk<MODE_RESID>(sh, x, q, lo, hi, vec, sh.cprime, xt, false, 0, 0, 0, nullptr);
+                Sweep s = sweep_chunk<MODE_RESID>(sh, x, q, se, sq, cta_lo, lo, hi, vec, cache_ok, sh.have_e != 0,
+                                                  sh.have_q != 0, sh.cprime, xt, false, 0, 0, 0, nullptr);
                 reduce_exchange(s.a, s.b);
             }
             if (tid == 0) {
@@ -345,6 +425,7 @@ accept_walk_kernel(const WalkArgs args)
                     sh.nrem++;
                 }
                 if (Dn > 0.0) sh.D = Dn;
+                sh.have_q = cache_ok;
             }
             __syncthreads();
         }
@@ -362,14 +443,12 @@ accept_walk_kernel(const WalkArgs args)
         const int cur = sh.cur;
         const float *x = lg + (size_t)cur * V;
         const float *q = dp + (size_t)cur * V;
-        if (!sh.exact) {
-            Sweep s = sweep_chunk<MODE_SUM>(sh, x, q, lo, hi, vec, 0.0, -1, false, 0, 0, 0, nullptr);
-            reduce_exchange(s.a, 0.0);
-            if (tid == 0) { sh.S = sh.tot[0]; sh.exact = 1; }
-            __syncthreads();
-        }
         const double c = sh.c;
-        Sweep s = sweep_chunk<MODE_CDF>(sh, x, q, lo, hi, vec, c, -1, false, 0, 0, 0, nullptr);
+        const bool have_e = sh.have_e != 0, have_q = sh.have_q != 0;
+        // with nothing rejected at this node (c == 0) the weights are the e_j themselves and the
+        // denominator cancels, so no separate exact-sum sweep is needed
+        Sweep s = sweep_chunk<MODE_CDF>(sh, x, q, se, sq, cta_lo, lo, hi, vec, cache_ok, have_e, have_q, c, -1,
+                                        false, 0, 0, 0, nullptr);
         // block-wide inclusive scan of the per-thread sums (index order)
         double incl = s.a;
         const int lane = tid & 31, wid = tid >> 5;
@@ -378,7 +457,7 @@ accept_walk_kernel(const WalkArgs args)
             const double t = __shfl_up_sync(0xffffffffu, incl, off);
             if (lane >= off) incl += t;
         }
-        double prev_incl = __shfl_up_sync(0xffffffffu, incl, 1);
+        const double prev_incl = __shfl_up_sync(0xffffffffu, incl, 1);
         if (lane == 31) sh.warp_a[wid] = incl;
         __syncthreads();
         if (tid == 0) {
@@ -399,7 +478,7 @@ accept_walk_kernel(const WalkArgs args)
             if (r == rank) base = Z;
             Z = Z + sh.cta_total[r];
         }
-        const double target = (double)un[N] * Z;
+        const double target = (double)sh.ubonus * Z;
         int owner = -1;
         {
             double cum = 0.0;
@@ -416,7 +495,8 @@ accept_walk_kernel(const WalkArgs args)
             __syncthreads();
             if (tid == sh.sel) {
                 int found = -1;
-                sweep_chunk<MODE_CDF>(sh, x, q, lo, hi, vec, c, -1, true, base, E, target, &found);
+                sweep_chunk<MODE_CDF>(sh, x, q, se, sq, cta_lo, lo, hi, vec, false, cache_ok, cache_ok && (c != 0.0),
+                                      c, -1, true, base, E, target, &found);
                 if (found < 0) found = min(lo, V - 1);
                 args.bonus[b] = found;
             }
@@ -434,29 +514,33 @@ accept_walk_kernel(const WalkArgs args)
 
 cudaError_t fspad_launch_accept_walk(fspad_ctx *ctx, const float *logits, const float *draft,
                                      const int *tokens, const int *parent, const float *temperature,
-                                     const float *uniforms, int N, int B, int V, int *path,
-                                     int *n_acc, int *bonus, cudaStream_t st)
+                                     const float *uniforms, const FspadStatsGeom &geom, int N, int B, int V,
+                                     int *path, int *n_acc, int *bonus, cudaStream_t st)
 {
     if (B == 0) return cudaSuccess;
     WalkArgs a;
     a.logits = logits; a.draft = draft; a.temperature = temperature; a.uniforms = uniforms;
     a.tokens = tokens; a.parent = parent;
-    a.row_max = ctx->row_max; a.row_sum = ctx->row_sum; a.row_arg = ctx->row_arg;
-    a.N = N; a.V = V; a.path_stride = ctx->cfg.max_nodes;
+    a.parts = ctx->st_part; a.geom = geom;
+    a.N = N; a.V = V; a.path_stride = ctx->cfg.max_nodes; a.cache_ok = 0;
     a.path = path; a.n_acc = n_acc; a.bonus = bonus; a.status = ctx->d_status;
 
     const bool sampling = draft != nullptr && uniforms != nullptr;
-    int cluster = 1, threads = 64;
+    int cluster = 1, threads = 256;
+    size_t smem = 0;
     if (sampling) {
         threads = kWalkThreads;
         if (ctx->walk_cluster == 0) {
-            // largest cluster the device can co-schedule for this kernel: 16 (opt-in), else 8
+            // once per context: raise the dynamic shared-memory limit and find the largest cluster
+            // the device can co-schedule for this kernel: 16 (opt-in), else 8
             ctx->walk_cluster = 8;
+            cudaFuncSetAttribute(accept_walk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
             if (cudaFuncSetAttribute(accept_walk_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) ==
                 cudaSuccess) {
                 cudaLaunchConfig_t probe = {};
                 probe.gridDim = dim3(kMaxCluster);
                 probe.blockDim = dim3(kWalkThreads);
+                probe.dynamicSmemBytes = kSmemBudget;
                 cudaLaunchAttribute at[1];
                 at[0].id = cudaLaunchAttributeClusterDimension;
                 at[0].val.clusterDim.x = kMaxCluster; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
@@ -469,12 +553,15 @@ cudaError_t fspad_launch_accept_walk(fspad_ctx *ctx, const float *logits, const 
         }
         cluster = ctx->walk_cluster;
         // small vocabularies do not need the whole cluster
-        while (cluster > 1 && (V + cluster - 1) / cluster < 1024) cluster >>= 1;
+        while (cluster > 1 && (V + cluster - 1) / cluster < 2048) cluster >>= 1;
+        const size_t per_cta = (size_t)((((V + cluster - 1) / cluster) + 3) & ~3);
+        const size_t need = per_cta * (sizeof(double) + sizeof(float));
+        if (need <= (size_t)kSmemBudget) { smem = need; a.cache_ok = 1; }
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(B * cluster));
     cfg.blockDim = dim3(threads);
-    cfg.dynamicSmemBytes = 0;
+    cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;

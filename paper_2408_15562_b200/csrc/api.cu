@@ -88,22 +88,17 @@ int fspad_create(const fspad_config *cfg, fspad_ctx **out)
         }
     ctx->attn_max_splits = max_splits;
     const size_t rows = B * Nmax;
-    ctx->stats_max_slices = 64;
+    ctx->stats_slots = 64;
 
     bool ok = dev_alloc(&ctx->d_status, 1);
     ok = ok && dev_alloc(&ctx->part_o, part_rows * FSPAD_HEAD_DIM);
     ok = ok && dev_alloc(&ctx->part_ml, part_rows * 2);
-    ok = ok && dev_alloc(&ctx->st_pmax, rows * ctx->stats_max_slices);
-    ok = ok && dev_alloc(&ctx->st_psum, rows * ctx->stats_max_slices);
-    ok = ok && dev_alloc(&ctx->st_parg, rows * ctx->stats_max_slices);
-    ok = ok && dev_alloc(&ctx->st_counter, rows);
+    ok = ok && dev_alloc(&ctx->st_part, rows * ctx->stats_slots);
     ok = ok && dev_alloc(&ctx->row_max, rows);
     ok = ok && dev_alloc(&ctx->row_sum, rows);
     ok = ok && dev_alloc(&ctx->row_arg, rows);
     if (ok) {
-        ok = cudaMemset(ctx->d_status, 0, sizeof(int)) == cudaSuccess &&
-             cudaMemset(ctx->st_counter, 0, rows * sizeof(unsigned)) == cudaSuccess &&
-             cudaDeviceSynchronize() == cudaSuccess;
+        ok = cudaMemset(ctx->d_status, 0, sizeof(int)) == cudaSuccess && cudaDeviceSynchronize() == cudaSuccess;
     }
     if (!ok) {
         fspad_destroy(ctx);
@@ -117,8 +112,7 @@ void fspad_destroy(fspad_ctx *ctx)
 {
     if (!ctx) return;
     cudaDeviceSynchronize();
-    void *ptrs[] = {ctx->d_status, ctx->part_o, ctx->part_ml, ctx->st_pmax, ctx->st_psum, ctx->st_parg,
-                    ctx->st_counter, ctx->row_max, ctx->row_sum, ctx->row_arg, ctx->h_q, ctx->h_tk,
+    void *ptrs[] = {ctx->d_status, ctx->part_o, ctx->part_ml, ctx->st_part, ctx->row_max, ctx->row_sum, ctx->row_arg, ctx->h_q, ctx->h_tk,
                     ctx->h_tv, ctx->h_out, ctx->h_parent, ctx->h_prefix, ctx->h_tokens, ctx->h_path,
                     ctx->h_nacc, ctx->h_bonus, ctx->h_newlen, ctx->h_logits, ctx->h_draft, ctx->h_temp,
                     ctx->h_unif};
@@ -192,11 +186,12 @@ int fspad_tree_accept(fspad_ctx *ctx, const float *target_logits, const float *d
     if (misaligned(target_logits) || misaligned(draft_probs)) return FSPAD_ERR_ALIGN;
     if (batch == 0) return FSPAD_OK;
     cudaStream_t st = fspad_stream(stream);
-    cudaError_t e = fspad_launch_accept_stats(ctx, target_logits, temperature, batch * n_nodes, n_nodes,
-                                              ctx->cfg.vocab, ctx->row_max, ctx->row_sum, ctx->row_arg, st);
+    FspadStatsGeom geom;
+    cudaError_t e = fspad_launch_stats_partials(ctx, target_logits, temperature, batch * n_nodes, n_nodes,
+                                                ctx->cfg.vocab, &geom, st);
     if (e != cudaSuccess) return FSPAD_ERR_CUDA;
     e = fspad_launch_accept_walk(ctx, target_logits, draft_probs, draft_tokens, parent, temperature,
-                                 uniforms, n_nodes, batch, ctx->cfg.vocab, accepted_path, n_accepted,
+                                 uniforms, geom, n_nodes, batch, ctx->cfg.vocab, accepted_path, n_accepted,
                                  bonus_token, st);
     return e == cudaSuccess ? FSPAD_OK : FSPAD_ERR_CUDA;
 }

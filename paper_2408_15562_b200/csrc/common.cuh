@@ -26,11 +26,8 @@ struct fspad_ctx {
     float *part_ml;           // [batch][Hkv][splits][M][2]  (running max in log2 units, sum)
 
     // per-node vocabulary scan
-    int stats_max_slices;
-    float *st_pmax;           // [rows][slices]
-    double *st_psum;
-    int *st_parg;
-    unsigned *st_counter;     // [rows], zero between calls
+    int stats_slots;          // partial slots per row in st_part
+    struct FspadStatsPart *st_part;   // [rows][stats_slots]
     float *row_max;           // [rows]
     double *row_sum;
     int *row_arg;
@@ -41,6 +38,86 @@ struct fspad_ctx {
     int *h_parent, *h_prefix, *h_tokens, *h_path, *h_nacc, *h_bonus, *h_newlen;
     float *h_logits, *h_draft, *h_temp, *h_unif;
 };
+
+// One CTA's contribution to a row of the vocabulary scan.
+struct FspadStatsPart {
+    float m;   // maximum over the CTA's part of the row
+    float s;   // sum of exp2((x - m) * log2(e) / T) over that part
+    int a;     // lowest index attaining m
+    int pad;
+};
+
+// How the flat [rows x V] logits array is cut into equal per-CTA ranges.
+struct FspadStatsGeom {
+    int unit;          // floats per load unit: 4 (128-bit loads) or 1
+    int upr;           // units per row
+    int n_cta;         // CTAs in the grid
+    int slots;         // partial slots per row (capacity)
+    long long chunk;   // units per CTA
+    long long total;   // rows * upr
+};
+
+static inline FspadStatsGeom fspad_stats_geom(int sm_count, int rows, int V, bool vec, int slots)
+{
+    FspadStatsGeom g;
+    g.unit = vec ? 4 : 1;
+    g.upr = V / g.unit;
+    g.slots = slots;
+    g.total = (long long)rows * g.upr;
+    long long n = (long long)sm_count * 4;                 // four 256-thread CTAs per SM, one wave
+    const long long by_size = (g.total + 255) / 256;       // at least one unit per thread
+    if (n > by_size) n = by_size;
+    if (n < 1) n = 1;
+    g.chunk = (g.total + n - 1) / n;
+    // a row may be shared by at most `slots` CTAs
+    const long long min_chunk = (g.upr + (slots - 2) - 1) / (slots - 2);
+    if (g.chunk < min_chunk) g.chunk = min_chunk;
+    g.n_cta = (int)((g.total + g.chunk - 1) / g.chunk);
+    return g;
+}
+
+#ifdef __CUDACC__
+// Merge the per-CTA partials of one row (warp-collective: all 32 lanes call it and all get
+// the result): maximum, its lowest index, and the sum of exponentials rescaled to that
+// maximum (k = log2(e)/T).  Every lane fetches up to two partial slots, so the loads of a
+// row are in flight together instead of one after another.
+__device__ __forceinline__ void fspad_stats_merge_warp(const FspadStatsPart *__restrict__ parts,
+                                                       const FspadStatsGeom &g, int row, float k, int lane,
+                                                       float &M, double &S, int &A)
+{
+    const long long r0 = (long long)row * g.upr;
+    const int first = (int)(r0 / g.chunk), last = (int)((r0 + g.upr - 1) / g.chunk);
+    const int cnt = last - first + 1;                       // <= g.slots <= 64
+    const FspadStatsPart *p = parts + (size_t)row * g.slots;
+    float m0 = -INFINITY, m1 = -INFINITY, s0 = 0.f, s1 = 0.f;
+    int a0 = 0x7fffffff, a1 = 0x7fffffff;
+    if (lane < cnt) {
+        const int4 v = __ldcg(reinterpret_cast<const int4 *>(p + lane));
+        m0 = __int_as_float(v.x); s0 = __int_as_float(v.y); a0 = v.z;
+    }
+    if (lane + 32 < cnt) {
+        const int4 v = __ldcg(reinterpret_cast<const int4 *>(p + lane + 32));
+        m1 = __int_as_float(v.x); s1 = __int_as_float(v.y); a1 = v.z;
+    }
+    float m = m0;
+    int a = a0;
+    if (m1 > m || (m1 == m && a1 < a)) { m = m1; a = a1; }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        const float om = __shfl_xor_sync(0xffffffffu, m, off);
+        const int oa = __shfl_xor_sync(0xffffffffu, a, off);
+        if (om > m || (om == m && oa < a)) { m = om; a = oa; }
+    }
+    double s = 0.0;
+    if (m0 != -INFINITY) s += (double)s0 * (double)exp2f((m0 - m) * k);
+    if (m1 != -INFINITY) s += (double)s1 * (double)exp2f((m1 - m) * k);
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
+    M = m;
+    S = s;
+    A = (a == 0x7fffffff) ? 0 : a;
+}
+#endif
 
 static inline cudaStream_t fspad_stream(void *s) { return reinterpret_cast<cudaStream_t>(s); }
 
@@ -56,8 +133,11 @@ cudaError_t fspad_launch_accept_stats(fspad_ctx *ctx, const float *logits, const
                                       double *row_sum, int *row_arg, cudaStream_t st);
 cudaError_t fspad_launch_accept_walk(fspad_ctx *ctx, const float *logits, const float *draft,
                                      const int *tokens, const int *parent, const float *temperature,
-                                     const float *uniforms, int N, int B, int V, int *path,
-                                     int *n_acc, int *bonus, cudaStream_t st);
+                                     const float *uniforms, const FspadStatsGeom &geom, int N, int B, int V,
+                                     int *path, int *n_acc, int *bonus, cudaStream_t st);
+cudaError_t fspad_launch_stats_partials(fspad_ctx *ctx, const float *logits, const float *temperature,
+                                        int rows, int rows_per_seq, int V, FspadStatsGeom *geom,
+                                        cudaStream_t st);
 cudaError_t fspad_launch_kv_compact(fspad_ctx *ctx, fspad_bf16 *cache, const int *path,
                                     const int *n_acc, const int *prefix_len, int B, int *new_len,
                                     cudaStream_t st);
@@ -69,4 +149,3 @@ cudaError_t fspad_launch_tree_scatter(fspad_ctx *ctx, fspad_bf16 *cache, const f
                                       const fspad_bf16 *tv, const int *prefix_len, int N, int B,
                                       cudaStream_t st);
 int fspad_attn_splits(const fspad_ctx *ctx, int N, int B);
-int fspad_stats_slices(const fspad_ctx *ctx, int rows, int V);
