@@ -46,6 +46,26 @@ constexpr int kSmemBudget = 200 * 1024;   // dynamic shared memory for the per-n
 constexpr double kAmbiguous = 1e-4;
 constexpr float kLog2eF = 1.4426950408889634f;
 
+// 2^(i/64), i = 0..63, correctly rounded
+__constant__ double kExp2Tbl[64] = {
+    1.0, 1.0108892860517005, 1.0218971486541166, 1.0330248790212284,
+    1.0442737824274138, 1.0556451783605572, 1.0671404006768237, 1.0787607977571199,
+    1.0905077326652577, 1.102382583307841, 1.1143867425958924, 1.1265216186082418,
+    1.1387886347566916, 1.1511892299529827, 1.1637248587775775, 1.1763969916502812,
+    1.189207115002721, 1.202156731452703, 1.215247359980469, 1.22848053610687,
+    1.241857812073484, 1.255380757024691, 1.2690509571917332, 1.2828700160787783,
+    1.2968395546510096, 1.3109612115247644, 1.3252366431597413, 1.339667524053303,
+    1.3542555469368927, 1.3690024229745905, 1.383909881963832, 1.3989796725383112,
+    1.4142135623730951, 1.42961333839197, 1.4451808069770467, 1.460917794180647,
+    1.4768261459394993, 1.4929077282912648, 1.5091644275934228, 1.5255981507445384,
+    1.5422108254079407, 1.559004400237837, 1.5759808451078865, 1.593142151342267,
+    1.6104903319492543, 1.6280274218573478, 1.645755478153965, 1.6636765803267364,
+    1.681792830507429, 1.7001063537185235, 1.718619298122478, 1.7373338352737062,
+    1.7562521603732995, 1.7753764925265212, 1.7947090750031072, 1.8142521755003989,
+    1.8340080864093424, 1.8539791250833855, 1.8741676341103, 1.8945759815869656,
+    1.9152065613971474, 1.9360617934922943, 1.9571441241754002, 1.978456026387951,
+};
+
 struct WalkArgs {
     const float *logits, *draft, *temperature, *uniforms;
     const int *tokens, *parent;
@@ -61,7 +81,8 @@ struct Shared {
     int tok[FSPAD_MAX_NODES];
     int path[FSPAD_MAX_NODES];
     // state of the current node (written by thread 0, read by all after a barrier)
-    double S, c, U, D, m, invT;
+    double S, invS, c, U, D, m, invT;
+    unsigned long long child_mask[FSPAD_MAX_NODES];   // bit c set in child_mask[i] iff parent[c] == i
     int exact, nrem, decision, xnew, ridx, next, len, cur, have_e, have_q, sel;
     double cprime, ex, qx;
     int rem_tok[FSPAD_MAX_NODES];
@@ -130,14 +151,14 @@ struct Sweep {
 // token where base + run exceeds target (else the last positive-weight token).
 template <int MODE>
 __device__ Sweep sweep_chunk(const Shared &sh, const float *__restrict__ x, const float *__restrict__ q,
-                             double *__restrict__ se, float *__restrict__ sq, int cta_lo, int lo, int hi,
+                             double *__restrict__ se, float *__restrict__ sq, int tid, int nthr, int lo, int hi,
                              bool vec, bool cache_ok, bool have_e, bool have_q, double c, int xnew,
                              bool locate, double base, double run0, double target, int *found)
 {
     const double m = sh.m, invT = sh.invT;
     const int nrem = sh.nrem;
     // bonus draw with nothing rejected at this node: the weights are the e_j themselves
-    const double invS = (MODE == MODE_CDF && c == 0.0 && nrem == 0) ? 1.0 : 1.0 / sh.S;
+    const double invS = (MODE == MODE_CDF && c == 0.0 && nrem == 0) ? 1.0 : sh.invS;
     const bool need_q = (MODE == MODE_RESID) || (MODE == MODE_CDF && c != 0.0);
     bool special = false;
     if (MODE != MODE_EXP) {
@@ -152,7 +173,7 @@ __device__ Sweep sweep_chunk(const Shared &sh, const float *__restrict__ x, cons
         float qv[4] = {0.f, 0.f, 0.f, 0.f};
         if (have_e) {
 #pragma unroll
-            for (int t = 0; t < 4; ++t) ev[t] = (t < n) ? se[j - cta_lo + t] : 0.0;
+            for (int t = 0; t < 4; ++t) ev[t] = (t < n) ? se[(j - lo + t) * nthr + tid] : 0.0;
         } else {
             float xv[4];
             if (vec && n == 4) {
@@ -165,13 +186,13 @@ __device__ Sweep sweep_chunk(const Shared &sh, const float *__restrict__ x, cons
 #pragma unroll
             for (int t = 0; t < 4; ++t) {
                 ev[t] = exp_neg(((double)xv[t] - m) * invT, sh.exp_tbl);
-                if (cache_ok && t < n) se[j - cta_lo + t] = ev[t];
+                if (cache_ok && t < n) se[(j - lo + t) * nthr + tid] = ev[t];
             }
         }
         if (need_q) {
             if (have_q) {
 #pragma unroll
-                for (int t = 0; t < 4; ++t) qv[t] = (t < n) ? sq[j - cta_lo + t] : 0.f;
+                for (int t = 0; t < 4; ++t) qv[t] = (t < n) ? sq[(j - lo + t) * nthr + tid] : 0.f;
             } else {
                 if (vec && n == 4) {
                     const float4 u4 = __ldg(reinterpret_cast<const float4 *>(q + j));
@@ -182,7 +203,7 @@ __device__ Sweep sweep_chunk(const Shared &sh, const float *__restrict__ x, cons
                 }
                 if (cache_ok) {
 #pragma unroll
-                    for (int t = 0; t < 4; ++t) if (t < n) sq[j - cta_lo + t] = qv[t];
+                    for (int t = 0; t < 4; ++t) if (t < n) sq[(j - lo + t) * nthr + tid] = qv[t];
                 }
             }
         }
@@ -228,26 +249,8 @@ accept_walk_kernel(const WalkArgs args)
     __shared__ Shared sh;
     extern __shared__ __align__(16) unsigned char dyn_smem[];
 
-    const int *par_g = args.parent + (size_t)b * N;
-    const int *tok_g = args.tokens + (size_t)b * N;
-    for (int i = tid; i < N; i += nthr) {
-        int p = par_g[i], t = tok_g[i];
-        if (i == 0) {
-            if (p != -1) fspad_report(args.status, FSPAD_ERR_BAD_TREE);
-            p = -1;
-        } else if (p < 0 || p >= i) {
-            fspad_report(args.status, FSPAD_ERR_BAD_TREE);
-            p = 0;
-        }
-        if (t < 0 || t >= V) {
-            fspad_report(args.status, FSPAD_ERR_RANGE);
-            t = 0;
-        }
-        sh.parent[i] = p;
-        sh.tok[i] = t;
-    }
-    if (tid < 64) sh.exp_tbl[tid] = exp2((double)tid * (1.0 / 64.0));
     float Tf = args.temperature[b];
+    if (tid < 64) { sh.exp_tbl[tid] = kExp2Tbl[tid]; sh.child_mask[tid] = 0ull; }
     if (!(Tf >= 0.0f)) {
         if (tid == 0 && rank == 0) fspad_report(args.status, FSPAD_ERR_RANGE);
         Tf = 0.0f;
@@ -261,24 +264,43 @@ accept_walk_kernel(const WalkArgs args)
     const float *un = args.uniforms ? args.uniforms + (size_t)b * (N + 1) : nullptr;
     int *out_path = args.path + (size_t)b * args.path_stride;
     const float kT = kLog2eF / (Tf > 0.0f ? Tf : 1.0f);
-    {
-        // every row's (max, sum, argmax): one warp per row, all partial slots fetched at once
-        const int lane = tid & 31, nwarps = nthr >> 5;
-        for (int row = tid >> 5; row < N; row += nwarps) {
-            float M; double S; int A;
-            fspad_stats_merge_warp(args.parts, args.geom, b * N + row, kT, lane, M, S, A);
-            if (lane == 0) { sh.rowM[row] = M; sh.rowS[row] = S; sh.rowA[row] = A; }
+
+    // Gathered once, in parallel: thread c owns node c (tree arrays, the child bit of its parent
+    // and the three scalars its accept test needs); half-warps merge the scan partials of the rows.
+    if (tid < N) {
+        int p = args.parent[(size_t)b * N + tid], t = args.tokens[(size_t)b * N + tid];
+        if (tid == 0) {
+            if (p != -1) fspad_report(args.status, FSPAD_ERR_BAD_TREE);
+            p = -1;
+        } else if (p < 0 || p >= tid) {
+            fspad_report(args.status, FSPAD_ERR_BAD_TREE);
+            p = 0;
         }
-        if (sampling) {
-            for (int c = tid; c < N; c += nthr) {
-                if (c >= 1) {
-                    const size_t at = (size_t)sh.parent[c] * V + sh.tok[c];
-                    sh.cx[c] = lg[at];
-                    sh.cq[c] = dp[at];
-                    sh.cu[c] = un[c];
-                }
+        if (t < 0 || t >= V) {
+            fspad_report(args.status, FSPAD_ERR_RANGE);
+            t = 0;
+        }
+        sh.parent[tid] = p;
+        sh.tok[tid] = t;
+        if (tid >= 1) {
+            atomicOr(&sh.child_mask[p], 1ull << tid);
+            if (sampling) {
+                const size_t at = (size_t)p * V + t;
+                sh.cx[tid] = lg[at];
+                sh.cq[tid] = dp[at];
+                sh.cu[tid] = un[tid];
             }
-            if (tid == 0) sh.ubonus = un[N];
+        } else if (sampling) {
+            sh.ubonus = un[N];
+        }
+    }
+    {
+        const int lane16 = tid & 15, n_half = nthr >> 4;
+        for (int r0 = 0; r0 < N; r0 += n_half) {                 // whole warps iterate together
+            const int row = r0 + (tid >> 4);
+            float M; double S; int A;
+            fspad_stats_merge_half(args.parts, args.geom, b * N + row, row < N, kT, lane16, M, S, A);
+            if (lane16 == 0 && row < N) { sh.rowM[row] = M; sh.rowS[row] = S; sh.rowA[row] = A; }
         }
     }
     __syncthreads();
@@ -291,8 +313,10 @@ accept_walk_kernel(const WalkArgs args)
             for (;;) {
                 const int want = sh.rowA[cur];
                 int next = -1;
-                for (int c = cur + 1; c < N; ++c)
-                    if (sh.parent[c] == cur && sh.tok[c] == want) { next = c; break; }
+                for (unsigned long long rem = sh.child_mask[cur]; rem; rem &= rem - 1) {
+                    const int c = __ffsll((long long)rem) - 1;
+                    if (sh.tok[c] == want) { next = c; break; }
+                }
                 if (next < 0) { args.bonus[b] = want; break; }
                 sh.path[len++] = next;
                 cur = next;
@@ -316,31 +340,37 @@ accept_walk_kernel(const WalkArgs args)
     const int lo = min(cta_hi, cta_lo + tid * per_thr), hi = min(cta_hi, lo + per_thr);
     const bool cache_ok = args.cache_ok != 0;
     double *se = reinterpret_cast<double *>(dyn_smem);
-    float *sq = reinterpret_cast<float *>(dyn_smem + (size_t)per_cta * sizeof(double));
+    // the cache is laid out [k][thread] (k-th token of each thread's chunk): conflict-free
+    float *sq = reinterpret_cast<float *>(dyn_smem + (size_t)per_thr * nthr * sizeof(double));
     int parity = 0;
 
-    // cluster-wide reduction of (a, b); result in sh.tot[] (read by thread 0 only)
+    // cluster-wide reduction of (a, b); result in sh.tot[] (read by thread 0 only).  Every level
+    // is a warp butterfly over values fetched in parallel (no serial chain of shared-memory or
+    // peer reads), and every CTA performs the same operations on the same values.
     auto reduce_exchange = [&](double a, double bb) {
+        const int lane = tid & 31, wid = tid >> 5, nwarps = nthr >> 5;
         a = warp_sum(a);
         bb = warp_sum(bb);
-        if ((tid & 31) == 0) { sh.warp_a[tid >> 5] = a; sh.warp_b[tid >> 5] = bb; }
+        if (lane == 0) { sh.warp_a[wid] = a; sh.warp_b[wid] = bb; }
         __syncthreads();
-        if (tid == 0) {
-            double sa = 0.0, sb = 0.0;
-            for (int w = 0; w < nthr / 32; ++w) { sa += sh.warp_a[w]; sb += sh.warp_b[w]; }
-            sh.slot[parity][0] = sa;
-            sh.slot[parity][1] = sb;
+        if (wid == 0) {
+            double sa = (lane < nwarps) ? sh.warp_a[lane] : 0.0;
+            double sb = (lane < nwarps) ? sh.warp_b[lane] : 0.0;
+            sa = warp_sum(sa);
+            sb = warp_sum(sb);
+            if (lane == 0) { sh.slot[parity][0] = sa; sh.slot[parity][1] = sb; }
         }
         cluster.sync();
-        if (tid == 0) {
+        if (wid == 0) {
             double ta = 0.0, tb = 0.0;
-            for (int r = 0; r < C; ++r) {
-                const double *peer = cluster.map_shared_rank(&sh.slot[parity][0], r);
-                ta += peer[0];
-                tb += peer[1];
+            if (lane < C) {
+                const double *peer = cluster.map_shared_rank(&sh.slot[parity][0], lane);
+                ta = peer[0];
+                tb = peer[1];
             }
-            sh.tot[0] = ta;
-            sh.tot[1] = tb;
+            ta = warp_sum(ta);
+            tb = warp_sum(tb);
+            if (lane == 0) { sh.tot[0] = ta; sh.tot[1] = tb; }
         }
         __syncthreads();
         parity ^= 1;
@@ -356,6 +386,7 @@ accept_walk_kernel(const WalkArgs args)
         if (tid == 0) {
             sh.m = (double)sh.rowM[cur];
             sh.S = sh.rowS[cur];
+            sh.invS = 1.0 / sh.S;
             sh.invT = 1.0 / (double)Tf;
             sh.exact = 0; sh.have_e = 0; sh.have_q = 0;
             sh.c = 0.0; sh.U = 1.0; sh.D = 1.0;
@@ -364,8 +395,8 @@ accept_walk_kernel(const WalkArgs args)
         }
         __syncthreads();
 
-        for (int ch = cur + 1; ch < N; ++ch) {
-            if (sh.parent[ch] != cur) continue;          // uniform: shared data
+        for (unsigned long long rem = sh.child_mask[cur]; rem; rem &= rem - 1) {   // uniform: shared data
+            const int ch = __ffsll((long long)rem) - 1;
             const int xt = sh.tok[ch];
             for (int attempt = 0; attempt < 2; ++attempt) {
                 if (tid == 0) {
@@ -376,7 +407,7 @@ accept_walk_kernel(const WalkArgs args)
                     for (int k = 0; k < sh.nrem; ++k) if (sh.rem_tok[k] == xt) ridx = k;
                     double qk, pk;
                     if (ridx >= 0) { qk = 0.0; pk = sh.rem_frozen[ridx] / sh.U; }
-                    else { qk = qx / sh.D; pk = weight(ex, qx, 1.0 / sh.S, sh.c) / sh.U; }
+                    else { qk = qx / sh.D; pk = weight(ex, qx, sh.invS, sh.c) / sh.U; }
                     const double lhs = r * qk;
                     int dec = (lhs < pk) ? 1 : 0;
                     if (!sh.exact) {
@@ -390,10 +421,10 @@ accept_walk_kernel(const WalkArgs args)
                 __syncthreads();
                 if (sh.decision != 2) break;
                 // exact softmax denominator of this node (parks e_j in shared memory)
-                Sweep s = sweep_chunk<MODE_EXP>(sh, x, q, se, sq, cta_lo, lo, hi, vec, cache_ok, false, false, 0.0,
+                Sweep s = sweep_chunk<MODE_EXP>(sh, x, q, se, sq, tid, nthr, lo, hi, vec, cache_ok, false, false, 0.0,
                                                 -1, false, 0, 0, 0, nullptr);
                 reduce_exchange(s.a, 0.0);
-                if (tid == 0) { sh.S = sh.tot[0]; sh.exact = 1; sh.have_e = cache_ok; }
+                if (tid == 0) { sh.S = sh.tot[0]; sh.invS = 1.0 / sh.S; sh.exact = 1; sh.have_e = cache_ok; }
                 __syncthreads();
             }
             if (sh.decision == 1) {
@@ -405,7 +436,7 @@ accept_walk_kernel(const WalkArgs args)
             if (tid == 0) sh.cprime = sh.c + sh.U / sh.D;
             __syncthreads();
             {
-                Sweep s = sweep_chunk<MODE_RESID>(sh, x, q, se, sq, cta_lo, lo, hi, vec, cache_ok, sh.have_e != 0,
+                Sweep s = sweep_chunk<MODE_RESID>(sh, x, q, se, sq, tid, nthr, lo, hi, vec, cache_ok, sh.have_e != 0,
                                                   sh.have_q != 0, sh.cprime, xt, false, 0, 0, 0, nullptr);
                 reduce_exchange(s.a, s.b);
             }
@@ -413,11 +444,11 @@ accept_walk_kernel(const WalkArgs args)
                 const double W = sh.tot[0], Dn = sh.tot[1];
                 double frozen;
                 if (W > 0.0) {
-                    frozen = weight(sh.ex, sh.qx, 1.0 / sh.S, sh.cprime);
+                    frozen = weight(sh.ex, sh.qx, sh.invS, sh.cprime);
                     sh.c = sh.cprime;
                     sh.U = W;
                 } else {
-                    frozen = weight(sh.ex, sh.qx, 1.0 / sh.S, sh.c);   // residual vanished: p is kept
+                    frozen = weight(sh.ex, sh.qx, sh.invS, sh.c);   // residual vanished: p is kept
                 }
                 if (sh.ridx < 0 && sh.nrem < FSPAD_MAX_NODES) {
                     sh.rem_tok[sh.nrem] = xt;
@@ -447,7 +478,7 @@ accept_walk_kernel(const WalkArgs args)
         const bool have_e = sh.have_e != 0, have_q = sh.have_q != 0;
         // with nothing rejected at this node (c == 0) the weights are the e_j themselves and the
         // denominator cancels, so no separate exact-sum sweep is needed
-        Sweep s = sweep_chunk<MODE_CDF>(sh, x, q, se, sq, cta_lo, lo, hi, vec, cache_ok, have_e, have_q, c, -1,
+        Sweep s = sweep_chunk<MODE_CDF>(sh, x, q, se, sq, tid, nthr, lo, hi, vec, cache_ok, have_e, have_q, c, -1,
                                         false, 0, 0, 0, nullptr);
         // block-wide inclusive scan of the per-thread sums (index order)
         double incl = s.a;
@@ -460,18 +491,26 @@ accept_walk_kernel(const WalkArgs args)
         const double prev_incl = __shfl_up_sync(0xffffffffu, incl, 1);
         if (lane == 31) sh.warp_a[wid] = incl;
         __syncthreads();
-        if (tid == 0) {
-            double off = 0.0;
-            for (int w = 0; w < nthr / 32; ++w) { sh.warp_off[w] = off; off = off + sh.warp_a[w]; }
-            sh.slot[parity][0] = off;                     // CTA total = inclusive prefix of the last thread
+        if (wid == 0) {
+            // exclusive scan of the warp totals; the last inclusive value is the CTA total
+            const int nwarps = nthr >> 5;
+            const double v = (lane < nwarps) ? sh.warp_a[lane] : 0.0;
+            double sc = v;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const double t = __shfl_up_sync(0xffffffffu, sc, off);
+                if (lane >= off) sc += t;
+            }
+            const double excl = __shfl_up_sync(0xffffffffu, sc, 1);
+            if (lane < nwarps) sh.warp_off[lane] = (lane == 0) ? 0.0 : excl;
+            if (lane == nwarps - 1) sh.slot[parity][0] = sc;
         }
         __syncthreads();
         const double woff = sh.warp_off[wid];
         const double P = woff + incl;
         const double E = (lane == 0) ? woff : woff + prev_incl;
         cluster.sync();
-        if (tid == 0)
-            for (int r = 0; r < C; ++r) sh.cta_total[r] = *cluster.map_shared_rank(&sh.slot[parity][0], r);
+        if (tid < C) sh.cta_total[tid] = *cluster.map_shared_rank(&sh.slot[parity][0], tid);
         __syncthreads();
         double Z = 0.0, base = 0.0;
         for (int r = 0; r < C; ++r) {
@@ -493,9 +532,13 @@ accept_walk_kernel(const WalkArgs args)
             __syncthreads();
             if (base + P > target) atomicMin(&sh.sel, tid);
             __syncthreads();
+            // rounding of the two-level prefix can leave no thread above the target although the
+            // CTA total is: the last non-empty chunk then takes the draw
+            if (tid == 0 && sh.sel == 0x7fffffff) sh.sel = max(0, (cta_hi - cta_lo - 1) / per_thr);
+            __syncthreads();
             if (tid == sh.sel) {
                 int found = -1;
-                sweep_chunk<MODE_CDF>(sh, x, q, se, sq, cta_lo, lo, hi, vec, false, cache_ok, cache_ok && (c != 0.0),
+                sweep_chunk<MODE_CDF>(sh, x, q, se, sq, tid, nthr, lo, hi, vec, false, cache_ok, cache_ok && (c != 0.0),
                                       c, -1, true, base, E, target, &found);
                 if (found < 0) found = min(lo, V - 1);
                 args.bonus[b] = found;
@@ -555,7 +598,8 @@ cudaError_t fspad_launch_accept_walk(fspad_ctx *ctx, const float *logits, const 
         // small vocabularies do not need the whole cluster
         while (cluster > 1 && (V + cluster - 1) / cluster < 2048) cluster >>= 1;
         const size_t per_cta = (size_t)((((V + cluster - 1) / cluster) + 3) & ~3);
-        const size_t need = per_cta * (sizeof(double) + sizeof(float));
+        const size_t per_thr = ((per_cta + kWalkThreads - 1) / kWalkThreads + 3) & ~(size_t)3;
+        const size_t need = per_thr * kWalkThreads * (sizeof(double) + sizeof(float));
         if (need <= (size_t)kSmemBudget) { smem = need; a.cache_ok = 1; }
     }
     cudaLaunchConfig_t cfg = {};

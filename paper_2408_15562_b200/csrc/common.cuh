@@ -117,6 +117,54 @@ __device__ __forceinline__ void fspad_stats_merge_warp(const FspadStatsPart *__r
     S = s;
     A = (a == 0x7fffffff) ? 0 : a;
 }
+
+// The same merge by a half-warp (16 lanes, up to four slots per lane), so that one warp
+// serves two rows at once.  Both halves of the warp must call it together; `valid` is false
+// for a half that has no row (it only takes part in the shuffles).
+__device__ __forceinline__ void fspad_stats_merge_half(const FspadStatsPart *__restrict__ parts,
+                                                       const FspadStatsGeom &g, int row, bool valid, float k,
+                                                       int lane16, float &M, double &S, int &A)
+{
+    int cnt = 0;
+    const FspadStatsPart *p = parts;
+    if (valid) {
+        const long long r0 = (long long)row * g.upr;
+        const int first = (int)(r0 / g.chunk), last = (int)((r0 + g.upr - 1) / g.chunk);
+        cnt = last - first + 1;
+        p = parts + (size_t)row * g.slots;
+    }
+    float mi[4], si[4];
+    int ai[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+        mi[u] = -INFINITY; si[u] = 0.f; ai[u] = 0x7fffffff;
+        const int sl = lane16 + 16 * u;
+        if (sl < cnt) {
+            const int4 v = __ldcg(reinterpret_cast<const int4 *>(p + sl));
+            mi[u] = __int_as_float(v.x); si[u] = __int_as_float(v.y); ai[u] = v.z;
+        }
+    }
+    float m = mi[0];
+    int a = ai[0];
+#pragma unroll
+    for (int u = 1; u < 4; ++u)
+        if (mi[u] > m || (mi[u] == m && ai[u] < a)) { m = mi[u]; a = ai[u]; }
+#pragma unroll
+    for (int off = 8; off > 0; off >>= 1) {
+        const float om = __shfl_xor_sync(0xffffffffu, m, off, 16);
+        const int oa = __shfl_xor_sync(0xffffffffu, a, off, 16);
+        if (om > m || (om == m && oa < a)) { m = om; a = oa; }
+    }
+    double s = 0.0;
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+        if (mi[u] != -INFINITY) s += (double)si[u] * (double)exp2f((mi[u] - m) * k);
+#pragma unroll
+    for (int off = 8; off > 0; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off, 16);
+    M = m;
+    S = s;
+    A = (a == 0x7fffffff) ? 0 : a;
+}
 #endif
 
 static inline cudaStream_t fspad_stream(void *s) { return reinterpret_cast<cudaStream_t>(s); }
