@@ -141,9 +141,8 @@ def main():
     import torch.distributed as dist
     from paper_2408_15562_b200 import binding
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    from paper_2408_15562_b200 import dist_util
+    rank, world, local = dist_util.rank_info()
     torch.cuda.set_device(local)
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
@@ -288,11 +287,8 @@ def main():
     d2h = sum(t.numel() * t.element_size() for t in (hout, hpath, hn, hb, hl))
 
     # max over ranks
-    vals = torch.tensor([step_us, attn_us, accept_us, compact_us, stats_us, e2e_us, eager_us], dtype=torch.float64,
-                        device="cuda")
-    if world > 1:
-        dist.all_reduce(vals, op=dist.ReduceOp.MAX)
-    step_us, attn_us, accept_us, compact_us, stats_us, e2e_us, eager_us = [float(x) for x in vals.cpu()]
+    step_us, attn_us, accept_us, compact_us, stats_us, e2e_us, eager_us = dist_util.max_over_ranks(
+        [step_us, attn_us, accept_us, compact_us, stats_us, e2e_us, eager_us], device="cuda")
 
     if rank == 0:
         peak, peak_kind = peaks()
@@ -310,7 +306,7 @@ def main():
                        "launch": "K steps captured in one CUDA graph, one replay timed",
                        "l2": "inputs rotated over %d copies (%.0f MB per copy, > 2x L2 in total)" % (R, one_set / 1e6),
                        "multi_gpu": "independent replicas, no collective"},
-            "steps_per_s_all_gpus": world * 1e6 / step_us,
+            "steps_per_s_all_gpus": dist_util.aggregate_replicas(step_us, world),
             "step_hbm_gbs_all_rows_definition": step_all / (step_us * 1e-6) / 1e9,
             "step_frac_of_hbm_peak": step_all / (step_us * 1e-6) / 1e9 / peak,
             "step_algorithmic_bytes": step_all,

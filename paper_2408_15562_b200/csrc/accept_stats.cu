@@ -9,9 +9,9 @@
 // equal contiguous ranges, one per CTA (four CTAs per SM, a single wave), so
 // the load is balanced whatever rows and V are.  A range may cross row
 // boundaries; each (row, CTA) piece yields one partial (max, argmax, sum).
-// A thread issues eight 128-bit loads before it touches the data, takes the
-// maximum of the 32 values in registers, rescales its running sum once and
-// adds the 32 exponentials: no per-element branch.  Partials are merged per
+// A thread works in batches of four 128-bit loads, with the next batch already
+// in flight: it takes the maximum of the 16 values in registers, rescales its
+// running sum once and adds the 16 exponentials: no per-element branch.  Partials are merged per
 // row by whoever needs them (the acceptance walk for the rows it visits, or
 // the small merge kernel behind fspad_accept_stats).
 #include "common.cuh"
@@ -19,7 +19,7 @@
 namespace {
 
 constexpr int kThreads = 256;
-constexpr int kDeep = 8;                  // load units in flight per thread
+constexpr int kDeep = 4;                  // load units per batch per thread (two batches in flight)
 constexpr float kLog2e = 1.4426950408889634f;
 
 __device__ __forceinline__ float ex2(float x)
@@ -44,11 +44,40 @@ __device__ __forceinline__ void acc_merge(Acc &p, float om, float os, int oa, fl
     p.s = sp + so;
 }
 
+// one load unit: a float4 (UNIT == 4) or a float (UNIT == 1)
+template <int UNIT> struct Unit;
+template <> struct Unit<4> {
+    typedef float4 T;
+    static __device__ __forceinline__ T pad() { return make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY); }
+    static __device__ __forceinline__ float vmax(const T &v) { return fmaxf(fmaxf(v.x, v.y), fmaxf(v.z, v.w)); }
+    static __device__ __forceinline__ float vsum(const T &v, float m, float k)
+    {
+        return (ex2((v.x - m) * k) + ex2((v.y - m) * k)) + (ex2((v.z - m) * k) + ex2((v.w - m) * k));
+    }
+    // lowest position inside the unit equal to bm, or keep `a`
+    static __device__ __forceinline__ int first_eq(const T &v, float bm, int j, int a)
+    {
+        if (v.w == bm) a = j + 3;
+        if (v.z == bm) a = j + 2;
+        if (v.y == bm) a = j + 1;
+        if (v.x == bm) a = j;
+        return a;
+    }
+};
+template <> struct Unit<1> {
+    typedef float T;
+    static __device__ __forceinline__ T pad() { return -INFINITY; }
+    static __device__ __forceinline__ float vmax(const T &v) { return v; }
+    static __device__ __forceinline__ float vsum(const T &v, float m, float k) { return ex2((v - m) * k); }
+    static __device__ __forceinline__ int first_eq(const T &v, float bm, int j, int a) { return v == bm ? j : a; }
+};
+
 template <int UNIT>
 __global__ void __launch_bounds__(kThreads, 4)
 accept_stats_kernel(const float *__restrict__ logits, const float *__restrict__ temperature,
                     int rows_per_seq, const FspadStatsGeom g, FspadStatsPart *__restrict__ parts)
 {
+    typedef typename Unit<UNIT>::T U;
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
     const long long lo = (long long)blockIdx.x * g.chunk;
     const long long hi = min(g.total, lo + g.chunk);
@@ -59,81 +88,60 @@ accept_stats_kernel(const float *__restrict__ logits, const float *__restrict__ 
         const int row = (int)(seg_lo / g.upr);
         const long long row_lo = (long long)row * g.upr;
         const long long seg_hi = min(hi, row_lo + g.upr);
+        const int n = (int)(seg_hi - seg_lo);                 // units in this piece of the row
+        const int off = (int)(seg_lo - row_lo);               // position of the piece inside the row
+        const U *px = reinterpret_cast<const U *>(logits) + seg_lo;
         float T = temperature ? temperature[row / rows_per_seq] : 1.0f;
         if (!(T > 0.0f)) T = 1.0f;
         const float k = kLog2e / T;
 
+        // software pipeline: the next batch of loads is in flight while this one is reduced
         Acc p{-INFINITY, 0.f, 0x7fffffff};
-        for (long long base = seg_lo; base < seg_hi; base += (long long)kThreads * kDeep) {
-            if (UNIT == 4) {
-                float4 v[kDeep];
-                const float4 *x4 = reinterpret_cast<const float4 *>(logits);
+        U cur[kDeep], nxt[kDeep];
+#pragma unroll
+        for (int u = 0; u < kDeep; ++u) {
+            const int i = u * kThreads + tid;
+            cur[u] = (i < n) ? __ldg(px + i) : Unit<UNIT>::pad();
+        }
+        for (int base = 0; base < n; base += kThreads * kDeep) {
+            const int nb = base + kThreads * kDeep;
+            if (nb < n) {
 #pragma unroll
                 for (int u = 0; u < kDeep; ++u) {
-                    const long long i = base + u * kThreads + tid;
-                    v[u] = (i < seg_hi) ? __ldg(x4 + i) : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+                    const int i = nb + u * kThreads + tid;
+                    nxt[u] = (i < n) ? __ldg(px + i) : Unit<UNIT>::pad();
                 }
-                float bm = -INFINITY;
+            }
+            float bm = Unit<UNIT>::vmax(cur[0]);
 #pragma unroll
-                for (int u = 0; u < kDeep; ++u) bm = fmaxf(bm, fmaxf(fmaxf(v[u].x, v[u].y), fmaxf(v[u].z, v[u].w)));
-                if (bm > p.m) {
-                    // lowest index attaining the new maximum: scan from the back so the first match wins
-                    int a = 0;
+            for (int u = 1; u < kDeep; ++u) bm = fmaxf(bm, Unit<UNIT>::vmax(cur[u]));
+            if (bm > p.m) {
+                // lowest index attaining the new maximum: scan from the back so the first match wins
+                int a = 0;
 #pragma unroll
-                    for (int u = kDeep - 1; u >= 0; --u) {
-                        const int j = (int)((base + u * kThreads + tid - row_lo) << 2);
-                        if (v[u].w == bm) a = j + 3;
-                        if (v[u].z == bm) a = j + 2;
-                        if (v[u].y == bm) a = j + 1;
-                        if (v[u].x == bm) a = j;
-                    }
-                    p.s = (p.m == -INFINITY) ? 0.f : p.s * ex2((p.m - bm) * k);
-                    p.m = bm;
-                    p.a = a;
-                }
-                if (p.m != -INFINITY) {
-                    const float m = p.m;
-                    float s0 = 0.f, s1 = 0.f;
+                for (int u = kDeep - 1; u >= 0; --u)
+                    a = Unit<UNIT>::first_eq(cur[u], bm, (off + base + u * kThreads + tid) * UNIT, a);
+                p.s = (p.m == -INFINITY) ? 0.f : p.s * ex2((p.m - bm) * k);
+                p.m = bm;
+                p.a = a;
+            }
+            if (p.m != -INFINITY) {
+                float s0 = 0.f;
 #pragma unroll
-                    for (int u = 0; u < kDeep; ++u) {
-                        s0 += ex2((v[u].x - m) * k) + ex2((v[u].y - m) * k);
-                        s1 += ex2((v[u].z - m) * k) + ex2((v[u].w - m) * k);
-                    }
-                    p.s += s0 + s1;
-                }
-            } else {
-                float v[kDeep];
+                for (int u = 0; u < kDeep; ++u) s0 += Unit<UNIT>::vsum(cur[u], p.m, k);
+                p.s += s0;
+            }
+            if (nb < n) {
 #pragma unroll
-                for (int u = 0; u < kDeep; ++u) {
-                    const long long i = base + u * kThreads + tid;
-                    v[u] = (i < seg_hi) ? __ldg(logits + i) : -INFINITY;
-                }
-                float bm = -INFINITY;
-#pragma unroll
-                for (int u = 0; u < kDeep; ++u) bm = fmaxf(bm, v[u]);
-                if (bm > p.m) {
-                    int a = 0;
-#pragma unroll
-                    for (int u = kDeep - 1; u >= 0; --u)
-                        if (v[u] == bm) a = (int)(base + u * kThreads + tid - row_lo);
-                    p.s = (p.m == -INFINITY) ? 0.f : p.s * ex2((p.m - bm) * k);
-                    p.m = bm;
-                    p.a = a;
-                }
-                if (p.m != -INFINITY) {
-                    float s0 = 0.f;
-#pragma unroll
-                    for (int u = 0; u < kDeep; ++u) s0 += ex2((v[u] - p.m) * k);
-                    p.s += s0;
-                }
+                for (int u = 0; u < kDeep; ++u) cur[u] = nxt[u];
             }
         }
         // block reduction of (m, s, a)
 #pragma unroll
-        for (int off = 16; off > 0; off >>= 1) {
-            const float om = __shfl_xor_sync(0xffffffffu, p.m, off);
-            const float os = __shfl_xor_sync(0xffffffffu, p.s, off);
-            const int oa = __shfl_xor_sync(0xffffffffu, p.a, off);
+        for (int o = 16; o > 0; o >>= 1) {
+            const float om = __shfl_xor_sync(0xffffffffu, p.m, o);
+            const float os = __shfl_xor_sync(0xffffffffu, p.s, o);
+            const int oa = __shfl_xor_sync(0xffffffffu, p.a, o);
             acc_merge(p, om, os, oa, k);
         }
         if (lane == 0) wacc[wid] = p;
@@ -141,10 +149,10 @@ accept_stats_kernel(const float *__restrict__ logits, const float *__restrict__ 
         if (wid == 0) {
             Acc q = (lane < kThreads / 32) ? wacc[lane] : Acc{-INFINITY, 0.f, 0x7fffffff};
 #pragma unroll
-            for (int off = 4; off > 0; off >>= 1) {
-                const float om = __shfl_xor_sync(0xffffffffu, q.m, off);
-                const float os = __shfl_xor_sync(0xffffffffu, q.s, off);
-                const int oa = __shfl_xor_sync(0xffffffffu, q.a, off);
+            for (int o = 4; o > 0; o >>= 1) {
+                const float om = __shfl_xor_sync(0xffffffffu, q.m, o);
+                const float os = __shfl_xor_sync(0xffffffffu, q.s, o);
+                const int oa = __shfl_xor_sync(0xffffffffu, q.a, o);
                 acc_merge(q, om, os, oa, k);
             }
             if (lane == 0) {

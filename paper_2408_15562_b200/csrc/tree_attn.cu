@@ -312,19 +312,42 @@ tree_attn_combine_kernel(const AttnArgs a, int B)
     const int g = (int)((row / a.M) % a.Hkv);
     const int b = (int)(row / ((long long)a.M * a.Hkv));
     const size_t pbase = ((size_t)b * a.Hkv + g) * a.n_splits;
-    float mmax = -INFINITY;
-    for (int sidx = 0; sidx < a.n_splits; ++sidx)
-        mmax = fmaxf(mmax, a.part_ml[((pbase + sidx) * a.M + gr) * 2]);
+    // all (max, sum) pairs of the row are fetched at once, two splits per lane (n_splits <= 64)
+    const int ns = a.n_splits;
+    float m0 = -INFINITY, l0 = 0.f, m1 = -INFINITY, l1 = 0.f;
+    if (lane < ns) {
+        const float2 t = __ldcg(reinterpret_cast<const float2 *>(a.part_ml + ((pbase + lane) * a.M + gr) * 2));
+        m0 = t.x; l0 = t.y;
+    }
+    if (lane + 32 < ns) {
+        const float2 t = __ldcg(reinterpret_cast<const float2 *>(a.part_ml + ((pbase + lane + 32) * a.M + gr) * 2));
+        m1 = t.x; l1 = t.y;
+    }
+    float mmax = fmaxf(m0, m1);
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) mmax = fmaxf(mmax, __shfl_xor_sync(0xffffffffu, mmax, off));
+    const float w0 = (m0 == -INFINITY) ? 0.f : exp2f(m0 - mmax);
+    const float w1 = (m1 == -INFINITY) ? 0.f : exp2f(m1 - mmax);
+    float denom = w0 * l0 + w1 * l1;
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) denom += __shfl_xor_sync(0xffffffffu, denom, off);
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    float denom = 0.f;
-    for (int sidx = 0; sidx < a.n_splits; ++sidx) {
-        const float *ml = a.part_ml + ((pbase + sidx) * a.M + gr) * 2;
-        const float ms = ml[0];
-        if (ms == -INFINITY) continue;
-        const float w = exp2f(ms - mmax);
-        denom += w * ml[1];
-        const float4 v = *reinterpret_cast<const float4 *>(a.part_o + ((pbase + sidx) * a.M + gr) * D + lane * 4);
-        acc.x += w * v.x; acc.y += w * v.y; acc.z += w * v.z; acc.w += w * v.w;
+    for (int s0 = 0; s0 < ns; s0 += 4) {
+        float4 v[4];
+        float w[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int sidx = s0 + u;
+            const float wa = __shfl_sync(0xffffffffu, w0, sidx & 31), wb = __shfl_sync(0xffffffffu, w1, sidx & 31);
+            w[u] = (sidx < ns) ? ((sidx < 32) ? wa : wb) : 0.f;
+            v[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (w[u] != 0.f)
+                v[u] = __ldcg(reinterpret_cast<const float4 *>(a.part_o + ((pbase + sidx) * a.M + gr) * D + lane * 4));
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            acc.x += w[u] * v[u].x; acc.y += w[u] * v[u].y; acc.z += w[u] * v[u].z; acc.w += w[u] * v[u].w;
+        }
     }
     const float inv = denom > 0.f ? 1.f / denom : 0.f;
     const int node = gr / a.G, hh = gr % a.G;
