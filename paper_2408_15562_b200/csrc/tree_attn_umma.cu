@@ -107,9 +107,11 @@ __device__ __forceinline__ uint32_t make_idesc(bool b_mn_major)
 __device__ __forceinline__ void mma_f16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
                                         uint32_t accumulate)
 {
+    const uint32_t zero = 0;                // no output lane is disabled
     asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}\n"
-                 :: "r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %6, %7, %8}, p;\n\t}\n"
+                 :: "r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(zero), "r"(zero),
+                    "r"(zero), "r"(zero) : "memory");
 }
 __device__ __forceinline__ void mma_commit(uint32_t bar)
 {
@@ -151,3 +153,249 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t *>(&v);
 }
+
+__global__ void __launch_bounds__(NT, 1)
+tree_attn_umma_kernel(const Args a)
+{
+    extern __shared__ unsigned char smem_raw[];
+    __shared__ __align__(8) unsigned long long s_bar[2];     // [0]: S ready, [1]: O updated
+    __shared__ uint32_t s_tmem;
+    __shared__ int s_fail;
+    __shared__ unsigned long long s_anc[FSPAD_MAX_NODES];
+
+    const int tid = threadIdx.x, warp = tid >> 5;
+    const int split = blockIdx.x;
+    const int g = blockIdx.y / a.mtiles, mt = blockIdx.y % a.mtiles;
+    const int b = blockIdx.z;
+    const int N = a.N, G = a.G, M = a.M;
+
+    int L = a.prefix_len[b];
+    if (L < 0 || L + N > a.max_len) {
+        if (tid == 0) fspad_report(a.status, FSPAD_ERR_RANGE);
+        L = max(0, min(L, a.max_len - N));
+    }
+    const int Ltot = L + N;
+    const int n_chunks = (Ltot + BK - 1) / BK;
+    const int per = (n_chunks + a.n_splits - 1) / a.n_splits;
+    const int c0 = split * per, c1 = min(n_chunks, c0 + per);
+
+    const int gr = mt * BM + tid;                 // this thread's row among the kv head's M rows
+    const bool row_ok = gr < M;
+    const int node = row_ok ? gr / G : 0;
+    const size_t prow = ((size_t)b * a.Hkv + g) * a.n_splits + split;
+
+    if (c0 >= c1) {                               // nothing to do for this split: empty partial
+        if (row_ok) { float *ml = a.part_ml + (prow * M + gr) * 2; ml[0] = -INFINITY; ml[1] = 0.f; }
+        return;
+    }
+
+    // 1024-byte aligned tiles: Q | K0 | K1 | V0 | V1 | P
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t sQ = base, sK = base + TILE, sV = base + 3 * TILE, sP = base + 5 * TILE;
+    const uint32_t barS = smem_u32(&s_bar[0]), barO = smem_u32(&s_bar[1]);
+
+    // ancestor-or-self masks
+    if (tid < N) {
+        const int *par = a.parent + (size_t)b * N;
+        unsigned long long mask = 0ull;
+        int cur = tid;
+        bool bad = false;
+        for (int step = 0; step <= N && cur >= 0; ++step) {
+            mask |= 1ull << cur;
+            const int p = par[cur];
+            if (cur == 0) { bad |= (p != -1); break; }
+            if (p < 0 || p >= cur) { bad = true; break; }
+            cur = p;
+        }
+        if (bad) fspad_report(a.status, FSPAD_ERR_BAD_TREE);
+        s_anc[tid] = mask;
+    }
+    if (tid == 0) {
+        mbar_init(barS, 1);
+        mbar_init(barO, 1);
+        s_fail = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+    }
+    if (warp == 0) {                              // one warp allocates the tensor memory
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n"
+                     :: "r"(smem_u32(&s_tmem)), "r"(TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
+    }
+
+    const fspad_bf16 *kcb = a.kc + ((size_t)b * a.Hkv + g) * (size_t)a.max_len * D;
+    const fspad_bf16 *vcb = a.vc + ((size_t)b * a.Hkv + g) * (size_t)a.max_len * D;
+    const fspad_bf16 *tkb = a.tk ? a.tk + ((size_t)b * a.Hkv + g) * (size_t)N * D : kcb + (size_t)L * D;
+    const fspad_bf16 *tvb = a.tv ? a.tv + ((size_t)b * a.Hkv + g) * (size_t)N * D : vcb + (size_t)L * D;
+
+    // ---- stage Q and the first chunks ----
+    for (int i = tid; i < BM * 16; i += NT) {
+        const int r = i >> 4, c = i & 15;
+        const int grr = mt * BM + r;
+        const bool ok = grr < M;
+        const int nd = ok ? grr / G : 0, hh = ok ? grr % G : 0;
+        const fspad_bf16 *src = a.q + (((size_t)b * N + nd) * a.Hq + g * G + hh) * D + c * 8;
+        cp_async16(sQ + tile_off(r, c), src, ok);
+    }
+    auto load_chunk = [&](int ch, int buf) {
+        const uint32_t dK = sK + buf * TILE, dV = sV + buf * TILE;
+        for (int i = tid; i < BK * 16; i += NT) {
+            const int r = i >> 4, c = i & 15;
+            const int key = ch * BK + r;
+            const bool ok = key < Ltot;
+            const fspad_bf16 *ks = kcb, *vs = vcb;
+            if (ok) {
+                if (key < L) { ks = kcb + (size_t)key * D + c * 8; vs = vcb + (size_t)key * D + c * 8; }
+                else { ks = tkb + (size_t)(key - L) * D + c * 8; vs = tvb + (size_t)(key - L) * D + c * 8; }
+            }
+            cp_async16(dK + tile_off(r, c), ks, ok);
+            cp_async16(dV + tile_off(r, c), vs, ok);
+        }
+    };
+    load_chunk(c0, 0);
+    cp_async_commit();
+    if (c0 + 1 < c1) load_chunk(c0 + 1, 1);
+    cp_async_commit();
+
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = s_tmem;
+    const uint32_t tS = tmem + ((uint32_t)(warp * 32) << 16);          // this warp's lanes, S columns
+    const uint32_t tO = tS + 128u;                                     // O columns
+    const uint32_t idesc_s = make_idesc(false), idesc_o = make_idesc(true);
+    const unsigned long long anc = s_anc[node];
+
+    float m_run = -INFINITY, l_run = 0.f;        // running maximum (base-2, scaled) and sum of this row
+    uint32_t phS = 0, phO = 0;
+    bool failed = false;
+
+    for (int ch = c0; ch < c1; ++ch) {
+        const int buf = (ch - c0) & 1;
+        // this chunk's copies have landed (the younger group, if any, may still be in flight)
+        if (ch + 1 < c1) cp_async_wait<1>(); else cp_async_wait<0>();
+        fence_async_smem();
+        __syncthreads();
+        if (tid == 0 && !failed) {
+            tc_fence_after();
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks) {     // K = 16 per instruction over d = 128
+                const uint32_t koff = (ks >> 2) * HALF + (ks & 3) * 32;
+                mma_f16(tmem, make_desc(sQ + koff, 16), make_desc(sK + buf * TILE + koff, 16), idesc_s, ks > 0);
+            }
+            mma_commit(barS);
+        }
+        if (!failed && !mbar_wait(barS, phS)) { failed = true; s_fail = 1; }
+        phS ^= 1;
+        tc_fence_after();
+
+        // ---- this row's 128 scores: mask, online softmax, P -> shared memory (bf16, swizzled) ----
+        const bool needs_mask = (ch + 1) * BK > L;
+        float mx = -INFINITY;
+        float sc[4][32];
+#pragma unroll
+        for (int q4 = 0; q4 < 4; ++q4) {
+            tmem_ld32(tS + q4 * 32, sc[q4]);
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+                float v = sc[q4][j] * a.scale_log2;
+                if (needs_mask) {
+                    const int key = ch * BK + q4 * 32 + j;
+                    if (key >= L) {
+                        const bool ok = (key < Ltot) && ((anc >> (key - L)) & 1ull);
+                        if (!ok) v = -INFINITY;
+                    }
+                }
+                sc[q4][j] = v;
+                mx = fmaxf(mx, v);
+            }
+        }
+        const float m_new = fmaxf(m_run, mx);
+        const float m_safe = (m_new == -INFINITY) ? 0.f : m_new;
+        const float alpha = exp2f(m_run - m_safe);
+        float rs = 0.f;
+#pragma unroll
+        for (int q4 = 0; q4 < 4; ++q4) {
+#pragma unroll
+            for (int c8 = 0; c8 < 4; ++c8) {     // 8 keys = one 16-byte chunk of the P row
+                uint32_t w[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const float p0 = exp2f(sc[q4][c8 * 8 + 2 * e] - m_safe);
+                    const float p1 = exp2f(sc[q4][c8 * 8 + 2 * e + 1] - m_safe);
+                    w[e] = pack_bf16(p0, p1);
+                    const float2 f = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162 *>(&w[e]));
+                    rs += f.x + f.y;             // the sum is taken over the rounded weights
+                }
+                const int c = q4 * 4 + c8;       // chunk 0..15 of this row of P
+                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};\n"
+                             :: "r"(sP + tile_off(tid, c)), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]) : "memory");
+            }
+        }
+        l_run = l_run * alpha + rs;
+        m_run = m_new;
+
+        // ---- rescale O in tensor memory when a previous chunk has contributed ----
+        if (ch > c0) {
+#pragma unroll
+            for (int q4 = 0; q4 < 4; ++q4) {
+                float o[32];
+                tmem_ld32(tO + q4 * 32, o);
+#pragma unroll
+                for (int j = 0; j < 32; ++j) o[j] *= alpha;
+                tmem_st32(tO + q4 * 32, o);
+            }
+            asm volatile("tcgen05.wait::st.sync.aligned;\n" ::: "memory");
+        }
+        fence_async_smem();
+        tc_fence_before();
+        __syncthreads();
+        if (tid == 0 && !failed) {
+            tc_fence_after();
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks) {     // K = 16 keys per instruction over the chunk's 128 keys
+                const uint64_t da = make_desc(sP + (ks >> 2) * HALF + (ks & 3) * 32, 16);
+                // V as an MN-major operand: d is contiguous, the two 64-wide halves are HALF bytes apart
+                const uint64_t db = make_desc(sV + buf * TILE + ks * 16 * 128, HALF);
+                mma_f16(tmem + 128u, da, db, idesc_o, (ch > c0) || (ks > 0));
+            }
+            mma_commit(barO);
+        }
+        // P, this K/V buffer and the S columns are free again once these products have completed
+        if (!failed && !mbar_wait(barO, phO)) { failed = true; s_fail = 1; }
+        phO ^= 1;
+        tc_fence_after();
+        __syncthreads();
+        failed = failed || (s_fail != 0);
+        if (ch + 2 < c1) load_chunk(ch + 2, buf);
+        cp_async_commit();
+    }
+
+    // ---- publish the partial: unnormalised O row, running max and sum ----
+    if (failed) {
+        if (tid == 0) fspad_report(a.status, FSPAD_ERR_TIMEOUT);
+    } else if (row_ok) {
+        float *po = a.part_o + (prow * M + gr) * D;
+#pragma unroll
+        for (int q4 = 0; q4 < 4; ++q4) {
+            float o[32];
+            tmem_ld32(tO + q4 * 32, o);
+#pragma unroll
+            for (int j = 0; j < 32; j += 4)
+                *reinterpret_cast<float4 *>(po + q4 * 32 + j) = make_float4(o[j], o[j + 1], o[j + 2], o[j + 3]);
+        }
+        float *ml = a.part_ml + (prow * M + gr) * 2;
+        ml[0] = m_run;
+        ml[1] = l_run;
+    } else {
+        // rows beyond M still take part in the warp-wide tensor-memory loads of their warp
+#pragma unroll
+        for (int q4 = 0; q4 < 4; ++q4) { float o[32]; tmem_ld32(tO + q4 * 32, o); }
+    }
+    cp_async_wait<0>();
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0)
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" :: "r"(tmem), "r"(TMEM_COLS) : "memory");
+}
+
+}  // namespace umma
