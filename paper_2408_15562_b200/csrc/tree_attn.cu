@@ -393,29 +393,12 @@ cudaError_t fspad_launch_tree_attn(fspad_ctx *ctx, const fspad_bf16 *q, const fs
     a.q = q; a.kc = kc; a.vc = vc; a.tk = tk; a.tv = tv; a.parent = parent; a.prefix_len = prefix_len;
     a.N = N; a.Hq = c.n_q_heads; a.Hkv = c.n_kv_heads; a.G = c.n_q_heads / c.n_kv_heads;
     a.M = N * a.G; a.max_len = c.max_len;
-    a.n_splits = fspad_attn_splits(ctx, N, B);
-    const int BM = attn_bm(a.M);
-    a.mtiles = (a.M + BM - 1) / BM;
+    a.n_splits = fspad_attn_umma_splits(ctx, N, B);
+    a.mtiles = (a.M + 127) / 128;
     a.scale_log2 = ctx->scale * kLog2e;
     a.part_o = ctx->part_o; a.part_ml = ctx->part_ml; a.out = out; a.status = ctx->d_status;
-
-    dim3 grid(a.n_splits, c.n_kv_heads * a.mtiles, B);
-    cudaError_t e;
-    if (!ctx->attn_attr_done) {
-        e = cudaFuncSetAttribute(tree_attn_splitkv_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 attn_smem_bytes<8>());
-        if (e != cudaSuccess) return e;
-        e = cudaFuncSetAttribute(tree_attn_splitkv_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 attn_smem_bytes<4>());
-        if (e != cudaSuccess) return e;
-        ctx->attn_attr_done = 1;
-    }
-    if (BM == 128)
-        tree_attn_splitkv_kernel<8><<<grid, 256, attn_smem_bytes<8>(), st>>>(a);
-    else
-        tree_attn_splitkv_kernel<4><<<grid, 128, attn_smem_bytes<4>(), st>>>(a);
-    ctx->launches++;
-    e = cudaGetLastError();
+    cudaError_t e = fspad_launch_attn_umma_split(ctx, q, kc, vc, tk, tv, parent, prefix_len, N, B, a.n_splits,
+                                                 a.scale_log2, st);
     if (e != cudaSuccess) return e;
     const long long rows = (long long)B * c.n_kv_heads * a.M;
     tree_attn_combine_kernel<<<(unsigned)((rows + 3) / 4), 128, 0, st>>>(a, B);

@@ -32,8 +32,6 @@ constexpr int TILE = 2 * HALF;         // bytes of one [128][128] bf16 tile
 constexpr int SMEM_BYTES = 6 * TILE + 1024;   // Q, K[2], V[2], P + alignment slack
 constexpr uint32_t TMEM_COLS = 256;    // S: columns 0..127, O: columns 128..255
 constexpr uint32_t WAIT_CAP = 4u << 20;
-constexpr float kLog2e = 1.4426950408889634f;
-
 struct Args {
     const fspad_bf16 *q, *kc, *vc, *tk, *tv;
     const int *parent, *prefix_len;
@@ -399,3 +397,41 @@ tree_attn_umma_kernel(const Args a)
 }
 
 }  // namespace umma
+
+int fspad_attn_umma_splits(const fspad_ctx *ctx, int N, int B)
+{
+    const int G = ctx->cfg.n_q_heads / ctx->cfg.n_kv_heads;
+    const int mtiles = (N * G + umma::BM - 1) / umma::BM;
+    const long long base = (long long)B * ctx->cfg.n_kv_heads * mtiles;
+    long long s = ctx->sm_count / base;           // one CTA per SM, never a partial second wave
+    const int max_chunks = (ctx->cfg.max_len + umma::BK - 1) / umma::BK;
+    if (s > max_chunks) s = max_chunks;
+    if (s > 64) s = 64;
+    if (s < 1) s = 1;
+    return (int)s;
+}
+
+cudaError_t fspad_launch_attn_umma_split(fspad_ctx *ctx, const fspad_bf16 *q, const fspad_bf16 *kc,
+                                         const fspad_bf16 *vc, const fspad_bf16 *tk, const fspad_bf16 *tv,
+                                         const int *parent, const int *prefix_len, int N, int B, int n_splits,
+                                         float scale_log2, cudaStream_t st)
+{
+    const fspad_config &c = ctx->cfg;
+    umma::Args a;
+    a.q = q; a.kc = kc; a.vc = vc; a.tk = tk; a.tv = tv; a.parent = parent; a.prefix_len = prefix_len;
+    a.N = N; a.Hq = c.n_q_heads; a.Hkv = c.n_kv_heads; a.G = c.n_q_heads / c.n_kv_heads;
+    a.M = N * a.G; a.max_len = c.max_len; a.n_splits = n_splits;
+    a.mtiles = (a.M + umma::BM - 1) / umma::BM;
+    a.scale_log2 = scale_log2;
+    a.part_o = ctx->part_o; a.part_ml = ctx->part_ml; a.status = ctx->d_status;
+    if (!ctx->attn_attr_done) {
+        cudaError_t e = cudaFuncSetAttribute(umma::tree_attn_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             umma::SMEM_BYTES);
+        if (e != cudaSuccess) return e;
+        ctx->attn_attr_done = 1;
+    }
+    dim3 grid(n_splits, c.n_kv_heads * a.mtiles, B);
+    umma::tree_attn_umma_kernel<<<grid, umma::NT, umma::SMEM_BYTES, st>>>(a);
+    ctx->launches++;
+    return cudaGetLastError();
+}
