@@ -31,7 +31,7 @@ constexpr int HALF = 128 * 128;        // bytes of one [128 rows][64 bf16] half 
 constexpr int TILE = 2 * HALF;         // bytes of one [128][128] bf16 tile
 constexpr int SMEM_BYTES = 6 * TILE + 1024;   // Q, K[2], V[2], P + alignment slack
 constexpr uint32_t TMEM_COLS = 256;    // S: columns 0..127, O: columns 128..255
-constexpr uint32_t WAIT_CAP = 4u << 20;
+constexpr uint32_t WAIT_CAP = 200000;   // polls of a bounded mbarrier wait
 struct Args {
     const fspad_bf16 *q, *kc, *vc, *tk, *tv;
     const int *parent, *prefix_len;
@@ -64,19 +64,27 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
 {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(bar), "r"(count));
 }
-__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity)
+__device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity)
 {
     uint32_t ok;
-    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}\n"
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}\n"
                  : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
-// bounded wait; false if the cap ran out
+// Bounded wait (non-blocking test + short sleep, about 20 ms in all); false if the cap ran out.
+// Lane 0 polls and the warp takes its verdict through a full-mask shuffle, so every lane leaves
+// together: the warp-collective tensor-memory instructions that follow need a converged warp.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
 {
-    for (uint32_t i = 0; i < WAIT_CAP; ++i)
-        if (mbar_try(bar, parity)) return true;
-    return false;
+    int ok = 0;
+    if ((threadIdx.x & 31) == 0) {
+        for (uint32_t i = 0; i < WAIT_CAP && !ok; ++i) {
+            ok = mbar_test(bar, parity) ? 1 : 0;
+            if (!ok) __nanosleep(40);
+        }
+    }
+    ok = __shfl_sync(0xffffffffu, ok, 0);
+    return ok != 0;
 }
 
 // shared-memory matrix descriptor, 128-byte swizzle, 8-row groups 1024 bytes apart
@@ -118,6 +126,7 @@ __device__ __forceinline__ void mma_commit(uint32_t bar)
 __device__ __forceinline__ void tmem_ld32(uint32_t addr, float (&v)[32])
 {
     uint32_t r[32];
+    __syncwarp();
     asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
                  "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
                  "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];\n"
@@ -132,6 +141,7 @@ __device__ __forceinline__ void tmem_ld32(uint32_t addr, float (&v)[32])
 }
 __device__ __forceinline__ void tmem_st32(uint32_t addr, const float (&v)[32])
 {
+    __syncwarp();
     asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
                  "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
                  "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};\n"
@@ -214,7 +224,8 @@ tree_attn_umma_kernel(const Args a)
         s_fail = 0;
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     }
-    if (warp == 0) {                              // one warp allocates the tensor memory
+    if (warp == 0) {                              // one (converged) warp allocates the tensor memory
+        __syncwarp();
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n"
                      :: "r"(smem_u32(&s_tmem)), "r"(TMEM_COLS) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
@@ -392,8 +403,10 @@ tree_attn_umma_kernel(const Args a)
     cp_async_wait<0>();
     tc_fence_before();
     __syncthreads();
-    if (warp == 0)
+    if (warp == 0) {
+        __syncwarp();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" :: "r"(tmem), "r"(TMEM_COLS) : "memory");
+    }
 }
 
 }  // namespace umma
