@@ -380,25 +380,27 @@ tree_attn_umma_kernel(const Args a)
     }
 
     // ---- publish the partial: unnormalised O row, running max and sum ----
-    if (failed) {
-        if (tid == 0) fspad_report(a.status, FSPAD_ERR_TIMEOUT);
-    } else if (row_ok) {
-        float *po = a.part_o + (prow * M + gr) * D;
+    // Every lane of every warp takes part in the tensor-memory loads (they are warp-collective);
+    // only the stores to global memory depend on whether the lane's row exists.
+    if (failed && tid == 0) fspad_report(a.status, FSPAD_ERR_TIMEOUT);
+    {
+        const bool store = row_ok && !failed;
+        float *po = a.part_o + (prow * M + (row_ok ? gr : 0)) * D;
 #pragma unroll
         for (int q4 = 0; q4 < 4; ++q4) {
             float o[32];
             tmem_ld32(tO + q4 * 32, o);
+            if (store) {
 #pragma unroll
-            for (int j = 0; j < 32; j += 4)
-                *reinterpret_cast<float4 *>(po + q4 * 32 + j) = make_float4(o[j], o[j + 1], o[j + 2], o[j + 3]);
+                for (int j = 0; j < 32; j += 4)
+                    *reinterpret_cast<float4 *>(po + q4 * 32 + j) = make_float4(o[j], o[j + 1], o[j + 2], o[j + 3]);
+            }
         }
-        float *ml = a.part_ml + (prow * M + gr) * 2;
-        ml[0] = m_run;
-        ml[1] = l_run;
-    } else {
-        // rows beyond M still take part in the warp-wide tensor-memory loads of their warp
-#pragma unroll
-        for (int q4 = 0; q4 < 4; ++q4) { float o[32]; tmem_ld32(tO + q4 * 32, o); }
+        if (store) {
+            float *ml = a.part_ml + (prow * M + gr) * 2;
+            ml[0] = m_run;
+            ml[1] = l_run;
+        }
     }
     cp_async_wait<0>();
     tc_fence_before();
