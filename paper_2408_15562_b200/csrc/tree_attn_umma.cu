@@ -5,10 +5,10 @@
 // Split-KV flash-decode with tcgen05: all query rows that share a kv head (tree
 // node x GQA group member) form the M = 128 operand of one CTA; keys are
 // consumed in chunks of 128.  Per chunk: S = Q K^T is one chain of eight
-// tcgen05.mma (128 x 128 x 16, bf16 -> fp32) into tensor memory; every thread
-// owns one query row, reads its 128 scores back with tcgen05.ld, applies the
-// ancestor mask (only on chunks that reach past the cached prefix) and the
-// softmax in registers with no cross-thread traffic, and writes P as bf16 into
+// tcgen05.mma (128 x 128 x 16, bf16 -> fp32) into tensor memory; two threads
+// share a query row, each reads 64 of its scores back with tcgen05.ld, applies
+// the ancestor mask (only on chunks that reach past the cached prefix) and the
+// softmax in registers (one shared-memory exchange of the row maximum), and writes P as bf16 into
 // a 128-byte-swizzled shared-memory tile; O += P V is a second chain of eight
 // tcgen05.mma with V read directly in its [key][d] layout (MN-major operand).
 // O stays in tensor memory across chunks and is rescaled there when the running
@@ -26,7 +26,7 @@ namespace umma {
 constexpr int D = FSPAD_HEAD_DIM;      // 128
 constexpr int BM = 128;                // query rows per CTA
 constexpr int BK = 128;                // keys per chunk
-constexpr int NT = 128;                // threads per CTA: one per query row
+constexpr int NT = 256;                // threads per CTA: two per query row
 constexpr int HALF = 128 * 128;        // bytes of one [128 rows][64 bf16] half tile
 constexpr int TILE = 2 * HALF;         // bytes of one [128][128] bf16 tile
 constexpr int SMEM_BYTES = 6 * TILE + 1024;   // Q, K[2], V[2], P + alignment slack
@@ -162,6 +162,16 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
     return *reinterpret_cast<uint32_t *>(&v);
 }
 
+__device__ __forceinline__ float ex2f(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// Two threads share a query row: thread (row, half) owns columns half*64 .. half*64+63 of the
+// row's scores, of its P row and of its O row.  Warps w and w+4 address the same 32 lanes of
+// tensor memory (a warp reaches the lane quarter given by its index modulo 4).
 __global__ void __launch_bounds__(NT, 1)
 tree_attn_umma_kernel(const Args a)
 {
@@ -169,9 +179,12 @@ tree_attn_umma_kernel(const Args a)
     __shared__ __align__(8) unsigned long long s_bar[2];     // [0]: S ready, [1]: O updated
     __shared__ uint32_t s_tmem;
     __shared__ int s_fail;
+    __shared__ int s_par[FSPAD_MAX_NODES];
     __shared__ unsigned long long s_anc[FSPAD_MAX_NODES];
+    __shared__ float s_mx[2][BM];                            // per-half row maxima / sums exchange
 
     const int tid = threadIdx.x, warp = tid >> 5;
+    const int row = tid & (BM - 1), half = tid >> 7;
     const int split = blockIdx.x;
     const int g = blockIdx.y / a.mtiles, mt = blockIdx.y % a.mtiles;
     const int b = blockIdx.z;
@@ -187,13 +200,13 @@ tree_attn_umma_kernel(const Args a)
     const int per = (n_chunks + a.n_splits - 1) / a.n_splits;
     const int c0 = split * per, c1 = min(n_chunks, c0 + per);
 
-    const int gr = mt * BM + tid;                 // this thread's row among the kv head's M rows
+    const int gr = mt * BM + row;                 // this thread's row among the kv head's M rows
     const bool row_ok = gr < M;
     const int node = row_ok ? gr / G : 0;
     const size_t prow = ((size_t)b * a.Hkv + g) * a.n_splits + split;
 
     if (c0 >= c1) {                               // nothing to do for this split: empty partial
-        if (row_ok) { float *ml = a.part_ml + (prow * M + gr) * 2; ml[0] = -INFINITY; ml[1] = 0.f; }
+        if (row_ok && half == 0) { float *ml = a.part_ml + (prow * M + gr) * 2; ml[0] = -INFINITY; ml[1] = 0.f; }
         return;
     }
 
@@ -202,53 +215,26 @@ tree_attn_umma_kernel(const Args a)
     const uint32_t sQ = base, sK = base + TILE, sV = base + 3 * TILE, sP = base + 5 * TILE;
     const uint32_t barS = smem_u32(&s_bar[0]), barO = smem_u32(&s_bar[1]);
 
-    // ancestor-or-self masks
-    if (tid < N) {
-        const int *par = a.parent + (size_t)b * N;
-        unsigned long long mask = 0ull;
-        int cur = tid;
-        bool bad = false;
-        for (int step = 0; step <= N && cur >= 0; ++step) {
-            mask |= 1ull << cur;
-            const int p = par[cur];
-            if (cur == 0) { bad |= (p != -1); break; }
-            if (p < 0 || p >= cur) { bad = true; break; }
-            cur = p;
-        }
-        if (bad) fspad_report(a.status, FSPAD_ERR_BAD_TREE);
-        s_anc[tid] = mask;
-    }
-    if (tid == 0) {
-        mbar_init(barS, 1);
-        mbar_init(barO, 1);
-        s_fail = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
-    }
-    if (warp == 0) {                              // one (converged) warp allocates the tensor memory
-        __syncwarp();
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n"
-                     :: "r"(smem_u32(&s_tmem)), "r"(TMEM_COLS) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
-    }
-
     const fspad_bf16 *kcb = a.kc + ((size_t)b * a.Hkv + g) * (size_t)a.max_len * D;
     const fspad_bf16 *vcb = a.vc + ((size_t)b * a.Hkv + g) * (size_t)a.max_len * D;
     const fspad_bf16 *tkb = a.tk ? a.tk + ((size_t)b * a.Hkv + g) * (size_t)N * D : kcb + (size_t)L * D;
     const fspad_bf16 *tvb = a.tv ? a.tv + ((size_t)b * a.Hkv + g) * (size_t)N * D : vcb + (size_t)L * D;
 
-    // ---- stage Q and the first chunks ----
-    for (int i = tid; i < BM * 16; i += NT) {
-        const int r = i >> 4, c = i & 15;
-        const int grr = mt * BM + r;
-        const bool ok = grr < M;
-        const int nd = ok ? grr / G : 0, hh = ok ? grr % G : 0;
-        const fspad_bf16 *src = a.q + (((size_t)b * N + nd) * a.Hq + g * G + hh) * D + c * 8;
-        cp_async16(sQ + tile_off(r, c), src, ok);
+    // ---- the copies go out first; everything else of the prologue hides under their latency ----
+    {
+        const int c = tid & 15;                   // 16-byte chunk of the row, fixed per thread
+        for (int r = tid >> 4; r < BM; r += NT / 16) {
+            const int grr = mt * BM + r;
+            const bool ok = grr < M;
+            const int nd = ok ? grr / G : 0, hh = ok ? grr % G : 0;
+            const fspad_bf16 *src = a.q + (((size_t)b * N + nd) * a.Hq + g * G + hh) * D + c * 8;
+            cp_async16(sQ + tile_off(r, c), src, ok);
+        }
     }
     auto load_chunk = [&](int ch, int buf) {
         const uint32_t dK = sK + buf * TILE, dV = sV + buf * TILE;
-        for (int i = tid; i < BK * 16; i += NT) {
-            const int r = i >> 4, c = i & 15;
+        const int c = tid & 15;
+        for (int r = tid >> 4; r < BK; r += NT / 16) {
             const int key = ch * BK + r;
             const bool ok = key < Ltot;
             const fspad_bf16 *ks = kcb, *vs = vcb;
@@ -265,16 +251,47 @@ tree_attn_umma_kernel(const Args a)
     if (c0 + 1 < c1) load_chunk(c0 + 1, 1);
     cp_async_commit();
 
+    // ---- tree -> ancestor-or-self masks (parents staged in shared memory, then walked there) ----
+    if (tid < N) s_par[tid] = a.parent[(size_t)b * N + tid];
+    if (tid == 0) {
+        mbar_init(barS, 1);
+        mbar_init(barO, 1);
+        s_fail = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+    }
+    if (warp == 1) {                              // one (converged) warp allocates the tensor memory
+        __syncwarp();
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n"
+                     :: "r"(smem_u32(&s_tmem)), "r"(TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
+    }
+    __syncthreads();
+    if (tid < N) {
+        unsigned long long mask = 0ull;
+        int cur = tid;
+        bool bad = false;
+        for (int step = 0; step <= N && cur >= 0; ++step) {
+            mask |= 1ull << cur;
+            const int p = s_par[cur];
+            if (cur == 0) { bad |= (p != -1); break; }
+            if (p < 0 || p >= cur) { bad = true; break; }
+            cur = p;
+        }
+        if (bad) fspad_report(a.status, FSPAD_ERR_BAD_TREE);
+        s_anc[tid] = mask;
+    }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = s_tmem;
-    const uint32_t tS = tmem + ((uint32_t)(warp * 32) << 16);          // this warp's lanes, S columns
-    const uint32_t tO = tS + 128u;                                     // O columns
+    const uint32_t lanes = (uint32_t)((row >> 5) * 32) << 16;
+    const uint32_t tS = tmem + lanes + (uint32_t)(half * 64);            // this thread's 64 score columns
+    const uint32_t tO = tmem + lanes + 128u + (uint32_t)(half * 64);     // and its 64 output columns
     const uint32_t idesc_s = make_idesc(false), idesc_o = make_idesc(true);
     const unsigned long long anc = s_anc[node];
+    const float scale = a.scale_log2;
 
-    float m_run = -INFINITY, l_run = 0.f;        // running maximum (base-2, scaled) and sum of this row
+    float m_run = -INFINITY, l_part = 0.f;       // row maximum (shared by both halves), this half's sum
     uint32_t phS = 0, phO = 0;
     bool failed = false;
 
@@ -297,61 +314,63 @@ tree_attn_umma_kernel(const Args a)
         phS ^= 1;
         tc_fence_after();
 
-        // ---- this row's 128 scores: mask, online softmax, P -> shared memory (bf16, swizzled) ----
-        const bool needs_mask = (ch + 1) * BK > L;
-        float mx = -INFINITY;
-        float sc[4][32];
+        // ---- this thread's 64 scores: mask, row maximum (exchanged with the other half) ----
+        float sc[2][32];
+        tmem_ld32(tS, sc[0]);
+        tmem_ld32(tS + 32, sc[1]);
+        if ((ch + 1) * BK > L) {                 // only chunks that reach past the cached prefix
 #pragma unroll
-        for (int q4 = 0; q4 < 4; ++q4) {
-            tmem_ld32(tS + q4 * 32, sc[q4]);
+            for (int q2 = 0; q2 < 2; ++q2)
 #pragma unroll
-            for (int j = 0; j < 32; ++j) {
-                float v = sc[q4][j] * a.scale_log2;
-                if (needs_mask) {
-                    const int key = ch * BK + q4 * 32 + j;
+                for (int j = 0; j < 32; ++j) {
+                    const int key = ch * BK + half * 64 + q2 * 32 + j;
                     if (key >= L) {
                         const bool ok = (key < Ltot) && ((anc >> (key - L)) & 1ull);
-                        if (!ok) v = -INFINITY;
+                        if (!ok) sc[q2][j] = -INFINITY;
                     }
                 }
-                sc[q4][j] = v;
-                mx = fmaxf(mx, v);
-            }
         }
-        const float m_new = fmaxf(m_run, mx);
+        float mx = -INFINITY;
+#pragma unroll
+        for (int q2 = 0; q2 < 2; ++q2)
+#pragma unroll
+            for (int j = 0; j < 32; ++j) mx = fmaxf(mx, sc[q2][j]);
+        s_mx[half][row] = mx;
+        __syncthreads();
+        mx = fmaxf(mx, s_mx[half ^ 1][row]);
+        const float m_new = fmaxf(m_run, mx * scale);
         const float m_safe = (m_new == -INFINITY) ? 0.f : m_new;
-        const float alpha = exp2f(m_run - m_safe);
+        const float alpha = ex2f(m_run - m_safe);
         float rs = 0.f;
 #pragma unroll
-        for (int q4 = 0; q4 < 4; ++q4) {
+        for (int q2 = 0; q2 < 2; ++q2) {
 #pragma unroll
             for (int c8 = 0; c8 < 4; ++c8) {     // 8 keys = one 16-byte chunk of the P row
                 uint32_t w[4];
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
-                    const float p0 = exp2f(sc[q4][c8 * 8 + 2 * e] - m_safe);
-                    const float p1 = exp2f(sc[q4][c8 * 8 + 2 * e + 1] - m_safe);
+                    const float p0 = ex2f(fmaf(sc[q2][c8 * 8 + 2 * e], scale, -m_safe));
+                    const float p1 = ex2f(fmaf(sc[q2][c8 * 8 + 2 * e + 1], scale, -m_safe));
+                    rs += p0 + p1;
                     w[e] = pack_bf16(p0, p1);
-                    const float2 f = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162 *>(&w[e]));
-                    rs += f.x + f.y;             // the sum is taken over the rounded weights
                 }
-                const int c = q4 * 4 + c8;       // chunk 0..15 of this row of P
+                const int c = half * 8 + q2 * 4 + c8;   // chunk 0..15 of this row of P
                 asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};\n"
-                             :: "r"(sP + tile_off(tid, c)), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]) : "memory");
+                             :: "r"(sP + tile_off(row, c)), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]) : "memory");
             }
         }
-        l_run = l_run * alpha + rs;
+        l_part = l_part * alpha + rs;
         m_run = m_new;
 
-        // ---- rescale O in tensor memory when a previous chunk has contributed ----
+        // ---- rescale this thread's half of the O row when a previous chunk has contributed ----
         if (ch > c0) {
 #pragma unroll
-            for (int q4 = 0; q4 < 4; ++q4) {
+            for (int q2 = 0; q2 < 2; ++q2) {
                 float o[32];
-                tmem_ld32(tO + q4 * 32, o);
+                tmem_ld32(tO + q2 * 32, o);
 #pragma unroll
                 for (int j = 0; j < 32; ++j) o[j] *= alpha;
-                tmem_st32(tO + q4 * 32, o);
+                tmem_st32(tO + q2 * 32, o);
             }
             asm volatile("tcgen05.wait::st.sync.aligned;\n" ::: "memory");
         }
@@ -383,29 +402,30 @@ tree_attn_umma_kernel(const Args a)
     // Every lane of every warp takes part in the tensor-memory loads (they are warp-collective);
     // only the stores to global memory depend on whether the lane's row exists.
     if (failed && tid == 0) fspad_report(a.status, FSPAD_ERR_TIMEOUT);
+    s_mx[half][row] = l_part;
     {
         const bool store = row_ok && !failed;
-        float *po = a.part_o + (prow * M + (row_ok ? gr : 0)) * D;
+        float *po = a.part_o + (prow * M + (row_ok ? gr : 0)) * D + half * 64;
 #pragma unroll
-        for (int q4 = 0; q4 < 4; ++q4) {
+        for (int q2 = 0; q2 < 2; ++q2) {
             float o[32];
-            tmem_ld32(tO + q4 * 32, o);
+            tmem_ld32(tO + q2 * 32, o);
             if (store) {
 #pragma unroll
                 for (int j = 0; j < 32; j += 4)
-                    *reinterpret_cast<float4 *>(po + q4 * 32 + j) = make_float4(o[j], o[j + 1], o[j + 2], o[j + 3]);
+                    *reinterpret_cast<float4 *>(po + q2 * 32 + j) = make_float4(o[j], o[j + 1], o[j + 2], o[j + 3]);
             }
         }
-        if (store) {
+        cp_async_wait<0>();
+        tc_fence_before();
+        __syncthreads();
+        if (store && half == 0) {
             float *ml = a.part_ml + (prow * M + gr) * 2;
             ml[0] = m_run;
-            ml[1] = l_run;
+            ml[1] = s_mx[0][row] + s_mx[1][row];
         }
     }
-    cp_async_wait<0>();
-    tc_fence_before();
-    __syncthreads();
-    if (warp == 0) {
+    if (warp == 1) {
         __syncwarp();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" :: "r"(tmem), "r"(TMEM_COLS) : "memory");
     }
