@@ -81,8 +81,7 @@ int fspad_create(const fspad_config *cfg, fspad_ctx **out)
     int max_splits = 1;
     for (int n = 1; n <= cfg->max_nodes; ++n)
         for (int b = 1; b <= cfg->max_batch; ++b) {
-            const int s1 = fspad_attn_splits(ctx, n, b), s2 = fspad_attn_umma_splits(ctx, n, b);
-            const int s = s1 > s2 ? s1 : s2;
+            const int s = fspad_attn_umma_splits(ctx, n, b);
             const size_t rows = (size_t)b * cfg->n_kv_heads * s * n * G;
             if (rows > part_rows) part_rows = rows;
             if (s > max_splits) max_splits = s;

@@ -196,7 +196,6 @@ cudaError_t fspad_launch_tree_attn(fspad_ctx *ctx, const fspad_bf16 *q, const fs
 cudaError_t fspad_launch_tree_scatter(fspad_ctx *ctx, fspad_bf16 *cache, const fspad_bf16 *tk,
                                       const fspad_bf16 *tv, const int *prefix_len, int N, int B,
                                       cudaStream_t st);
-int fspad_attn_splits(const fspad_ctx *ctx, int N, int B);
 int fspad_attn_umma_splits(const fspad_ctx *ctx, int N, int B);
 cudaError_t fspad_launch_attn_umma_split(fspad_ctx *ctx, const fspad_bf16 *q, const fspad_bf16 *kc,
                                          const fspad_bf16 *vc, const fspad_bf16 *tk, const fspad_bf16 *tv,
