@@ -19,12 +19,7 @@ struct fspad_ctx {
 
     int *d_status;            // first device-detected error (0 = none)
 
-    // split-KV attention partials
-    int attn_max_splits;
-    int attn_attr_done;       // dynamic shared-memory limit raised for the attention kernels
-    float *part_o;            // [batch][Hkv][splits][M][d]
-    float *part_ml;           // [batch][Hkv][splits][M][2]  (running max in log2 units, sum)
-    int *attn_counter;        // [batch][Hkv][row tiles] arrivals of the key ranges, zero between calls
+    int attn_attr_done;       // dynamic shared-memory limit raised for the attention kernel
 
     // per-node vocabulary scan
     int stats_slots;          // partial slots per row in st_part

@@ -13,15 +13,21 @@
 // tcgen05.mma with V read directly in its [key][d] layout (MN-major operand).
 // O stays in tensor memory across chunks and is rescaled there when the running
 // maximum moves.  K/V chunks are double buffered with 16-byte asynchronous
-// copies into the swizzled layout the matrix descriptors expect.  Every key
-// range leaves a partial (unnormalised O row, running maximum, sum) in scratch;
-// the CTA that finishes last for a (sequence, kv head, row tile) merges them by
-// log-sum-exp and writes bf16 (arrival counter, no second launch).
+// copies into the swizzled layout the matrix descriptors expect.  The key
+// ranges of one (sequence, kv head, row tile) form a thread-block cluster: each
+// CTA parks its partial (unnormalised O rows, running maxima, sums) in its own
+// shared memory and then merges a slice of the rows by log-sum-exp, reading the
+// peers' partials through distributed shared memory, and writes bf16.  No
+// partial ever goes to global memory and there is no second launch.
 //
 // Every wait on an mbarrier is bounded; on expiry the CTA records
 // FSPAD_ERR_TIMEOUT, skips the remaining tensor-core work, frees its tensor
 // memory and returns.
+#include <cooperative_groups.h>
+
 #include "common.cuh"
+
+namespace cg = cooperative_groups;
 
 namespace umma {
 
@@ -39,9 +45,7 @@ struct Args {
     const int *parent, *prefix_len;
     int N, Hq, Hkv, G, M, max_len, n_splits, mtiles;
     float scale_log2;
-    float *part_o, *part_ml;
     fspad_bf16 *out;
-    int *counter;          // [batch][Hkv][mtiles] arrivals, zero between calls
     int *status;
 };
 
@@ -176,7 +180,8 @@ __device__ __forceinline__ float ex2f(float x)
 // Two threads share a query row: thread (row, half) owns columns half*64 .. half*64+63 of the
 // row's scores, of its P row and of its O row.  Warps w and w+4 address the same 32 lanes of
 // tensor memory (a warp reaches the lane quarter given by its index modulo 4).
-__device__ __forceinline__ void run_split(const Args &a, unsigned char *smem_raw, int L, int c0, int c1)
+__device__ __forceinline__ void run_split(const Args &a, unsigned char *smem_raw, int L, int c0, int c1,
+                                          float *s_m, float *s_l)
 {
     __shared__ __align__(8) unsigned long long s_bar[2];     // [0]: S ready, [1]: O updated
     __shared__ uint32_t s_tmem;
@@ -187,7 +192,6 @@ __device__ __forceinline__ void run_split(const Args &a, unsigned char *smem_raw
 
     const int tid = threadIdx.x, warp = tid >> 5;
     const int row = tid & (BM - 1), half = tid >> 7;
-    const int split = blockIdx.x;
     const int g = blockIdx.y / a.mtiles, mt = blockIdx.y % a.mtiles;
     const int b = blockIdx.z;
     const int N = a.N, G = a.G, M = a.M;
@@ -195,8 +199,6 @@ __device__ __forceinline__ void run_split(const Args &a, unsigned char *smem_raw
     const int gr = mt * BM + row;                 // this thread's row among the kv head's M rows
     const bool row_ok = gr < M;
     const int node = row_ok ? gr / G : 0;
-    const size_t prow = ((size_t)b * a.Hkv + g) * a.n_splits + split;
-
     // 1024-byte aligned tiles: Q | K0 | K1 | V0 | V1 | P
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t sQ = base, sK = base + TILE, sV = base + 3 * TILE, sP = base + 5 * TILE;
@@ -385,31 +387,30 @@ __device__ __forceinline__ void run_split(const Args &a, unsigned char *smem_raw
         cp_async_commit();
     }
 
-    // ---- publish the partial: unnormalised O row, running max and sum ----
-    // Every lane of every warp takes part in the tensor-memory loads (they are warp-collective);
-    // only the stores to global memory depend on whether the lane's row exists.
+    // ---- park the partial in shared memory: unnormalised O row (the K buffers are free now),
+    // running maximum and sum.  Every lane of every warp takes part in the tensor-memory loads
+    // (they are warp-collective).  Row r, 16-byte group c sits at group c ^ (r & 31): lanes of a
+    // warp hold different rows, so their stores spread over all banks.
     if (failed && tid == 0) fspad_report(a.status, FSPAD_ERR_TIMEOUT);
     s_mx[half][row] = l_part;
     {
-        const bool store = row_ok && !failed;
-        float *po = a.part_o + (prow * M + (row_ok ? gr : 0)) * D + half * 64;
+        float4 *so = reinterpret_cast<float4 *>(smem_raw + (base - smem_u32(smem_raw)) + TILE);
 #pragma unroll
         for (int q2 = 0; q2 < 2; ++q2) {
             float o[32];
             tmem_ld32(tO + q2 * 32, o);
-            if (store) {
 #pragma unroll
-                for (int j = 0; j < 32; j += 4)
-                    *reinterpret_cast<float4 *>(po + q2 * 32 + j) = make_float4(o[j], o[j + 1], o[j + 2], o[j + 3]);
+            for (int j = 0; j < 32; j += 4) {
+                const int c4 = half * 16 + q2 * 8 + (j >> 2);
+                so[row * 32 + (c4 ^ (row & 31))] = make_float4(o[j], o[j + 1], o[j + 2], o[j + 3]);
             }
         }
         cp_async_wait<0>();
         tc_fence_before();
         __syncthreads();
-        if (store && half == 0) {
-            float *ml = a.part_ml + (prow * M + gr) * 2;
-            ml[0] = m_run;
-            ml[1] = s_mx[0][row] + s_mx[1][row];
+        if (half == 0) {
+            s_m[row] = (row_ok && !failed) ? m_run : -INFINITY;
+            s_l[row] = s_mx[0][row] + s_mx[1][row];
         }
     }
     if (warp == 1) {
@@ -419,63 +420,15 @@ __device__ __forceinline__ void run_split(const Args &a, unsigned char *smem_raw
 }
 
 
-// Merge the partials of one output row by log-sum-exp and write it as bf16 (one warp).
-__device__ __forceinline__ void combine_row(const Args &a, int b, int g, int gr, int lane)
-{
-    const size_t pbase = ((size_t)b * a.Hkv + g) * a.n_splits;
-    const int ns = a.n_splits, M = a.M;
-    // all (max, sum) pairs of the row are fetched at once, two key ranges per lane (n_splits <= 64)
-    float m0 = -INFINITY, l0 = 0.f, m1 = -INFINITY, l1 = 0.f;
-    if (lane < ns) {
-        const float2 t = __ldcg(reinterpret_cast<const float2 *>(a.part_ml + ((pbase + lane) * M + gr) * 2));
-        m0 = t.x; l0 = t.y;
-    }
-    if (lane + 32 < ns) {
-        const float2 t = __ldcg(reinterpret_cast<const float2 *>(a.part_ml + ((pbase + lane + 32) * M + gr) * 2));
-        m1 = t.x; l1 = t.y;
-    }
-    float mmax = fmaxf(m0, m1);
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) mmax = fmaxf(mmax, __shfl_xor_sync(0xffffffffu, mmax, off));
-    const float w0 = (m0 == -INFINITY) ? 0.f : ex2f(m0 - mmax);
-    const float w1 = (m1 == -INFINITY) ? 0.f : ex2f(m1 - mmax);
-    float denom = w0 * l0 + w1 * l1;
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) denom += __shfl_xor_sync(0xffffffffu, denom, off);
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int s0 = 0; s0 < ns; s0 += 4) {
-        float4 v[4];
-        float w[4];
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            const int sidx = s0 + u;
-            const float wa = __shfl_sync(0xffffffffu, w0, sidx & 31), wb = __shfl_sync(0xffffffffu, w1, sidx & 31);
-            w[u] = (sidx < ns) ? ((sidx < 32) ? wa : wb) : 0.f;
-            v[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (w[u] != 0.f)
-                v[u] = __ldcg(reinterpret_cast<const float4 *>(a.part_o + ((pbase + sidx) * M + gr) * D + lane * 4));
-        }
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            acc.x += w[u] * v[u].x; acc.y += w[u] * v[u].y; acc.z += w[u] * v[u].z; acc.w += w[u] * v[u].w;
-        }
-    }
-    const float inv = denom > 0.f ? 1.f / denom : 0.f;
-    const int node = gr / a.G, hh = gr % a.G;
-    fspad_bf16 *dst = a.out + (((size_t)b * a.N + node) * a.Hq + g * a.G + hh) * D + lane * 4;
-    uint2 pk;
-    pk.x = pack_bf16(acc.x * inv, acc.y * inv);
-    pk.y = pack_bf16(acc.z * inv, acc.w * inv);
-    *reinterpret_cast<uint2 *>(dst) = pk;
-}
-
 __global__ void __launch_bounds__(NT, 1)
 tree_attn_kernel(const Args a)
 {
     extern __shared__ unsigned char smem_raw[];
-    __shared__ int s_last;
+    __shared__ float s_m[BM], s_l[BM];            // this CTA's running maxima (base 2) and sums
+    cg::cluster_group cluster = cg::this_cluster();
+    const int S = (int)cluster.num_blocks();      // key ranges = CTAs of the cluster
+    const int rank = (int)cluster.block_rank();
     const int tid = threadIdx.x;
-    const int split = blockIdx.x;
     const int g = blockIdx.y / a.mtiles, mt = blockIdx.y % a.mtiles;
     const int b = blockIdx.z;
 
@@ -486,49 +439,76 @@ tree_attn_kernel(const Args a)
     }
     // key chunks are dealt out as evenly as possible: range s gets chunks [s*n/S, (s+1)*n/S)
     const int n_chunks = (L + a.N + BK - 1) / BK;
-    const int c0 = (int)(((long long)split * n_chunks) / a.n_splits);
-    const int c1 = (int)(((long long)(split + 1) * n_chunks) / a.n_splits);
+    const int c0 = (int)(((long long)rank * n_chunks) / S);
+    const int c1 = (int)(((long long)(rank + 1) * n_chunks) / S);
     if (c0 < c1) {
-        run_split(a, smem_raw, L, c0, c1);
-    } else {
-        // no chunk for this range: an empty partial
-        const int gr = mt * BM + (tid & (BM - 1));
-        if (gr < a.M && tid < BM) {
-            float *ml = a.part_ml + ((((size_t)b * a.Hkv + g) * a.n_splits + split) * a.M + gr) * 2;
-            ml[0] = -INFINITY;
-            ml[1] = 0.f;
-        }
+        run_split(a, smem_raw, L, c0, c1, s_m, s_l);
+    } else if (tid < BM) {                        // no chunk for this range: an empty partial
+        s_m[tid] = -INFINITY;
+        s_l[tid] = 0.f;
     }
 
-    // ---- the last CTA to arrive for this (sequence, kv head, row tile) merges the partials ----
-    __threadfence();
-    __syncthreads();
-    int *cnt = a.counter + ((size_t)b * a.Hkv + g) * a.mtiles + mt;
-    if (tid == 0) s_last = (atomicAdd(cnt, 1) == a.n_splits - 1);
-    __syncthreads();
-    if (!s_last) return;
-    __threadfence();
-    const int lane = tid & 31;
-    for (int r = tid >> 5; r < BM; r += NT / 32) {
+    // ---- merge across the cluster: this CTA finishes rows rank*BM/S .. (rank+1)*BM/S - 1 ----
+    cluster.sync();
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const float4 *so = reinterpret_cast<const float4 *>(smem_raw + (base - smem_u32(smem_raw)) + TILE);
+    const int rows_per = BM / S;                  // S is a power of two <= 8
+    const int c = tid & 15;                       // eight output columns: 16-byte groups 2c, 2c+1
+    for (int rl = tid >> 4; rl < rows_per; rl += NT / 16) {
+        const int r = rank * rows_per + rl;
         const int gr = mt * BM + r;
-        if (gr < a.M) combine_row(a, b, g, gr, lane);
+        if (gr >= a.M) continue;
+        float mp[8], lp[8];
+        float mmax = -INFINITY;
+#pragma unroll
+        for (int p = 0; p < 8; ++p) {
+            mp[p] = -INFINITY; lp[p] = 0.f;
+            if (p < S) {
+                mp[p] = *cluster.map_shared_rank(&s_m[r], p);
+                lp[p] = *cluster.map_shared_rank(&s_l[r], p);
+            }
+            mmax = fmaxf(mmax, mp[p]);
+        }
+        float denom = 0.f;
+        float4 acc0 = make_float4(0.f, 0.f, 0.f, 0.f), acc1 = acc0;
+#pragma unroll
+        for (int p = 0; p < 8; ++p) {
+            if (p < S && mp[p] != -INFINITY) {
+                const float w = ex2f(mp[p] - mmax);
+                denom += w * lp[p];
+                const float4 *peer = cluster.map_shared_rank(so, p);
+                const float4 v0 = peer[r * 32 + ((2 * c) ^ (r & 31))];
+                const float4 v1 = peer[r * 32 + ((2 * c + 1) ^ (r & 31))];
+                acc0.x += w * v0.x; acc0.y += w * v0.y; acc0.z += w * v0.z; acc0.w += w * v0.w;
+                acc1.x += w * v1.x; acc1.y += w * v1.y; acc1.z += w * v1.z; acc1.w += w * v1.w;
+            }
+        }
+        const float inv = denom > 0.f ? 1.f / denom : 0.f;
+        const int node = gr / a.G, hh = gr % a.G;
+        fspad_bf16 *dst = a.out + (((size_t)b * a.N + node) * a.Hq + g * a.G + hh) * D + c * 8;
+        uint4 pk;
+        pk.x = pack_bf16(acc0.x * inv, acc0.y * inv);
+        pk.y = pack_bf16(acc0.z * inv, acc0.w * inv);
+        pk.z = pack_bf16(acc1.x * inv, acc1.y * inv);
+        pk.w = pack_bf16(acc1.z * inv, acc1.w * inv);
+        *reinterpret_cast<uint4 *>(dst) = pk;
     }
-    if (tid == 0) *cnt = 0;                       // ready for the next call
+    cluster.sync();                               // nobody leaves while a peer may still read its partial
 }
 
 }  // namespace umma
 
 int fspad_attn_splits(const fspad_ctx *ctx, int N, int B)
 {
+    // key ranges per (sequence, kv head, row tile) = CTAs of one cluster: the largest power of
+    // two (at most 8, the portable cluster size) that keeps the grid within one wave of the SMs
     const int G = ctx->cfg.n_q_heads / ctx->cfg.n_kv_heads;
     const int mtiles = (N * G + umma::BM - 1) / umma::BM;
     const long long base = (long long)B * ctx->cfg.n_kv_heads * mtiles;
-    long long s = ctx->sm_count / base;           // one CTA per SM, never a partial second wave
     const int max_chunks = (ctx->cfg.max_len + umma::BK - 1) / umma::BK;
-    if (s > max_chunks) s = max_chunks;
-    if (s > 64) s = 64;
-    if (s < 1) s = 1;
-    return (int)s;
+    int s = 1;
+    while (s < 8 && 2 * s * base <= ctx->sm_count && 2 * s <= max_chunks) s *= 2;
+    return s;
 }
 
 cudaError_t fspad_launch_tree_attn(fspad_ctx *ctx, const fspad_bf16 *q, const fspad_bf16 *kc,
@@ -544,7 +524,7 @@ cudaError_t fspad_launch_tree_attn(fspad_ctx *ctx, const fspad_bf16 *q, const fs
     a.M = N * a.G; a.max_len = c.max_len; a.n_splits = fspad_attn_splits(ctx, N, B);
     a.mtiles = (a.M + umma::BM - 1) / umma::BM;
     a.scale_log2 = ctx->scale * 1.4426950408889634f;
-    a.part_o = ctx->part_o; a.part_ml = ctx->part_ml; a.out = out; a.counter = ctx->attn_counter;
+    a.out = out;
     a.status = ctx->d_status;
     if (!ctx->attn_attr_done) {
         cudaError_t e = cudaFuncSetAttribute(umma::tree_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -552,8 +532,15 @@ cudaError_t fspad_launch_tree_attn(fspad_ctx *ctx, const fspad_bf16 *q, const fs
         if (e != cudaSuccess) return e;
         ctx->attn_attr_done = 1;
     }
-    dim3 grid(a.n_splits, c.n_kv_heads * a.mtiles, B);
-    umma::tree_attn_kernel<<<grid, umma::NT, umma::SMEM_BYTES, st>>>(a);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(a.n_splits, c.n_kv_heads * a.mtiles, B);
+    cfg.blockDim = dim3(umma::NT);
+    cfg.dynamicSmemBytes = umma::SMEM_BYTES;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = a.n_splits; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
     ctx->launches++;
-    return cudaGetLastError();
+    return cudaLaunchKernelEx(&cfg, umma::tree_attn_kernel, a);
 }
