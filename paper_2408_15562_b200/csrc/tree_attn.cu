@@ -16,8 +16,9 @@
 // copies into the swizzled layout the matrix descriptors expect.  The key
 // ranges of one (sequence, kv head, row tile) form a thread-block cluster: each
 // CTA parks its partial (unnormalised O rows, running maxima, sums) in its own
-// shared memory and then merges a slice of the rows by log-sum-exp, reading the
-// peers' partials through distributed shared memory, and writes bf16.  No
+// shared memory, sends each row to the CTA that finishes it (remote stores over
+// distributed shared memory), merges its slice of the rows by log-sum-exp from
+// local memory and writes bf16.  No
 // partial ever goes to global memory and there is no second launch.
 //
 // Every wait on an mbarrier is bounded; on expiry the CTA records
@@ -425,6 +426,7 @@ tree_attn_kernel(const Args a)
 {
     extern __shared__ unsigned char smem_raw[];
     __shared__ float s_m[BM], s_l[BM];            // this CTA's running maxima (base 2) and sums
+    __shared__ float r_m[8][BM], r_l[8][BM];      // received from the peers: [source CTA][row of my slice]
     cg::cluster_group cluster = cg::this_cluster();
     const int S = (int)cluster.num_blocks();      // key ranges = CTAs of the cluster
     const int rank = (int)cluster.block_rank();
@@ -448,37 +450,49 @@ tree_attn_kernel(const Args a)
         s_l[tid] = 0.f;
     }
 
-    // ---- merge across the cluster: this CTA finishes rows rank*BM/S .. (rank+1)*BM/S - 1 ----
+    // ---- merge across the cluster: this CTA finishes rows rank*rows_per .. ----
+    // After the first barrier every pipeline of the cluster has finished, so each CTA may send
+    // the rows of its partial to the CTA that finishes them (remote shared-memory stores into
+    // the peers' idle V buffers); after the second barrier the merge reads local memory only.
     cluster.sync();
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    const float4 *so = reinterpret_cast<const float4 *>(smem_raw + (base - smem_u32(smem_raw)) + TILE);
-    const int rows_per = BM / S;                  // S is a power of two <= 8
+    unsigned char *tiles = smem_raw + (base - smem_u32(smem_raw));
+    const float4 *so = reinterpret_cast<const float4 *>(tiles + TILE);        // own partial (K buffers)
+    float4 *rv = reinterpret_cast<float4 *>(tiles + 3 * TILE);                // received rows (V buffers)
+    const int rows_per = (BM + S - 1) / S;        // 1 <= S <= 8
+    {
+        const int r = tid >> 1, h = tid & 1;      // row of the partial, half of its 32 16-byte groups
+        const int dst = r / rows_per, rl = r - dst * rows_per;
+        float4 *peer = cluster.map_shared_rank(rv, dst) + ((size_t)rank * rows_per + rl) * 32;
+#pragma unroll
+        for (int k = 0; k < 16; ++k) {
+            const int c4 = h * 16 + k;
+            peer[c4] = so[r * 32 + (c4 ^ (r & 31))];
+        }
+        if (h == 0) {
+            *cluster.map_shared_rank(&r_m[rank][rl], dst) = s_m[r];
+            *cluster.map_shared_rank(&r_l[rank][rl], dst) = s_l[r];
+        }
+    }
+    cluster.sync();
     const int c = tid & 15;                       // eight output columns: 16-byte groups 2c, 2c+1
     for (int rl = tid >> 4; rl < rows_per; rl += NT / 16) {
         const int r = rank * rows_per + rl;
         const int gr = mt * BM + r;
-        if (gr >= a.M) continue;
-        float mp[8], lp[8];
+        if (r >= BM || gr >= a.M) continue;
         float mmax = -INFINITY;
 #pragma unroll
-        for (int p = 0; p < 8; ++p) {
-            mp[p] = -INFINITY; lp[p] = 0.f;
-            if (p < S) {
-                mp[p] = *cluster.map_shared_rank(&s_m[r], p);
-                lp[p] = *cluster.map_shared_rank(&s_l[r], p);
-            }
-            mmax = fmaxf(mmax, mp[p]);
-        }
+        for (int p = 0; p < 8; ++p)
+            if (p < S) mmax = fmaxf(mmax, r_m[p][rl]);
         float denom = 0.f;
         float4 acc0 = make_float4(0.f, 0.f, 0.f, 0.f), acc1 = acc0;
 #pragma unroll
         for (int p = 0; p < 8; ++p) {
-            if (p < S && mp[p] != -INFINITY) {
-                const float w = ex2f(mp[p] - mmax);
-                denom += w * lp[p];
-                const float4 *peer = cluster.map_shared_rank(so, p);
-                const float4 v0 = peer[r * 32 + ((2 * c) ^ (r & 31))];
-                const float4 v1 = peer[r * 32 + ((2 * c + 1) ^ (r & 31))];
+            if (p < S && r_m[p][rl] != -INFINITY) {
+                const float w = ex2f(r_m[p][rl] - mmax);
+                denom += w * r_l[p][rl];
+                const float4 v0 = rv[((size_t)p * rows_per + rl) * 32 + 2 * c];
+                const float4 v1 = rv[((size_t)p * rows_per + rl) * 32 + 2 * c + 1];
                 acc0.x += w * v0.x; acc0.y += w * v0.y; acc0.z += w * v0.z; acc0.w += w * v0.w;
                 acc1.x += w * v1.x; acc1.y += w * v1.y; acc1.z += w * v1.z; acc1.w += w * v1.w;
             }
@@ -493,22 +507,48 @@ tree_attn_kernel(const Args a)
         pk.w = pack_bf16(acc1.z * inv, acc1.w * inv);
         *reinterpret_cast<uint4 *>(dst) = pk;
     }
-    cluster.sync();                               // nobody leaves while a peer may still read its partial
 }
 
 }  // namespace umma
 
-int fspad_attn_splits(const fspad_ctx *ctx, int N, int B)
+// How many clusters of `size` CTAs of the attention kernel the device can hold at once (cached).
+static int max_active_clusters(fspad_ctx *ctx, int size)
 {
-    // key ranges per (sequence, kv head, row tile) = CTAs of one cluster: the largest power of
-    // two (at most 8, the portable cluster size) that keeps the grid within one wave of the SMs
+    if (ctx->attn_max_clusters[size] == 0) {
+        cudaLaunchConfig_t probe = {};
+        probe.gridDim = dim3(size);
+        probe.blockDim = dim3(umma::NT);
+        probe.dynamicSmemBytes = umma::SMEM_BYTES;
+        cudaLaunchAttribute at[1];
+        at[0].id = cudaLaunchAttributeClusterDimension;
+        at[0].val.clusterDim.x = size; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+        probe.attrs = at; probe.numAttrs = 1;
+        int n = 0;
+        if (cudaOccupancyMaxActiveClusters(&n, umma::tree_attn_kernel, &probe) != cudaSuccess || n < 1) {
+            (void)cudaGetLastError();
+            n = -1;
+        }
+        ctx->attn_max_clusters[size] = n;
+    }
+    return ctx->attn_max_clusters[size];
+}
+
+// Key ranges per (sequence, kv head, row tile) = CTAs of one cluster (1..8, the portable sizes).
+// Among the sizes for which every cluster of the grid is resident at once, take the one that
+// leaves the fewest key chunks to the busiest CTA; the smallest such size on ties.
+int fspad_attn_splits(fspad_ctx *ctx, int N, int B)
+{
     const int G = ctx->cfg.n_q_heads / ctx->cfg.n_kv_heads;
     const int mtiles = (N * G + umma::BM - 1) / umma::BM;
     const long long base = (long long)B * ctx->cfg.n_kv_heads * mtiles;
     const int max_chunks = (ctx->cfg.max_len + umma::BK - 1) / umma::BK;
-    int s = 1;
-    while (s < 8 && 2 * s * base <= ctx->sm_count && 2 * s <= max_chunks) s *= 2;
-    return s;
+    int best = 1, best_cost = max_chunks;
+    for (int size = 2; size <= 8 && size <= max_chunks; ++size) {
+        if (base > max_active_clusters(ctx, size)) continue;
+        const int cost = (max_chunks + size - 1) / size;
+        if (cost < best_cost) { best = size; best_cost = cost; }
+    }
+    return best;
 }
 
 cudaError_t fspad_launch_tree_attn(fspad_ctx *ctx, const fspad_bf16 *q, const fspad_bf16 *kc,
@@ -521,7 +561,7 @@ cudaError_t fspad_launch_tree_attn(fspad_ctx *ctx, const fspad_bf16 *q, const fs
     umma::Args a;
     a.q = q; a.kc = kc; a.vc = vc; a.tk = tk; a.tv = tv; a.parent = parent; a.prefix_len = prefix_len;
     a.N = N; a.Hq = c.n_q_heads; a.Hkv = c.n_kv_heads; a.G = c.n_q_heads / c.n_kv_heads;
-    a.M = N * a.G; a.max_len = c.max_len; a.n_splits = fspad_attn_splits(ctx, N, B);
+    a.M = N * a.G; a.max_len = c.max_len;
     a.mtiles = (a.M + umma::BM - 1) / umma::BM;
     a.scale_log2 = ctx->scale * 1.4426950408889634f;
     a.out = out;
@@ -532,6 +572,7 @@ cudaError_t fspad_launch_tree_attn(fspad_ctx *ctx, const fspad_bf16 *q, const fs
         if (e != cudaSuccess) return e;
         ctx->attn_attr_done = 1;
     }
+    a.n_splits = fspad_attn_splits(ctx, N, B);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(a.n_splits, c.n_kv_heads * a.mtiles, B);
     cfg.blockDim = dim3(umma::NT);
