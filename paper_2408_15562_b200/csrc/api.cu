@@ -74,11 +74,25 @@ int fspad_create(const fspad_config *cfg, fspad_ctx **out)
         return FSPAD_ERR_CUDA;
     }
 
+    const int G = cfg->n_q_heads / cfg->n_kv_heads;
     const size_t B = (size_t)cfg->max_batch, Nmax = (size_t)cfg->max_nodes;
+    // split-KV partials: worst case over every (n_nodes, batch) a call may pass
+    size_t part_rows = 0;
+    int max_splits = 1;
+    for (int n = 1; n <= cfg->max_nodes; ++n)
+        for (int b = 1; b <= cfg->max_batch; ++b) {
+            const int s = fspad_attn_umma_splits(ctx, n, b);
+            const size_t rows = (size_t)b * cfg->n_kv_heads * s * n * G;
+            if (rows > part_rows) part_rows = rows;
+            if (s > max_splits) max_splits = s;
+        }
+    ctx->attn_max_splits = max_splits;
     const size_t rows = B * Nmax;
     ctx->stats_slots = 64;
 
     bool ok = dev_alloc(&ctx->d_status, 1);
+    ok = ok && dev_alloc(&ctx->part_o, part_rows * FSPAD_HEAD_DIM);
+    ok = ok && dev_alloc(&ctx->part_ml, part_rows * 2);
     ok = ok && dev_alloc(&ctx->st_part, rows * ctx->stats_slots);
     ok = ok && dev_alloc(&ctx->row_max, rows);
     ok = ok && dev_alloc(&ctx->row_sum, rows);
@@ -98,7 +112,7 @@ void fspad_destroy(fspad_ctx *ctx)
 {
     if (!ctx) return;
     cudaDeviceSynchronize();
-    void *ptrs[] = {ctx->d_status, ctx->st_part, ctx->row_max, ctx->row_sum, ctx->row_arg, ctx->h_q, ctx->h_tk,
+    void *ptrs[] = {ctx->d_status, ctx->part_o, ctx->part_ml, ctx->st_part, ctx->row_max, ctx->row_sum, ctx->row_arg, ctx->h_q, ctx->h_tk,
                     ctx->h_tv, ctx->h_out, ctx->h_parent, ctx->h_prefix, ctx->h_tokens, ctx->h_path,
                     ctx->h_nacc, ctx->h_bonus, ctx->h_newlen, ctx->h_logits, ctx->h_draft, ctx->h_temp,
                     ctx->h_unif};

@@ -19,8 +19,11 @@ struct fspad_ctx {
 
     int *d_status;            // first device-detected error (0 = none)
 
-    int attn_attr_done;       // dynamic shared-memory limit raised for the attention kernel
-    int attn_max_clusters[9]; // resident clusters of 1..8 CTAs, by size (0 = not queried, -1 = none)
+    // split-KV attention partials
+    int attn_max_splits;
+    int attn_attr_done;       // dynamic shared-memory limit raised for the attention kernels
+    float *part_o;            // [batch][Hkv][splits][M][d]
+    float *part_ml;           // [batch][Hkv][splits][M][2]  (running max in log2 units, sum)
 
     // per-node vocabulary scan
     int stats_slots;          // partial slots per row in st_part
@@ -193,4 +196,8 @@ cudaError_t fspad_launch_tree_attn(fspad_ctx *ctx, const fspad_bf16 *q, const fs
 cudaError_t fspad_launch_tree_scatter(fspad_ctx *ctx, fspad_bf16 *cache, const fspad_bf16 *tk,
                                       const fspad_bf16 *tv, const int *prefix_len, int N, int B,
                                       cudaStream_t st);
-int fspad_attn_splits(fspad_ctx *ctx, int N, int B);
+int fspad_attn_umma_splits(const fspad_ctx *ctx, int N, int B);
+cudaError_t fspad_launch_attn_umma_split(fspad_ctx *ctx, const fspad_bf16 *q, const fspad_bf16 *kc,
+                                         const fspad_bf16 *vc, const fspad_bf16 *tk, const fspad_bf16 *tv,
+                                         const int *parent, const int *prefix_len, int N, int B, int n_splits,
+                                         float scale_log2, cudaStream_t st);

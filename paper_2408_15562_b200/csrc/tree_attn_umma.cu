@@ -1,0 +1,473 @@
+// Tree-masked verify attention on the 5th-generation tensor cores (paper,
+// Section "Preliminaries": the target processes the flattened token tree under
+// the attention mask built from the tree).
+//
+// Split-KV flash-decode with tcgen05: all query rows that share a kv head (tree
+// node x GQA group member) form the M = 128 operand of one CTA; keys are
+// consumed in chunks of 128.  Per chunk: S = Q K^T is one chain of eight
+// tcgen05.mma (128 x 128 x 16, bf16 -> fp32) into tensor memory; two threads
+// share a query row, each reads 64 of its scores back with tcgen05.ld, applies
+// the ancestor mask (only on chunks that reach past the cached prefix) and the
+// softmax in registers (one shared-memory exchange of the row maximum), and writes P as bf16 into
+// a 128-byte-swizzled shared-memory tile; O += P V is a second chain of eight
+// tcgen05.mma with V read directly in its [key][d] layout (MN-major operand).
+// O stays in tensor memory across chunks and is rescaled there when the running
+// maximum moves.  K/V chunks are double buffered with 16-byte asynchronous
+// copies into the swizzled layout the matrix descriptors expect.  Per-split
+// partials are merged by the combine kernel.
+//
+// Every wait on an mbarrier is bounded; on expiry the CTA records
+// FSPAD_ERR_TIMEOUT, skips the remaining tensor-core work, frees its tensor
+// memory and returns.
+#include "common.cuh"
+
+namespace umma {
+
+constexpr int D = FSPAD_HEAD_DIM;      // 128
+constexpr int BM = 128;                // query rows per CTA
+constexpr int BK = 128;                // keys per chunk
+constexpr int NT = 256;                // threads per CTA: two per query row
+constexpr int HALF = 128 * 128;        // bytes of one [128 rows][64 bf16] half tile
+constexpr int TILE = 2 * HALF;         // bytes of one [128][128] bf16 tile
+constexpr int SMEM_BYTES = 6 * TILE + 1024;   // Q, K[2], V[2], P + alignment slack
+constexpr uint32_t TMEM_COLS = 256;    // S: columns 0..127, O: columns 128..255
+constexpr uint32_t WAIT_CAP = 200000;   // polls of a bounded mbarrier wait
+struct Args {
+    const fspad_bf16 *q, *kc, *vc, *tk, *tv;
+    const int *parent, *prefix_len;
+    int N, Hq, Hkv, G, M, max_len, n_splits, mtiles;
+    float scale_log2;
+    float *part_o, *part_ml;
+    int *status;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+// byte offset of 16-byte chunk c (0..15) of row r inside a [128][128] bf16 tile stored as two
+// 128-byte-swizzled halves (columns 0..63 | 64..127), each [128 rows][128 bytes]
+__device__ __forceinline__ uint32_t tile_off(int r, int c)
+{
+    return (uint32_t)((c >> 3) * HALF + r * 128 + (((c & 7) ^ (r & 7)) << 4));
+}
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src, bool valid)
+{
+    const int sz = valid ? 16 : 0;   // 0: destination zero-filled, source not read
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(src), "r"(sz));
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::); }
+template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N)); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory"); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}\n"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait (non-blocking test + short sleep, about 20 ms in all); false if the cap ran out.
+// Lane 0 polls and the warp takes its verdict through a full-mask shuffle, so every lane leaves
+// together: the warp-collective tensor-memory instructions that follow need a converged warp.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
+{
+    int ok = 0;
+    if ((threadIdx.x & 31) == 0) {
+        for (uint32_t i = 0; i < WAIT_CAP && !ok; ++i) {
+            ok = mbar_test(bar, parity) ? 1 : 0;
+            if (!ok) __nanosleep(40);
+        }
+    }
+    ok = __shfl_sync(0xffffffffu, ok, 0);
+    return ok != 0;
+}
+
+// shared-memory matrix descriptor, 128-byte swizzle, 8-row groups 1024 bytes apart
+__device__ __forceinline__ uint64_t make_desc(uint32_t addr, uint32_t lbo_bytes)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((addr >> 4) & 0x3FFF);
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFF) << 16;
+    d |= (uint64_t)((1024u >> 4) & 0x3FFF) << 32;
+    d |= (uint64_t)1 << 46;                 // descriptor version
+    d |= (uint64_t)2 << 61;                 // SWIZZLE_128B
+    return d;
+}
+// instruction descriptor: bf16 x bf16 -> fp32, M = 128, N = 128
+__device__ __forceinline__ uint32_t make_idesc(bool b_mn_major)
+{
+    uint32_t d = 0;
+    d |= 1u << 4;                           // accumulator fp32
+    d |= 1u << 7;                           // A bf16
+    d |= 1u << 10;                          // B bf16
+    d |= (b_mn_major ? 1u : 0u) << 16;      // B major: 0 = K, 1 = MN
+    d |= (128u >> 3) << 17;                 // N
+    d |= (128u >> 4) << 24;                 // M
+    return d;
+}
+__device__ __forceinline__ void mma_f16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                        uint32_t accumulate)
+{
+    const uint32_t zero = 0;                // no output lane is disabled
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %6, %7, %8}, p;\n\t}\n"
+                 :: "r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(zero), "r"(zero),
+                    "r"(zero), "r"(zero) : "memory");
+}
+__device__ __forceinline__ void mma_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t addr, float (&v)[32])
+{
+    uint32_t r[32];
+    __syncwarp();
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+                 "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+                 "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];\n"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                   "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+                   "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+                   "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+                 : "r"(addr) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void tmem_st32(uint32_t addr, const float (&v)[32])
+{
+    __syncwarp();
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+                 "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
+                 "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};\n"
+                 :: "r"(addr),
+                    "r"(__float_as_uint(v[0])), "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])), "r"(__float_as_uint(v[3])),
+                    "r"(__float_as_uint(v[4])), "r"(__float_as_uint(v[5])), "r"(__float_as_uint(v[6])), "r"(__float_as_uint(v[7])),
+                    "r"(__float_as_uint(v[8])), "r"(__float_as_uint(v[9])), "r"(__float_as_uint(v[10])), "r"(__float_as_uint(v[11])),
+                    "r"(__float_as_uint(v[12])), "r"(__float_as_uint(v[13])), "r"(__float_as_uint(v[14])), "r"(__float_as_uint(v[15])),
+                    "r"(__float_as_uint(v[16])), "r"(__float_as_uint(v[17])), "r"(__float_as_uint(v[18])), "r"(__float_as_uint(v[19])),
+                    "r"(__float_as_uint(v[20])), "r"(__float_as_uint(v[21])), "r"(__float_as_uint(v[22])), "r"(__float_as_uint(v[23])),
+                    "r"(__float_as_uint(v[24])), "r"(__float_as_uint(v[25])), "r"(__float_as_uint(v[26])), "r"(__float_as_uint(v[27])),
+                    "r"(__float_as_uint(v[28])), "r"(__float_as_uint(v[29])), "r"(__float_as_uint(v[30])), "r"(__float_as_uint(v[31]))
+                 : "memory");
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
+{
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t *>(&v);
+}
+
+__device__ __forceinline__ float ex2f(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// Two threads share a query row: thread (row, half) owns columns half*64 .. half*64+63 of the
+// row's scores, of its P row and of its O row.  Warps w and w+4 address the same 32 lanes of
+// tensor memory (a warp reaches the lane quarter given by its index modulo 4).
+__global__ void __launch_bounds__(NT, 1)
+tree_attn_umma_kernel(const Args a)
+{
+    extern __shared__ unsigned char smem_raw[];
+    __shared__ __align__(8) unsigned long long s_bar[2];     // [0]: S ready, [1]: O updated
+    __shared__ uint32_t s_tmem;
+    __shared__ int s_fail;
+    __shared__ int s_par[FSPAD_MAX_NODES];
+    __shared__ unsigned long long s_anc[FSPAD_MAX_NODES];
+    __shared__ float s_mx[2][BM];                            // per-half row maxima / sums exchange
+
+    const int tid = threadIdx.x, warp = tid >> 5;
+    const int row = tid & (BM - 1), half = tid >> 7;
+    const int split = blockIdx.x;
+    const int g = blockIdx.y / a.mtiles, mt = blockIdx.y % a.mtiles;
+    const int b = blockIdx.z;
+    const int N = a.N, G = a.G, M = a.M;
+
+    int L = a.prefix_len[b];
+    if (L < 0 || L + N > a.max_len) {
+        if (tid == 0) fspad_report(a.status, FSPAD_ERR_RANGE);
+        L = max(0, min(L, a.max_len - N));
+    }
+    const int Ltot = L + N;
+    const int n_chunks = (Ltot + BK - 1) / BK;
+    // key chunks are dealt out as evenly as possible: range s gets chunks [s*n/S, (s+1)*n/S)
+    const int c0 = (int)(((long long)split * n_chunks) / a.n_splits);
+    const int c1 = (int)(((long long)(split + 1) * n_chunks) / a.n_splits);
+
+    const int gr = mt * BM + row;                 // this thread's row among the kv head's M rows
+    const bool row_ok = gr < M;
+    const int node = row_ok ? gr / G : 0;
+    const size_t prow = ((size_t)b * a.Hkv + g) * a.n_splits + split;
+
+    if (c0 >= c1) {                               // nothing to do for this split: empty partial
+        if (row_ok && half == 0) { float *ml = a.part_ml + (prow * M + gr) * 2; ml[0] = -INFINITY; ml[1] = 0.f; }
+        return;
+    }
+
+    // 1024-byte aligned tiles: Q | K0 | K1 | V0 | V1 | P
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t sQ = base, sK = base + TILE, sV = base + 3 * TILE, sP = base + 5 * TILE;
+    const uint32_t barS = smem_u32(&s_bar[0]), barO = smem_u32(&s_bar[1]);
+
+    const fspad_bf16 *kcb = a.kc + ((size_t)b * a.Hkv + g) * (size_t)a.max_len * D;
+    const fspad_bf16 *vcb = a.vc + ((size_t)b * a.Hkv + g) * (size_t)a.max_len * D;
+    const fspad_bf16 *tkb = a.tk ? a.tk + ((size_t)b * a.Hkv + g) * (size_t)N * D : kcb + (size_t)L * D;
+    const fspad_bf16 *tvb = a.tv ? a.tv + ((size_t)b * a.Hkv + g) * (size_t)N * D : vcb + (size_t)L * D;
+
+    // ---- the copies go out first; everything else of the prologue hides under their latency ----
+    {
+        const int c = tid & 15;                   // 16-byte chunk of the row, fixed per thread
+        for (int r = tid >> 4; r < BM; r += NT / 16) {
+            const int grr = mt * BM + r;
+            const bool ok = grr < M;
+            const int nd = ok ? grr / G : 0, hh = ok ? grr % G : 0;
+            const fspad_bf16 *src = a.q + (((size_t)b * N + nd) * a.Hq + g * G + hh) * D + c * 8;
+            cp_async16(sQ + tile_off(r, c), src, ok);
+        }
+    }
+    auto load_chunk = [&](int ch, int buf) {
+        const uint32_t dK = sK + buf * TILE, dV = sV + buf * TILE;
+        const int c = tid & 15;
+        for (int r = tid >> 4; r < BK; r += NT / 16) {
+            const int key = ch * BK + r;
+            const bool ok = key < Ltot;
+            const fspad_bf16 *ks = kcb, *vs = vcb;
+            if (ok) {
+                if (key < L) { ks = kcb + (size_t)key * D + c * 8; vs = vcb + (size_t)key * D + c * 8; }
+                else { ks = tkb + (size_t)(key - L) * D + c * 8; vs = tvb + (size_t)(key - L) * D + c * 8; }
+            }
+            cp_async16(dK + tile_off(r, c), ks, ok);
+            cp_async16(dV + tile_off(r, c), vs, ok);
+        }
+    };
+    load_chunk(c0, 0);
+    cp_async_commit();
+    if (c0 + 1 < c1) load_chunk(c0 + 1, 1);
+    cp_async_commit();
+
+    // ---- tree -> ancestor-or-self masks (parents staged in shared memory, then walked there) ----
+    if (tid < N) s_par[tid] = a.parent[(size_t)b * N + tid];
+    if (tid == 0) {
+        mbar_init(barS, 1);
+        mbar_init(barO, 1);
+        s_fail = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+    }
+    if (warp == 1) {                              // one (converged) warp allocates the tensor memory
+        __syncwarp();
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n"
+                     :: "r"(smem_u32(&s_tmem)), "r"(TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
+    }
+    __syncthreads();
+    if (tid < N) {
+        unsigned long long mask = 0ull;
+        int cur = tid;
+        bool bad = false;
+        for (int step = 0; step <= N && cur >= 0; ++step) {
+            mask |= 1ull << cur;
+            const int p = s_par[cur];
+            if (cur == 0) { bad |= (p != -1); break; }
+            if (p < 0 || p >= cur) { bad = true; break; }
+            cur = p;
+        }
+        if (bad) fspad_report(a.status, FSPAD_ERR_BAD_TREE);
+        s_anc[tid] = mask;
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = s_tmem;
+    const uint32_t lanes = (uint32_t)((row >> 5) * 32) << 16;
+    const uint32_t tS = tmem + lanes + (uint32_t)(half * 64);            // this thread's 64 score columns
+    const uint32_t tO = tmem + lanes + 128u + (uint32_t)(half * 64);     // and its 64 output columns
+    const uint32_t idesc_s = make_idesc(false), idesc_o = make_idesc(true);
+    const unsigned long long anc = s_anc[node];
+    const float scale = a.scale_log2;
+
+    float m_run = -INFINITY, l_part = 0.f;       // row maximum (shared by both halves), this half's sum
+    uint32_t phS = 0, phO = 0;
+    bool failed = false;
+
+    for (int ch = c0; ch < c1; ++ch) {
+        const int buf = (ch - c0) & 1;
+        // this chunk's copies have landed (the younger group, if any, may still be in flight)
+        if (ch + 1 < c1) cp_async_wait<1>(); else cp_async_wait<0>();
+        fence_async_smem();
+        __syncthreads();
+        if (tid == 0 && !failed) {
+            tc_fence_after();
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks) {     // K = 16 per instruction over d = 128
+                const uint32_t koff = (ks >> 2) * HALF + (ks & 3) * 32;
+                mma_f16(tmem, make_desc(sQ + koff, 16), make_desc(sK + buf * TILE + koff, 16), idesc_s, ks > 0);
+            }
+            mma_commit(barS);
+        }
+        if (!failed && !mbar_wait(barS, phS)) { failed = true; s_fail = 1; }
+        phS ^= 1;
+        tc_fence_after();
+
+        // ---- this thread's 64 scores: mask, row maximum (exchanged with the other half) ----
+        float sc[2][32];
+        tmem_ld32(tS, sc[0]);
+        tmem_ld32(tS + 32, sc[1]);
+        if ((ch + 1) * BK > L) {                 // only chunks that reach past the cached prefix
+#pragma unroll
+            for (int q2 = 0; q2 < 2; ++q2)
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    const int key = ch * BK + half * 64 + q2 * 32 + j;
+                    if (key >= L) {
+                        const bool ok = (key < Ltot) && ((anc >> (key - L)) & 1ull);
+                        if (!ok) sc[q2][j] = -INFINITY;
+                    }
+                }
+        }
+        float mx = -INFINITY;
+#pragma unroll
+        for (int q2 = 0; q2 < 2; ++q2)
+#pragma unroll
+            for (int j = 0; j < 32; ++j) mx = fmaxf(mx, sc[q2][j]);
+        s_mx[half][row] = mx;
+        __syncthreads();
+        mx = fmaxf(mx, s_mx[half ^ 1][row]);
+        const float m_new = fmaxf(m_run, mx * scale);
+        const float m_safe = (m_new == -INFINITY) ? 0.f : m_new;
+        const float alpha = ex2f(m_run - m_safe);
+        float rs = 0.f;
+#pragma unroll
+        for (int q2 = 0; q2 < 2; ++q2) {
+#pragma unroll
+            for (int c8 = 0; c8 < 4; ++c8) {     // 8 keys = one 16-byte chunk of the P row
+                uint32_t w[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const float p0 = ex2f(fmaf(sc[q2][c8 * 8 + 2 * e], scale, -m_safe));
+                    const float p1 = ex2f(fmaf(sc[q2][c8 * 8 + 2 * e + 1], scale, -m_safe));
+                    rs += p0 + p1;
+                    w[e] = pack_bf16(p0, p1);
+                }
+                const int c = half * 8 + q2 * 4 + c8;   // chunk 0..15 of this row of P
+                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};\n"
+                             :: "r"(sP + tile_off(row, c)), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]) : "memory");
+            }
+        }
+        l_part = l_part * alpha + rs;
+        m_run = m_new;
+
+        // ---- rescale this thread's half of the O row when a previous chunk has contributed ----
+        if (ch > c0) {
+#pragma unroll
+            for (int q2 = 0; q2 < 2; ++q2) {
+                float o[32];
+                tmem_ld32(tO + q2 * 32, o);
+#pragma unroll
+                for (int j = 0; j < 32; ++j) o[j] *= alpha;
+                tmem_st32(tO + q2 * 32, o);
+            }
+            asm volatile("tcgen05.wait::st.sync.aligned;\n" ::: "memory");
+        }
+        fence_async_smem();
+        tc_fence_before();
+        __syncthreads();
+        if (tid == 0 && !failed) {
+            tc_fence_after();
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks) {     // K = 16 keys per instruction over the chunk's 128 keys
+                const uint64_t da = make_desc(sP + (ks >> 2) * HALF + (ks & 3) * 32, 16);
+                // V as an MN-major operand: d is contiguous, the two 64-wide halves are HALF bytes apart
+                const uint64_t db = make_desc(sV + buf * TILE + ks * 16 * 128, HALF);
+                mma_f16(tmem + 128u, da, db, idesc_o, (ch > c0) || (ks > 0));
+            }
+            mma_commit(barO);
+        }
+        // P, this K/V buffer and the S columns are free again once these products have completed
+        if (!failed && !mbar_wait(barO, phO)) { failed = true; s_fail = 1; }
+        phO ^= 1;
+        tc_fence_after();
+        __syncthreads();
+        failed = failed || (s_fail != 0);
+        if (ch + 2 < c1) load_chunk(ch + 2, buf);
+        cp_async_commit();
+    }
+
+    // ---- publish the partial: unnormalised O row, running max and sum ----
+    // Every lane of every warp takes part in the tensor-memory loads (they are warp-collective);
+    // only the stores to global memory depend on whether the lane's row exists.
+    if (failed && tid == 0) fspad_report(a.status, FSPAD_ERR_TIMEOUT);
+    s_mx[half][row] = l_part;
+    {
+        const bool store = row_ok && !failed;
+        float *po = a.part_o + (prow * M + (row_ok ? gr : 0)) * D + half * 64;
+#pragma unroll
+        for (int q2 = 0; q2 < 2; ++q2) {
+            float o[32];
+            tmem_ld32(tO + q2 * 32, o);
+            if (store) {
+#pragma unroll
+                for (int j = 0; j < 32; j += 4)
+                    *reinterpret_cast<float4 *>(po + q2 * 32 + j) = make_float4(o[j], o[j + 1], o[j + 2], o[j + 3]);
+            }
+        }
+        cp_async_wait<0>();
+        tc_fence_before();
+        __syncthreads();
+        if (store && half == 0) {
+            float *ml = a.part_ml + (prow * M + gr) * 2;
+            ml[0] = m_run;
+            ml[1] = s_mx[0][row] + s_mx[1][row];
+        }
+    }
+    if (warp == 1) {
+        __syncwarp();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" :: "r"(tmem), "r"(TMEM_COLS) : "memory");
+    }
+}
+
+}  // namespace umma
+
+int fspad_attn_umma_splits(const fspad_ctx *ctx, int N, int B)
+{
+    const int G = ctx->cfg.n_q_heads / ctx->cfg.n_kv_heads;
+    const int mtiles = (N * G + umma::BM - 1) / umma::BM;
+    const long long base = (long long)B * ctx->cfg.n_kv_heads * mtiles;
+    long long s = ctx->sm_count / base;           // one CTA per SM, never a partial second wave
+    const int max_chunks = (ctx->cfg.max_len + umma::BK - 1) / umma::BK;
+    if (s > max_chunks) s = max_chunks;
+    if (s > 64) s = 64;
+    if (s < 1) s = 1;
+    return (int)s;
+}
+
+cudaError_t fspad_launch_attn_umma_split(fspad_ctx *ctx, const fspad_bf16 *q, const fspad_bf16 *kc,
+                                         const fspad_bf16 *vc, const fspad_bf16 *tk, const fspad_bf16 *tv,
+                                         const int *parent, const int *prefix_len, int N, int B, int n_splits,
+                                         float scale_log2, cudaStream_t st)
+{
+    const fspad_config &c = ctx->cfg;
+    umma::Args a;
+    a.q = q; a.kc = kc; a.vc = vc; a.tk = tk; a.tv = tv; a.parent = parent; a.prefix_len = prefix_len;
+    a.N = N; a.Hq = c.n_q_heads; a.Hkv = c.n_kv_heads; a.G = c.n_q_heads / c.n_kv_heads;
+    a.M = N * a.G; a.max_len = c.max_len; a.n_splits = n_splits;
+    a.mtiles = (a.M + umma::BM - 1) / umma::BM;
+    a.scale_log2 = scale_log2;
+    a.part_o = ctx->part_o; a.part_ml = ctx->part_ml; a.status = ctx->d_status;
+    if (!ctx->attn_attr_done) {
+        cudaError_t e = cudaFuncSetAttribute(umma::tree_attn_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             umma::SMEM_BYTES);
+        if (e != cudaSuccess) return e;
+        ctx->attn_attr_done = 1;
+    }
+    dim3 grid(n_splits, c.n_kv_heads * a.mtiles, B);
+    umma::tree_attn_umma_kernel<<<grid, umma::NT, umma::SMEM_BYTES, st>>>(a);
+    ctx->launches++;
+    return cudaGetLastError();
+}
