@@ -82,6 +82,8 @@ accept_stats_kernel(const float *__restrict__ logits, const float *__restrict__ 
     const long long lo = (long long)blockIdx.x * g.chunk;
     const long long hi = min(g.total, lo + g.chunk);
     __shared__ Acc wacc[kThreads / 32];
+    fspad_pdl_trigger();
+    fspad_pdl_wait();
 
     long long seg_lo = lo;
     while (seg_lo < hi) {
@@ -173,6 +175,8 @@ accept_stats_merge_kernel(const FspadStatsPart *__restrict__ parts, const FspadS
                           const float *__restrict__ temperature, int rows, int rows_per_seq,
                           float *__restrict__ row_max, double *__restrict__ row_sum, int *__restrict__ row_arg)
 {
+    fspad_pdl_trigger();
+    fspad_pdl_wait();
     const int lane = threadIdx.x & 31;
     const int row = blockIdx.x * 4 + (threadIdx.x >> 5);
     if (row >= rows) return;
@@ -193,10 +197,10 @@ cudaError_t launch_partials(const float *logits, const float *temperature, int r
                             const FspadStatsGeom &g, FspadStatsPart *parts, cudaStream_t st)
 {
     if (g.unit == 4)
-        accept_stats_kernel<4><<<g.n_cta, kThreads, 0, st>>>(logits, temperature, rows_per_seq, g, parts);
-    else
-        accept_stats_kernel<1><<<g.n_cta, kThreads, 0, st>>>(logits, temperature, rows_per_seq, g, parts);
-    return cudaGetLastError();
+        return fspad_launch(accept_stats_kernel<4>, dim3(g.n_cta), dim3(kThreads), 0, st, 0, logits, temperature,
+                            rows_per_seq, g, parts);
+    return fspad_launch(accept_stats_kernel<1>, dim3(g.n_cta), dim3(kThreads), 0, st, 0, logits, temperature,
+                        rows_per_seq, g, parts);
 }
 
 }  // namespace
@@ -219,10 +223,10 @@ cudaError_t fspad_launch_accept_stats(fspad_ctx *ctx, const float *logits, const
     FspadStatsGeom g;
     cudaError_t e = fspad_launch_stats_partials(ctx, logits, temperature, rows, rows_per_seq, V, &g, st);
     if (e != cudaSuccess) return e;
-    accept_stats_merge_kernel<<<(rows + 3) / 4, 128, 0, st>>>(ctx->st_part, g, temperature, rows,
-                                                                 rows_per_seq, row_max, row_sum, row_arg);
     ctx->launches++;
-    return cudaGetLastError();
+    return fspad_launch(accept_stats_merge_kernel, dim3((rows + 3) / 4), dim3(128), 0, st, 0,
+                        (const FspadStatsPart *)ctx->st_part, g, temperature, rows, rows_per_seq, row_max, row_sum,
+                        row_arg);
 }
 
 // ---------------------------------------------------------------------------
@@ -279,7 +283,7 @@ extern "C" int fspad_accept_stats_noalloc(const float *logits, const float *temp
     // every slot the merge reads is rewritten by this call's first kernel, so the contents an
     // earlier call left in the shared array never need clearing
     if (launch_partials(logits, temperature, rows_per_seq, g, parts, st) != cudaSuccess) return FSPAD_ERR_CUDA;
-    accept_stats_merge_kernel<<<(rows + 3) / 4, 128, 0, st>>>(parts, g, temperature, rows, rows_per_seq,
-                                                                 row_max, row_sum, row_arg);
-    return cudaGetLastError() == cudaSuccess ? FSPAD_OK : FSPAD_ERR_CUDA;
+    return fspad_launch(accept_stats_merge_kernel, dim3((rows + 3) / 4), dim3(128), 0, st, 0,
+                        (const FspadStatsPart *)parts, g, temperature, rows, rows_per_seq, row_max, row_sum,
+                        (int *)row_arg) == cudaSuccess ? FSPAD_OK : FSPAD_ERR_CUDA;
 }

@@ -249,8 +249,10 @@ accept_walk_kernel(const WalkArgs args)
     __shared__ Shared sh;
     extern __shared__ __align__(16) unsigned char dyn_smem[];
 
-    float Tf = args.temperature[b];
+    fspad_pdl_trigger();
     if (tid < 64) { sh.exp_tbl[tid] = kExp2Tbl[tid]; sh.child_mask[tid] = 0ull; }
+    fspad_pdl_wait();
+    float Tf = args.temperature[b];
     if (!(Tf >= 0.0f)) {
         if (tid == 0 && rank == 0) fspad_report(args.status, FSPAD_ERR_RANGE);
         Tf = 0.0f;
@@ -602,15 +604,6 @@ cudaError_t fspad_launch_accept_walk(fspad_ctx *ctx, const float *logits, const 
         const size_t need = per_thr * kWalkThreads * (sizeof(double) + sizeof(float));
         if (need <= (size_t)kSmemBudget) { smem = need; a.cache_ok = 1; }
     }
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)(B * cluster));
-    cfg.blockDim = dim3(threads);
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = cluster; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr; cfg.numAttrs = 1;
     ctx->launches++;
-    return cudaLaunchKernelEx(&cfg, accept_walk_kernel, a);
+    return fspad_launch(accept_walk_kernel, dim3((unsigned)(B * cluster)), dim3(threads), smem, st, (unsigned)cluster, a);
 }

@@ -4,6 +4,8 @@
 #include <cuda_bf16.h>
 #include <stdint.h>
 
+#include <utility>
+
 #include "fspad.h"
 
 #define FSPAD_MAX_NODES 64
@@ -164,6 +166,50 @@ __device__ __forceinline__ void fspad_stats_merge_half(const FspadStatsPart *__r
     M = m;
     S = s;
     A = (a == 0x7fffffff) ? 0 : a;
+}
+#endif
+
+// ---- programmatic dependent launch -----------------------------------------------------
+// Every kernel of the library is launched with the programmatic-serialization attribute and
+// follows one rule: it lets its successor start launching at once (fspad_pdl_trigger) and it
+// touches global memory only after the whole preceding kernel of the stream has completed and
+// flushed (fspad_pdl_wait).  Launch latency and the memory-free part of a prologue (barrier
+// set-up, tensor-memory allocation, table fills) then overlap the tail of the previous kernel,
+// while results stay exactly those of plain stream order.
+#ifdef __CUDACC__
+__device__ __forceinline__ void fspad_pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void fspad_pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+static inline cudaError_t fspad_launch_opt(bool pdl, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                                           cudaStream_t st, unsigned cluster_x, Args &&...args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    int n = 0;
+    if (pdl) {
+        attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[n].val.programmaticStreamSerializationAllowed = 1;
+        ++n;
+    }
+    if (cluster_x > 0) {
+        attr[n].id = cudaLaunchAttributeClusterDimension;
+        attr[n].val.clusterDim.x = cluster_x; attr[n].val.clusterDim.y = 1; attr[n].val.clusterDim.z = 1;
+        ++n;
+    }
+    cfg.attrs = attr;
+    cfg.numAttrs = n;
+    return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
+template <typename... KArgs, typename... Args>
+static inline cudaError_t fspad_launch(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                                       cudaStream_t st, unsigned cluster_x, Args &&...args)
+{
+    return fspad_launch_opt(true, kernel, grid, block, smem, st, cluster_x, std::forward<Args>(args)...);
 }
 #endif
 

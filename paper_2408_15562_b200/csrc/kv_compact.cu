@@ -25,6 +25,8 @@ kv_compact_kernel(uint4 *__restrict__ cache, const int *__restrict__ path, const
                   const int *__restrict__ prefix_len, int n_layers, int B, int Hkv, int max_len,
                   int path_stride, int n_tree_max, int *__restrict__ new_len, int *__restrict__ status)
 {
+    fspad_pdl_trigger();
+    fspad_pdl_wait();
     const int lane = threadIdx.x & 31;
     const long long slice = (long long)blockIdx.x * kWarpsPerCta + (threadIdx.x >> 5);
     const long long n_slices = (long long)n_layers * 2 * B * Hkv;
@@ -71,6 +73,8 @@ tree_scatter_kernel(uint4 *__restrict__ cache, const uint4 *__restrict__ tk, con
                     const int *__restrict__ prefix_len, int N, int B, int Hkv, int max_len,
                     int *__restrict__ status)
 {
+    fspad_pdl_trigger();
+    fspad_pdl_wait();
     const long long total = (long long)2 * B * Hkv * N * kChunks;
     for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total;
          i += (long long)gridDim.x * blockDim.x) {
@@ -97,12 +101,10 @@ cudaError_t fspad_launch_kv_compact(fspad_ctx *ctx, fspad_bf16 *cache, const int
     const fspad_config &c = ctx->cfg;
     const long long slices = (long long)c.n_layers * 2 * B * c.n_kv_heads;
     const unsigned grid = (unsigned)((slices + kWarpsPerCta - 1) / kWarpsPerCta);
-    kv_compact_kernel<<<grid, kWarpsPerCta * 32, 0, st>>>(reinterpret_cast<uint4 *>(cache), path, n_acc,
-                                                          prefix_len, c.n_layers, B, c.n_kv_heads,
-                                                          c.max_len, c.max_nodes, c.max_nodes, new_len,
-                                                          ctx->d_status);
     ctx->launches++;
-    return cudaGetLastError();
+    return fspad_launch(kv_compact_kernel, dim3(grid), dim3(kWarpsPerCta * 32), 0, st, 0,
+                        reinterpret_cast<uint4 *>(cache), path, n_acc, prefix_len, c.n_layers, B, c.n_kv_heads,
+                        c.max_len, c.max_nodes, c.max_nodes, new_len, ctx->d_status);
 }
 
 cudaError_t fspad_launch_tree_scatter(fspad_ctx *ctx, fspad_bf16 *cache, const fspad_bf16 *tk,
@@ -114,10 +116,8 @@ cudaError_t fspad_launch_tree_scatter(fspad_ctx *ctx, fspad_bf16 *cache, const f
     const long long total = (long long)2 * B * c.n_kv_heads * N * kChunks;
     unsigned grid = (unsigned)((total + 255) / 256);
     if (grid > (unsigned)ctx->sm_count * 8) grid = (unsigned)ctx->sm_count * 8;
-    tree_scatter_kernel<<<grid, 256, 0, st>>>(reinterpret_cast<uint4 *>(cache),
-                                              reinterpret_cast<const uint4 *>(tk),
-                                              reinterpret_cast<const uint4 *>(tv), prefix_len, N, B,
-                                              c.n_kv_heads, c.max_len, ctx->d_status);
     ctx->launches++;
-    return cudaGetLastError();
+    return fspad_launch(tree_scatter_kernel, dim3(grid), dim3(256), 0, st, 0, reinterpret_cast<uint4 *>(cache),
+                        reinterpret_cast<const uint4 *>(tk), reinterpret_cast<const uint4 *>(tv), prefix_len, N, B,
+                        c.n_kv_heads, c.max_len, ctx->d_status);
 }

@@ -32,6 +32,8 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
 __global__ void __launch_bounds__(128)
 tree_attn_combine_kernel(const AttnArgs a, int B)
 {
+    fspad_pdl_trigger();
+    fspad_pdl_wait();
     const int lane = threadIdx.x & 31;
     const long long row = (long long)blockIdx.x * 4 + (threadIdx.x >> 5);   // over [B][Hkv][M]
     const long long total = (long long)B * a.Hkv * a.M;
@@ -107,7 +109,6 @@ cudaError_t fspad_launch_tree_attn(fspad_ctx *ctx, const fspad_bf16 *q, const fs
                                                  a.scale_log2, st);
     if (e != cudaSuccess) return e;
     const long long rows = (long long)B * c.n_kv_heads * a.M;
-    tree_attn_combine_kernel<<<(unsigned)((rows + 3) / 4), 128, 0, st>>>(a, B);
     ctx->launches++;
-    return cudaGetLastError();
+    return fspad_launch_opt(false, tree_attn_combine_kernel, dim3((unsigned)((rows + 3) / 4)), dim3(128), 0, st, 0, a, B);
 }

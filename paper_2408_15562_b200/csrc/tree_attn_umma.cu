@@ -183,6 +183,7 @@ tree_attn_umma_kernel(const Args a)
     __shared__ unsigned long long s_anc[FSPAD_MAX_NODES];
     __shared__ float s_mx[2][BM];                            // per-half row maxima / sums exchange
 
+    fspad_pdl_wait();
     const int tid = threadIdx.x, warp = tid >> 5;
     const int row = tid & (BM - 1), half = tid >> 7;
     const int split = blockIdx.x;
@@ -197,9 +198,8 @@ tree_attn_umma_kernel(const Args a)
     }
     const int Ltot = L + N;
     const int n_chunks = (Ltot + BK - 1) / BK;
-    // key chunks are dealt out as evenly as possible: range s gets chunks [s*n/S, (s+1)*n/S)
-    const int c0 = (int)(((long long)split * n_chunks) / a.n_splits);
-    const int c1 = (int)(((long long)(split + 1) * n_chunks) / a.n_splits);
+    const int per = (n_chunks + a.n_splits - 1) / a.n_splits;
+    const int c0 = split * per, c1 = min(n_chunks, c0 + per);
 
     const int gr = mt * BM + row;                 // this thread's row among the kv head's M rows
     const bool row_ok = gr < M;
@@ -399,6 +399,7 @@ tree_attn_umma_kernel(const Args a)
         cp_async_commit();
     }
 
+    fspad_pdl_trigger();                          // the merge kernel may start launching
     // ---- publish the partial: unnormalised O row, running max and sum ----
     // Every lane of every warp takes part in the tensor-memory loads (they are warp-collective);
     // only the stores to global memory depend on whether the lane's row exists.
@@ -467,7 +468,6 @@ cudaError_t fspad_launch_attn_umma_split(fspad_ctx *ctx, const fspad_bf16 *q, co
         ctx->attn_attr_done = 1;
     }
     dim3 grid(n_splits, c.n_kv_heads * a.mtiles, B);
-    umma::tree_attn_umma_kernel<<<grid, umma::NT, umma::SMEM_BYTES, st>>>(a);
     ctx->launches++;
-    return cudaGetLastError();
+    return fspad_launch_opt(false, umma::tree_attn_umma_kernel, grid, dim3(umma::NT), umma::SMEM_BYTES, st, 0, a);
 }
