@@ -93,12 +93,14 @@ struct Shared {
     double rowS[FSPAD_MAX_NODES];
     int rowA[FSPAD_MAX_NODES];
     float cx[FSPAD_MAX_NODES], cq[FSPAD_MAX_NODES], cu[FSPAD_MAX_NODES];
+    double cex[FSPAD_MAX_NODES];    // exp((logit - row max)/T) of each node's token in its parent's row
     float ubonus;
+    int want_q;
     // reductions
     double warp_a[kWarps], warp_b[kWarps], warp_off[kWarps];
-    double slot[2][2];              // this CTA's partial sums, by pass parity (read by peers)
+    double slot[2][kMaxCluster][2]; // partial sums received from every CTA of the cluster, by pass parity
     double tot[2];                  // cluster totals
-    double cta_total[kMaxCluster];
+    double cta_total[kMaxCluster];  // bonus draw: every CTA's total, received from the peers
 };
 
 // exp(a) for a <= 0 in double precision: a = (64 n + i) ln2/64 + r, |r| <= ln2/128,
@@ -159,7 +161,8 @@ __device__ Sweep sweep_chunk(const Shared &sh, const float *__restrict__ x, cons
     const int nrem = sh.nrem;
     // bonus draw with nothing rejected at this node: the weights are the e_j themselves
     const double invS = (MODE == MODE_CDF && c == 0.0 && nrem == 0) ? 1.0 : sh.invS;
-    const bool need_q = (MODE == MODE_RESID) || (MODE == MODE_CDF && c != 0.0);
+    // the exact-sum sweep that precedes a rejection also parks the draft row for the sweeps to come
+    const bool need_q = (MODE == MODE_RESID) || (MODE == MODE_CDF && c != 0.0) || (MODE == MODE_EXP && xnew == -2);
     bool special = false;
     if (MODE != MODE_EXP) {
         for (int r = 0; r < nrem; ++r) special |= (sh.rem_tok[r] >= lo && sh.rem_tok[r] < hi);
@@ -306,6 +309,9 @@ accept_walk_kernel(const WalkArgs args)
         }
     }
     __syncthreads();
+    if (sampling && tid >= 1 && tid < N)
+        sh.cex[tid] = exp_neg(((double)sh.cx[tid] - (double)sh.rowM[sh.parent[tid]]) * (1.0 / (double)Tf), sh.exp_tbl);
+    __syncthreads();
 
     if (!sampling) {
         // ---- greedy: strict token comparison against the target argmax ----
@@ -347,8 +353,9 @@ accept_walk_kernel(const WalkArgs args)
     int parity = 0;
 
     // cluster-wide reduction of (a, b); result in sh.tot[] (read by thread 0 only).  Every level
-    // is a warp butterfly over values fetched in parallel (no serial chain of shared-memory or
-    // peer reads), and every CTA performs the same operations on the same values.
+    // is a warp butterfly; the CTAs exchange by remote stores (each writes its pair into every
+    // peer's slot before the barrier), so after the barrier all reads are local, and every CTA
+    // performs the same operations on the same values.
     auto reduce_exchange = [&](double a, double bb) {
         const int lane = tid & 31, wid = tid >> 5, nwarps = nthr >> 5;
         a = warp_sum(a);
@@ -360,16 +367,16 @@ accept_walk_kernel(const WalkArgs args)
             double sb = (lane < nwarps) ? sh.warp_b[lane] : 0.0;
             sa = warp_sum(sa);
             sb = warp_sum(sb);
-            if (lane == 0) { sh.slot[parity][0] = sa; sh.slot[parity][1] = sb; }
+            if (lane < C) {
+                double *peer = cluster.map_shared_rank(&sh.slot[parity][rank][0], lane);
+                peer[0] = sa;
+                peer[1] = sb;
+            }
         }
         cluster.sync();
         if (wid == 0) {
-            double ta = 0.0, tb = 0.0;
-            if (lane < C) {
-                const double *peer = cluster.map_shared_rank(&sh.slot[parity][0], lane);
-                ta = peer[0];
-                tb = peer[1];
-            }
+            double ta = (lane < C) ? sh.slot[parity][lane][0] : 0.0;
+            double tb = (lane < C) ? sh.slot[parity][lane][1] : 0.0;
             ta = warp_sum(ta);
             tb = warp_sum(tb);
             if (lane == 0) { sh.tot[0] = ta; sh.tot[1] = tb; }
@@ -404,17 +411,19 @@ accept_walk_kernel(const WalkArgs args)
                 if (tid == 0) {
                     const double r = (double)sh.cu[ch];
                     const double qx = (double)sh.cq[ch];
-                    const double ex = exp_neg(((double)sh.cx[ch] - sh.m) * sh.invT, sh.exp_tbl);
+                    const double ex = sh.cex[ch];
                     int ridx = -1;
                     for (int k = 0; k < sh.nrem; ++k) if (sh.rem_tok[k] == xt) ridx = k;
-                    double qk, pk;
-                    if (ridx >= 0) { qk = 0.0; pk = sh.rem_frozen[ridx] / sh.U; }
-                    else { qk = qx / sh.D; pk = weight(ex, qx, sh.invS, sh.c) / sh.U; }
-                    const double lhs = r * qk;
-                    int dec = (lhs < pk) ? 1 : 0;
+                    // accept iff r * q_k(x) < p_k(x) with q_k = qx / D and p_k = u / U: compared as
+                    // r * qx * U < u * D (both normalisers are positive), so no division is needed
+                    const double u = (ridx >= 0) ? sh.rem_frozen[ridx] : weight(ex, qx, sh.invS, sh.c);
+                    const double lhs = (ridx >= 0) ? 0.0 : r * qx * sh.U;
+                    const double rhs = u * sh.D;
+                    int dec = (lhs < rhs) ? 1 : 0;
+                    sh.want_q = (dec == 0);
                     if (!sh.exact) {
-                        const double big = fmax(lhs, pk);
-                        if (big > 0.0 && fabs(lhs - pk) <= kAmbiguous * big) dec = 2;
+                        const double big = fmax(lhs, rhs);
+                        if (big > 0.0 && fabs(lhs - rhs) <= kAmbiguous * big) dec = 2;
                         else if (dec == 0) dec = 2;      // a rejection needs the exact denominator anyway
                     }
                     sh.decision = dec;
@@ -423,10 +432,14 @@ accept_walk_kernel(const WalkArgs args)
                 __syncthreads();
                 if (sh.decision != 2) break;
                 // exact softmax denominator of this node (parks e_j in shared memory)
+                const bool with_q = sh.want_q != 0;
                 Sweep s = sweep_chunk<MODE_EXP>(sh, x, q, se, sq, tid, nthr, lo, hi, vec, cache_ok, false, false, 0.0,
-                                                -1, false, 0, 0, 0, nullptr);
+                                                with_q ? -2 : -1, false, 0, 0, 0, nullptr);
                 reduce_exchange(s.a, 0.0);
-                if (tid == 0) { sh.S = sh.tot[0]; sh.invS = 1.0 / sh.S; sh.exact = 1; sh.have_e = cache_ok; }
+                if (tid == 0) {
+                    sh.S = sh.tot[0]; sh.invS = 1.0 / sh.S; sh.exact = 1; sh.have_e = cache_ok;
+                    if (with_q) sh.have_q = cache_ok;
+                }
                 __syncthreads();
             }
             if (sh.decision == 1) {
@@ -505,15 +518,15 @@ accept_walk_kernel(const WalkArgs args)
             }
             const double excl = __shfl_up_sync(0xffffffffu, sc, 1);
             if (lane < nwarps) sh.warp_off[lane] = (lane == 0) ? 0.0 : excl;
-            if (lane == nwarps - 1) sh.slot[parity][0] = sc;
+            // the CTA total goes to every CTA of the cluster (remote stores; read locally after the barrier)
+            const double total = __shfl_sync(0xffffffffu, sc, nwarps - 1);
+            if (lane < C) *cluster.map_shared_rank(&sh.cta_total[rank], lane) = total;
         }
         __syncthreads();
         const double woff = sh.warp_off[wid];
         const double P = woff + incl;
         const double E = (lane == 0) ? woff : woff + prev_incl;
         cluster.sync();
-        if (tid < C) sh.cta_total[tid] = *cluster.map_shared_rank(&sh.slot[parity][0], tid);
-        __syncthreads();
         double Z = 0.0, base = 0.0;
         for (int r = 0; r < C; ++r) {
             if (r == rank) base = Z;
@@ -551,7 +564,7 @@ accept_walk_kernel(const WalkArgs args)
             if (tid == 0) args.n_acc[b] = sh.len;
             for (int i = tid; i < args.path_stride; i += nthr) out_path[i] = (i < sh.len) ? sh.path[i] : -1;
         }
-        cluster.sync();    // nobody leaves while a peer may still read its shared memory
+        // no CTA touches a peer's shared memory after the barrier above, so each may leave on its own
     }
 }
 
