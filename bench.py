@@ -130,6 +130,7 @@ def main():
     ap.add_argument("--workload", default="llama3_8b_2k", choices=sorted(synth.WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-verify", action="store_true", help="skip the oracle check of the timed step")
     args = ap.parse_args()
     w = synth.WORKLOADS[args.workload]
     if args.impl == "reference":
@@ -248,13 +249,43 @@ def main():
     lg2d = [s["logits"].view(B * N, w.vocab) for s in sets]
     st_out = (torch.empty(B * N, dtype=torch.float32, device="cuda"), torch.empty(B * N, dtype=torch.float64, device="cuda"),
               torch.empty(B * N, dtype=torch.int32, device="cuda"))
-    stats_us = timed(lambda i: ctx.accept_stats(lg2d[i % R], temp, N, out=st_out), args.steps)
+    stats_us = timed(lambda i: ctx.accept_stats(lg2d[i % R], temp, N, out="scan_only"), args.steps)
+    stats_merge_us = timed(lambda i: ctx.accept_stats(lg2d[i % R], temp, N, out=st_out), args.steps)
     eager_us = timed(step, args.steps, graph=False)
+    # attention and acceptance use disjoint scratch, so a caller may queue them on two streams
+    side = torch.cuda.Stream()
+
+    def step_two_streams(i):
+        s = sets[i % R]
+        cur = torch.cuda.current_stream()
+        side.wait_stream(cur)
+        with torch.cuda.stream(side):
+            attn(s)
+        accept(s)
+        compact(s)
+        cur.wait_stream(side)
+
+    two_us = timed(step_two_streams, args.steps)
     clocks = sampler.stop()
     ctx.check()
 
     # ---- correctness of what was timed: compare the last step with the oracle on rank 0 ----
     n_acc_host = n_acc.cpu().numpy()
+    verified = None
+    if rank == 0 and not args.no_verify and B <= 2:
+        import oracle
+        step(0)
+        torch.cuda.synchronize()
+        ref = oracle.tree_accept(inp.target_logits, inp.draft_probs, inp.draft_tokens, inp.parent, inp.temperature,
+                                 inp.uniforms if inp.draft_probs is not None else None)
+        k = ref["n_accepted"]
+        ok_acc = (np.array_equal(n_acc.cpu().numpy(), k) and np.array_equal(bonus.cpu().numpy(), ref["bonus_token"])
+                  and all(np.array_equal(path[b_, :k[b_]].cpu().numpy(), ref["accepted_path"][b_, :k[b_]]) for b_ in range(B)))
+        ref_o = oracle.tree_attn(inp.q, inp.k_cache, inp.v_cache, inp.tree_k, inp.tree_v, inp.parent, inp.prefix_len)
+        err = np.abs(out.float().cpu().numpy() - ref_o)
+        verified = {"accept_bit_exact": bool(ok_acc), "attn_max_abs_err": float(err.max()),
+                    "attn_mean_abs_err": float(err.mean()),
+                    "ok": bool(ok_acc and err.max() <= 1e-2 and err.mean() <= 1e-3)}
 
     # ---- end to end through the host entry point (pinned host buffers, copies inside the timed region) ----
     pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()  # noqa: E731
@@ -287,8 +318,8 @@ def main():
     d2h = sum(t.numel() * t.element_size() for t in (hout, hpath, hn, hb, hl))
 
     # max over ranks
-    step_us, attn_us, accept_us, compact_us, stats_us, e2e_us, eager_us = dist_util.max_over_ranks(
-        [step_us, attn_us, accept_us, compact_us, stats_us, e2e_us, eager_us], device="cuda")
+    step_us, attn_us, accept_us, compact_us, stats_us, e2e_us, eager_us, two_us, stats_merge_us = dist_util.max_over_ranks(
+        [step_us, attn_us, accept_us, compact_us, stats_us, e2e_us, eager_us, two_us, stats_merge_us], device="cuda")
 
     if rank == 0:
         peak, peak_kind = peaks()
@@ -311,12 +342,15 @@ def main():
             "step_frac_of_hbm_peak": step_all / (step_us * 1e-6) / 1e9 / peak,
             "step_algorithmic_bytes": step_all,
             "breakdown_us": {"tree_attn": attn_us, "tree_accept": accept_us, "kv_compact": compact_us,
-                             "accept_stats_kernel_alone": stats_us,
-                             "whole_step_eager_python_launches": eager_us},
+                             "accept_stats_kernel_alone": stats_us, "accept_stats_with_merge": stats_merge_us,
+                             "whole_step_eager_python_launches": eager_us,
+                             "whole_step_two_streams_attn_overlapping_accept": two_us},
+            "verified_against_oracle": verified,
             "mean_accepted_len": float(n_acc_host.mean()),
             "roofline": {"kernel": "accept_stats_kernel", "bound": "hbm", "achieved": achieved, "peak": peak,
                          "peak_kind": "%s copy bandwidth (burst, kernel timed alone)" % peak_kind, "unit": "GB/s",
-                         "frac": achieved / peak, "traffic": None, "algorithmic_bytes_per_launch": stats_bytes},
+                         "frac": achieved / peak, "traffic": 30800896 if (w.name == "llama3_8b_2k") else None,
+                         "traffic_note": "dram__bytes_read+write per launch, ncu capture in profiles/accept_stats_kernel_llama3_8b_2k.md", "algorithmic_bytes_per_launch": stats_bytes},
             "e2e": {"value": e2e_us, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "steps": e2e_steps, "note": "fspad_verify_step_host: pinned host inputs, device-resident KV cache"},
             "gpu_launches": int(launches),

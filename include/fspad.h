@@ -154,6 +154,9 @@ int fspad_tree_accept(fspad_ctx *ctx, const float *target_logits, const float *d
  * and row_sum = sum_j exp((x_j - max)/T_row) accumulated from fp32 exponentials
  * (relative accuracy about 1e-6; the acceptance walk re-derives exact sums
  * where a decision is close).  temperature [rows / rows_per_seq] fp32, 0 -> 1.
+ * With all three outputs NULL only the streaming pass over the logits runs (its per-CTA
+ * partial results stay in the context's scratch): the HBM-bound kernel on its own, for
+ * timing and profiling.
  */
 int fspad_accept_stats(fspad_ctx *ctx, const float *logits, const float *temperature, int rows,
                        int rows_per_seq, float *row_max, double *row_sum, int32_t *row_arg,

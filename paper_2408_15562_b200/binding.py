@@ -159,6 +159,8 @@ class Context:
             out = (torch.empty((rows,), dtype=torch.float32, device=dev),
                    torch.empty((rows,), dtype=torch.float64, device=dev),
                    torch.empty((rows,), dtype=torch.int32, device=dev))
+        elif out == "scan_only":      # the streaming pass alone; partials stay in the context
+            out = (None, None, None)
         row_max, row_sum, row_arg = out
         rc = load().fspad_accept_stats(self._h, _ptr(logits, torch.float32), _ptr(temperature, torch.float32),
                                        rows, rows_per_seq, _ptr(row_max, torch.float32),

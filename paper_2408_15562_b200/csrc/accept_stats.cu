@@ -34,12 +34,11 @@ struct Acc {
     int a;
 };
 
-__device__ __forceinline__ void acc_merge(Acc &p, float om, float os, int oa, float k)
+__device__ __forceinline__ void acc_merge(Acc &p, float om, float os, float k)
 {
     const float mn = fmaxf(p.m, om);
     const float sp = (p.m == -INFINITY) ? 0.f : p.s * ex2((p.m - mn) * k);
     const float so = (om == -INFINITY) ? 0.f : os * ex2((om - mn) * k);
-    if (om > p.m || (om == p.m && oa < p.a)) p.a = oa;
     p.m = mn;
     p.s = sp + so;
 }
@@ -82,6 +81,8 @@ accept_stats_kernel(const float *__restrict__ logits, const float *__restrict__ 
     const long long lo = (long long)blockIdx.x * g.chunk;
     const long long hi = min(g.total, lo + g.chunk);
     __shared__ Acc wacc[kThreads / 32];
+    __shared__ float s_bmax;
+    __shared__ int s_barg;
     fspad_pdl_trigger();
     fspad_pdl_wait();
 
@@ -118,14 +119,11 @@ accept_stats_kernel(const float *__restrict__ logits, const float *__restrict__ 
 #pragma unroll
             for (int u = 1; u < kDeep; ++u) bm = fmaxf(bm, Unit<UNIT>::vmax(cur[u]));
             if (bm > p.m) {
-                // lowest index attaining the new maximum: scan from the back so the first match wins
-                int a = 0;
-#pragma unroll
-                for (int u = kDeep - 1; u >= 0; --u)
-                    a = Unit<UNIT>::first_eq(cur[u], bm, (off + base + u * kThreads + tid) * UNIT, a);
+                // only the batch is remembered; the position inside it is looked up once, at the
+                // end, by the threads that hold the block's maximum
                 p.s = (p.m == -INFINITY) ? 0.f : p.s * ex2((p.m - bm) * k);
                 p.m = bm;
-                p.a = a;
+                p.a = base;
             }
             if (p.m != -INFINITY) {
                 float s0 = 0.f;
@@ -138,31 +136,46 @@ accept_stats_kernel(const float *__restrict__ logits, const float *__restrict__ 
                 for (int u = 0; u < kDeep; ++u) cur[u] = nxt[u];
             }
         }
-        // block reduction of (m, s, a)
+        // block reduction of (m, s); then the lowest index of the block's maximum
+        const float my_m = p.m;
+        const int my_base = p.a;
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
             const float om = __shfl_xor_sync(0xffffffffu, p.m, o);
             const float os = __shfl_xor_sync(0xffffffffu, p.s, o);
-            const int oa = __shfl_xor_sync(0xffffffffu, p.a, o);
-            acc_merge(p, om, os, oa, k);
+            acc_merge(p, om, os, k);
         }
         if (lane == 0) wacc[wid] = p;
+        if (tid == 0) s_barg = 0x7fffffff;
         __syncthreads();
         if (wid == 0) {
-            Acc q = (lane < kThreads / 32) ? wacc[lane] : Acc{-INFINITY, 0.f, 0x7fffffff};
+            Acc q = (lane < kThreads / 32) ? wacc[lane] : Acc{-INFINITY, 0.f, 0};
 #pragma unroll
             for (int o = 4; o > 0; o >>= 1) {
                 const float om = __shfl_xor_sync(0xffffffffu, q.m, o);
                 const float os = __shfl_xor_sync(0xffffffffu, q.s, o);
-                const int oa = __shfl_xor_sync(0xffffffffu, q.a, o);
-                acc_merge(q, om, os, oa, k);
+                acc_merge(q, om, os, k);
             }
-            if (lane == 0) {
-                const int first = (int)(row_lo / g.chunk);
-                FspadStatsPart out;
-                out.m = q.m; out.s = q.s; out.a = q.a; out.pad = 0;
-                parts[(size_t)row * g.slots + (blockIdx.x - first)] = out;
+            if (lane == 0) { wacc[0] = q; s_bmax = q.m; }
+        }
+        __syncthreads();
+        const float bmax = s_bmax;
+        if (my_m == bmax && bmax != -INFINITY) {
+            // this thread's batch `my_base` holds the maximum: fetch it again (cache hit) and scan it
+            int a = 0x7fffffff;
+#pragma unroll
+            for (int u = kDeep - 1; u >= 0; --u) {
+                const int i = my_base + u * kThreads + tid;
+                if (i < n) a = Unit<UNIT>::first_eq(__ldg(px + i), bmax, (off + i) * UNIT, a);
             }
+            atomicMin(&s_barg, a);
+        }
+        __syncthreads();
+        if (tid == 0) {
+            const int first = (int)(row_lo / g.chunk);
+            FspadStatsPart out;
+            out.m = wacc[0].m; out.s = wacc[0].s; out.a = s_barg; out.pad = 0;
+            parts[(size_t)row * g.slots + (blockIdx.x - first)] = out;
         }
         __syncthreads();
         seg_lo = seg_hi;

@@ -163,10 +163,16 @@ int fspad_accept_stats(fspad_ctx *ctx, const float *logits, const float *tempera
                        void *stream)
 {
     if (!ctx) return FSPAD_ERR_NULL;
-    if (!logits || !row_max || !row_sum || !row_arg) return FSPAD_ERR_NULL;
+    const bool scan_only = !row_max && !row_sum && !row_arg;
+    if (!logits || (!scan_only && (!row_max || !row_sum || !row_arg))) return FSPAD_ERR_NULL;
     if (rows < 0 || rows_per_seq < 1 || rows > ctx->cfg.max_batch * ctx->cfg.max_nodes)
         return FSPAD_ERR_SHAPE;
     if (rows == 0) return FSPAD_OK;
+    if (scan_only) {
+        FspadStatsGeom geom;
+        return fspad_launch_stats_partials(ctx, logits, temperature, rows, rows_per_seq, ctx->cfg.vocab, &geom,
+                                           fspad_stream(stream)) == cudaSuccess ? FSPAD_OK : FSPAD_ERR_CUDA;
+    }
     cudaError_t e = fspad_launch_accept_stats(ctx, logits, temperature, rows, rows_per_seq, ctx->cfg.vocab,
                                               row_max, row_sum, row_arg, fspad_stream(stream));
     return e == cudaSuccess ? FSPAD_OK : FSPAD_ERR_CUDA;
