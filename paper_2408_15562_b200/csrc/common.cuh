@@ -24,6 +24,11 @@ struct fspad_ctx {
     // split-KV attention partials
     int attn_max_splits;
     int attn_attr_done;       // dynamic shared-memory limit raised for the attention kernels
+    // TMA descriptors of the K and V cache planes last seen (re-encoded when they change)
+    alignas(64) unsigned char attn_tmap_k[128];
+    alignas(64) unsigned char attn_tmap_v[128];
+    const void *attn_tmap_kptr, *attn_tmap_vptr;
+    int attn_tmap_batch, attn_tmap_ok;
     float *part_o;            // [batch][Hkv][splits][M][d]
     float *part_ml;           // [batch][Hkv][splits][M][2]  (running max in log2 units, sum)
 

@@ -12,13 +12,18 @@
 // a 128-byte-swizzled shared-memory tile; O += P V is a second chain of eight
 // tcgen05.mma with V read directly in its [key][d] layout (MN-major operand).
 // O stays in tensor memory across chunks and is rescaled there when the running
-// maximum moves.  K/V chunks are double buffered with 16-byte asynchronous
-// copies into the swizzled layout the matrix descriptors expect.  Per-split
+// maximum moves.  K/V chunks are double buffered in the 128-byte-swizzled layout
+// the matrix descriptors expect: chunks that lie inside the cached prefix arrive
+// by TMA (four cp.async.bulk.tensor boxes of 64 x 128 per chunk, one issuing
+// thread, completion on an mbarrier); Q and the one chunk that mixes prefix,
+// tree rows and zero padding use 16-byte asynchronous copies.  Per-split
 // partials are merged by the combine kernel.
 //
 // Every wait on an mbarrier is bounded; on expiry the CTA records
 // FSPAD_ERR_TIMEOUT, skips the remaining tensor-core work, frees its tensor
 // memory and returns.
+#include <cuda.h>
+
 #include "common.cuh"
 
 namespace umma {
@@ -35,7 +40,7 @@ constexpr uint32_t WAIT_CAP = 200000;   // polls of a bounded mbarrier wait
 struct Args {
     const fspad_bf16 *q, *kc, *vc, *tk, *tv;
     const int *parent, *prefix_len;
-    int N, Hq, Hkv, G, M, max_len, n_splits, mtiles;
+    int N, Hq, Hkv, G, M, max_len, n_splits, mtiles, use_tma;
     float scale_log2;
     float *part_o, *part_ml;
     int *status;
@@ -85,6 +90,18 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
     }
     ok = __shfl_sync(0xffffffffu, ok, 0);
     return ok != 0;
+}
+
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(bytes) : "memory");
+}
+// one box of a 2-D tensor map -> shared memory; x counts elements of the inner dimension
+// (here 0 or 64 bf16 = 0 or 128 bytes, a multiple of the 16 bytes TMA requires), y counts rows
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];\n"
+                 :: "r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(x), "r"(y) : "memory");
 }
 
 // shared-memory matrix descriptor, 128-byte swizzle, 8-row groups 1024 bytes apart
@@ -173,10 +190,10 @@ __device__ __forceinline__ float ex2f(float x)
 // row's scores, of its P row and of its O row.  Warps w and w+4 address the same 32 lanes of
 // tensor memory (a warp reaches the lane quarter given by its index modulo 4).
 __global__ void __launch_bounds__(NT, 1)
-tree_attn_umma_kernel(const Args a)
+tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV)
 {
     extern __shared__ unsigned char smem_raw[];
-    __shared__ __align__(8) unsigned long long s_bar[2];     // [0]: S ready, [1]: O updated
+    __shared__ __align__(8) unsigned long long s_bar[4];     // [0]: S ready, [1]: O updated, [2],[3]: chunk buffer filled by TMA
     __shared__ uint32_t s_tmem;
     __shared__ int s_fail;
     __shared__ int s_par[FSPAD_MAX_NODES];
@@ -215,6 +232,17 @@ tree_attn_umma_kernel(const Args a)
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t sQ = base, sK = base + TILE, sV = base + 3 * TILE, sP = base + 5 * TILE;
     const uint32_t barS = smem_u32(&s_bar[0]), barO = smem_u32(&s_bar[1]);
+    const uint32_t barF[2] = {smem_u32(&s_bar[2]), smem_u32(&s_bar[3])};
+    const bool tma_ok = a.use_tma != 0;
+    if (tid == 0) {
+        mbar_init(barS, 1);
+        mbar_init(barO, 1);
+        mbar_init(barF[0], 1);
+        mbar_init(barF[1], 1);
+        s_fail = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+    }
+    __syncthreads();
 
     const fspad_bf16 *kcb = a.kc + ((size_t)b * a.Hkv + g) * (size_t)a.max_len * D;
     const fspad_bf16 *vcb = a.vc + ((size_t)b * a.Hkv + g) * (size_t)a.max_len * D;
@@ -232,8 +260,22 @@ tree_attn_umma_kernel(const Args a)
             cp_async16(sQ + tile_off(r, c), src, ok);
         }
     }
+    // row of the cache planes (as one [batch*Hkv*max_len][128] matrix) where this kv head starts
+    const int plane_row0 = (b * a.Hkv + g) * a.max_len;
     auto load_chunk = [&](int ch, int buf) {
         const uint32_t dK = sK + buf * TILE, dV = sV + buf * TILE;
+        if (tma_ok && (ch + 1) * BK <= L) {
+            // the whole chunk is cached prefix: four 64 x 128 boxes, one thread, no register traffic
+            if (tid == 0) {
+                mbar_expect_tx(barF[buf], 2 * TILE);
+                const int y = plane_row0 + ch * BK;
+                tma_load_2d(dK, &tmK, 0, y, barF[buf]);
+                tma_load_2d(dK + HALF, &tmK, 64, y, barF[buf]);
+                tma_load_2d(dV, &tmV, 0, y, barF[buf]);
+                tma_load_2d(dV + HALF, &tmV, 64, y, barF[buf]);
+            }
+            return;
+        }
         const int c = tid & 15;
         for (int r = tid >> 4; r < BK; r += NT / 16) {
             const int key = ch * BK + r;
@@ -254,12 +296,6 @@ tree_attn_umma_kernel(const Args a)
 
     // ---- tree -> ancestor-or-self masks (parents staged in shared memory, then walked there) ----
     if (tid < N) s_par[tid] = a.parent[(size_t)b * N + tid];
-    if (tid == 0) {
-        mbar_init(barS, 1);
-        mbar_init(barO, 1);
-        s_fail = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
-    }
     if (warp == 1) {                              // one (converged) warp allocates the tensor memory
         __syncwarp();
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n"
@@ -293,13 +329,17 @@ tree_attn_umma_kernel(const Args a)
     const float scale = a.scale_log2;
 
     float m_run = -INFINITY, l_part = 0.f;       // row maximum (shared by both halves), this half's sum
-    uint32_t phS = 0, phO = 0;
+    uint32_t phS = 0, phO = 0, phF[2] = {0, 0};
     bool failed = false;
 
     for (int ch = c0; ch < c1; ++ch) {
         const int buf = (ch - c0) & 1;
         // this chunk's copies have landed (the younger group, if any, may still be in flight)
         if (ch + 1 < c1) cp_async_wait<1>(); else cp_async_wait<0>();
+        if (tma_ok && (ch + 1) * BK <= L) {
+            if (!failed && !mbar_wait(barF[buf], phF[buf])) { failed = true; s_fail = 1; }
+            phF[buf] ^= 1;
+        }
         fence_async_smem();
         __syncthreads();
         if (tid == 0 && !failed) {
@@ -448,6 +488,42 @@ int fspad_attn_umma_splits(const fspad_ctx *ctx, int N, int B)
     return (int)s;
 }
 
+// ---- TMA descriptors of the K and V cache planes ----------------------------------------
+// Each plane is viewed as one row-major matrix [batch * Hkv * max_len][128] bf16; a box is
+// 64 columns (128 bytes, the swizzle span) by 128 rows and lands as one half tile.
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_tiled_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+        (void)cudaGetLastError();
+    }
+    return fn;
+}
+
+static bool make_plane_map(CUtensorMap *map, const fspad_bf16 *plane, size_t rows)
+{
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn || rows == 0 || rows > 0x7fffffffull) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)umma::D, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)umma::D * sizeof(fspad_bf16)};
+    const cuuint32_t box[2] = {64u, (cuuint32_t)umma::BK};
+    const cuuint32_t estr[2] = {1u, 1u};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<fspad_bf16 *>(plane), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 cudaError_t fspad_launch_attn_umma_split(fspad_ctx *ctx, const fspad_bf16 *q, const fspad_bf16 *kc,
                                          const fspad_bf16 *vc, const fspad_bf16 *tk, const fspad_bf16 *tv,
                                          const int *parent, const int *prefix_len, int N, int B, int n_splits,
@@ -467,7 +543,17 @@ cudaError_t fspad_launch_attn_umma_split(fspad_ctx *ctx, const fspad_bf16 *q, co
         if (e != cudaSuccess) return e;
         ctx->attn_attr_done = 1;
     }
+    // descriptors are re-encoded only when a plane pointer or the batch changes
+    static_assert(sizeof(CUtensorMap) <= sizeof(ctx->attn_tmap_k), "tensor map storage");
+    CUtensorMap *mk = reinterpret_cast<CUtensorMap *>(ctx->attn_tmap_k);
+    CUtensorMap *mv = reinterpret_cast<CUtensorMap *>(ctx->attn_tmap_v);
+    if (ctx->attn_tmap_kptr != kc || ctx->attn_tmap_vptr != vc || ctx->attn_tmap_batch != B) {
+        const size_t rows = (size_t)B * c.n_kv_heads * c.max_len;
+        ctx->attn_tmap_ok = make_plane_map(mk, kc, rows) && make_plane_map(mv, vc, rows);
+        ctx->attn_tmap_kptr = kc; ctx->attn_tmap_vptr = vc; ctx->attn_tmap_batch = B;
+    }
+    a.use_tma = ctx->attn_tmap_ok ? 1 : 0;
     dim3 grid(n_splits, c.n_kv_heads * a.mtiles, B);
     ctx->launches++;
-    return fspad_launch_opt(false, umma::tree_attn_umma_kernel, grid, dim3(umma::NT), umma::SMEM_BYTES, st, 0, a);
+    return fspad_launch_opt(false, umma::tree_attn_umma_kernel, grid, dim3(umma::NT), umma::SMEM_BYTES, st, 0, a, *mk, *mv);
 }
