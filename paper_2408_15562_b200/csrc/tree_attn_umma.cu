@@ -35,7 +35,7 @@ constexpr int NT = 256;                // threads per CTA: two per query row
 constexpr int HALF = 128 * 128;        // bytes of one [128 rows][64 bf16] half tile
 constexpr int TILE = 2 * HALF;         // bytes of one [128][128] bf16 tile
 constexpr int SMEM_BYTES = 6 * TILE + 1024;   // Q, K[2], V[2], P + alignment slack
-constexpr uint32_t TMEM_COLS = 512;    // S buffers: columns 0..127 and 128..255, O: columns 256..383
+constexpr uint32_t TMEM_COLS = 256;    // S: columns 0..127, O: columns 128..255
 constexpr uint32_t WAIT_CAP = 200000;   // polls of a bounded mbarrier wait
 struct Args {
     const fspad_bf16 *q, *kc, *vc, *tk, *tv;
@@ -193,7 +193,7 @@ __global__ void __launch_bounds__(NT, 1)
 tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV)
 {
     extern __shared__ unsigned char smem_raw[];
-    __shared__ __align__(8) unsigned long long s_bar[7];     // S done x2, PV done, K filled x2, V filled x2
+    __shared__ __align__(8) unsigned long long s_bar[4];     // [0]: S ready, [1]: O updated, [2],[3]: chunk buffer filled by TMA
     __shared__ uint32_t s_tmem;
     __shared__ int s_fail;
     __shared__ int s_par[FSPAD_MAX_NODES];
@@ -231,15 +231,14 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
     // 1024-byte aligned tiles: Q | K0 | K1 | V0 | V1 | P
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t sQ = base, sK = base + TILE, sV = base + 3 * TILE, sP = base + 5 * TILE;
-    // mbarriers: S chain done (one per S buffer), PV chain done, K / V buffer filled by TMA
-    const uint32_t barS[2] = {smem_u32(&s_bar[0]), smem_u32(&s_bar[1])};
-    const uint32_t barO = smem_u32(&s_bar[2]);
-    const uint32_t barK[2] = {smem_u32(&s_bar[3]), smem_u32(&s_bar[4])};
-    const uint32_t barV[2] = {smem_u32(&s_bar[5]), smem_u32(&s_bar[6])};
+    const uint32_t barS = smem_u32(&s_bar[0]), barO = smem_u32(&s_bar[1]);
+    const uint32_t barF[2] = {smem_u32(&s_bar[2]), smem_u32(&s_bar[3])};
     const bool tma_ok = a.use_tma != 0;
     if (tid == 0) {
-#pragma unroll
-        for (int i = 0; i < 7; ++i) mbar_init(smem_u32(&s_bar[i]), 1);
+        mbar_init(barS, 1);
+        mbar_init(barO, 1);
+        mbar_init(barF[0], 1);
+        mbar_init(barF[1], 1);
         s_fail = 0;
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     }
@@ -263,39 +262,37 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
     }
     // row of the cache planes (as one [batch*Hkv*max_len][128] matrix) where this kv head starts
     const int plane_row0 = (b * a.Hkv + g) * a.max_len;
-    // A chunk that lies inside the cached prefix comes by TMA (two 64 x 128 boxes per operand, one
-    // issuing thread, completion on the buffer's mbarrier); the chunk that mixes prefix, tree rows
-    // and zero padding is gathered with 16-byte asynchronous copies by all threads.
-    auto is_tma = [&](int ch) { return tma_ok && (ch + 1) * BK <= L; };
-    auto load_operand = [&](int ch, int buf, bool is_v) {
-        const uint32_t dst = (is_v ? sV : sK) + buf * TILE;
-        if (is_tma(ch)) {
+    auto load_chunk = [&](int ch, int buf) {
+        const uint32_t dK = sK + buf * TILE, dV = sV + buf * TILE;
+        if (tma_ok && (ch + 1) * BK <= L) {
+            // the whole chunk is cached prefix: four 64 x 128 boxes, one thread, no register traffic
             if (tid == 0) {
-                const uint32_t bar = is_v ? barV[buf] : barK[buf];
-                const CUtensorMap *map = is_v ? &tmV : &tmK;
-                mbar_expect_tx(bar, TILE);
+                mbar_expect_tx(barF[buf], 2 * TILE);
                 const int y = plane_row0 + ch * BK;
-                tma_load_2d(dst, map, 0, y, bar);
-                tma_load_2d(dst + HALF, map, 64, y, bar);
+                tma_load_2d(dK, &tmK, 0, y, barF[buf]);
+                tma_load_2d(dK + HALF, &tmK, 64, y, barF[buf]);
+                tma_load_2d(dV, &tmV, 0, y, barF[buf]);
+                tma_load_2d(dV + HALF, &tmV, 64, y, barF[buf]);
             }
             return;
         }
         const int c = tid & 15;
-        const fspad_bf16 *cb = is_v ? vcb : kcb, *tb = is_v ? tvb : tkb;
         for (int r = tid >> 4; r < BK; r += NT / 16) {
             const int key = ch * BK + r;
             const bool ok = key < Ltot;
-            const fspad_bf16 *src = cb;
-            if (ok) src = (key < L) ? cb + (size_t)key * D + c * 8 : tb + (size_t)(key - L) * D + c * 8;
-            cp_async16(dst + tile_off(r, c), src, ok);
+            const fspad_bf16 *ks = kcb, *vs = vcb;
+            if (ok) {
+                if (key < L) { ks = kcb + (size_t)key * D + c * 8; vs = vcb + (size_t)key * D + c * 8; }
+                else { ks = tkb + (size_t)(key - L) * D + c * 8; vs = tvb + (size_t)(key - L) * D + c * 8; }
+            }
+            cp_async16(dK + tile_off(r, c), ks, ok);
+            cp_async16(dV + tile_off(r, c), vs, ok);
         }
-        cp_async_commit();
     };
-    const int n_ch = c1 - c0;
-    cp_async_commit();                            // Q
-    load_operand(c0, 0, false);
-    load_operand(c0, 0, true);
-    if (n_ch > 1) { load_operand(c0 + 1, 1, false); load_operand(c0 + 1, 1, true); }
+    load_chunk(c0, 0);
+    cp_async_commit();
+    if (c0 + 1 < c1) load_chunk(c0 + 1, 1);
+    cp_async_commit();
 
     // ---- tree -> ancestor-or-self masks (parents staged in shared memory, then walked there) ----
     if (tid < N) s_par[tid] = a.parent[(size_t)b * N + tid];
@@ -325,71 +322,43 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
     tc_fence_after();
     const uint32_t tmem = s_tmem;
     const uint32_t lanes = (uint32_t)((row >> 5) * 32) << 16;
-    const uint32_t tSrow = tmem + lanes + (uint32_t)(half * 64);         // + 128 * (S buffer): this thread's 64 score columns
-    const uint32_t tO = tmem + lanes + 256u + (uint32_t)(half * 64);     // its 64 output columns
+    const uint32_t tS = tmem + lanes + (uint32_t)(half * 64);            // this thread's 64 score columns
+    const uint32_t tO = tmem + lanes + 128u + (uint32_t)(half * 64);     // and its 64 output columns
     const uint32_t idesc_s = make_idesc(false), idesc_o = make_idesc(true);
     const unsigned long long anc = s_anc[node];
     const float scale = a.scale_log2;
 
     float m_run = -INFINITY, l_part = 0.f;       // row maximum (shared by both halves), this half's sum
-    uint32_t phS[2] = {0, 0}, phO = 0, phK[2] = {0, 0}, phV[2] = {0, 0};
+    uint32_t phS = 0, phO = 0, phF[2] = {0, 0};
     bool failed = false;
 
-    // Wait until an operand buffer holds chunk `ch`.  TMA chunks: the buffer's mbarrier (only the
-    // waiting warp needs it); gathered chunks: all of this thread's copies, then a CTA barrier.
-    auto operand_ready = [&](int ch, int buf, bool is_v, bool whole_cta) {
-        if (is_tma(ch)) {
-            uint32_t &ph = is_v ? phV[buf] : phK[buf];
-            if (!failed && !mbar_wait(is_v ? barV[buf] : barK[buf], ph)) { failed = true; s_fail = 1; }
-            ph ^= 1;
-        } else if (whole_cta) {
-            cp_async_wait<0>();
-            fence_async_smem();
-            __syncthreads();
+    for (int ch = c0; ch < c1; ++ch) {
+        const int buf = (ch - c0) & 1;
+        // this chunk's copies have landed (the younger group, if any, may still be in flight)
+        if (ch + 1 < c1) cp_async_wait<1>(); else cp_async_wait<0>();
+        if (tma_ok && (ch + 1) * BK <= L) {
+            if (!failed && !mbar_wait(barF[buf], phF[buf])) { failed = true; s_fail = 1; }
+            phF[buf] ^= 1;
         }
-    };
-    auto issue_s = [&](int i) {                   // S[i & 1] = Q K(i)^T, by one thread
+        fence_async_smem();
+        __syncthreads();
         if (tid == 0 && !failed) {
             tc_fence_after();
-            const int sb = i & 1;
 #pragma unroll
             for (int ks = 0; ks < 8; ++ks) {     // K = 16 per instruction over d = 128
                 const uint32_t koff = (ks >> 2) * HALF + (ks & 3) * 32;
-                mma_f16(tmem + 128u * sb, make_desc(sQ + koff, 16), make_desc(sK + sb * TILE + koff, 16), idesc_s,
-                        ks > 0);
+                mma_f16(tmem, make_desc(sQ + koff, 16), make_desc(sK + buf * TILE + koff, 16), idesc_s, ks > 0);
             }
-            mma_commit(barS[sb]);
+            mma_commit(barS);
         }
-    };
-
-    // Q (and a gathered first chunk) must have landed before the first product
-    cp_async_wait<0>();
-    fence_async_smem();
-    __syncthreads();
-    if (is_tma(c0)) operand_ready(c0, 0, false, false);
-    issue_s(0);
-    int s_issued = 1;
-
-    for (int i = 0; i < n_ch; ++i) {
-        const int ch = c0 + i, buf = i & 1;
-        // ---- (1) the next chunk's QK^T goes to the tensor cores before this chunk's softmax ----
-        // (TMA chunks only: the wait is a single warp's business; a gathered chunk is issued in (7))
-        if (i + 1 < n_ch && is_tma(ch + 1) && warp == 0) {
-            operand_ready(ch + 1, buf ^ 1, false, false);
-            issue_s(i + 1);
-        }
-        if (i + 1 < n_ch && is_tma(ch + 1)) s_issued = i + 2;
-
-        // ---- (2) this chunk's scores are complete: its K buffer is free for chunk i + 2 ----
-        if (!failed && !mbar_wait(barS[buf], phS[buf])) { failed = true; s_fail = 1; }
-        phS[buf] ^= 1;
+        if (!failed && !mbar_wait(barS, phS)) { failed = true; s_fail = 1; }
+        phS ^= 1;
         tc_fence_after();
-        if (i + 2 < n_ch && is_tma(ch + 2)) load_operand(ch + 2, buf, false);
 
-        // ---- (3) this thread's 64 scores: mask, row maximum (exchanged with the other half) ----
+        // ---- this thread's 64 scores: mask, row maximum (exchanged with the other half) ----
         float sc[2][32];
-        tmem_ld32(tSrow + 128u * buf, sc[0]);
-        tmem_ld32(tSrow + 128u * buf + 32, sc[1]);
+        tmem_ld32(tS, sc[0]);
+        tmem_ld32(tS + 32, sc[1]);
         if ((ch + 1) * BK > L) {                 // only chunks that reach past the cached prefix
 #pragma unroll
             for (int q2 = 0; q2 < 2; ++q2)
@@ -414,37 +383,28 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
         const float m_safe = (m_new == -INFINITY) ? 0.f : m_new;
         const float alpha = ex2f(m_run - m_safe);
         float rs = 0.f;
-        uint32_t pw[2][16];
 #pragma unroll
-        for (int q2 = 0; q2 < 2; ++q2)
+        for (int q2 = 0; q2 < 2; ++q2) {
 #pragma unroll
-            for (int e = 0; e < 16; ++e) {
-                const float p0 = ex2f(fmaf(sc[q2][2 * e], scale, -m_safe));
-                const float p1 = ex2f(fmaf(sc[q2][2 * e + 1], scale, -m_safe));
-                rs += p0 + p1;
-                pw[q2][e] = pack_bf16(p0, p1);
+            for (int c8 = 0; c8 < 4; ++c8) {     // 8 keys = one 16-byte chunk of the P row
+                uint32_t w[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const float p0 = ex2f(fmaf(sc[q2][c8 * 8 + 2 * e], scale, -m_safe));
+                    const float p1 = ex2f(fmaf(sc[q2][c8 * 8 + 2 * e + 1], scale, -m_safe));
+                    rs += p0 + p1;
+                    w[e] = pack_bf16(p0, p1);
+                }
+                const int c = half * 8 + q2 * 4 + c8;   // chunk 0..15 of this row of P
+                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};\n"
+                             :: "r"(sP + tile_off(row, c)), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]) : "memory");
             }
+        }
         l_part = l_part * alpha + rs;
         m_run = m_new;
 
-        // ---- (4) the previous chunk's PV has finished: P and that V buffer are free ----
-        if (i > 0) {
-            if (!failed && !mbar_wait(barO, phO)) { failed = true; s_fail = 1; }
-            phO ^= 1;
-            tc_fence_after();
-            if (i + 1 < n_ch && is_tma(ch + 1)) load_operand(ch + 1, buf ^ 1, true);
-        }
-        // ---- (5) P -> shared memory (bf16, swizzled); rescale this thread's half of the O row ----
-#pragma unroll
-        for (int q2 = 0; q2 < 2; ++q2)
-#pragma unroll
-            for (int c8 = 0; c8 < 4; ++c8) {     // 8 keys = one 16-byte chunk of the P row
-                const int c = half * 8 + q2 * 4 + c8;
-                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};\n"
-                             :: "r"(sP + tile_off(row, c)), "r"(pw[q2][c8 * 4]), "r"(pw[q2][c8 * 4 + 1]),
-                                "r"(pw[q2][c8 * 4 + 2]), "r"(pw[q2][c8 * 4 + 3]) : "memory");
-            }
-        if (i > 0) {
+        // ---- rescale this thread's half of the O row when a previous chunk has contributed ----
+        if (ch > c0) {
 #pragma unroll
             for (int q2 = 0; q2 < 2; ++q2) {
                 float o[32];
@@ -455,17 +415,9 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
             }
             asm volatile("tcgen05.wait::st.sync.aligned;\n" ::: "memory");
         }
-        // gathered (non-TMA) operands of the chunks to come are fetched here by all threads; their
-        // buffers are free: K[buf ^ 1 .. ] after S(i), V[buf ^ 1] after PV(i - 1)
-        if (i + 1 < n_ch && !is_tma(ch + 1) && i > 0) load_operand(ch + 1, buf ^ 1, true);
-        if (i + 2 < n_ch && !is_tma(ch + 2)) load_operand(ch + 2, buf, false);
-        // ---- (6) O += P V(i) ----
-        if (warp == 0) operand_ready(ch, buf, true, false);   // TMA chunk: V(i) has landed
-        if (!is_tma(ch)) cp_async_wait<0>();                   // gathered chunk: this thread's copies
         fence_async_smem();
         tc_fence_before();
         __syncthreads();
-        failed = failed || (s_fail != 0);
         if (tid == 0 && !failed) {
             tc_fence_after();
 #pragma unroll
@@ -473,24 +425,19 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
                 const uint64_t da = make_desc(sP + (ks >> 2) * HALF + (ks & 3) * 32, 16);
                 // V as an MN-major operand: d is contiguous, the two 64-wide halves are HALF bytes apart
                 const uint64_t db = make_desc(sV + buf * TILE + ks * 16 * 128, HALF);
-                mma_f16(tmem + 256u, da, db, idesc_o, (i > 0) || (ks > 0));
+                mma_f16(tmem + 128u, da, db, idesc_o, (ch > c0) || (ks > 0));
             }
             mma_commit(barO);
         }
-        // ---- (7) a gathered next chunk: its QK^T is issued now (its copies were waited for above) ----
-        if (i + 1 < n_ch && s_issued == i + 1) {
-            cp_async_wait<0>();
-            fence_async_smem();
-            __syncthreads();
-            issue_s(i + 1);
-            s_issued = i + 2;
-        }
+        // P, this K/V buffer and the S columns are free again once these products have completed
+        if (!failed && !mbar_wait(barO, phO)) { failed = true; s_fail = 1; }
+        phO ^= 1;
+        tc_fence_after();
+        __syncthreads();
+        failed = failed || (s_fail != 0);
+        if (ch + 2 < c1) load_chunk(ch + 2, buf);
+        cp_async_commit();
     }
-    // the last PV
-    if (!failed && !mbar_wait(barO, phO)) { failed = true; s_fail = 1; }
-    tc_fence_after();
-    __syncthreads();
-    failed = failed || (s_fail != 0);
 
     fspad_pdl_trigger();                          // the merge kernel may start launching
     // ---- publish the partial: unnormalised O row, running max and sum ----
