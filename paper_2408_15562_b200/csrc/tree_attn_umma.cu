@@ -31,11 +31,11 @@ namespace umma {
 constexpr int D = FSPAD_HEAD_DIM;      // 128
 constexpr int BM = 128;                // query rows per CTA
 constexpr int BK = 128;                // keys per chunk
-constexpr int NT = 256;                // threads per CTA: two per query row
+constexpr int NT = 288;                // threads per CTA: two per query row + one producer warp
 constexpr int HALF = 128 * 128;        // bytes of one [128 rows][64 bf16] half tile
 constexpr int TILE = 2 * HALF;         // bytes of one [128][128] bf16 tile
 constexpr int SMEM_BYTES = 6 * TILE + 1024;   // Q, K[2], V[2], P + alignment slack
-constexpr uint32_t TMEM_COLS = 256;    // S: columns 0..127, O: columns 128..255
+constexpr uint32_t TMEM_COLS = 512;    // S (two buffers): columns 0..255, O: columns 256..383
 constexpr uint32_t WAIT_CAP = 200000;   // polls of a bounded mbarrier wait
 struct Args {
     const fspad_bf16 *q, *kc, *vc, *tk, *tv;
@@ -85,7 +85,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
     if ((threadIdx.x & 31) == 0) {
         for (uint32_t i = 0; i < WAIT_CAP && !ok; ++i) {
             ok = mbar_test(bar, parity) ? 1 : 0;
-            if (!ok) __nanosleep(40);
+            if (!ok && i >= 64) __nanosleep(40);      // the first polls spin: hand-offs are short
         }
     }
     ok = __shfl_sync(0xffffffffu, ok, 0);
@@ -186,23 +186,40 @@ __device__ __forceinline__ float ex2f(float x)
     return y;
 }
 
-// Two threads share a query row: thread (row, half) owns columns half*64 .. half*64+63 of the
-// row's scores, of its P row and of its O row.  Warps w and w+4 address the same 32 lanes of
-// tensor memory (a warp reaches the lane quarter given by its index modulo 4).
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];\n" ::"r"(bar) : "memory");
+}
+// barrier among the 256 softmax threads only (hardware barrier 1; barrier 0 is __syncthreads)
+__device__ __forceinline__ void softmax_sync() { asm volatile("bar.sync 1, 256;\n" ::: "memory"); }
+
+// Roles.  Warps 0-7 (256 threads) are the softmax warps: two threads share a query row, thread
+// (row, half) owns columns half*64 .. half*64+63 of the row's scores, of its P row and of its O
+// row; warps w and w+4 address the same 32 lanes of tensor memory (a warp reaches the lane
+// quarter given by its index modulo 4).  Warp 8 is the producer: it issues every TMA copy and
+// every tcgen05.mma, gathers the one chunk TMA cannot describe, and owns the tensor memory.
+// The two sides meet only on mbarriers, never on a CTA-wide barrier inside the loop:
+//   kfull/vfull(b)  K / V buffer b filled (TMA transaction count)           producer waits
+//   sfull(b)        S buffer b holds Q K^T of its chunk (tcgen05.commit)     softmax + producer wait
+//   pfull           P written, O rescaled and S read by all 8 softmax warps  producer waits
+//   odone           O += P V of the chunk complete (tcgen05.commit)          softmax + producer wait
+// Tensor-core order: S(0) S(1) | PV(0) S(2) | PV(1) S(3) | ...  so the scores of the next chunk
+// are ready before the softmax warps ask for them and PV(i) runs under the softmax of chunk i+1.
 __global__ void __launch_bounds__(NT, 1)
 tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV)
 {
     extern __shared__ unsigned char smem_raw[];
-    __shared__ __align__(8) unsigned long long s_bar[4];     // [0]: S ready, [1]: O updated, [2],[3]: chunk buffer filled by TMA
+    __shared__ __align__(8) unsigned long long s_bar[8];
     __shared__ uint32_t s_tmem;
     __shared__ int s_fail;
     __shared__ int s_par[FSPAD_MAX_NODES];
     __shared__ unsigned long long s_anc[FSPAD_MAX_NODES];
-    __shared__ float s_mx[2][BM];                            // per-half row maxima / sums exchange
+    __shared__ float s_mx[2][2][BM];                         // [chunk parity][half][row]: row maxima / sums exchange
 
     fspad_pdl_wait();
-    const int tid = threadIdx.x, warp = tid >> 5;
-    const int row = tid & (BM - 1), half = tid >> 7;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const bool producer = warp == 8;
+    const int row = tid & (BM - 1), half = (tid >> 7) & 1;
     const int split = blockIdx.x;
     const int g = blockIdx.y / a.mtiles, mt = blockIdx.y % a.mtiles;
     const int b = blockIdx.z;
@@ -217,9 +234,10 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
     const int n_chunks = (Ltot + BK - 1) / BK;
     const int per = (n_chunks + a.n_splits - 1) / a.n_splits;
     const int c0 = split * per, c1 = min(n_chunks, c0 + per);
+    const int n_ch = c1 - c0;
 
     const int gr = mt * BM + row;                 // this thread's row among the kv head's M rows
-    const bool row_ok = gr < M;
+    const bool row_ok = gr < M && !producer;
     const int node = row_ok ? gr / G : 0;
     const size_t prow = ((size_t)b * a.Hkv + g) * a.n_splits + split;
 
@@ -231,79 +249,84 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
     // 1024-byte aligned tiles: Q | K0 | K1 | V0 | V1 | P
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t sQ = base, sK = base + TILE, sV = base + 3 * TILE, sP = base + 5 * TILE;
-    const uint32_t barS = smem_u32(&s_bar[0]), barO = smem_u32(&s_bar[1]);
-    const uint32_t barF[2] = {smem_u32(&s_bar[2]), smem_u32(&s_bar[3])};
+    const uint32_t bar0 = smem_u32(&s_bar[0]);
+    auto kfull = [&](int buf) { return bar0 + 8u * (uint32_t)buf; };
+    auto vfull = [&](int buf) { return bar0 + 16u + 8u * (uint32_t)buf; };
+    auto sfull = [&](int buf) { return bar0 + 32u + 8u * (uint32_t)buf; };
+    const uint32_t pfull = bar0 + 48u, odone = bar0 + 56u;
     const bool tma_ok = a.use_tma != 0;
     if (tid == 0) {
-        mbar_init(barS, 1);
-        mbar_init(barO, 1);
-        mbar_init(barF[0], 1);
-        mbar_init(barF[1], 1);
+#pragma unroll
+        for (int i = 0; i < 6; ++i) mbar_init(bar0 + 8u * i, 1);
+        mbar_init(pfull, 8);
+        mbar_init(odone, 1);
         s_fail = 0;
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     }
+    if (tid < N) s_par[tid] = a.parent[(size_t)b * N + tid];
     __syncthreads();
 
     const fspad_bf16 *kcb = a.kc + ((size_t)b * a.Hkv + g) * (size_t)a.max_len * D;
     const fspad_bf16 *vcb = a.vc + ((size_t)b * a.Hkv + g) * (size_t)a.max_len * D;
     const fspad_bf16 *tkb = a.tk ? a.tk + ((size_t)b * a.Hkv + g) * (size_t)N * D : kcb + (size_t)L * D;
     const fspad_bf16 *tvb = a.tv ? a.tv + ((size_t)b * a.Hkv + g) * (size_t)N * D : vcb + (size_t)L * D;
+    const int plane_row0 = (b * a.Hkv + g) * a.max_len;   // first row of this kv head in the cache planes
+    auto is_tma = [&](int ch) { return tma_ok && (ch + 1) * BK <= L; };
 
-    // ---- the copies go out first; everything else of the prologue hides under their latency ----
-    {
-        const int c = tid & 15;                   // 16-byte chunk of the row, fixed per thread
-        for (int r = tid >> 4; r < BM; r += NT / 16) {
-            const int grr = mt * BM + r;
-            const bool ok = grr < M;
-            const int nd = ok ? grr / G : 0, hh = ok ? grr % G : 0;
-            const fspad_bf16 *src = a.q + (((size_t)b * N + nd) * a.Hq + g * G + hh) * D + c * 8;
-            cp_async16(sQ + tile_off(r, c), src, ok);
-        }
-    }
-    // row of the cache planes (as one [batch*Hkv*max_len][128] matrix) where this kv head starts
-    const int plane_row0 = (b * a.Hkv + g) * a.max_len;
-    auto load_chunk = [&](int ch, int buf) {
-        const uint32_t dK = sK + buf * TILE, dV = sV + buf * TILE;
-        if (tma_ok && (ch + 1) * BK <= L) {
-            // the whole chunk is cached prefix: four 64 x 128 boxes, one thread, no register traffic
-            if (tid == 0) {
-                mbar_expect_tx(barF[buf], 2 * TILE);
-                const int y = plane_row0 + ch * BK;
-                tma_load_2d(dK, &tmK, 0, y, barF[buf]);
-                tma_load_2d(dK + HALF, &tmK, 64, y, barF[buf]);
-                tma_load_2d(dV, &tmV, 0, y, barF[buf]);
-                tma_load_2d(dV + HALF, &tmV, 64, y, barF[buf]);
-            }
-            return;
-        }
-        const int c = tid & 15;
-        for (int r = tid >> 4; r < BK; r += NT / 16) {
+    // Start the fill of an operand buffer with chunk `ch`.  A chunk inside the cached prefix comes
+    // by TMA (two 64 x 128 boxes, issued by one lane of the producer warp, completion counted on
+    // the buffer's mbarrier); the chunk that mixes prefix, tree rows and zero padding is gathered
+    // with 16-byte asynchronous copies by the threads t0, t0 + nt, ... that the caller names (the
+    // whole CTA in the prologue, the producer warp alone inside the loop).
+    auto gather = [&](int ch, int buf, bool is_v, int t0, int nt) {
+        const uint32_t dst = (is_v ? sV : sK) + buf * TILE;
+        const fspad_bf16 *cb = is_v ? vcb : kcb, *tb = is_v ? tvb : tkb;
+        for (int i = t0; i < BK * 16; i += nt) {
+            const int r = i >> 4, c = i & 15;
             const int key = ch * BK + r;
             const bool ok = key < Ltot;
-            const fspad_bf16 *ks = kcb, *vs = vcb;
-            if (ok) {
-                if (key < L) { ks = kcb + (size_t)key * D + c * 8; vs = vcb + (size_t)key * D + c * 8; }
-                else { ks = tkb + (size_t)(key - L) * D + c * 8; vs = tvb + (size_t)(key - L) * D + c * 8; }
-            }
-            cp_async16(dK + tile_off(r, c), ks, ok);
-            cp_async16(dV + tile_off(r, c), vs, ok);
+            const fspad_bf16 *src = cb;
+            if (ok) src = (key < L) ? cb + (size_t)key * D + c * 8 : tb + (size_t)(key - L) * D + c * 8;
+            cp_async16(dst + tile_off(r, c), src, ok);
         }
     };
-    load_chunk(c0, 0);
-    cp_async_commit();
-    if (c0 + 1 < c1) load_chunk(c0 + 1, 1);
-    cp_async_commit();
+    auto tma_fill = [&](int ch, int buf, bool is_v) {       // one lane
+        const uint32_t dst = (is_v ? sV : sK) + buf * TILE;
+        const uint32_t bar = is_v ? vfull(buf) : kfull(buf);
+        const CUtensorMap *map = is_v ? &tmV : &tmK;
+        mbar_expect_tx(bar, TILE);
+        const int y = plane_row0 + ch * BK;
+        tma_load_2d(dst, map, 0, y, bar);
+        tma_load_2d(dst + HALF, map, 64, y, bar);
+    };
 
-    // ---- tree -> ancestor-or-self masks (parents staged in shared memory, then walked there) ----
-    if (tid < N) s_par[tid] = a.parent[(size_t)b * N + tid];
-    if (warp == 1) {                              // one (converged) warp allocates the tensor memory
+    // ---- prologue: the first two chunks and Q go out first, the rest hides under their latency ----
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+        if (u >= n_ch) break;
+        if (is_tma(c0 + u)) {
+            if (producer && lane == 0) { tma_fill(c0 + u, u, false); tma_fill(c0 + u, u, true); }
+        } else {
+            gather(c0 + u, u, false, tid, NT);
+            gather(c0 + u, u, true, tid, NT);
+        }
+    }
+    for (int i = tid; i < BM * 16; i += NT) {
+        const int r = i >> 4, c = i & 15;
+        const int grr = mt * BM + r;
+        const bool ok = grr < M;
+        const int nd = ok ? grr / G : 0, hh = ok ? grr % G : 0;
+        const fspad_bf16 *src = a.q + (((size_t)b * N + nd) * a.Hq + g * G + hh) * D + c * 8;
+        cp_async16(sQ + tile_off(r, c), src, ok);
+    }
+    cp_async_commit();
+    if (producer) {
         __syncwarp();
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n"
                      :: "r"(smem_u32(&s_tmem)), "r"(TMEM_COLS) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
-    }
-    __syncthreads();
-    if (tid < N) {
+    } else if (tid < N) {
+        // tree -> ancestor-or-self masks (parents were staged in shared memory above)
         unsigned long long mask = 0ull;
         int cur = tid;
         bool bad = false;
@@ -317,136 +340,183 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
         if (bad) fspad_report(a.status, FSPAD_ERR_BAD_TREE);
         s_anc[tid] = mask;
     }
+    cp_async_wait<0>();                           // Q and any gathered chunk
+    fence_async_smem();
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = s_tmem;
-    const uint32_t lanes = (uint32_t)((row >> 5) * 32) << 16;
-    const uint32_t tS = tmem + lanes + (uint32_t)(half * 64);            // this thread's 64 score columns
-    const uint32_t tO = tmem + lanes + 128u + (uint32_t)(half * 64);     // and its 64 output columns
     const uint32_t idesc_s = make_idesc(false), idesc_o = make_idesc(true);
-    const unsigned long long anc = s_anc[node];
-    const float scale = a.scale_log2;
-
-    float m_run = -INFINITY, l_part = 0.f;       // row maximum (shared by both halves), this half's sum
-    uint32_t phS = 0, phO = 0, phF[2] = {0, 0};
     bool failed = false;
 
-    for (int ch = c0; ch < c1; ++ch) {
-        const int buf = (ch - c0) & 1;
-        // this chunk's copies have landed (the younger group, if any, may still be in flight)
-        if (ch + 1 < c1) cp_async_wait<1>(); else cp_async_wait<0>();
-        if (tma_ok && (ch + 1) * BK <= L) {
-            if (!failed && !mbar_wait(barF[buf], phF[buf])) { failed = true; s_fail = 1; }
-            phF[buf] ^= 1;
-        }
-        fence_async_smem();
-        __syncthreads();
-        if (tid == 0 && !failed) {
-            tc_fence_after();
-#pragma unroll
-            for (int ks = 0; ks < 8; ++ks) {     // K = 16 per instruction over d = 128
-                const uint32_t koff = (ks >> 2) * HALF + (ks & 3) * 32;
-                mma_f16(tmem, make_desc(sQ + koff, 16), make_desc(sK + buf * TILE + koff, 16), idesc_s, ks > 0);
+    if (producer) {
+        // ================= producer warp: copies and tensor-core issue =================
+        uint32_t ph_fill = 0;                    // phase bits: K buffers 0,1 then V buffers 0,1
+        // warp-uniform: chunk `ch` has landed in K (or V) buffer `buf`
+        auto wait_fill = [&](int ch, int buf, bool is_v) -> bool {
+            if (is_tma(ch)) {
+                const uint32_t bit = (uint32_t)buf + (is_v ? 2u : 0u);
+                const bool ok = mbar_wait(is_v ? vfull(buf) : kfull(buf), (ph_fill >> bit) & 1u);
+                ph_fill ^= 1u << bit;
+                return ok;
             }
-            mma_commit(barS);
+            cp_async_wait<0>();                  // gathered by this warp (or in the prologue)
+            fence_async_smem();
+            __syncwarp();
+            return true;
+        };
+        auto fill = [&](int ch, int buf, bool is_v) {
+            if (is_tma(ch)) {
+                if (lane == 0) tma_fill(ch, buf, is_v);
+            } else {
+                gather(ch, buf, is_v, lane, 32);
+                cp_async_commit();
+            }
+        };
+        auto issue_s = [&](int i) {              // S[i & 1] = Q K(i)^T
+            const int buf = i & 1;
+            if (!failed && !wait_fill(c0 + i, buf, false)) failed = true;
+            if (lane == 0 && !failed) {
+                tc_fence_after();
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) { // K = 16 per instruction over d = 128
+                    const uint32_t koff = (ks >> 2) * HALF + (ks & 3) * 32;
+                    mma_f16(tmem + (uint32_t)buf * 128u, make_desc(sQ + koff, 16),
+                            make_desc(sK + buf * TILE + koff, 16), idesc_s, ks > 0);
+                }
+                mma_commit(sfull(buf));
+            }
+            __syncwarp();
+        };
+        issue_s(0);
+        if (n_ch > 1) issue_s(1);
+        for (int i = 0; i < n_ch; ++i) {
+            const int buf = i & 1;
+            const bool more = i + 2 < n_ch;
+            if (more) {                          // K buffer is free once S(i) has completed
+                if (!failed && !mbar_wait(sfull(buf), (uint32_t)(i >> 1) & 1u)) failed = true;
+                if (!failed) fill(c0 + i + 2, buf, false);
+            }
+            // O += P(i) V(i): needs P from all softmax warps and the V chunk
+            if (!failed && !mbar_wait(pfull, (uint32_t)i & 1u)) failed = true;
+            if (!failed && !wait_fill(c0 + i, buf, true)) failed = true;
+            if (lane == 0 && !failed) {
+                tc_fence_after();
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) { // K = 16 keys per instruction over the chunk's 128 keys
+                    const uint64_t da = make_desc(sP + (ks >> 2) * HALF + (ks & 3) * 32, 16);
+                    // V as an MN-major operand: d is contiguous, the two 64-wide halves are HALF bytes apart
+                    const uint64_t db = make_desc(sV + buf * TILE + ks * 16 * 128, HALF);
+                    mma_f16(tmem + 256u, da, db, idesc_o, (i > 0) || (ks > 0));
+                }
+                mma_commit(odone);
+            }
+            __syncwarp();
+            // the S buffer of chunk i was read before P(i) was announced, so it can take chunk i + 2
+            if (more) issue_s(i + 2);
+            // V buffer and P are free once the products have completed
+            if (!failed && !mbar_wait(odone, (uint32_t)i & 1u)) failed = true;
+            if (more && !failed) fill(c0 + i + 2, buf, true);
         }
-        if (!failed && !mbar_wait(barS, phS)) { failed = true; s_fail = 1; }
-        phS ^= 1;
-        tc_fence_after();
+        cp_async_wait<0>();
+        if (failed) s_fail = 1;
+    } else {
+        // ================= softmax warps =================
+        const uint32_t lanes = (uint32_t)((row >> 5) * 32) << 16;
+        const uint32_t tO = tmem + lanes + 256u + (uint32_t)(half * 64);     // this thread's 64 output columns
+        const unsigned long long anc = s_anc[node];
+        const float scale = a.scale_log2;
+        float m_run = -INFINITY, l_part = 0.f;   // row maximum (shared by both halves), this half's sum
 
-        // ---- this thread's 64 scores: mask, row maximum (exchanged with the other half) ----
-        float sc[2][32];
-        tmem_ld32(tS, sc[0]);
-        tmem_ld32(tS + 32, sc[1]);
-        if ((ch + 1) * BK > L) {                 // only chunks that reach past the cached prefix
+        for (int i = 0; i < n_ch; ++i) {
+            const int ch = c0 + i, sb = i & 1;
+            if (!failed && !mbar_wait(sfull(sb), (uint32_t)(i >> 1) & 1u)) failed = true;
+            tc_fence_after();
+            // ---- this thread's 64 scores: mask, row maximum (exchanged with the other half) ----
+            const uint32_t tS = tmem + lanes + (uint32_t)(sb * 128 + half * 64);
+            float sc[2][32];
+            tmem_ld32(tS, sc[0]);
+            tmem_ld32(tS + 32, sc[1]);
+            if ((ch + 1) * BK > L) {             // only chunks that reach past the cached prefix
+#pragma unroll
+                for (int q2 = 0; q2 < 2; ++q2)
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        const int key = ch * BK + half * 64 + q2 * 32 + j;
+                        if (key >= L) {
+                            const bool ok = (key < Ltot) && ((anc >> (key - L)) & 1ull);
+                            if (!ok) sc[q2][j] = -INFINITY;
+                        }
+                    }
+            }
+            float mx = -INFINITY;
 #pragma unroll
             for (int q2 = 0; q2 < 2; ++q2)
 #pragma unroll
-                for (int j = 0; j < 32; ++j) {
-                    const int key = ch * BK + half * 64 + q2 * 32 + j;
-                    if (key >= L) {
-                        const bool ok = (key < Ltot) && ((anc >> (key - L)) & 1ull);
-                        if (!ok) sc[q2][j] = -INFINITY;
-                    }
-                }
-        }
-        float mx = -INFINITY;
+                for (int j = 0; j < 32; ++j) mx = fmaxf(mx, sc[q2][j]);
+            s_mx[sb][half][row] = mx;
+            softmax_sync();
+            mx = fmaxf(mx, s_mx[sb][half ^ 1][row]);
+            const float m_new = fmaxf(m_run, mx * scale);
+            const float m_safe = (m_new == -INFINITY) ? 0.f : m_new;
+            const float alpha = ex2f(m_run - m_safe);
+            float rs = 0.f;
+            uint32_t w[32];
 #pragma unroll
-        for (int q2 = 0; q2 < 2; ++q2)
+            for (int q2 = 0; q2 < 2; ++q2)
 #pragma unroll
-            for (int j = 0; j < 32; ++j) mx = fmaxf(mx, sc[q2][j]);
-        s_mx[half][row] = mx;
-        __syncthreads();
-        mx = fmaxf(mx, s_mx[half ^ 1][row]);
-        const float m_new = fmaxf(m_run, mx * scale);
-        const float m_safe = (m_new == -INFINITY) ? 0.f : m_new;
-        const float alpha = ex2f(m_run - m_safe);
-        float rs = 0.f;
-#pragma unroll
-        for (int q2 = 0; q2 < 2; ++q2) {
-#pragma unroll
-            for (int c8 = 0; c8 < 4; ++c8) {     // 8 keys = one 16-byte chunk of the P row
-                uint32_t w[4];
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const float p0 = ex2f(fmaf(sc[q2][c8 * 8 + 2 * e], scale, -m_safe));
-                    const float p1 = ex2f(fmaf(sc[q2][c8 * 8 + 2 * e + 1], scale, -m_safe));
+                for (int e = 0; e < 16; ++e) {
+                    const float p0 = ex2f(fmaf(sc[q2][2 * e], scale, -m_safe));
+                    const float p1 = ex2f(fmaf(sc[q2][2 * e + 1], scale, -m_safe));
                     rs += p0 + p1;
-                    w[e] = pack_bf16(p0, p1);
+                    w[q2 * 16 + e] = pack_bf16(p0, p1);
                 }
-                const int c = half * 8 + q2 * 4 + c8;   // chunk 0..15 of this row of P
+            l_part = l_part * alpha + rs;
+            m_run = m_new;
+            // P (single tile) and O may be touched once the products of the previous chunk are done
+            if (i > 0) {
+                if (!failed && !mbar_wait(odone, (uint32_t)(i - 1) & 1u)) failed = true;
+                tc_fence_after();
+            }
+#pragma unroll
+            for (int c8 = 0; c8 < 8; ++c8) {     // 8 keys = one 16-byte chunk of the P row
+                const int c = half * 8 + c8;
                 asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};\n"
-                             :: "r"(sP + tile_off(row, c)), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]) : "memory");
+                             :: "r"(sP + tile_off(row, c)), "r"(w[c8 * 4]), "r"(w[c8 * 4 + 1]), "r"(w[c8 * 4 + 2]),
+                                "r"(w[c8 * 4 + 3]) : "memory");
             }
-        }
-        l_part = l_part * alpha + rs;
-        m_run = m_new;
-
-        // ---- rescale this thread's half of the O row when a previous chunk has contributed ----
-        if (ch > c0) {
+            // rescale this thread's half of the O row; skipped (warp-uniformly) when no row of the
+            // warp moved its maximum, since the factor is then exactly one
+            if (i > 0 && !__all_sync(0xffffffffu, alpha == 1.f)) {
 #pragma unroll
-            for (int q2 = 0; q2 < 2; ++q2) {
-                float o[32];
-                tmem_ld32(tO + q2 * 32, o);
+                for (int q2 = 0; q2 < 2; ++q2) {
+                    float o[32];
+                    tmem_ld32(tO + q2 * 32, o);
 #pragma unroll
-                for (int j = 0; j < 32; ++j) o[j] *= alpha;
-                tmem_st32(tO + q2 * 32, o);
+                    for (int j = 0; j < 32; ++j) o[j] *= alpha;
+                    tmem_st32(tO + q2 * 32, o);
+                }
+                asm volatile("tcgen05.wait::st.sync.aligned;\n" ::: "memory");
             }
-            asm volatile("tcgen05.wait::st.sync.aligned;\n" ::: "memory");
+            fence_async_smem();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(pfull);
         }
-        fence_async_smem();
+        if (!failed && !mbar_wait(odone, (uint32_t)(n_ch - 1) & 1u)) failed = true;
+        tc_fence_after();
+        if (failed) s_fail = 1;
+        s_mx[0][half][row] = l_part;
+        fspad_pdl_trigger();                      // the merge kernel may start launching
         tc_fence_before();
         __syncthreads();
-        if (tid == 0 && !failed) {
-            tc_fence_after();
-#pragma unroll
-            for (int ks = 0; ks < 8; ++ks) {     // K = 16 keys per instruction over the chunk's 128 keys
-                const uint64_t da = make_desc(sP + (ks >> 2) * HALF + (ks & 3) * 32, 16);
-                // V as an MN-major operand: d is contiguous, the two 64-wide halves are HALF bytes apart
-                const uint64_t db = make_desc(sV + buf * TILE + ks * 16 * 128, HALF);
-                mma_f16(tmem + 128u, da, db, idesc_o, (ch > c0) || (ks > 0));
-            }
-            mma_commit(barO);
-        }
-        // P, this K/V buffer and the S columns are free again once these products have completed
-        if (!failed && !mbar_wait(barO, phO)) { failed = true; s_fail = 1; }
-        phO ^= 1;
         tc_fence_after();
-        __syncthreads();
-        failed = failed || (s_fail != 0);
-        if (ch + 2 < c1) load_chunk(ch + 2, buf);
-        cp_async_commit();
-    }
-
-    fspad_pdl_trigger();                          // the merge kernel may start launching
-    // ---- publish the partial: unnormalised O row, running max and sum ----
-    // Every lane of every warp takes part in the tensor-memory loads (they are warp-collective);
-    // only the stores to global memory depend on whether the lane's row exists.
-    if (failed && tid == 0) fspad_report(a.status, FSPAD_ERR_TIMEOUT);
-    s_mx[half][row] = l_part;
-    {
-        const bool store = row_ok && !failed;
+        // ---- publish the partial: unnormalised O row, running max and sum ----
+        // Every lane of every softmax warp takes part in the tensor-memory loads (they are
+        // warp-collective); only the stores to global memory depend on whether the lane's row exists.
+        const bool any_fail = s_fail != 0;
+        if (any_fail && tid == 0) fspad_report(a.status, FSPAD_ERR_TIMEOUT);
+        const bool store = row_ok && !any_fail;
         float *po = a.part_o + (prow * M + (row_ok ? gr : 0)) * D + half * 64;
 #pragma unroll
         for (int q2 = 0; q2 < 2; ++q2) {
@@ -458,19 +528,23 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
                     *reinterpret_cast<float4 *>(po + q2 * 32 + j) = make_float4(o[j], o[j + 1], o[j + 2], o[j + 3]);
             }
         }
-        cp_async_wait<0>();
-        tc_fence_before();
-        __syncthreads();
         if (store && half == 0) {
             float *ml = a.part_ml + (prow * M + gr) * 2;
             ml[0] = m_run;
-            ml[1] = s_mx[0][row] + s_mx[1][row];
+            ml[1] = s_mx[0][0][row] + s_mx[0][1][row];
         }
+        tc_fence_before();
+        __syncthreads();
+        return;
     }
-    if (warp == 1) {
-        __syncwarp();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" :: "r"(tmem), "r"(TMEM_COLS) : "memory");
-    }
+    // producer: meet the softmax warps at their two CTA-wide barriers, then free the tensor memory
+    fspad_pdl_trigger();
+    tc_fence_before();
+    __syncthreads();
+    __syncthreads();
+    tc_fence_after();
+    __syncwarp();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" :: "r"(tmem), "r"(TMEM_COLS) : "memory");
 }
 
 }  // namespace umma
