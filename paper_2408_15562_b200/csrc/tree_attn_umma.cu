@@ -31,7 +31,7 @@ namespace umma {
 constexpr int D = FSPAD_HEAD_DIM;      // 128
 constexpr int BM = 128;                // query rows per CTA
 constexpr int BK = 128;                // keys per chunk
-constexpr int NT = 288;                // threads per CTA: two per query row + one producer warp
+constexpr int NT = 320;                // threads per CTA: two per query row + a copy warp + a tensor-core warp
 constexpr int HALF = 128 * 128;        // bytes of one [128 rows][64 bf16] half tile
 constexpr int TILE = 2 * HALF;         // bytes of one [128][128] bf16 tile
 constexpr int SMEM_BYTES = 6 * TILE + 1024;   // Q, K[2], V[2], P + alignment slack
@@ -136,6 +136,25 @@ __device__ __forceinline__ void mma_f16(uint32_t d_tmem, uint64_t a_desc, uint64
                  :: "r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(zero), "r"(zero),
                     "r"(zero), "r"(zero) : "memory");
 }
+// same instruction, descriptors handed over as (low, high) words so the issuing thread can keep
+// the precomputed low words in registers and add a tile offset with one integer add
+__device__ __forceinline__ void mma_f16_lo(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
+                                           uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile("{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\tsetp.ne.b32 p, %6, 0;\n\t"
+                 "mov.b64 da, {%1, %2};\n\tmov.b64 db, {%3, %4};\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, p;\n\t}\n"
+                 :: "r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate) : "memory");
+}
+// single-thread bounded wait (the tensor-core thread polls alone; nothing warp-collective follows)
+__device__ __forceinline__ bool mbar_wait_one(uint32_t bar, uint32_t parity)
+{
+    for (uint32_t i = 0; i < WAIT_CAP; ++i) {
+        if (mbar_test(bar, parity)) return true;
+        if (i >= 64) __nanosleep(40);
+    }
+    return false;
+}
 __device__ __forceinline__ void mma_commit(uint32_t bar)
 {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(bar) : "memory");
@@ -196,13 +215,14 @@ __device__ __forceinline__ void softmax_sync() { asm volatile("bar.sync 1, 256;\
 // Roles.  Warps 0-7 (256 threads) are the softmax warps: two threads share a query row, thread
 // (row, half) owns columns half*64 .. half*64+63 of the row's scores, of its P row and of its O
 // row; warps w and w+4 address the same 32 lanes of tensor memory (a warp reaches the lane
-// quarter given by its index modulo 4).  Warp 8 is the producer: it issues every TMA copy and
-// every tcgen05.mma, gathers the one chunk TMA cannot describe, and owns the tensor memory.
+// quarter given by its index modulo 4).  Warp 8 is the copy warp: it issues every TMA copy of
+// the loop and gathers the one chunk TMA cannot describe.  Warp 9 is the tensor-core warp: one
+// of its threads issues every tcgen05.mma; the warp owns the tensor memory.
 // The two sides meet only on mbarriers, never on a CTA-wide barrier inside the loop:
-//   kfull/vfull(b)  K / V buffer b filled (TMA transaction count)           producer waits
-//   sfull(b)        S buffer b holds Q K^T of its chunk (tcgen05.commit)     softmax + producer wait
-//   pfull           P written, O rescaled and S read by all 8 softmax warps  producer waits
-//   odone           O += P V of the chunk complete (tcgen05.commit)          softmax + producer wait
+//   kfull/vfull(b)  K / V buffer b filled (TMA bytes, or one arrival)        tensor-core warp waits
+//   sfull(b)        S buffer b holds Q K^T of its chunk (tcgen05.commit)     softmax + copy warps wait
+//   pfull           P written, O rescaled and S read by all 8 softmax warps  tensor-core warp waits
+//   odone           O += P V of the chunk complete (tcgen05.commit)          softmax + copy warps wait
 // Tensor-core order: S(0) S(1) | PV(0) S(2) | PV(1) S(3) | ...  so the scores of the next chunk
 // are ready before the softmax warps ask for them and PV(i) runs under the softmax of chunk i+1.
 __global__ void __launch_bounds__(NT, 1)
@@ -218,7 +238,7 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
 
     fspad_pdl_wait();
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const bool producer = warp == 8;
+    const bool producer = warp >= 8;         // warp 8 copies, warp 9 drives the tensor cores
     const int row = tid & (BM - 1), half = (tid >> 7) & 1;
     const int split = blockIdx.x;
     const int g = blockIdx.y / a.mtiles, mt = blockIdx.y % a.mtiles;
@@ -305,7 +325,7 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
     for (int u = 0; u < 2; ++u) {
         if (u >= n_ch) break;
         if (is_tma(c0 + u)) {
-            if (producer && lane == 0) { tma_fill(c0 + u, u, false); tma_fill(c0 + u, u, true); }
+            if (tid == 256) { tma_fill(c0 + u, u, false); tma_fill(c0 + u, u, true); }
         } else {
             gather(c0 + u, u, false, tid, NT);
             gather(c0 + u, u, true, tid, NT);
@@ -320,7 +340,7 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
         cp_async16(sQ + tile_off(r, c), src, ok);
     }
     cp_async_commit();
-    if (producer) {
+    if (warp == 9) {
         __syncwarp();
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n"
                      :: "r"(smem_u32(&s_tmem)), "r"(TMEM_COLS) : "memory");
@@ -349,77 +369,81 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
     const uint32_t idesc_s = make_idesc(false), idesc_o = make_idesc(true);
     bool failed = false;
 
-    if (producer) {
-        // ================= producer warp: copies and tensor-core issue =================
-        uint32_t ph_fill = 0;                    // phase bits: K buffers 0,1 then V buffers 0,1
-        // warp-uniform: chunk `ch` has landed in K (or V) buffer `buf`
-        auto wait_fill = [&](int ch, int buf, bool is_v) -> bool {
-            if (is_tma(ch)) {
-                const uint32_t bit = (uint32_t)buf + (is_v ? 2u : 0u);
-                const bool ok = mbar_wait(is_v ? vfull(buf) : kfull(buf), (ph_fill >> bit) & 1u);
-                ph_fill ^= 1u << bit;
-                return ok;
-            }
-            cp_async_wait<0>();                  // gathered by this warp (or in the prologue)
-            fence_async_smem();
-            __syncwarp();
-            return true;
-        };
+    if (warp == 8) {
+        // ================= copy warp: refills the K / V buffers =================
+        // chunks gathered by the whole CTA in the prologue are announced here
+        if (lane == 0) {
+            for (int u = 0; u < 2 && u < n_ch; ++u)
+                if (!is_tma(c0 + u)) { mbar_arrive(kfull(u)); mbar_arrive(vfull(u)); }
+        }
         auto fill = [&](int ch, int buf, bool is_v) {
             if (is_tma(ch)) {
                 if (lane == 0) tma_fill(ch, buf, is_v);
             } else {
                 gather(ch, buf, is_v, lane, 32);
                 cp_async_commit();
+                cp_async_wait<0>();
+                fence_async_smem();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(is_v ? vfull(buf) : kfull(buf));
             }
+            __syncwarp();
         };
-        auto issue_s = [&](int i) {              // S[i & 1] = Q K(i)^T
+        for (int i = 0; i + 2 < n_ch; ++i) {
             const int buf = i & 1;
-            if (!failed && !wait_fill(c0 + i, buf, false)) failed = true;
-            if (lane == 0 && !failed) {
+            // K buffer is free once S(i) has completed, V buffer once O += P(i) V(i) has
+            if (!failed && !mbar_wait(sfull(buf), (uint32_t)(i >> 1) & 1u)) failed = true;
+            if (!failed) fill(c0 + i + 2, buf, false);
+            if (!failed && !mbar_wait(odone, (uint32_t)i & 1u)) failed = true;
+            if (!failed) fill(c0 + i + 2, buf, true);
+        }
+        if (failed) s_fail = 1;
+    } else if (warp == 9) {
+        // ================= tensor-core warp: one thread issues every tcgen05.mma =================
+        if (lane == 0) {
+            // low words of the shared-memory descriptors (start address and leading byte offset);
+            // the high word (8-row group stride, version, swizzle mode) is the same for all
+            const uint32_t hi = (uint32_t)(make_desc(0, 16) >> 32);
+            const uint32_t q_lo = (uint32_t)make_desc(sQ, 16), k_lo = (uint32_t)make_desc(sK, 16);
+            const uint32_t p_lo = (uint32_t)make_desc(sP, 16), v_lo = (uint32_t)make_desc(sV, HALF);
+            auto issue_s = [&](int i) {          // S[i & 1] = Q K(i)^T
+                const int buf = i & 1;
+                if (!failed && !mbar_wait_one(kfull(buf), (uint32_t)(i >> 1) & 1u)) failed = true;
+                if (failed) return;
                 tc_fence_after();
+                const uint32_t kb = k_lo + (uint32_t)buf * (TILE >> 4);
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) { // K = 16 per instruction over d = 128
-                    const uint32_t koff = (ks >> 2) * HALF + (ks & 3) * 32;
-                    mma_f16(tmem + (uint32_t)buf * 128u, make_desc(sQ + koff, 16),
-                            make_desc(sK + buf * TILE + koff, 16), idesc_s, ks > 0);
+                    const uint32_t koff = ((ks >> 2) * HALF + (ks & 3) * 32) >> 4;
+                    mma_f16_lo(tmem + (uint32_t)buf * 128u, q_lo + koff, hi, kb + koff, hi, idesc_s, ks > 0);
                 }
                 mma_commit(sfull(buf));
-            }
-            __syncwarp();
-        };
-        issue_s(0);
-        if (n_ch > 1) issue_s(1);
-        for (int i = 0; i < n_ch; ++i) {
-            const int buf = i & 1;
-            const bool more = i + 2 < n_ch;
-            if (more) {                          // K buffer is free once S(i) has completed
-                if (!failed && !mbar_wait(sfull(buf), (uint32_t)(i >> 1) & 1u)) failed = true;
-                if (!failed) fill(c0 + i + 2, buf, false);
-            }
-            // O += P(i) V(i): needs P from all softmax warps and the V chunk
-            if (!failed && !mbar_wait(pfull, (uint32_t)i & 1u)) failed = true;
-            if (!failed && !wait_fill(c0 + i, buf, true)) failed = true;
-            if (lane == 0 && !failed) {
-                tc_fence_after();
+            };
+            issue_s(0);
+            if (n_ch > 1) issue_s(1);
+            for (int i = 0; i < n_ch; ++i) {
+                const int buf = i & 1;
+                // O += P(i) V(i): needs P from all softmax warps and the V chunk
+                if (!failed && !mbar_wait_one(pfull, (uint32_t)i & 1u)) failed = true;
+                if (!failed && !mbar_wait_one(vfull(buf), (uint32_t)(i >> 1) & 1u)) failed = true;
+                if (!failed) {
+                    tc_fence_after();
+                    const uint32_t vb = v_lo + (uint32_t)buf * (TILE >> 4);
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks) { // K = 16 keys per instruction over the chunk's 128 keys
-                    const uint64_t da = make_desc(sP + (ks >> 2) * HALF + (ks & 3) * 32, 16);
-                    // V as an MN-major operand: d is contiguous, the two 64-wide halves are HALF bytes apart
-                    const uint64_t db = make_desc(sV + buf * TILE + ks * 16 * 128, HALF);
-                    mma_f16(tmem + 256u, da, db, idesc_o, (i > 0) || (ks > 0));
+                    for (int ks = 0; ks < 8; ++ks) { // K = 16 keys per instruction over the chunk's 128 keys
+                        const uint32_t poff = ((ks >> 2) * HALF + (ks & 3) * 32) >> 4;
+                        // V as an MN-major operand: d is contiguous, the two 64-wide halves are HALF bytes apart
+                        mma_f16_lo(tmem + 256u, p_lo + poff, hi, vb + (uint32_t)(ks * 16 * 128 >> 4), hi, idesc_o,
+                                   (i > 0) || (ks > 0));
+                    }
+                    mma_commit(odone);
                 }
-                mma_commit(odone);
+                // the S buffer of chunk i was read before P(i) was announced, so it can take chunk i + 2
+                if (i + 2 < n_ch) issue_s(i + 2);
             }
-            __syncwarp();
-            // the S buffer of chunk i was read before P(i) was announced, so it can take chunk i + 2
-            if (more) issue_s(i + 2);
-            // V buffer and P are free once the products have completed
-            if (!failed && !mbar_wait(odone, (uint32_t)i & 1u)) failed = true;
-            if (more && !failed) fill(c0 + i + 2, buf, true);
+            if (failed) s_fail = 1;
         }
-        cp_async_wait<0>();
-        if (failed) s_fail = 1;
+        __syncwarp();
     } else {
         // ================= softmax warps =================
         const uint32_t lanes = (uint32_t)((row >> 5) * 32) << 16;
@@ -537,11 +561,13 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
         __syncthreads();
         return;
     }
-    // producer: meet the softmax warps at their two CTA-wide barriers, then free the tensor memory
+    // copy and tensor-core warps: meet the softmax warps at their two CTA-wide barriers; the warp
+    // that allocated the tensor memory then frees it
     fspad_pdl_trigger();
     tc_fence_before();
     __syncthreads();
     __syncthreads();
+    if (warp != 9) return;
     tc_fence_after();
     __syncwarp();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" :: "r"(tmem), "r"(TMEM_COLS) : "memory");
