@@ -34,8 +34,8 @@ constexpr int BK = 128;                // keys per chunk
 constexpr int NT = 320;                // threads per CTA: two per query row + a copy warp + a tensor-core warp
 constexpr int HALF = 128 * 128;        // bytes of one [128 rows][64 bf16] half tile
 constexpr int TILE = 2 * HALF;         // bytes of one [128][128] bf16 tile
-constexpr int SMEM_BYTES = 6 * TILE + 1024;   // Q, K[2], V[2], P + alignment slack
-constexpr uint32_t TMEM_COLS = 512;    // S (two buffers): columns 0..255, O: columns 256..383
+constexpr int SMEM_BYTES = 5 * TILE + 1024;   // Q, K[2], V[2] + alignment slack
+constexpr uint32_t TMEM_COLS = 512;    // S/P of group 0, of group 1: columns 0..255; O of group 0, of group 1: 256..511
 constexpr uint32_t WAIT_CAP = 200000;   // polls of a bounded mbarrier wait
 struct Args {
     const fspad_bf16 *q, *kc, *vc, *tk, *tv;
@@ -209,37 +209,58 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar)
 {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];\n" ::"r"(bar) : "memory");
 }
-// barrier among the 256 softmax threads only (hardware barrier 1; barrier 0 is __syncthreads)
-__device__ __forceinline__ void softmax_sync() { asm volatile("bar.sync 1, 256;\n" ::: "memory"); }
+// D[tmem] (+)= A[tmem] * B[smem]: the A operand (here P, bf16 pairs packed into 32-bit columns, one
+// query row per lane) is read from tensor memory
+__device__ __forceinline__ void mma_f16_ts(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t b_hi, uint32_t idesc,
+                                           uint32_t accumulate)
+{
+    asm volatile("{\n\t.reg .pred p;\n\t.reg .b64 db;\n\tsetp.ne.b32 p, %5, 0;\n\t"
+                 "mov.b64 db, {%2, %3};\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n\t}\n"
+                 :: "r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void tmem_st16(uint32_t addr, const uint32_t (&v)[16])
+{
+    __syncwarp();
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+                 "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};\n"
+                 :: "r"(addr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
+                    "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15])
+                 : "memory");
+}
 
-// Roles.  Warps 0-7 (256 threads) are the softmax warps: two threads share a query row, thread
-// (row, half) owns columns half*64 .. half*64+63 of the row's scores, of its P row and of its O
-// row; warps w and w+4 address the same 32 lanes of tensor memory (a warp reaches the lane
-// quarter given by its index modulo 4).  Warp 8 is the copy warp: it issues every TMA copy of
-// the loop and gathers the one chunk TMA cannot describe.  Warp 9 is the tensor-core warp: one
-// of its threads issues every tcgen05.mma; the warp owns the tensor memory.
-// The two sides meet only on mbarriers, never on a CTA-wide barrier inside the loop:
+// Roles.  Warps 0-7 are the softmax warps, in two groups of four (128 threads, one query row per
+// thread, a warp reaching the tensor-memory lane quarter given by its index modulo 4).  The groups
+// take the chunks alternately - group 0 the even ones, group 1 the odd ones - and each keeps its
+// own running maximum, sum and O accumulator, so the exponentials of one chunk run while the other
+// group is waiting for, loading or storing its operands; the two accumulators are merged by
+// log-sum-exp when the loop ends.  Warp 8 is the copy warp: it issues every TMA copy of the loop
+// and gathers the one chunk TMA cannot describe.  Warp 9 is the tensor-core warp: one of its
+// threads issues every tcgen05.mma; the warp owns the tensor memory.
+// Tensor memory: columns [128 g, 128 g + 128) hold the fp32 scores S of group g's current chunk
+// and then, written over their first 64 columns, P as packed bf16 pairs, which the second product
+// reads directly as its A operand; columns [256 + 128 g, 384 + 128 g) hold O of group g.
+// The sides meet only on mbarriers, never on a CTA-wide barrier inside the loop:
 //   kfull/vfull(b)  K / V buffer b filled (TMA bytes, or one arrival)        tensor-core warp waits
-//   sfull(b)        S buffer b holds Q K^T of its chunk (tcgen05.commit)     softmax + copy warps wait
-//   pfull           P written, O rescaled and S read by all 8 softmax warps  tensor-core warp waits
-//   odone           O += P V of the chunk complete (tcgen05.commit)          softmax + copy warps wait
-// Tensor-core order: S(0) S(1) | PV(0) S(2) | PV(1) S(3) | ...  so the scores of the next chunk
-// are ready before the softmax warps ask for them and PV(i) runs under the softmax of chunk i+1.
+//   sfull(g)        S of group g's chunk complete (tcgen05.commit)           group g + copy warp wait
+//   pfull(g)        P written and O rescaled by the 4 warps of group g       tensor-core warp waits
+//   odone(g)        O[g] += P V of the chunk complete (tcgen05.commit)       copy warp waits (and all at the end)
+// Tensor-core order: S(0) S(1) | PV(0) S(2) | PV(1) S(3) | ...
 __global__ void __launch_bounds__(NT, 1)
 tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV)
 {
     extern __shared__ unsigned char smem_raw[];
-    __shared__ __align__(8) unsigned long long s_bar[8];
+    __shared__ __align__(8) unsigned long long s_bar[10];
     __shared__ uint32_t s_tmem;
     __shared__ int s_fail;
     __shared__ int s_par[FSPAD_MAX_NODES];
     __shared__ unsigned long long s_anc[FSPAD_MAX_NODES];
-    __shared__ float s_mx[2][2][BM];                         // [chunk parity][half][row]: row maxima / sums exchange
+    __shared__ float2 s_ml[2][BM];                           // [group][row]: (max, sum) of each group at the end
 
     fspad_pdl_wait();
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const bool producer = warp >= 8;         // warp 8 copies, warp 9 drives the tensor cores
-    const int row = tid & (BM - 1), half = (tid >> 7) & 1;
+    const int row = tid & (BM - 1), grp = (tid >> 7) & 1;
     const int split = blockIdx.x;
     const int g = blockIdx.y / a.mtiles, mt = blockIdx.y % a.mtiles;
     const int b = blockIdx.z;
@@ -262,24 +283,27 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
     const size_t prow = ((size_t)b * a.Hkv + g) * a.n_splits + split;
 
     if (c0 >= c1) {                               // nothing to do for this split: empty partial
-        if (row_ok && half == 0) { float *ml = a.part_ml + (prow * M + gr) * 2; ml[0] = -INFINITY; ml[1] = 0.f; }
+        if (row_ok && grp == 0) { float *ml = a.part_ml + (prow * M + gr) * 2; ml[0] = -INFINITY; ml[1] = 0.f; }
         return;
     }
 
-    // 1024-byte aligned tiles: Q | K0 | K1 | V0 | V1 | P
+    // 1024-byte aligned tiles: Q | K0 | K1 | V0 | V1
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    const uint32_t sQ = base, sK = base + TILE, sV = base + 3 * TILE, sP = base + 5 * TILE;
+    const uint32_t sQ = base, sK = base + TILE, sV = base + 3 * TILE;
     const uint32_t bar0 = smem_u32(&s_bar[0]);
     auto kfull = [&](int buf) { return bar0 + 8u * (uint32_t)buf; };
     auto vfull = [&](int buf) { return bar0 + 16u + 8u * (uint32_t)buf; };
     auto sfull = [&](int buf) { return bar0 + 32u + 8u * (uint32_t)buf; };
-    const uint32_t pfull = bar0 + 48u, odone = bar0 + 56u;
+    auto pfull = [&](int grp2) { return bar0 + 48u + 8u * (uint32_t)grp2; };
+    auto odone = [&](int grp2) { return bar0 + 64u + 8u * (uint32_t)grp2; };
     const bool tma_ok = a.use_tma != 0;
     if (tid == 0) {
 #pragma unroll
         for (int i = 0; i < 6; ++i) mbar_init(bar0 + 8u * i, 1);
-        mbar_init(pfull, 8);
-        mbar_init(odone, 1);
+        mbar_init(pfull(0), 4);
+        mbar_init(pfull(1), 4);
+        mbar_init(odone(0), 1);
+        mbar_init(odone(1), 1);
         s_fail = 0;
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     }
@@ -367,6 +391,7 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
     tc_fence_after();
     const uint32_t tmem = s_tmem;
     const uint32_t idesc_s = make_idesc(false), idesc_o = make_idesc(true);
+    const uint32_t tO = tmem + ((uint32_t)((warp & 3) * 32) << 16) + 256u + (uint32_t)grp * 128u;   // this group's O row
     bool failed = false;
 
     if (warp == 8) {
@@ -391,10 +416,11 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
         };
         for (int i = 0; i + 2 < n_ch; ++i) {
             const int buf = i & 1;
+            const uint32_t ph = (uint32_t)(i >> 1) & 1u;
             // K buffer is free once S(i) has completed, V buffer once O += P(i) V(i) has
-            if (!failed && !mbar_wait(sfull(buf), (uint32_t)(i >> 1) & 1u)) failed = true;
+            if (!failed && !mbar_wait(sfull(buf), ph)) failed = true;
             if (!failed) fill(c0 + i + 2, buf, false);
-            if (!failed && !mbar_wait(odone, (uint32_t)i & 1u)) failed = true;
+            if (!failed && !mbar_wait(odone(buf), ph)) failed = true;
             if (!failed) fill(c0 + i + 2, buf, true);
         }
         if (failed) s_fail = 1;
@@ -405,7 +431,7 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
             // the high word (8-row group stride, version, swizzle mode) is the same for all
             const uint32_t hi = (uint32_t)(make_desc(0, 16) >> 32);
             const uint32_t q_lo = (uint32_t)make_desc(sQ, 16), k_lo = (uint32_t)make_desc(sK, 16);
-            const uint32_t p_lo = (uint32_t)make_desc(sP, 16), v_lo = (uint32_t)make_desc(sV, HALF);
+            const uint32_t v_lo = (uint32_t)make_desc(sV, HALF);
             auto issue_s = [&](int i) {          // S[i & 1] = Q K(i)^T
                 const int buf = i & 1;
                 if (!failed && !mbar_wait_one(kfull(buf), (uint32_t)(i >> 1) & 1u)) failed = true;
@@ -422,23 +448,24 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
             issue_s(0);
             if (n_ch > 1) issue_s(1);
             for (int i = 0; i < n_ch; ++i) {
-                const int buf = i & 1;
-                // O += P(i) V(i): needs P from all softmax warps and the V chunk
-                if (!failed && !mbar_wait_one(pfull, (uint32_t)i & 1u)) failed = true;
-                if (!failed && !mbar_wait_one(vfull(buf), (uint32_t)(i >> 1) & 1u)) failed = true;
+                const int g2 = i & 1;
+                const uint32_t ph = (uint32_t)(i >> 1) & 1u;
+                // O[g2] += P(i) V(i): P from the four warps of group g2 (in tensor memory, over the
+                // scores it was computed from) and the V chunk
+                if (!failed && !mbar_wait_one(pfull(g2), ph)) failed = true;
+                if (!failed && !mbar_wait_one(vfull(g2), ph)) failed = true;
                 if (!failed) {
                     tc_fence_after();
-                    const uint32_t vb = v_lo + (uint32_t)buf * (TILE >> 4);
+                    const uint32_t vb = v_lo + (uint32_t)g2 * (TILE >> 4);
 #pragma unroll
-                    for (int ks = 0; ks < 8; ++ks) { // K = 16 keys per instruction over the chunk's 128 keys
-                        const uint32_t poff = ((ks >> 2) * HALF + (ks & 3) * 32) >> 4;
+                    for (int ks = 0; ks < 8; ++ks) { // K = 16 keys per instruction = 8 columns of packed bf16 pairs
                         // V as an MN-major operand: d is contiguous, the two 64-wide halves are HALF bytes apart
-                        mma_f16_lo(tmem + 256u, p_lo + poff, hi, vb + (uint32_t)(ks * 16 * 128 >> 4), hi, idesc_o,
-                                   (i > 0) || (ks > 0));
+                        mma_f16_ts(tmem + 256u + (uint32_t)g2 * 128u, tmem + (uint32_t)g2 * 128u + (uint32_t)ks * 8u,
+                                   vb + (uint32_t)(ks * 16 * 128 >> 4), hi, idesc_o, (i >= 2) || (ks > 0));
                     }
-                    mma_commit(odone);
+                    mma_commit(odone(g2));
                 }
-                // the S buffer of chunk i was read before P(i) was announced, so it can take chunk i + 2
+                // tensor-core work completes in issue order, so the scores of chunk i + 2 may replace P(i)
                 if (i + 2 < n_ch) issue_s(i + 2);
             }
             if (failed) s_fail = 1;
@@ -446,116 +473,128 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
         __syncwarp();
     } else {
         // ================= softmax warps =================
-        const uint32_t lanes = (uint32_t)((row >> 5) * 32) << 16;
-        const uint32_t tO = tmem + lanes + 256u + (uint32_t)(half * 64);     // this thread's 64 output columns
+        const uint32_t lanes = (uint32_t)((warp & 3) * 32) << 16;
+        const uint32_t tS = tmem + lanes + (uint32_t)grp * 128u;             // this group's scores, then its P
         const unsigned long long anc = s_anc[node];
         const float scale = a.scale_log2;
-        float m_run = -INFINITY, l_part = 0.f;   // row maximum (shared by both halves), this half's sum
+        float m_run = -INFINITY, l_run = 0.f;
 
-        for (int i = 0; i < n_ch; ++i) {
-            const int ch = c0 + i, sb = i & 1;
-            if (!failed && !mbar_wait(sfull(sb), (uint32_t)(i >> 1) & 1u)) failed = true;
+        for (int i = grp; i < n_ch; i += 2) {
+            const int ch = c0 + i;
+            if (!failed && !mbar_wait(sfull(grp), (uint32_t)(i >> 1) & 1u)) failed = true;
             tc_fence_after();
-            // ---- this thread's 64 scores: mask, row maximum (exchanged with the other half) ----
-            const uint32_t tS = tmem + lanes + (uint32_t)(sb * 128 + half * 64);
-            float sc[2][32];
-            tmem_ld32(tS, sc[0]);
-            tmem_ld32(tS + 32, sc[1]);
-            if ((ch + 1) * BK > L) {             // only chunks that reach past the cached prefix
-#pragma unroll
-                for (int q2 = 0; q2 < 2; ++q2)
+            const bool masked = (ch + 1) * BK > L;   // only chunks that reach past the cached prefix
+            // 32 scores of this thread's row, with the tree mask applied where it matters
+            auto load_scores = [&](int blk, float (&v)[32]) {
+                tmem_ld32(tS + (uint32_t)blk * 32u, v);
+                if (masked) {
 #pragma unroll
                     for (int j = 0; j < 32; ++j) {
-                        const int key = ch * BK + half * 64 + q2 * 32 + j;
+                        const int key = ch * BK + blk * 32 + j;
                         if (key >= L) {
                             const bool ok = (key < Ltot) && ((anc >> (key - L)) & 1ull);
-                            if (!ok) sc[q2][j] = -INFINITY;
+                            if (!ok) v[j] = -INFINITY;
                         }
                     }
-            }
+                }
+            };
+            // ---- pass 1: row maximum ----
             float mx = -INFINITY;
 #pragma unroll
-            for (int q2 = 0; q2 < 2; ++q2)
+            for (int blk = 0; blk < 4; ++blk) {
+                float v[32];
+                load_scores(blk, v);
 #pragma unroll
-                for (int j = 0; j < 32; ++j) mx = fmaxf(mx, sc[q2][j]);
-            s_mx[sb][half][row] = mx;
-            softmax_sync();
-            mx = fmaxf(mx, s_mx[sb][half ^ 1][row]);
+                for (int j = 0; j < 32; ++j) mx = fmaxf(mx, v[j]);
+            }
             const float m_new = fmaxf(m_run, mx * scale);
             const float m_safe = (m_new == -INFINITY) ? 0.f : m_new;
             const float alpha = ex2f(m_run - m_safe);
-            float rs = 0.f;
-            uint32_t w[32];
+            // ---- rescale this row of O[grp]; skipped (warp-uniformly) when no row of the warp moved its
+            // maximum, the factor then being exactly one.  The products of this group's previous chunk are
+            // complete: the scores just read were issued after them and complete in order. ----
+            if (i >= 2 && !__all_sync(0xffffffffu, alpha == 1.f)) {
 #pragma unroll
-            for (int q2 = 0; q2 < 2; ++q2)
-#pragma unroll
-                for (int e = 0; e < 16; ++e) {
-                    const float p0 = ex2f(fmaf(sc[q2][2 * e], scale, -m_safe));
-                    const float p1 = ex2f(fmaf(sc[q2][2 * e + 1], scale, -m_safe));
-                    rs += p0 + p1;
-                    w[q2 * 16 + e] = pack_bf16(p0, p1);
-                }
-            l_part = l_part * alpha + rs;
-            m_run = m_new;
-            // P (single tile) and O may be touched once the products of the previous chunk are done
-            if (i > 0) {
-                if (!failed && !mbar_wait(odone, (uint32_t)(i - 1) & 1u)) failed = true;
-                tc_fence_after();
-            }
-#pragma unroll
-            for (int c8 = 0; c8 < 8; ++c8) {     // 8 keys = one 16-byte chunk of the P row
-                const int c = half * 8 + c8;
-                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};\n"
-                             :: "r"(sP + tile_off(row, c)), "r"(w[c8 * 4]), "r"(w[c8 * 4 + 1]), "r"(w[c8 * 4 + 2]),
-                                "r"(w[c8 * 4 + 3]) : "memory");
-            }
-            // rescale this thread's half of the O row; skipped (warp-uniformly) when no row of the
-            // warp moved its maximum, since the factor is then exactly one
-            if (i > 0 && !__all_sync(0xffffffffu, alpha == 1.f)) {
-#pragma unroll
-                for (int q2 = 0; q2 < 2; ++q2) {
+                for (int blk = 0; blk < 4; ++blk) {
                     float o[32];
-                    tmem_ld32(tO + q2 * 32, o);
+                    tmem_ld32(tO + (uint32_t)blk * 32u, o);
 #pragma unroll
                     for (int j = 0; j < 32; ++j) o[j] *= alpha;
-                    tmem_st32(tO + q2 * 32, o);
+                    tmem_st32(tO + (uint32_t)blk * 32u, o);
                 }
-                asm volatile("tcgen05.wait::st.sync.aligned;\n" ::: "memory");
             }
-            fence_async_smem();
+            // ---- pass 2: P = exp2(s * scale - m) as bf16 pairs, written over the scores already consumed
+            // (block blk of P takes columns 16 blk .. 16 blk + 15, all below the 32 (blk + 1) columns read) ----
+            float rs = 0.f;
+#pragma unroll
+            for (int blk = 0; blk < 4; ++blk) {
+                float v[32];
+                load_scores(blk, v);
+                uint32_t w[16];
+#pragma unroll
+                for (int e = 0; e < 16; ++e) {
+                    const float p0 = ex2f(fmaf(v[2 * e], scale, -m_safe));
+                    const float p1 = ex2f(fmaf(v[2 * e + 1], scale, -m_safe));
+                    rs += p0 + p1;
+                    w[e] = pack_bf16(p0, p1);
+                }
+                tmem_st16(tS + (uint32_t)blk * 16u, w);
+            }
+            l_run = l_run * alpha + rs;
+            m_run = m_new;
+            asm volatile("tcgen05.wait::st.sync.aligned;\n" ::: "memory");
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(pfull);
+            if (lane == 0) mbar_arrive(pfull(grp));
         }
-        if (!failed && !mbar_wait(odone, (uint32_t)(n_ch - 1) & 1u)) failed = true;
+        // ---- both groups' last products must be complete before the two accumulators are merged ----
+        {
+            const int last0 = (n_ch - 1) & ~1, last1 = ((n_ch - 2) & ~1) + 1;   // last chunk index of each group
+            if (!failed && !mbar_wait(odone(0), (uint32_t)(last0 >> 1) & 1u)) failed = true;
+            if (n_ch >= 2 && !failed && !mbar_wait(odone(1), (uint32_t)(last1 >> 1) & 1u)) failed = true;
+        }
         tc_fence_after();
         if (failed) s_fail = 1;
-        s_mx[0][half][row] = l_part;
+        s_ml[grp][row] = make_float2(m_run, l_run);
         fspad_pdl_trigger();                      // the merge kernel may start launching
         tc_fence_before();
         __syncthreads();
         tc_fence_after();
-        // ---- publish the partial: unnormalised O row, running max and sum ----
-        // Every lane of every softmax warp takes part in the tensor-memory loads (they are
-        // warp-collective); only the stores to global memory depend on whether the lane's row exists.
+        // ---- publish the partial: the two groups' (max, sum, O row) merged by log-sum-exp ----
+        // Thread (row, grp) owns output columns grp*64 .. grp*64+63.  Every lane of every softmax warp
+        // takes part in the tensor-memory loads (they are warp-collective); only the stores to global
+        // memory depend on whether the lane's row exists.
         const bool any_fail = s_fail != 0;
         if (any_fail && tid == 0) fspad_report(a.status, FSPAD_ERR_TIMEOUT);
         const bool store = row_ok && !any_fail;
-        float *po = a.part_o + (prow * M + (row_ok ? gr : 0)) * D + half * 64;
+        const float2 ml0 = s_ml[0][row], ml1 = s_ml[1][row];
+        const float m_all = fmaxf(ml0.x, ml1.x);
+        const float m_fin = (m_all == -INFINITY) ? 0.f : m_all;
+        const float f0 = ex2f(ml0.x - m_fin), f1 = ex2f(ml1.x - m_fin);     // exp2(-inf) = 0 for an idle group
+        float *po = a.part_o + (prow * M + (row_ok ? gr : 0)) * D + grp * 64;
+        const uint32_t tO0 = tmem + lanes + 256u + (uint32_t)grp * 64u, tO1 = tO0 + 128u;
 #pragma unroll
         for (int q2 = 0; q2 < 2; ++q2) {
             float o[32];
-            tmem_ld32(tO + q2 * 32, o);
+            tmem_ld32(tO0 + q2 * 32, o);
+#pragma unroll
+            for (int j = 0; j < 32; ++j) o[j] *= f0;
+            if (n_ch >= 2) {                      // group 1 has accumulated something (uniform over the CTA)
+                float o1[32];
+                tmem_ld32(tO1 + q2 * 32, o1);
+#pragma unroll
+                for (int j = 0; j < 32; ++j) o[j] = fmaf(o1[j], f1, o[j]);
+            }
             if (store) {
 #pragma unroll
                 for (int j = 0; j < 32; j += 4)
                     *reinterpret_cast<float4 *>(po + q2 * 32 + j) = make_float4(o[j], o[j + 1], o[j + 2], o[j + 3]);
             }
         }
-        if (store && half == 0) {
+        if (store && grp == 0) {
             float *ml = a.part_ml + (prow * M + gr) * 2;
-            ml[0] = m_run;
-            ml[1] = s_mx[0][0][row] + s_mx[0][1][row];
+            ml[0] = m_all;
+            ml[1] = ml0.y * f0 + ml1.y * f1;
         }
         tc_fence_before();
         __syncthreads();
