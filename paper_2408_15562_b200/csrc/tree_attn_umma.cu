@@ -484,18 +484,30 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
             if (!failed && !mbar_wait(sfull(grp), (uint32_t)(i >> 1) & 1u)) failed = true;
             tc_fence_after();
             const bool masked = (ch + 1) * BK > L;   // only chunks that reach past the cached prefix
+            // Validity of the chunk's 128 keys for this row as four 32-bit words: prefix keys are
+            // valid, tree key L + t is valid iff bit t of the row's ancestor mask is set (bits at and
+            // beyond the tree size are clear, which also rules out the zero padding).
+            uint32_t valid[4] = {~0u, ~0u, ~0u, ~0u};
+            if (masked) {
+#pragma unroll
+                for (int blk = 0; blk < 4; ++blk) {
+                    const int off = ch * BK + blk * 32 - L;      // tree index of the word's first key
+                    uint32_t wv;
+                    if (off >= 64) wv = 0u;
+                    else if (off >= 0) wv = (uint32_t)(anc >> off);
+                    else if (off <= -32) wv = ~0u;
+                    else wv = ((1u << (-off)) - 1u) | (uint32_t)(anc << (-off));
+                    valid[blk] = wv;
+                }
+            }
             // 32 scores of this thread's row, with the tree mask applied where it matters
             auto load_scores = [&](int blk, float (&v)[32]) {
                 tmem_ld32(tS + (uint32_t)blk * 32u, v);
                 if (masked) {
+                    const uint32_t wv = valid[blk];
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        const int key = ch * BK + blk * 32 + j;
-                        if (key >= L) {
-                            const bool ok = (key < Ltot) && ((anc >> (key - L)) & 1ull);
-                            if (!ok) v[j] = -INFINITY;
-                        }
-                    }
+                    for (int j = 0; j < 32; ++j)
+                        if (!((wv >> j) & 1u)) v[j] = -INFINITY;
                 }
             };
             // ---- pass 1: row maximum ----
