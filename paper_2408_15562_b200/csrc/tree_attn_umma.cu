@@ -34,7 +34,8 @@ constexpr int BK = 128;                // keys per chunk
 constexpr int NT = 320;                // threads per CTA: two per query row + a copy warp + a tensor-core warp
 constexpr int HALF = 128 * 128;        // bytes of one [128 rows][64 bf16] half tile
 constexpr int TILE = 2 * HALF;         // bytes of one [128][128] bf16 tile
-constexpr int SMEM_BYTES = 5 * TILE + 1024;   // Q, K[2], V[2] + alignment slack
+constexpr int NS = 3;                  // K / V chunks in flight per CTA
+constexpr int SMEM_BYTES = (1 + 2 * NS) * TILE + 1024;   // Q, K[NS], V[NS] + alignment slack
 constexpr uint32_t TMEM_COLS = 512;    // S/P of group 0, of group 1: columns 0..255; O of group 0, of group 1: 256..511
 constexpr uint32_t WAIT_CAP = 200000;   // polls of a bounded mbarrier wait
 struct Args {
@@ -242,20 +243,21 @@ __device__ __forceinline__ void tmem_st16(uint32_t addr, const uint32_t (&v)[16]
 // reads directly as its A operand; columns [256 + 128 g, 384 + 128 g) hold O of group g.
 // The sides meet only on mbarriers, never on a CTA-wide barrier inside the loop:
 //   kfull/vfull(b)  K / V buffer b filled (TMA bytes, or one arrival)        tensor-core warp waits
-//   sfull(g)        S of group g's chunk complete (tcgen05.commit)           group g + copy warp wait
+//   kfree/vfree(b)  S (P V) of the chunk in buffer b complete (tcgen05.commit) copy warp waits
+//   sfull(g)        S of group g's chunk complete (tcgen05.commit)           group g waits
 //   pfull(g)        P written and O rescaled by the 4 warps of group g       tensor-core warp waits
-//   odone(g)        O[g] += P V of the chunk complete (tcgen05.commit)       copy warp waits (and all at the end)
+//   odone(g)        O[g] += P V of the chunk complete (tcgen05.commit)       group g waits, after its last chunk
+// Every barrier has exactly one waiting side, which waits on each of its phases in order.
 // Tensor-core order: S(0) S(1) | PV(0) S(2) | PV(1) S(3) | ...
 __global__ void __launch_bounds__(NT, 1)
 tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV)
 {
     extern __shared__ unsigned char smem_raw[];
-    __shared__ __align__(8) unsigned long long s_bar[10];
+    __shared__ __align__(8) unsigned long long s_bar[4 * NS + 6];
     __shared__ uint32_t s_tmem;
     __shared__ int s_fail;
     __shared__ int s_par[FSPAD_MAX_NODES];
     __shared__ unsigned long long s_anc[FSPAD_MAX_NODES];
-    __shared__ float2 s_ml[2][BM];                           // [group][row]: (max, sum) of each group at the end
 
     fspad_pdl_wait();
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -287,19 +289,21 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
         return;
     }
 
-    // 1024-byte aligned tiles: Q | K0 | K1 | V0 | V1
+    // 1024-byte aligned tiles: Q | K[NS] | V[NS]
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    const uint32_t sQ = base, sK = base + TILE, sV = base + 3 * TILE;
+    const uint32_t sQ = base, sK = base + TILE, sV = base + (1 + NS) * TILE;
     const uint32_t bar0 = smem_u32(&s_bar[0]);
     auto kfull = [&](int buf) { return bar0 + 8u * (uint32_t)buf; };
-    auto vfull = [&](int buf) { return bar0 + 16u + 8u * (uint32_t)buf; };
-    auto sfull = [&](int buf) { return bar0 + 32u + 8u * (uint32_t)buf; };
-    auto pfull = [&](int grp2) { return bar0 + 48u + 8u * (uint32_t)grp2; };
-    auto odone = [&](int grp2) { return bar0 + 64u + 8u * (uint32_t)grp2; };
+    auto vfull = [&](int buf) { return bar0 + 8u * (uint32_t)(NS + buf); };
+    auto kfree = [&](int buf) { return bar0 + 8u * (uint32_t)(2 * NS + buf); };
+    auto vfree = [&](int buf) { return bar0 + 8u * (uint32_t)(3 * NS + buf); };
+    auto sfull = [&](int grp2) { return bar0 + 8u * (uint32_t)(4 * NS + grp2); };
+    auto pfull = [&](int grp2) { return bar0 + 8u * (uint32_t)(4 * NS + 2 + grp2); };
+    auto odone = [&](int grp2) { return bar0 + 8u * (uint32_t)(4 * NS + 4 + grp2); };
     const bool tma_ok = a.use_tma != 0;
     if (tid == 0) {
 #pragma unroll
-        for (int i = 0; i < 6; ++i) mbar_init(bar0 + 8u * i, 1);
+        for (int i = 0; i < 4 * NS + 2; ++i) mbar_init(bar0 + 8u * i, 1);
         mbar_init(pfull(0), 4);
         mbar_init(pfull(1), 4);
         mbar_init(odone(0), 1);
@@ -344,9 +348,9 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
         tma_load_2d(dst + HALF, map, 64, y, bar);
     };
 
-    // ---- prologue: the first two chunks and Q go out first, the rest hides under their latency ----
+    // ---- prologue: the first NS chunks and Q go out first, the rest hides under their latency ----
 #pragma unroll
-    for (int u = 0; u < 2; ++u) {
+    for (int u = 0; u < NS; ++u) {
         if (u >= n_ch) break;
         if (is_tma(c0 + u)) {
             if (tid == 256) { tma_fill(c0 + u, u, false); tma_fill(c0 + u, u, true); }
@@ -398,7 +402,7 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
         // ================= copy warp: refills the K / V buffers =================
         // chunks gathered by the whole CTA in the prologue are announced here
         if (lane == 0) {
-            for (int u = 0; u < 2 && u < n_ch; ++u)
+            for (int u = 0; u < NS && u < n_ch; ++u)
                 if (!is_tma(c0 + u)) { mbar_arrive(kfull(u)); mbar_arrive(vfull(u)); }
         }
         auto fill = [&](int ch, int buf, bool is_v) {
@@ -414,14 +418,15 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
             }
             __syncwarp();
         };
-        for (int i = 0; i + 2 < n_ch; ++i) {
-            const int buf = i & 1;
-            const uint32_t ph = (uint32_t)(i >> 1) & 1u;
-            // K buffer is free once S(i) has completed, V buffer once O += P(i) V(i) has
-            if (!failed && !mbar_wait(sfull(buf), ph)) failed = true;
-            if (!failed) fill(c0 + i + 2, buf, false);
-            if (!failed && !mbar_wait(odone(buf), ph)) failed = true;
-            if (!failed) fill(c0 + i + 2, buf, true);
+        int buf = 0;                             // i modulo NS
+        uint32_t ph = 0;                         // flips each time the ring wraps
+        for (int i = 0; i + NS < n_ch; ++i) {
+            // the K buffer of chunk i is free once S(i) has completed, its V buffer once O += P(i) V(i) has
+            if (!failed && !mbar_wait(kfree(buf), ph)) failed = true;
+            if (!failed) fill(c0 + i + NS, buf, false);
+            if (!failed && !mbar_wait(vfree(buf), ph)) failed = true;
+            if (!failed) fill(c0 + i + NS, buf, true);
+            if (++buf == NS) { buf = 0; ph ^= 1u; }
         }
         if (failed) s_fail = 1;
     } else if (warp == 9) {
@@ -432,18 +437,22 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
             const uint32_t hi = (uint32_t)(make_desc(0, 16) >> 32);
             const uint32_t q_lo = (uint32_t)make_desc(sQ, 16), k_lo = (uint32_t)make_desc(sK, 16);
             const uint32_t v_lo = (uint32_t)make_desc(sV, HALF);
+            int kbuf = 0, vbuf = 0;              // buffers of the next S and of the next P V
+            uint32_t kph = 0, vph = 0;           // and their phases (flip each time the ring wraps)
             auto issue_s = [&](int i) {          // S[i & 1] = Q K(i)^T
-                const int buf = i & 1;
-                if (!failed && !mbar_wait_one(kfull(buf), (uint32_t)(i >> 1) & 1u)) failed = true;
+                const int buf = kbuf;
+                if (!failed && !mbar_wait_one(kfull(buf), kph)) failed = true;
+                if (++kbuf == NS) { kbuf = 0; kph ^= 1u; }
                 if (failed) return;
                 tc_fence_after();
                 const uint32_t kb = k_lo + (uint32_t)buf * (TILE >> 4);
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) { // K = 16 per instruction over d = 128
                     const uint32_t koff = ((ks >> 2) * HALF + (ks & 3) * 32) >> 4;
-                    mma_f16_lo(tmem + (uint32_t)buf * 128u, q_lo + koff, hi, kb + koff, hi, idesc_s, ks > 0);
+                    mma_f16_lo(tmem + (uint32_t)(i & 1) * 128u, q_lo + koff, hi, kb + koff, hi, idesc_s, ks > 0);
                 }
-                mma_commit(sfull(buf));
+                mma_commit(sfull(i & 1));
+                mma_commit(kfree(buf));
             };
             issue_s(0);
             if (n_ch > 1) issue_s(1);
@@ -453,10 +462,12 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
                 // O[g2] += P(i) V(i): P from the four warps of group g2 (in tensor memory, over the
                 // scores it was computed from) and the V chunk
                 if (!failed && !mbar_wait_one(pfull(g2), ph)) failed = true;
-                if (!failed && !mbar_wait_one(vfull(g2), ph)) failed = true;
+                if (!failed && !mbar_wait_one(vfull(vbuf), vph)) failed = true;
+                const uint32_t vb = v_lo + (uint32_t)vbuf * (TILE >> 4);
+                const uint32_t vfree_bar = vfree(vbuf);
+                if (++vbuf == NS) { vbuf = 0; vph ^= 1u; }
                 if (!failed) {
                     tc_fence_after();
-                    const uint32_t vb = v_lo + (uint32_t)g2 * (TILE >> 4);
 #pragma unroll
                     for (int ks = 0; ks < 8; ++ks) { // K = 16 keys per instruction = 8 columns of packed bf16 pairs
                         // V as an MN-major operand: d is contiguous, the two 64-wide halves are HALF bytes apart
@@ -464,6 +475,7 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
                                    vb + (uint32_t)(ks * 16 * 128 >> 4), hi, idesc_o, (i >= 2) || (ks > 0));
                     }
                     mma_commit(odone(g2));
+                    mma_commit(vfree_bar);
                 }
                 // tensor-core work completes in issue order, so the scores of chunk i + 2 may replace P(i)
                 if (i + 2 < n_ch) issue_s(i + 2);
@@ -559,15 +571,20 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
             __syncwarp();
             if (lane == 0) mbar_arrive(pfull(grp));
         }
-        // ---- both groups' last products must be complete before the two accumulators are merged ----
-        {
-            const int last0 = (n_ch - 1) & ~1, last1 = ((n_ch - 2) & ~1) + 1;   // last chunk index of each group
-            if (!failed && !mbar_wait(odone(0), (uint32_t)(last0 >> 1) & 1u)) failed = true;
-            if (n_ch >= 2 && !failed && !mbar_wait(odone(1), (uint32_t)(last1 >> 1) & 1u)) failed = true;
+        // ---- each group waits for its own last product; the CTA-wide barrier below then orders both
+        // accumulators before the merge (a group's barrier is only ever waited on by that group, in
+        // phase order, so a parity wait can never see it a phase behind) ----
+        if (grp < n_ch) {
+            const int last = grp ? ((n_ch - 2) & ~1) + 1 : (n_ch - 1) & ~1;    // last chunk index of the group
+            if (!failed && !mbar_wait(odone(grp), (uint32_t)(last >> 1) & 1u)) failed = true;
         }
         tc_fence_after();
         if (failed) s_fail = 1;
-        s_ml[grp][row] = make_float2(m_run, l_run);
+        // For a group that has waited for its last product the Q tile is dead (every S was issued
+        // before that product and completes before it): it carries the groups' (max, sum) exchange.
+        // A group without a chunk has waited for nothing and must not touch it.
+        float2 *s_ml = reinterpret_cast<float2 *>(smem_raw + (base - smem_u32(smem_raw)));
+        if (grp < n_ch) s_ml[grp * BM + row] = make_float2(m_run, l_run);
         fspad_pdl_trigger();                      // the merge kernel may start launching
         tc_fence_before();
         __syncthreads();
@@ -579,7 +596,7 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
         const bool any_fail = s_fail != 0;
         if (any_fail && tid == 0) fspad_report(a.status, FSPAD_ERR_TIMEOUT);
         const bool store = row_ok && !any_fail;
-        const float2 ml0 = s_ml[0][row], ml1 = s_ml[1][row];
+        const float2 ml0 = s_ml[row], ml1 = (n_ch >= 2) ? s_ml[BM + row] : make_float2(-INFINITY, 0.f);
         const float m_all = fmaxf(ml0.x, ml1.x);
         const float m_fin = (m_all == -INFINITY) ? 0.f : m_all;
         const float f0 = ex2f(ml0.x - m_fin), f1 = ex2f(ml1.x - m_fin);     // exp2(-inf) = 0 for an idle group
