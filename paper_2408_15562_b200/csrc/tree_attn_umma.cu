@@ -38,6 +38,7 @@ constexpr int NS = 3;                  // K / V chunks in flight per CTA
 constexpr int SMEM_BYTES = (1 + 2 * NS) * TILE + 1024;   // Q, K[NS], V[NS] + alignment slack
 constexpr uint32_t TMEM_COLS = 512;    // S/P of group 0, of group 1: columns 0..255; O of group 0, of group 1: 256..511
 constexpr uint32_t WAIT_CAP = 200000;   // polls of a bounded mbarrier wait
+constexpr float kLazyLog2 = 8.f;        // a row's reference maximum may lag its true maximum by this much (log2)
 struct Args {
     const fspad_bf16 *q, *kc, *vc, *tk, *tv;
     const int *parent, *prefix_len;
@@ -531,13 +532,19 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
 #pragma unroll
                 for (int j = 0; j < 32; ++j) mx = fmaxf(mx, v[j]);
             }
-            const float m_new = fmaxf(m_run, mx * scale);
+            // The reference value m of a row (P = exp2(s * scale - m), O and the sum are relative to it)
+            // only has to bound the scores loosely: it follows the row maximum when some row of the warp
+            // would otherwise see a P above 2^kLazyLog2, and stays put - no pass over O - when not.
+            // (The decision is taken per warp because the tensor-memory accesses are warp-collective;
+            // a comparison with -inf - -inf = NaN is false and so counts as a move.)
+            const float m_cand = fmaxf(m_run, mx * scale);
+            const bool move = !__all_sync(0xffffffffu, m_cand - m_run <= kLazyLog2);
+            const float m_new = move ? m_cand : m_run;
             const float m_safe = (m_new == -INFINITY) ? 0.f : m_new;
-            const float alpha = ex2f(m_run - m_safe);
-            // ---- rescale this row of O[grp]; skipped (warp-uniformly) when no row of the warp moved its
-            // maximum, the factor then being exactly one.  The products of this group's previous chunk are
-            // complete: the scores just read were issued after them and complete in order. ----
-            if (i >= 2 && !__all_sync(0xffffffffu, alpha == 1.f)) {
+            const float alpha = move ? ex2f(m_run - m_safe) : 1.f;
+            // ---- rescale this row of O[grp].  The products of this group's previous chunk are complete:
+            // the scores just read were issued after them and complete in order. ----
+            if (i >= 2 && move) {
 #pragma unroll
                 for (int blk = 0; blk < 4; ++blk) {
                     float o[32];
