@@ -5,19 +5,18 @@
 // Split-KV flash-decode with tcgen05: all query rows that share a kv head (tree
 // node x GQA group member) form the M = 128 operand of one CTA; keys are
 // consumed in chunks of 128.  Per chunk: S = Q K^T is one chain of eight
-// tcgen05.mma (128 x 128 x 16, bf16 -> fp32) into tensor memory; two threads
-// share a query row, each reads 64 of its scores back with tcgen05.ld, applies
-// the ancestor mask (only on chunks that reach past the cached prefix) and the
-// softmax in registers (one shared-memory exchange of the row maximum), and writes P as bf16 into
-// a 128-byte-swizzled shared-memory tile; O += P V is a second chain of eight
-// tcgen05.mma with V read directly in its [key][d] layout (MN-major operand).
-// O stays in tensor memory across chunks and is rescaled there when the running
-// maximum moves.  K/V chunks are double buffered in the 128-byte-swizzled layout
-// the matrix descriptors expect: chunks that lie inside the cached prefix arrive
-// by TMA (four cp.async.bulk.tensor boxes of 64 x 128 per chunk, one issuing
-// thread, completion on an mbarrier); Q and the one chunk that mixes prefix,
-// tree rows and zero padding use 16-byte asynchronous copies.  Per-split
-// partials are merged by the combine kernel.
+// tcgen05.mma (128 x 128 x 16, bf16 -> fp32) into tensor memory; a softmax
+// thread per query row reads its scores back with tcgen05.ld, applies the
+// ancestor mask (only on chunks that reach past the cached prefix) and the
+// softmax in registers, and writes P as packed bf16 pairs back into tensor
+// memory, over the scores; O += P V is a second chain of eight tcgen05.mma whose
+// A operand is read from tensor memory and whose B operand is V in its
+// [key][d] layout (MN-major).  O stays in tensor memory across chunks.  The
+// work is split over three kinds of warps that meet only on mbarriers (see the
+// kernel's comment); K/V chunks go through a three-deep ring of 128-byte-swizzled
+// tiles, filled by TMA for chunks inside the cached prefix and by 16-byte
+// asynchronous copies for Q and the one chunk that mixes prefix, tree rows and
+// zero padding.  Per-split partials are merged by the combine kernel.
 //
 // Every wait on an mbarrier is bounded; on expiry the CTA records
 // FSPAD_ERR_TIMEOUT, skips the remaining tensor-core work, frees its tensor
