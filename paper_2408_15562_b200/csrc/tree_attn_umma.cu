@@ -116,15 +116,15 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t addr, uint32_t lbo_bytes)
     d |= (uint64_t)2 << 61;                 // SWIZZLE_128B
     return d;
 }
-// instruction descriptor: bf16 x bf16 -> fp32, M = 128, N = 128
-__device__ __forceinline__ uint32_t make_idesc(bool b_mn_major)
+// instruction descriptor: bf16 x bf16 -> fp32, M = 128, N = n
+__device__ __forceinline__ uint32_t make_idesc(bool b_mn_major, uint32_t n)
 {
     uint32_t d = 0;
     d |= 1u << 4;                           // accumulator fp32
     d |= 1u << 7;                           // A bf16
     d |= 1u << 10;                          // B bf16
     d |= (b_mn_major ? 1u : 0u) << 16;      // B major: 0 = K, 1 = MN
-    d |= (128u >> 3) << 17;                 // N
+    d |= (n >> 3) << 17;                    // N
     d |= (128u >> 4) << 24;                 // M
     return d;
 }
@@ -231,29 +231,32 @@ __device__ __forceinline__ void tmem_st16(uint32_t addr, const uint32_t (&v)[16]
 }
 
 // Roles.  Warps 0-7 are the softmax warps, in two groups of four (128 threads, one query row per
-// thread, a warp reaching the tensor-memory lane quarter given by its index modulo 4).  The groups
-// take the chunks alternately - group 0 the even ones, group 1 the odd ones - and each keeps its
-// own running maximum, sum and O accumulator, so the exponentials of one chunk run while the other
-// group is waiting for, loading or storing its operands; the two accumulators are merged by
-// log-sum-exp when the loop ends.  Warp 8 is the copy warp: it issues every TMA copy of the loop
-// and gathers the one chunk TMA cannot describe.  Warp 9 is the tensor-core warp: one of its
-// threads issues every tcgen05.mma; the warp owns the tensor memory.
-// Tensor memory: columns [128 g, 128 g + 128) hold the fp32 scores S of group g's current chunk
-// and then, written over their first 64 columns, P as packed bf16 pairs, which the second product
-// reads directly as its A operand; columns [256 + 128 g, 384 + 128 g) hold O of group g.
+// thread, a warp reaching the tensor-memory lane quarter given by its index modulo 4).  Group g
+// owns keys 64 g .. 64 g + 63 of every chunk: its own score buffers (two, used alternately),
+// running reference maximum, sum and O accumulator, merged with the other group's by log-sum-exp
+// when the loop ends.  Warp 8 is the copy warp: it issues every TMA copy of the loop and gathers
+// the one chunk TMA cannot describe.  Warp 9 is the tensor-core warp: one of its threads issues
+// every tcgen05.mma; the warp owns the tensor memory.
+// Tensor memory: columns [128 g + 64 p, 128 g + 64 p + 64) hold the fp32 scores S_g of the group's
+// chunks of parity p and then, written over their first 32 columns, P as packed bf16 pairs, which
+// the second product reads directly as its A operand; columns [256 + 128 g, 384 + 128 g) hold O_g.
+// With two score buffers per group the scores of chunk c + 1 are complete long before the group
+// has finished chunk c, and O_g += P V runs under the group's next softmax: a group never waits for
+// the tensor cores unless it has to rescale O.
 // The sides meet only on mbarriers, never on a CTA-wide barrier inside the loop:
-//   kfull/vfull(b)  K / V buffer b filled (TMA bytes, or one arrival)        tensor-core warp waits
-//   kfree/vfree(b)  S (P V) of the chunk in buffer b complete (tcgen05.commit) copy warp waits
-//   sfull(g)        S of group g's chunk complete (tcgen05.commit)           group g waits
-//   pfull(g)        P written and O rescaled by the 4 warps of group g       tensor-core warp waits
-//   odone(g)        O[g] += P V of the chunk complete (tcgen05.commit)       group g waits, after its last chunk
-// Every barrier has exactly one waiting side, which waits on each of its phases in order.
-// Tensor-core order: S(0) S(1) | PV(0) S(2) | PV(1) S(3) | ...
+//   kfull/vfull(b)  K / V ring slot b filled (TMA bytes, or one arrival)     tensor-core warp waits
+//   kfree/vfree(b)  both S (both P V) of the chunk in slot b complete        copy warp waits
+//   sfull(g, p)     S_g of a chunk of parity p complete (tcgen05.commit)     group g waits
+//   pfull(g, p)     P_g written and O_g rescaled by the 4 warps of group g   tensor-core warp waits
+//   odone(g, p)     O_g += P_g V of a chunk of parity p complete             group g waits (rescale, end)
+// Every barrier has exactly one waiting side, and a new phase of it can only begin after that
+// side has seen the previous one (a parity wait must never fall two phases behind).
+// Tensor-core order: S_0(0) S_1(0) S_0(1) S_1(1) | PV_0(0) S_0(2) PV_1(0) S_1(2) | PV_0(1) S_0(3) ...
 __global__ void __launch_bounds__(NT, 1)
 tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV)
 {
     extern __shared__ unsigned char smem_raw[];
-    __shared__ __align__(8) unsigned long long s_bar[4 * NS + 6];
+    __shared__ __align__(8) unsigned long long s_bar[4 * NS + 12];
     __shared__ uint32_t s_tmem;
     __shared__ int s_fail;
     __shared__ int s_par[FSPAD_MAX_NODES];
@@ -297,17 +300,13 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
     auto vfull = [&](int buf) { return bar0 + 8u * (uint32_t)(NS + buf); };
     auto kfree = [&](int buf) { return bar0 + 8u * (uint32_t)(2 * NS + buf); };
     auto vfree = [&](int buf) { return bar0 + 8u * (uint32_t)(3 * NS + buf); };
-    auto sfull = [&](int grp2) { return bar0 + 8u * (uint32_t)(4 * NS + grp2); };
-    auto pfull = [&](int grp2) { return bar0 + 8u * (uint32_t)(4 * NS + 2 + grp2); };
-    auto odone = [&](int grp2) { return bar0 + 8u * (uint32_t)(4 * NS + 4 + grp2); };
+    auto sfull = [&](int grp2, int par) { return bar0 + 8u * (uint32_t)(4 * NS + 2 * grp2 + par); };
+    auto pfull = [&](int grp2, int par) { return bar0 + 8u * (uint32_t)(4 * NS + 4 + 2 * grp2 + par); };
+    auto odone = [&](int grp2, int par) { return bar0 + 8u * (uint32_t)(4 * NS + 8 + 2 * grp2 + par); };
     const bool tma_ok = a.use_tma != 0;
     if (tid == 0) {
 #pragma unroll
-        for (int i = 0; i < 4 * NS + 2; ++i) mbar_init(bar0 + 8u * i, 1);
-        mbar_init(pfull(0), 4);
-        mbar_init(pfull(1), 4);
-        mbar_init(odone(0), 1);
-        mbar_init(odone(1), 1);
+        for (int i = 0; i < 4 * NS + 12; ++i) mbar_init(bar0 + 8u * i, (i >= 4 * NS + 4 && i < 4 * NS + 8) ? 4 : 1);
         s_fail = 0;
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     }
@@ -394,7 +393,7 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = s_tmem;
-    const uint32_t idesc_s = make_idesc(false), idesc_o = make_idesc(true);
+    const uint32_t idesc_s = make_idesc(false, 64), idesc_o = make_idesc(true, 128);
     const uint32_t tO = tmem + ((uint32_t)((warp & 3) * 32) << 16) + 256u + (uint32_t)grp * 128u;   // this group's O row
     bool failed = false;
 
@@ -437,48 +436,62 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
             const uint32_t hi = (uint32_t)(make_desc(0, 16) >> 32);
             const uint32_t q_lo = (uint32_t)make_desc(sQ, 16), k_lo = (uint32_t)make_desc(sK, 16);
             const uint32_t v_lo = (uint32_t)make_desc(sV, HALF);
-            int kbuf = 0, vbuf = 0;              // buffers of the next S and of the next P V
+            int kbuf = 0, vbuf = 0;              // ring slots of the next chunk to score / to multiply by V
             uint32_t kph = 0, vph = 0;           // and their phases (flip each time the ring wraps)
-            auto issue_s = [&](int i) {          // S[i & 1] = Q K(i)^T
-                const int buf = kbuf;
-                if (!failed && !mbar_wait_one(kfull(buf), kph)) failed = true;
-                if (++kbuf == NS) { kbuf = 0; kph ^= 1u; }
+            // S_g(c) = Q K(c)[64 g .. 64 g + 63]^T into buffer c & 1 of group g; K(c) sits in slot kbuf
+            auto issue_s = [&](int c, int g2) {
                 if (failed) return;
                 tc_fence_after();
-                const uint32_t kb = k_lo + (uint32_t)buf * (TILE >> 4);
+                const uint32_t kb = k_lo + (uint32_t)kbuf * (TILE >> 4) + (uint32_t)g2 * (64u * 128u >> 4);
+                const uint32_t d = tmem + (uint32_t)g2 * 128u + (uint32_t)(c & 1) * 64u;
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) { // K = 16 per instruction over d = 128
                     const uint32_t koff = ((ks >> 2) * HALF + (ks & 3) * 32) >> 4;
-                    mma_f16_lo(tmem + (uint32_t)(i & 1) * 128u, q_lo + koff, hi, kb + koff, hi, idesc_s, ks > 0);
+                    mma_f16_lo(d, q_lo + koff, hi, kb + koff, hi, idesc_s, ks > 0);
                 }
-                mma_commit(sfull(i & 1));
-                mma_commit(kfree(buf));
+                mma_commit(sfull(g2, c & 1));
             };
-            issue_s(0);
-            if (n_ch > 1) issue_s(1);
-            for (int i = 0; i < n_ch; ++i) {
-                const int g2 = i & 1;
-                const uint32_t ph = (uint32_t)(i >> 1) & 1u;
-                // O[g2] += P(i) V(i): P from the four warps of group g2 (in tensor memory, over the
-                // scores it was computed from) and the V chunk
-                if (!failed && !mbar_wait_one(pfull(g2), ph)) failed = true;
-                if (!failed && !mbar_wait_one(vfull(vbuf), vph)) failed = true;
+            // both halves of the scores of chunk c (the K slot is released by the second commit)
+            auto issue_s_first = [&](int c) {
+                if (!failed && !mbar_wait_one(kfull(kbuf), kph)) failed = true;
+                issue_s(c, 0);
+            };
+            auto issue_s_second = [&](int c) {
+                issue_s(c, 1);
+                if (!failed) mma_commit(kfree(kbuf));
+                if (++kbuf == NS) { kbuf = 0; kph ^= 1u; }
+            };
+            issue_s_first(0);
+            issue_s_second(0);
+            if (n_ch > 1) { issue_s_first(1); issue_s_second(1); }
+            for (int c = 0; c < n_ch; ++c) {
+                const int p = c & 1;
+                const uint32_t ph = (uint32_t)(c >> 1) & 1u;
                 const uint32_t vb = v_lo + (uint32_t)vbuf * (TILE >> 4);
-                const uint32_t vfree_bar = vfree(vbuf);
-                if (++vbuf == NS) { vbuf = 0; vph ^= 1u; }
-                if (!failed) {
-                    tc_fence_after();
 #pragma unroll
-                    for (int ks = 0; ks < 8; ++ks) { // K = 16 keys per instruction = 8 columns of packed bf16 pairs
-                        // V as an MN-major operand: d is contiguous, the two 64-wide halves are HALF bytes apart
-                        mma_f16_ts(tmem + 256u + (uint32_t)g2 * 128u, tmem + (uint32_t)g2 * 128u + (uint32_t)ks * 8u,
-                                   vb + (uint32_t)(ks * 16 * 128 >> 4), hi, idesc_o, (i >= 2) || (ks > 0));
+                for (int g2 = 0; g2 < 2; ++g2) {
+                    // O[g2] += P_g2(c) V(c)[64 g2 .. 64 g2 + 63]: P from the four warps of group g2 (in tensor
+                    // memory, over the scores it was computed from) and the V chunk
+                    if (!failed && !mbar_wait_one(pfull(g2, p), ph)) failed = true;
+                    if (g2 == 0 && !failed && !mbar_wait_one(vfull(vbuf), vph)) failed = true;
+                    if (!failed) {
+                        tc_fence_after();
+                        const uint32_t a_t = tmem + (uint32_t)g2 * 128u + (uint32_t)p * 64u;
+#pragma unroll
+                        for (int ks = 0; ks < 4; ++ks) { // K = 16 keys per instruction = 8 columns of packed bf16 pairs
+                            // V as an MN-major operand: d is contiguous, the two 64-wide halves are HALF bytes apart
+                            mma_f16_ts(tmem + 256u + (uint32_t)g2 * 128u, a_t + (uint32_t)ks * 8u,
+                                       vb + (uint32_t)((g2 * 64 + ks * 16) * 128 >> 4), hi, idesc_o, (c > 0) || (ks > 0));
+                        }
+                        mma_commit(odone(g2, p));
+                        if (g2 == 1) mma_commit(vfree(vbuf));
                     }
-                    mma_commit(odone(g2));
-                    mma_commit(vfree_bar);
+                    // tensor-core work completes in issue order, so the scores of chunk c + 2 may replace P_g2(c)
+                    if (c + 2 < n_ch) {
+                        if (g2 == 0) issue_s_first(c + 2); else issue_s_second(c + 2);
+                    }
                 }
-                // tensor-core work completes in issue order, so the scores of chunk i + 2 may replace P(i)
-                if (i + 2 < n_ch) issue_s(i + 2);
+                if (++vbuf == NS) { vbuf = 0; vph ^= 1u; }
             }
             if (failed) s_fail = 1;
         }
@@ -486,24 +499,24 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
     } else {
         // ================= softmax warps =================
         const uint32_t lanes = (uint32_t)((warp & 3) * 32) << 16;
-        const uint32_t tS = tmem + lanes + (uint32_t)grp * 128u;             // this group's scores, then its P
         const unsigned long long anc = s_anc[node];
         const float scale = a.scale_log2;
         float m_run = -INFINITY, l_run = 0.f;
 
-        for (int i = grp; i < n_ch; i += 2) {
-            const int ch = c0 + i;
-            if (!failed && !mbar_wait(sfull(grp), (uint32_t)(i >> 1) & 1u)) failed = true;
+        for (int c = 0; c < n_ch; ++c) {
+            const int ch = c0 + c, p = c & 1;
+            const uint32_t tS = tmem + lanes + (uint32_t)grp * 128u + (uint32_t)p * 64u;   // scores, then P
+            if (!failed && !mbar_wait(sfull(grp, p), (uint32_t)(c >> 1) & 1u)) failed = true;
             tc_fence_after();
             const bool masked = (ch + 1) * BK > L;   // only chunks that reach past the cached prefix
-            // Validity of the chunk's 128 keys for this row as four 32-bit words: prefix keys are
+            // Validity of this group's 64 keys for this row as two 32-bit words: prefix keys are
             // valid, tree key L + t is valid iff bit t of the row's ancestor mask is set (bits at and
             // beyond the tree size are clear, which also rules out the zero padding).
-            uint32_t valid[4] = {~0u, ~0u, ~0u, ~0u};
+            uint32_t valid[2] = {~0u, ~0u};
             if (masked) {
 #pragma unroll
-                for (int blk = 0; blk < 4; ++blk) {
-                    const int off = ch * BK + blk * 32 - L;      // tree index of the word's first key
+                for (int blk = 0; blk < 2; ++blk) {
+                    const int off = ch * BK + grp * 64 + blk * 32 - L;      // tree index of the word's first key
                     uint32_t wv;
                     if (off >= 64) wv = 0u;
                     else if (off >= 0) wv = (uint32_t)(anc >> off);
@@ -525,7 +538,7 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
             // ---- pass 1: row maximum ----
             float mx = -INFINITY;
 #pragma unroll
-            for (int blk = 0; blk < 4; ++blk) {
+            for (int blk = 0; blk < 2; ++blk) {
                 float v[32];
                 load_scores(blk, v);
 #pragma unroll
@@ -541,9 +554,10 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
             const float m_new = move ? m_cand : m_run;
             const float m_safe = (m_new == -INFINITY) ? 0.f : m_new;
             const float alpha = move ? ex2f(m_run - m_safe) : 1.f;
-            // ---- rescale this row of O[grp].  The products of this group's previous chunk are complete:
-            // the scores just read were issued after them and complete in order. ----
-            if (i >= 2 && move) {
+            // ---- rescale this row of O[grp], once the group's product of the previous chunk is complete ----
+            if (c >= 1 && move) {
+                if (!failed && !mbar_wait(odone(grp, (c - 1) & 1), (uint32_t)((c - 1) >> 1) & 1u)) failed = true;
+                tc_fence_after();
 #pragma unroll
                 for (int blk = 0; blk < 4; ++blk) {
                     float o[32];
@@ -557,7 +571,7 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
             // (block blk of P takes columns 16 blk .. 16 blk + 15, all below the 32 (blk + 1) columns read) ----
             float rs = 0.f;
 #pragma unroll
-            for (int blk = 0; blk < 4; ++blk) {
+            for (int blk = 0; blk < 2; ++blk) {
                 float v[32];
                 load_scores(blk, v);
                 uint32_t w[16];
@@ -575,22 +589,18 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
             asm volatile("tcgen05.wait::st.sync.aligned;\n" ::: "memory");
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(pfull(grp));
+            if (lane == 0) mbar_arrive(pfull(grp, p));
         }
-        // ---- each group waits for its own last product; the CTA-wide barrier below then orders both
-        // accumulators before the merge (a group's barrier is only ever waited on by that group, in
-        // phase order, so a parity wait can never see it a phase behind) ----
-        if (grp < n_ch) {
-            const int last = grp ? ((n_ch - 2) & ~1) + 1 : (n_ch - 1) & ~1;    // last chunk index of the group
-            if (!failed && !mbar_wait(odone(grp), (uint32_t)(last >> 1) & 1u)) failed = true;
-        }
+        // ---- each group waits for its own last product (tensor-core work completes in order, so the
+        // one before it is complete too); the CTA-wide barrier below then orders both accumulators
+        // before the merge ----
+        if (!failed && !mbar_wait(odone(grp, (n_ch - 1) & 1), (uint32_t)((n_ch - 1) >> 1) & 1u)) failed = true;
         tc_fence_after();
         if (failed) s_fail = 1;
-        // For a group that has waited for its last product the Q tile is dead (every S was issued
-        // before that product and completes before it): it carries the groups' (max, sum) exchange.
-        // A group without a chunk has waited for nothing and must not touch it.
+        // the Q tile is dead (every S was issued before that product and completes before it): it
+        // carries the groups' (max, sum) exchange
         float2 *s_ml = reinterpret_cast<float2 *>(smem_raw + (base - smem_u32(smem_raw)));
-        if (grp < n_ch) s_ml[grp * BM + row] = make_float2(m_run, l_run);
+        s_ml[grp * BM + row] = make_float2(m_run, l_run);
         fspad_pdl_trigger();                      // the merge kernel may start launching
         tc_fence_before();
         __syncthreads();
@@ -602,24 +612,19 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
         const bool any_fail = s_fail != 0;
         if (any_fail && tid == 0) fspad_report(a.status, FSPAD_ERR_TIMEOUT);
         const bool store = row_ok && !any_fail;
-        const float2 ml0 = s_ml[row], ml1 = (n_ch >= 2) ? s_ml[BM + row] : make_float2(-INFINITY, 0.f);
+        const float2 ml0 = s_ml[row], ml1 = s_ml[BM + row];
         const float m_all = fmaxf(ml0.x, ml1.x);
         const float m_fin = (m_all == -INFINITY) ? 0.f : m_all;
-        const float f0 = ex2f(ml0.x - m_fin), f1 = ex2f(ml1.x - m_fin);     // exp2(-inf) = 0 for an idle group
+        const float f0 = ex2f(ml0.x - m_fin), f1 = ex2f(ml1.x - m_fin);     // exp2(-inf) = 0 for a fully masked half
         float *po = a.part_o + (prow * M + (row_ok ? gr : 0)) * D + grp * 64;
         const uint32_t tO0 = tmem + lanes + 256u + (uint32_t)grp * 64u, tO1 = tO0 + 128u;
 #pragma unroll
         for (int q2 = 0; q2 < 2; ++q2) {
-            float o[32];
+            float o[32], o1[32];
             tmem_ld32(tO0 + q2 * 32, o);
+            tmem_ld32(tO1 + q2 * 32, o1);
 #pragma unroll
-            for (int j = 0; j < 32; ++j) o[j] *= f0;
-            if (n_ch >= 2) {                      // group 1 has accumulated something (uniform over the CTA)
-                float o1[32];
-                tmem_ld32(tO1 + q2 * 32, o1);
-#pragma unroll
-                for (int j = 0; j < 32; ++j) o[j] = fmaf(o1[j], f1, o[j]);
-            }
+            for (int j = 0; j < 32; ++j) o[j] = fmaf(o1[j], f1, o[j] * f0);
             if (store) {
 #pragma unroll
                 for (int j = 0; j < 32; j += 4)
