@@ -139,13 +139,16 @@ __device__ __forceinline__ void mma_f16(uint32_t d_tmem, uint64_t a_desc, uint64
 }
 // same instruction, descriptors handed over as (low, high) words so the issuing thread can keep
 // the precomputed low words in registers and add a tile offset with one integer add
+// The whole warp runs the issue loop so that descriptors and addresses stay warp-uniform values;
+// `elect` is non-zero in the one lane whose instruction is actually issued.
 __device__ __forceinline__ void mma_f16_lo(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
-                                           uint32_t idesc, uint32_t accumulate)
+                                           uint32_t idesc, uint32_t accumulate, uint32_t elect)
 {
-    asm volatile("{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\tsetp.ne.b32 p, %6, 0;\n\t"
+    asm volatile("{\n\t.reg .pred p, e;\n\t.reg .b64 da, db;\n\tsetp.ne.b32 p, %6, 0;\n\tsetp.ne.b32 e, %7, 0;\n\t"
                  "mov.b64 da, {%1, %2};\n\tmov.b64 db, {%3, %4};\n\t"
-                 "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, p;\n\t}\n"
-                 :: "r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate) : "memory");
+                 "@e tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, p;\n\t}\n"
+                 :: "r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate), "r"(elect)
+                 : "memory");
 }
 // single-thread bounded wait (the tensor-core thread polls alone; nothing warp-collective follows)
 __device__ __forceinline__ bool mbar_wait_one(uint32_t bar, uint32_t parity)
@@ -213,12 +216,18 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar)
 // D[tmem] (+)= A[tmem] * B[smem]: the A operand (here P, bf16 pairs packed into 32-bit columns, one
 // query row per lane) is read from tensor memory
 __device__ __forceinline__ void mma_f16_ts(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t b_hi, uint32_t idesc,
-                                           uint32_t accumulate)
+                                           uint32_t accumulate, uint32_t elect)
 {
-    asm volatile("{\n\t.reg .pred p;\n\t.reg .b64 db;\n\tsetp.ne.b32 p, %5, 0;\n\t"
+    asm volatile("{\n\t.reg .pred p, e;\n\t.reg .b64 db;\n\tsetp.ne.b32 p, %5, 0;\n\tsetp.ne.b32 e, %6, 0;\n\t"
                  "mov.b64 db, {%2, %3};\n\t"
-                 "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n\t}\n"
-                 :: "r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate) : "memory");
+                 "@e tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n\t}\n"
+                 :: "r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate), "r"(elect) : "memory");
+}
+__device__ __forceinline__ void mma_commit_if(uint32_t bar, uint32_t elect)
+{
+    asm volatile("{\n\t.reg .pred e;\n\tsetp.ne.b32 e, %1, 0;\n\t"
+                 "@e tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}\n"
+                 :: "r"(bar), "r"(elect) : "memory");
 }
 __device__ __forceinline__ void tmem_st16(uint32_t addr, const uint32_t (&v)[16])
 {
@@ -430,7 +439,8 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
         if (failed) s_fail = 1;
     } else if (warp == 9) {
         // ================= tensor-core warp: one thread issues every tcgen05.mma =================
-        if (lane == 0) {
+        {
+            const uint32_t elect = lane == 0;     // every lane runs the loop, this one issues
             // low words of the shared-memory descriptors (start address and leading byte offset);
             // the high word (8-row group stride, version, swizzle mode) is the same for all
             const uint32_t hi = (uint32_t)(make_desc(0, 16) >> 32);
@@ -447,9 +457,9 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) { // K = 16 per instruction over d = 128
                     const uint32_t koff = ((ks >> 2) * HALF + (ks & 3) * 32) >> 4;
-                    mma_f16_lo(d, q_lo + koff, hi, kb + koff, hi, idesc_s, ks > 0);
+                    mma_f16_lo(d, q_lo + koff, hi, kb + koff, hi, idesc_s, ks > 0, elect);
                 }
-                mma_commit(sfull(g2, c & 1));
+                mma_commit_if(sfull(g2, c & 1), elect);
             };
             // both halves of the scores of chunk c (the K slot is released by the second commit)
             auto issue_s_first = [&](int c) {
@@ -458,7 +468,7 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
             };
             auto issue_s_second = [&](int c) {
                 issue_s(c, 1);
-                if (!failed) mma_commit(kfree(kbuf));
+                if (!failed) mma_commit_if(kfree(kbuf), elect);
                 if (++kbuf == NS) { kbuf = 0; kph ^= 1u; }
             };
             issue_s_first(0);
@@ -481,10 +491,10 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
                         for (int ks = 0; ks < 4; ++ks) { // K = 16 keys per instruction = 8 columns of packed bf16 pairs
                             // V as an MN-major operand: d is contiguous, the two 64-wide halves are HALF bytes apart
                             mma_f16_ts(tmem + 256u + (uint32_t)g2 * 128u, a_t + (uint32_t)ks * 8u,
-                                       vb + (uint32_t)((g2 * 64 + ks * 16) * 128 >> 4), hi, idesc_o, (c > 0) || (ks > 0));
+                                       vb + (uint32_t)((g2 * 64 + ks * 16) * 128 >> 4), hi, idesc_o, (c > 0) || (ks > 0), elect);
                         }
-                        mma_commit(odone(g2, p));
-                        if (g2 == 1) mma_commit(vfree(vbuf));
+                        mma_commit_if(odone(g2, p), elect);
+                        if (g2 == 1) mma_commit_if(vfree(vbuf), elect);
                     }
                     // tensor-core work completes in issue order, so the scores of chunk c + 2 may replace P_g2(c)
                     if (c + 2 < n_ch) {
