@@ -246,21 +246,22 @@ __device__ __forceinline__ void tmem_st16(uint32_t addr, const uint32_t (&v)[16]
 // when the loop ends.  Warp 8 is the copy warp: it issues every TMA copy of the loop and gathers
 // the one chunk TMA cannot describe.  Warp 9 is the tensor-core warp: one of its threads issues
 // every tcgen05.mma; the warp owns the tensor memory.
-// Tensor memory: columns [128 g + 64 p, 128 g + 64 p + 64) hold the fp32 scores S_g of the group's
-// chunks of parity p and then, written over their first 32 columns, P as packed bf16 pairs, which
-// the second product reads directly as its A operand; columns [256 + 128 g, 384 + 128 g) hold O_g.
+// Tensor memory: columns [128 p, 128 p + 128) hold the fp32 scores S of the chunks of parity p, the
+// 64 columns at 128 p + 64 g being group g's, and then, written over the first 32 of those, P_g as
+// packed bf16 pairs, which the second product reads directly as its A operand; columns
+// [256 + 128 g, 384 + 128 g) hold O_g.
 // With two score buffers per group the scores of chunk c + 1 are complete long before the group
 // has finished chunk c, and O_g += P V runs under the group's next softmax: a group never waits for
 // the tensor cores unless it has to rescale O.
 // The sides meet only on mbarriers, never on a CTA-wide barrier inside the loop:
 //   kfull/vfull(b)  K / V ring slot b filled (TMA bytes, or one arrival)     tensor-core warp waits
 //   kfree/vfree(b)  both S (both P V) of the chunk in slot b complete        copy warp waits
-//   sfull(g, p)     S_g of a chunk of parity p complete (tcgen05.commit)     group g waits
+//   sfull(p)        S of a chunk of parity p complete (tcgen05.commit)       both groups wait
 //   pfull(g, p)     P_g written and O_g rescaled by the 4 warps of group g   tensor-core warp waits
 //   odone(g, p)     O_g += P_g V of a chunk of parity p complete             group g waits (rescale, end)
-// Every barrier has exactly one waiting side, and a new phase of it can only begin after that
-// side has seen the previous one (a parity wait must never fall two phases behind).
-// Tensor-core order: S_0(0) S_1(0) S_0(1) S_1(1) | PV_0(0) S_0(2) PV_1(0) S_1(2) | PV_0(1) S_0(3) ...
+// A new phase of a barrier can only begin after every side that waits on it has seen the previous
+// one (a parity wait must never fall two phases behind).
+// Tensor-core order: S(0) S(1) | PV_0(0) PV_1(0) S(2) | PV_0(1) PV_1(1) S(3) | ...
 __global__ void __launch_bounds__(NT, 1)
 tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV)
 {
@@ -309,7 +310,7 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
     auto vfull = [&](int buf) { return bar0 + 8u * (uint32_t)(NS + buf); };
     auto kfree = [&](int buf) { return bar0 + 8u * (uint32_t)(2 * NS + buf); };
     auto vfree = [&](int buf) { return bar0 + 8u * (uint32_t)(3 * NS + buf); };
-    auto sfull = [&](int grp2, int par) { return bar0 + 8u * (uint32_t)(4 * NS + 2 * grp2 + par); };
+    auto sfull = [&](int par) { return bar0 + 8u * (uint32_t)(4 * NS + par); };
     auto pfull = [&](int grp2, int par) { return bar0 + 8u * (uint32_t)(4 * NS + 4 + 2 * grp2 + par); };
     auto odone = [&](int grp2, int par) { return bar0 + 8u * (uint32_t)(4 * NS + 8 + 2 * grp2 + par); };
     const bool tma_ok = a.use_tma != 0;
@@ -402,7 +403,7 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = s_tmem;
-    const uint32_t idesc_s = make_idesc(false, 64), idesc_o = make_idesc(true, 128);
+    const uint32_t idesc_s = make_idesc(false, 128), idesc_o = make_idesc(true, 128);
     const uint32_t tO = tmem + ((uint32_t)((warp & 3) * 32) << 16) + 256u + (uint32_t)grp * 128u;   // this group's O row
     bool failed = false;
 
@@ -448,32 +449,26 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
             const uint32_t v_lo = (uint32_t)make_desc(sV, HALF);
             int kbuf = 0, vbuf = 0;              // ring slots of the next chunk to score / to multiply by V
             uint32_t kph = 0, vph = 0;           // and their phases (flip each time the ring wraps)
-            // S_g(c) = Q K(c)[64 g .. 64 g + 63]^T into buffer c & 1 of group g; K(c) sits in slot kbuf
-            auto issue_s = [&](int c, int g2) {
-                if (failed) return;
-                tc_fence_after();
-                const uint32_t kb = k_lo + (uint32_t)kbuf * (TILE >> 4) + (uint32_t)g2 * (64u * 128u >> 4);
-                const uint32_t d = tmem + (uint32_t)g2 * 128u + (uint32_t)(c & 1) * 64u;
-#pragma unroll
-                for (int ks = 0; ks < 8; ++ks) { // K = 16 per instruction over d = 128
-                    const uint32_t koff = ((ks >> 2) * HALF + (ks & 3) * 32) >> 4;
-                    mma_f16_lo(d, q_lo + koff, hi, kb + koff, hi, idesc_s, ks > 0, elect);
-                }
-                mma_commit_if(sfull(g2, c & 1), elect);
-            };
-            // both halves of the scores of chunk c (the K slot is released by the second commit)
-            auto issue_s_first = [&](int c) {
+            // S(c) = Q K(c)^T into score buffer c & 1 (columns 0..63 of it belong to group 0, 64..127 to
+            // group 1); K(c) sits in ring slot kbuf, which the second commit releases
+            auto issue_s = [&](int c) {
                 if (!failed && !mbar_wait_one(kfull(kbuf), kph)) failed = true;
-                issue_s(c, 0);
-            };
-            auto issue_s_second = [&](int c) {
-                issue_s(c, 1);
-                if (!failed) mma_commit_if(kfree(kbuf), elect);
+                if (!failed) {
+                    tc_fence_after();
+                    const uint32_t kb = k_lo + (uint32_t)kbuf * (TILE >> 4);
+                    const uint32_t d = tmem + (uint32_t)(c & 1) * 128u;
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks) { // K = 16 per instruction over d = 128
+                        const uint32_t koff = ((ks >> 2) * HALF + (ks & 3) * 32) >> 4;
+                        mma_f16_lo(d, q_lo + koff, hi, kb + koff, hi, idesc_s, ks > 0, elect);
+                    }
+                    mma_commit_if(sfull(c & 1), elect);
+                    mma_commit_if(kfree(kbuf), elect);
+                }
                 if (++kbuf == NS) { kbuf = 0; kph ^= 1u; }
             };
-            issue_s_first(0);
-            issue_s_second(0);
-            if (n_ch > 1) { issue_s_first(1); issue_s_second(1); }
+            issue_s(0);
+            if (n_ch > 1) issue_s(1);
             for (int c = 0; c < n_ch; ++c) {
                 const int p = c & 1;
                 const uint32_t ph = (uint32_t)(c >> 1) & 1u;
@@ -486,7 +481,7 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
                     if (g2 == 0 && !failed && !mbar_wait_one(vfull(vbuf), vph)) failed = true;
                     if (!failed) {
                         tc_fence_after();
-                        const uint32_t a_t = tmem + (uint32_t)g2 * 128u + (uint32_t)p * 64u;
+                        const uint32_t a_t = tmem + (uint32_t)p * 128u + (uint32_t)g2 * 64u;
 #pragma unroll
                         for (int ks = 0; ks < 4; ++ks) { // K = 16 keys per instruction = 8 columns of packed bf16 pairs
                             // V as an MN-major operand: d is contiguous, the two 64-wide halves are HALF bytes apart
@@ -496,11 +491,9 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
                         mma_commit_if(odone(g2, p), elect);
                         if (g2 == 1) mma_commit_if(vfree(vbuf), elect);
                     }
-                    // tensor-core work completes in issue order, so the scores of chunk c + 2 may replace P_g2(c)
-                    if (c + 2 < n_ch) {
-                        if (g2 == 0) issue_s_first(c + 2); else issue_s_second(c + 2);
-                    }
                 }
+                // tensor-core work completes in issue order, so the scores of chunk c + 2 may replace P(c)
+                if (c + 2 < n_ch) issue_s(c + 2);
                 if (++vbuf == NS) { vbuf = 0; vph ^= 1u; }
             }
             if (failed) s_fail = 1;
@@ -515,8 +508,8 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
 
         for (int c = 0; c < n_ch; ++c) {
             const int ch = c0 + c, p = c & 1;
-            const uint32_t tS = tmem + lanes + (uint32_t)grp * 128u + (uint32_t)p * 64u;   // scores, then P
-            if (!failed && !mbar_wait(sfull(grp, p), (uint32_t)(c >> 1) & 1u)) failed = true;
+            const uint32_t tS = tmem + lanes + (uint32_t)p * 128u + (uint32_t)grp * 64u;   // scores, then P
+            if (!failed && !mbar_wait(sfull(p), (uint32_t)(c >> 1) & 1u)) failed = true;
             tc_fence_after();
             const bool masked = (ch + 1) * BK > L;   // only chunks that reach past the cached prefix
             // Validity of this group's 64 keys for this row as two 32-bit words: prefix keys are
