@@ -28,7 +28,10 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
     return *reinterpret_cast<uint32_t *>(&v);
 }
 
-// Merge the split partials of one output row by log-sum-exp; one warp per row.
+// Merge the split partials of one output row by log-sum-exp; one warp per row.  kBatch = how many
+// ranges' rows a lane requests at once (few ranges: a small batch keeps the kernel light; many:
+// a large one saves dependent round trips through L2).
+template <int kBatch>
 __global__ void __launch_bounds__(128)
 tree_attn_combine_kernel(const AttnArgs a, int B)
 {
@@ -61,22 +64,25 @@ tree_attn_combine_kernel(const AttnArgs a, int B)
     float denom = w0 * l0 + w1 * l1;
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) denom += __shfl_xor_sync(0xffffffffu, denom, off);
+    // The partial rows are requested before the weights are known (one round trip through L2 for up
+    // to kBatch ranges instead of one per dependent step); a range that saw no key left its row
+    // unwritten, so what was loaded for a zero weight is discarded, not multiplied.
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int s0 = 0; s0 < ns; s0 += 4) {
-        float4 v[4];
-        float w[4];
+    for (int s0 = 0; s0 < ns; s0 += kBatch) {
+        float4 v[kBatch];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
+        for (int u = 0; u < kBatch; ++u) {
             const int sidx = s0 + u;
-            const float wa = __shfl_sync(0xffffffffu, w0, sidx & 31), wb = __shfl_sync(0xffffffffu, w1, sidx & 31);
-            w[u] = (sidx < ns) ? ((sidx < 32) ? wa : wb) : 0.f;
             v[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (w[u] != 0.f)
+            if (sidx < ns)
                 v[u] = __ldcg(reinterpret_cast<const float4 *>(a.part_o + ((pbase + sidx) * a.M + gr) * D + lane * 4));
         }
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            acc.x += w[u] * v[u].x; acc.y += w[u] * v[u].y; acc.z += w[u] * v[u].z; acc.w += w[u] * v[u].w;
+        for (int u = 0; u < kBatch; ++u) {
+            const int sidx = s0 + u;
+            const float wa = __shfl_sync(0xffffffffu, w0, sidx & 31), wb = __shfl_sync(0xffffffffu, w1, sidx & 31);
+            const float w = (sidx < ns) ? ((sidx < 32) ? wa : wb) : 0.f;
+            if (w != 0.f) { acc.x += w * v[u].x; acc.y += w * v[u].y; acc.z += w * v[u].z; acc.w += w * v[u].w; }
         }
     }
     const float inv = denom > 0.f ? 1.f / denom : 0.f;
@@ -110,5 +116,7 @@ cudaError_t fspad_launch_tree_attn(fspad_ctx *ctx, const fspad_bf16 *q, const fs
     if (e != cudaSuccess) return e;
     const long long rows = (long long)B * c.n_kv_heads * a.M;
     ctx->launches++;
-    return fspad_launch_opt(false, tree_attn_combine_kernel, dim3((unsigned)((rows + 3) / 4)), dim3(128), 0, st, 0, a, B);
+    const dim3 grid((unsigned)((rows + 3) / 4));
+    if (a.n_splits <= 4) return fspad_launch_opt(false, tree_attn_combine_kernel<4>, grid, dim3(128), 0, st, 0, a, B);
+    return fspad_launch_opt(false, tree_attn_combine_kernel<12>, grid, dim3(128), 0, st, 0, a, B);
 }
