@@ -255,25 +255,36 @@ accept_walk_kernel(const WalkArgs args)
     fspad_pdl_trigger();
     if (tid < 64) { sh.exp_tbl[tid] = kExp2Tbl[tid]; sh.child_mask[tid] = 0ull; }
     fspad_pdl_wait();
+    // The prologue is a chain of dependent global loads; it is kept to two round trips.
+    // Round trip 1: everything that depends on nothing - temperature, tree arrays, uniforms.
     float Tf = args.temperature[b];
+    int p = -1, t = 0;
+    float uval = 0.f;
+    if (tid < N) {
+        p = args.parent[(size_t)b * N + tid];
+        t = args.tokens[(size_t)b * N + tid];
+    }
+    if (args.uniforms != nullptr && tid <= N)      // thread c: node c's uniform; thread 0: the bonus uniform
+        uval = args.uniforms[(size_t)b * (N + 1) + (tid == 0 ? N : tid)];
     if (!(Tf >= 0.0f)) {
         if (tid == 0 && rank == 0) fspad_report(args.status, FSPAD_ERR_RANGE);
         Tf = 0.0f;
     }
     const bool sampling = Tf > 0.0f && args.draft != nullptr && args.uniforms != nullptr;
     if (Tf > 0.0f && !sampling && tid == 0 && rank == 0) fspad_report(args.status, FSPAD_ERR_NULL);
-    __syncthreads();
+    __syncthreads();                             // child masks are zeroed
 
     const float *lg = args.logits + (size_t)b * N * V;
     const float *dp = args.draft ? args.draft + (size_t)b * N * V : nullptr;
-    const float *un = args.uniforms ? args.uniforms + (size_t)b * (N + 1) : nullptr;
     int *out_path = args.path + (size_t)b * args.path_stride;
     const float kT = kLog2eF / (Tf > 0.0f ? Tf : 1.0f);
 
-    // Gathered once, in parallel: thread c owns node c (tree arrays, the child bit of its parent
-    // and the three scalars its accept test needs); half-warps merge the scan partials of the rows.
+    // Round trip 2: thread c owns node c (tree arrays, the child bit of its parent and the scalars
+    // its accept test needs: target logit and draft probability of its token in its parent's row);
+    // half-warps merge the scan partials of the rows.  The gathered scalars stay in registers until
+    // the merge has issued its own loads.
+    float xv = 0.f, qv = 0.f;
     if (tid < N) {
-        int p = args.parent[(size_t)b * N + tid], t = args.tokens[(size_t)b * N + tid];
         if (tid == 0) {
             if (p != -1) fspad_report(args.status, FSPAD_ERR_BAD_TREE);
             p = -1;
@@ -291,12 +302,9 @@ accept_walk_kernel(const WalkArgs args)
             atomicOr(&sh.child_mask[p], 1ull << tid);
             if (sampling) {
                 const size_t at = (size_t)p * V + t;
-                sh.cx[tid] = lg[at];
-                sh.cq[tid] = dp[at];
-                sh.cu[tid] = un[tid];
+                xv = lg[at];
+                qv = dp[at];
             }
-        } else if (sampling) {
-            sh.ubonus = un[N];
         }
     }
     {
@@ -307,6 +315,10 @@ accept_walk_kernel(const WalkArgs args)
             fspad_stats_merge_half(args.parts, args.geom, b * N + row, row < N, kT, lane16, M, S, A);
             if (lane16 == 0 && row < N) { sh.rowM[row] = M; sh.rowS[row] = S; sh.rowA[row] = A; }
         }
+    }
+    if (sampling && tid < N) {
+        if (tid >= 1) { sh.cx[tid] = xv; sh.cq[tid] = qv; sh.cu[tid] = uval; }
+        else sh.ubonus = uval;
     }
     __syncthreads();
     if (sampling && tid >= 1 && tid < N)
