@@ -91,6 +91,7 @@ struct Shared {
     // every node, its parent's logit and draft probability at the node's token and its uniform
     float rowM[FSPAD_MAX_NODES];
     double rowS[FSPAD_MAX_NODES];
+    double rowInvS[FSPAD_MAX_NODES];   // 1 / rowS, so that no division sits on the serial path
     int rowA[FSPAD_MAX_NODES];
     float cx[FSPAD_MAX_NODES], cq[FSPAD_MAX_NODES], cu[FSPAD_MAX_NODES];
     double cex[FSPAD_MAX_NODES];    // exp((logit - row max)/T) of each node's token in its parent's row
@@ -313,7 +314,7 @@ accept_walk_kernel(const WalkArgs args)
             const int row = r0 + (tid >> 4);
             float M; double S; int A;
             fspad_stats_merge_half(args.parts, args.geom, b * N + row, row < N, kT, lane16, M, S, A);
-            if (lane16 == 0 && row < N) { sh.rowM[row] = M; sh.rowS[row] = S; sh.rowA[row] = A; }
+            if (lane16 == 0 && row < N) { sh.rowM[row] = M; sh.rowS[row] = S; sh.rowInvS[row] = 1.0 / S; sh.rowA[row] = A; }
         }
     }
     if (sampling && tid < N) {
@@ -397,6 +398,7 @@ accept_walk_kernel(const WalkArgs args)
         parity ^= 1;
     };
 
+    const double invT = 1.0 / (double)Tf;        // every thread: off the serial path of thread 0
     if (tid == 0) { sh.cur = 0; sh.len = 1; sh.path[0] = 0; }
     __syncthreads();
 
@@ -407,8 +409,8 @@ accept_walk_kernel(const WalkArgs args)
         if (tid == 0) {
             sh.m = (double)sh.rowM[cur];
             sh.S = sh.rowS[cur];
-            sh.invS = 1.0 / sh.S;
-            sh.invT = 1.0 / (double)Tf;
+            sh.invS = sh.rowInvS[cur];
+            sh.invT = invT;
             sh.exact = 0; sh.have_e = 0; sh.have_q = 0;
             sh.c = 0.0; sh.U = 1.0; sh.D = 1.0;
             sh.nrem = 0;
