@@ -349,7 +349,7 @@ def main():
             "mean_accepted_len": float(n_acc_host.mean()),
             "roofline": {"kernel": "accept_stats_kernel", "bound": "hbm", "achieved": achieved, "peak": peak,
                          "peak_kind": "%s copy bandwidth (burst, kernel timed alone)" % peak_kind, "unit": "GB/s",
-                         "frac": achieved / peak, "traffic": 30800896 if (w.name == "llama3_8b_2k") else None,
+                         "frac": achieved / peak, "traffic": 30800128 if (w.name == "llama3_8b_2k") else None,
                          "traffic_note": "dram__bytes_read+write per launch, ncu capture in profiles/accept_stats_kernel_llama3_8b_2k.md", "algorithmic_bytes_per_launch": stats_bytes},
             "e2e": {"value": e2e_us, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "steps": e2e_steps, "note": "fspad_verify_step_host: pinned host inputs, device-resident KV cache"},
