@@ -241,17 +241,17 @@ __device__ __forceinline__ void tmem_st16(uint32_t addr, const uint32_t (&v)[16]
 
 // Roles.  Warps 0-7 are the softmax warps, in two groups of four (128 threads, one query row per
 // thread, a warp reaching the tensor-memory lane quarter given by its index modulo 4).  Group g
-// owns keys 64 g .. 64 g + 63 of every chunk: its own score buffers (two, used alternately),
-// running reference maximum, sum and O accumulator, merged with the other group's by log-sum-exp
-// when the loop ends.  Warp 8 is the copy warp: it issues every TMA copy of the loop and gathers
+// owns keys 64 g .. 64 g + 63 of every chunk: its half of each score buffer, its own running
+// reference maximum, sum and O accumulator, merged with the other group's by log-sum-exp when the
+// loop ends.  Warp 8 is the copy warp: it issues every TMA copy of the loop and gathers
 // the one chunk TMA cannot describe.  Warp 9 is the tensor-core warp: one of its threads issues
 // every tcgen05.mma; the warp owns the tensor memory.
 // Tensor memory: columns [128 p, 128 p + 128) hold the fp32 scores S of the chunks of parity p, the
 // 64 columns at 128 p + 64 g being group g's, and then, written over the first 32 of those, P_g as
 // packed bf16 pairs, which the second product reads directly as its A operand; columns
 // [256 + 128 g, 384 + 128 g) hold O_g.
-// With two score buffers per group the scores of chunk c + 1 are complete long before the group
-// has finished chunk c, and O_g += P V runs under the group's next softmax: a group never waits for
+// With two score buffers the scores of chunk c + 1 are complete long before the groups have
+// finished chunk c, and O_g += P V runs under the group's next softmax: a group never waits for
 // the tensor cores unless it has to rescale O.
 // The sides meet only on mbarriers, never on a CTA-wide barrier inside the loop:
 //   kfull/vfull(b)  K / V ring slot b filled (TMA bytes, or one arrival)     tensor-core warp waits
