@@ -68,6 +68,27 @@ def test_tree_rows_taken_from_cache_when_no_tree_arrays():
     assert torch.equal(a, b)
 
 
+@pytest.mark.parametrize("prefix", [0, 100, 128, 200, 256, 300, 511, 640, 1000])
+def test_every_chunk_count_per_cta(prefix):
+    """80 kv heads fill the GPU with one key range per head, so a CTA walks all of the sequence's
+    1 .. 9 chunks itself: every wrap state of the three-deep K/V ring and of the parity-doubled
+    score barriers, with the gathered boundary chunk first, in the middle of the ring, or last."""
+    w = synth.scaled(W["llama3_8b_2k"], n_q_heads=80, n_kv_heads=80, prefix=(prefix, prefix), n_nodes=9,
+                     depth=3, branch=3, vocab=16)
+    inp = synth.generate(w, 3, with_accept=False)
+    if prefix < 64:
+        _shrink_values(inp)
+    _check(inp)
+
+
+@pytest.mark.parametrize("hq,hkv,n", [(16, 2, 60), (24, 2, 33), (12, 4, 64)])
+def test_gqa_row_tiles(hq, hkv, n):
+    """Rows per kv head beyond one 128-row tile: 480 (four tiles, the last ragged), 396, 192."""
+    w = synth.scaled(W["llama3_8b_2k"], n_q_heads=hq, n_kv_heads=hkv, prefix=(700, 700), n_nodes=n,
+                     depth=6, branch=4, vocab=16)
+    _check(synth.generate(w, 4, with_accept=False))
+
+
 def test_batched_ragged_small():
     w = synth.scaled(W["batch16_ragged"], batch=5, prefix=(10, 700), temperatures=(0.0,) * 5, vocab=16)
     _check(synth.generate(w, 0, with_accept=False))
