@@ -314,14 +314,14 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
     auto pfull = [&](int grp2, int par) { return bar0 + 8u * (uint32_t)(4 * NS + 4 + 2 * grp2 + par); };
     auto odone = [&](int grp2, int par) { return bar0 + 8u * (uint32_t)(4 * NS + 8 + 2 * grp2 + par); };
     const bool tma_ok = a.use_tma != 0;
-    if (tid == 0) {
+    // The thread that issues the first TMA copies also initialises the barriers, so those copies
+    // leave as soon as the prefix length is known, ahead of the CTA's first barrier.
+    if (tid == 256) {
 #pragma unroll
         for (int i = 0; i < 4 * NS + 12; ++i) mbar_init(bar0 + 8u * i, (i >= 4 * NS + 4 && i < 4 * NS + 8) ? 4 : 1);
         s_fail = 0;
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     }
-    if (tid < N) s_par[tid] = a.parent[(size_t)b * N + tid];
-    __syncthreads();
 
     const fspad_bf16 *kcb = a.kc + ((size_t)b * a.Hkv + g) * (size_t)a.max_len * D;
     const fspad_bf16 *vcb = a.vc + ((size_t)b * a.Hkv + g) * (size_t)a.max_len * D;
@@ -377,6 +377,8 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
         cp_async16(sQ + tile_off(r, c), src, ok);
     }
     cp_async_commit();
+    if (tid < N) s_par[tid] = a.parent[(size_t)b * N + tid];
+    __syncthreads();                              // barriers initialised, parents staged
     if (warp == 9) {
         __syncwarp();
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n"
