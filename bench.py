@@ -50,6 +50,28 @@ def peaks():
     return 6650.0, "fallback"
 
 
+def tensor_peak():
+    """Dense bf16 TFLOP/s (burst figure: the attention call is timed alone)."""
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            return float(json.load(f)["bf16_tflops"]), "measured"
+    return 1590.0, "fallback"
+
+
+def attention_report(w, L_mean, attn_us, attn_bytes, hbm_peak):
+    """The attention call (range kernel + merge kernel) against both of its roofs: bytes of Q, K, V and
+    the output once, and the dense-tile flops 4 * N * Hq * d * (L + N) of the two products."""
+    flops = 4.0 * w.n_nodes * w.n_q_heads * w.head_dim * (L_mean + w.n_nodes) * w.batch
+    tpeak, tkind = tensor_peak()
+    gbs, tfl = attn_bytes / (attn_us * 1e-6) / 1e9, flops / (attn_us * 1e-6) / 1e12
+    g = w.n_q_heads // w.n_kv_heads
+    return {"us": attn_us, "algorithmic_bytes": attn_bytes, "gbs": gbs, "frac_of_hbm_peak": gbs / hbm_peak,
+            "dense_tile_flops": flops, "tflops": tfl, "frac_of_bf16_peak": tfl / tpeak, "bf16_peak_tflops": tpeak,
+            "bf16_peak_kind": tkind, "flop_per_byte": w.n_nodes * g,
+            "bound": "hbm" if w.n_nodes * g < 200 else ("tensor" if w.n_nodes * g > 300 else "ridge")}
+
+
 class ClockSampler:
     FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
               "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
@@ -351,6 +373,7 @@ def main():
                          "peak_kind": "%s copy bandwidth (burst, kernel timed alone)" % peak_kind, "unit": "GB/s",
                          "frac": achieved / peak, "traffic": 30800128 if (w.name == "llama3_8b_2k") else None,
                          "traffic_note": "dram__bytes_read+write per launch, ncu capture in profiles/accept_stats_kernel_llama3_8b_2k.md", "algorithmic_bytes_per_launch": stats_bytes},
+            "tree_attn_call": attention_report(w, L_mean, attn_us, bytes_real["attention"], peak),
             "e2e": {"value": e2e_us, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "steps": e2e_steps, "note": "fspad_verify_step_host: pinned host inputs, device-resident KV cache"},
             "gpu_launches": int(launches),
