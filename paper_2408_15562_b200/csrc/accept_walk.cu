@@ -97,6 +97,7 @@ struct Shared {
     double cex[FSPAD_MAX_NODES];    // exp((logit - row max)/T) of each node's token in its parent's row
     float ubonus;
     int want_q;
+    int bonus_ok;                   // the last residual sweep already holds the bonus draw's per-thread sums
     // reductions
     double warp_a[kWarps], warp_b[kWarps], warp_off[kWarps];
     double slot[2][kMaxCluster][2]; // partial sums received from every CTA of the cluster, by pass parity
@@ -400,6 +401,7 @@ accept_walk_kernel(const WalkArgs args)
 
     const double invT = 1.0 / (double)Tf;        // every thread: off the serial path of thread 0
     if (tid == 0) { sh.cur = 0; sh.len = 1; sh.path[0] = 0; }
+    double last_a = 0.0;                         // this thread's sum of weights in the latest residual sweep
     __syncthreads();
 
     for (;;) {   // one iteration per node on the path
@@ -415,6 +417,7 @@ accept_walk_kernel(const WalkArgs args)
             sh.c = 0.0; sh.U = 1.0; sh.D = 1.0;
             sh.nrem = 0;
             sh.next = -1;
+            sh.bonus_ok = 0;
         }
         __syncthreads();
 
@@ -467,8 +470,13 @@ accept_walk_kernel(const WalkArgs args)
             {
                 Sweep s = sweep_chunk<MODE_RESID>(sh, x, q, se, sq, tid, nthr, lo, hi, vec, cache_ok, sh.have_e != 0,
                                                   sh.have_q != 0, sh.cprime, xt, false, 0, 0, 0, nullptr);
+                last_a = s.a;
                 reduce_exchange(s.a, s.b);
             }
+            // When this was the node's last child, the weights just summed (residual at the new
+            // coefficient, the rejected tokens at their frozen values) are the ones the bonus token is
+            // drawn from, thread by thread in the same order: the draw can reuse the sums.
+            const bool last_child = (rem & (rem - 1)) == 0;
             if (tid == 0) {
                 const double W = sh.tot[0], Dn = sh.tot[1];
                 double frozen;
@@ -476,6 +484,7 @@ accept_walk_kernel(const WalkArgs args)
                     frozen = weight(sh.ex, sh.qx, sh.invS, sh.cprime);
                     sh.c = sh.cprime;
                     sh.U = W;
+                    sh.bonus_ok = last_child ? 1 : 0;
                 } else {
                     frozen = weight(sh.ex, sh.qx, sh.invS, sh.c);   // residual vanished: p is kept
                 }
@@ -507,8 +516,10 @@ accept_walk_kernel(const WalkArgs args)
         const bool have_e = sh.have_e != 0, have_q = sh.have_q != 0;
         // with nothing rejected at this node (c == 0) the weights are the e_j themselves and the
         // denominator cancels, so no separate exact-sum sweep is needed
-        Sweep s = sweep_chunk<MODE_CDF>(sh, x, q, se, sq, tid, nthr, lo, hi, vec, cache_ok, have_e, have_q, c, -1,
-                                        false, 0, 0, 0, nullptr);
+        Sweep s{last_a, 0.0};
+        if (!sh.bonus_ok)
+            s = sweep_chunk<MODE_CDF>(sh, x, q, se, sq, tid, nthr, lo, hi, vec, cache_ok, have_e, have_q, c, -1, false, 0, 0,
+                                      0, nullptr);
         // block-wide inclusive scan of the per-thread sums (index order)
         double incl = s.a;
         const int lane = tid & 31, wid = tid >> 5;
