@@ -44,6 +44,8 @@ constexpr int kWalkThreads = 1024;
 constexpr int kWarps = kWalkThreads / 32;
 constexpr int kSmemBudget = 200 * 1024;   // dynamic shared memory for the per-node cache
 constexpr double kAmbiguous = 1e-4;
+constexpr double kScanRel = 1e-6;          // bound taken for the relative error of the scan's sum of exponentials
+constexpr double kFusedTol = 1e-9;         // relative error the fused first-rejection sweep may leave in the residual mass
 constexpr float kLog2eF = 1.4426950408889634f;
 
 // 2^(i/64), i = 0..63, correctly rounded
@@ -102,6 +104,8 @@ struct Shared {
     double warp_a[kWarps], warp_b[kWarps], warp_off[kWarps];
     double slot[2][kMaxCluster][2]; // partial sums received from every CTA of the cluster, by pass parity
     double tot[2];                  // cluster totals
+    double warp5[kWarps][5], slot5[2][kMaxCluster][5], tot5[5];   // the same exchange for five values
+    int fused_fallback;
     double cta_total[kMaxCluster];  // bonus draw: every CTA's total, received from the peers
 };
 
@@ -239,6 +243,60 @@ __device__ Sweep sweep_chunk(const Shared &sh, const float *__restrict__ x, cons
     }
     if (locate) *found = (hit >= 0) ? hit : last_pos;
     return Sweep{a, b};
+}
+
+// The first rejection at a node, in one sweep instead of two.  The exact denominator S is not known
+// yet, but the residual sum_j max(e_j / S - c q_j, 0) is linear in 1 / S over a fixed set of positive
+// terms: with P = { j : e_j / S' - c q_j > 0 } taken at the scan's S' it equals (sum_P e_j) / S -
+// c sum_P q_j for every S that leaves P unchanged.  The sweep returns
+//   v[0] = sum e_j (= S)      v[1] = sum_P e_j      v[2] = sum_P q_j
+//   v[3] = sum of q_j over j != xnew (the next draft mass)
+//   v[4] = sum of e_j / S' over the tokens whose sign a relative error kScanRel of S' could flip;
+// a flipped token changes the result by at most kScanRel times its probability, so kScanRel * v[4]
+// bounds the error and the caller falls back to the two-sweep path when that is not negligible.
+// e_j and q_j are parked in shared memory as in the exact-sum sweep.
+struct Sweep5 {
+    double v[5];
+};
+__device__ Sweep5 fused_reject_sweep(const Shared &sh, const float *__restrict__ x, const float *__restrict__ q,
+                                     double *__restrict__ se, float *__restrict__ sq, int tid, int nthr, int lo, int hi,
+                                     bool vec, bool cache_ok, double inv_s_scan, double c, int xnew)
+{
+    const double m = sh.m, invT = sh.invT;
+    Sweep5 r{{0.0, 0.0, 0.0, 0.0, 0.0}};
+    for (int j = lo; j < hi; j += 4) {
+        const int n = min(4, hi - j);
+        float xv[4], qv[4];
+        if (vec && n == 4) {
+            const float4 t4 = __ldg(reinterpret_cast<const float4 *>(x + j));
+            const float4 u4 = __ldg(reinterpret_cast<const float4 *>(q + j));
+            xv[0] = t4.x; xv[1] = t4.y; xv[2] = t4.z; xv[3] = t4.w;
+            qv[0] = u4.x; qv[1] = u4.y; qv[2] = u4.z; qv[3] = u4.w;
+        } else {
+#pragma unroll
+            for (int t = 0; t < 4; ++t) {
+                xv[t] = (t < n) ? x[j + t] : -INFINITY;
+                qv[t] = (t < n) ? q[j + t] : 0.f;
+            }
+        }
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+            if (t >= n) break;
+            const double e = exp_neg(((double)xv[t] - m) * invT, sh.exp_tbl);
+            const double qd = (double)qv[t];
+            if (cache_ok) {
+                se[(j - lo + t) * nthr + tid] = e;
+                sq[(j - lo + t) * nthr + tid] = qv[t];
+            }
+            const double pe = e * inv_s_scan;
+            const double w = pe - c * qd;
+            r.v[0] += e;
+            if (w > 0.0) { r.v[1] += e; r.v[2] += qd; }
+            if (j + t != xnew) r.v[3] += qd;
+            if (pe > 0.0 && fabs(w) <= kScanRel * pe) r.v[4] += pe;
+        }
+    }
+    return r;
 }
 
 __global__ void __launch_bounds__(kWalkThreads, 1)
@@ -400,6 +458,38 @@ accept_walk_kernel(const WalkArgs args)
     };
 
     const double invT = 1.0 / (double)Tf;        // every thread: off the serial path of thread 0
+    // the same exchange for the five sums of the fused sweep; result in sh.tot5[]
+    auto reduce_exchange5 = [&](const Sweep5 &in) {
+        const int lane = tid & 31, wid = tid >> 5, nwarps = nthr >> 5;
+        double v[5];
+#pragma unroll
+        for (int k = 0; k < 5; ++k) v[k] = warp_sum(in.v[k]);
+        if (lane == 0) {
+#pragma unroll
+            for (int k = 0; k < 5; ++k) sh.warp5[wid][k] = v[k];
+        }
+        __syncthreads();
+        if (wid == 0) {
+#pragma unroll
+            for (int k = 0; k < 5; ++k) v[k] = warp_sum((lane < nwarps) ? sh.warp5[lane][k] : 0.0);
+            if (lane < C) {
+                double *peer = cluster.map_shared_rank(&sh.slot5[parity][rank][0], lane);
+#pragma unroll
+                for (int k = 0; k < 5; ++k) peer[k] = v[k];
+            }
+        }
+        cluster.sync();
+        if (wid == 0) {
+#pragma unroll
+            for (int k = 0; k < 5; ++k) {
+                const double t = warp_sum((lane < C) ? sh.slot5[parity][lane][k] : 0.0);
+                if (lane == 0) sh.tot5[k] = t;
+            }
+        }
+        __syncthreads();
+        parity ^= 1;
+    };
+
     if (tid == 0) { sh.cur = 0; sh.len = 1; sh.path[0] = 0; }
     double last_a = 0.0;                         // this thread's sum of weights in the latest residual sweep
     __syncthreads();
@@ -441,13 +531,13 @@ accept_walk_kernel(const WalkArgs args)
                     if (!sh.exact) {
                         const double big = fmax(lhs, rhs);
                         if (big > 0.0 && fabs(lhs - rhs) <= kAmbiguous * big) dec = 2;
-                        else if (dec == 0) dec = 2;      // a rejection needs the exact denominator anyway
+                        else if (dec == 0) dec = 3;      // clear rejection: exact denominator and residual in one sweep
                     }
                     sh.decision = dec;
                     sh.ex = ex; sh.qx = qx; sh.ridx = ridx; sh.xnew = xt;
                 }
                 __syncthreads();
-                if (sh.decision != 2) break;
+                if (sh.decision != 2) break;                  // 0, 1 or 3
                 // exact softmax denominator of this node (parks e_j in shared memory)
                 const bool with_q = sh.want_q != 0;
                 Sweep s = sweep_chunk<MODE_EXP>(sh, x, q, se, sq, tid, nthr, lo, hi, vec, cache_ok, false, false, 0.0,
@@ -467,7 +557,28 @@ accept_walk_kernel(const WalkArgs args)
             // -- rejected: one sweep gives the new residual mass and the new draft mass
             if (tid == 0) sh.cprime = sh.c + sh.U / sh.D;
             __syncthreads();
-            {
+            const bool last_child = (rem & (rem - 1)) == 0;
+            bool fused_done = false;
+            if (sh.decision == 3) {
+                // first rejection at this node, nothing exact yet (c = 0, U = D = 1, nothing removed)
+                const double cp = sh.cprime;
+                const Sweep5 f = fused_reject_sweep(sh, x, q, se, sq, tid, nthr, lo, hi, vec, cache_ok, sh.invS, cp, xt);
+                reduce_exchange5(f);
+                if (tid == 0) {
+                    const double S = sh.tot5[0], invS = 1.0 / S;
+                    const double W = sh.tot5[1] * invS - cp * sh.tot5[2];
+                    sh.S = S; sh.invS = invS; sh.exact = 1; sh.have_e = cache_ok; sh.have_q = cache_ok;
+                    sh.fused_fallback = !(W > 0.0 && kScanRel * sh.tot5[4] <= kFusedTol * W);
+                    if (!sh.fused_fallback) {
+                        sh.tot[0] = W;
+                        sh.tot[1] = sh.tot5[3];
+                    }
+                }
+                __syncthreads();
+                fused_done = !sh.fused_fallback;
+                if (fused_done) last_a = f.v[1] * sh.invS - cp * f.v[2];
+            }
+            if (!fused_done) {
                 Sweep s = sweep_chunk<MODE_RESID>(sh, x, q, se, sq, tid, nthr, lo, hi, vec, cache_ok, sh.have_e != 0,
                                                   sh.have_q != 0, sh.cprime, xt, false, 0, 0, 0, nullptr);
                 last_a = s.a;
@@ -475,8 +586,7 @@ accept_walk_kernel(const WalkArgs args)
             }
             // When this was the node's last child, the weights just summed (residual at the new
             // coefficient, the rejected tokens at their frozen values) are the ones the bonus token is
-            // drawn from, thread by thread in the same order: the draw can reuse the sums.
-            const bool last_child = (rem & (rem - 1)) == 0;
+            // drawn from, thread by thread in the same order: the draw reuses the sums (last_a).
             if (tid == 0) {
                 const double W = sh.tot[0], Dn = sh.tot[1];
                 double frozen;
