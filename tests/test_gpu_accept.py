@@ -83,6 +83,30 @@ def test_draft_far_from_target_forces_many_rejections():
     assert rejected_somewhere > 20
 
 
+def test_draft_equal_to_target_up_to_fp32_rounding():
+    """q = softmax(logits) up to a few fp32 ulps: every token sits inside the band where the scan's approximate
+    denominator cannot fix the sign of p - q, so the one-sweep first rejection must hand over to the
+    exact two-sweep path; the residual mass itself is of the order of fp32 rounding."""
+    w = synth.scaled(W["llama3_8b_2k"], batch=6, vocab=5000, n_nodes=24, depth=3, branch=8,
+                     temperatures=(1.0, 1.0, 0.7, 0.7, 1.3, 1.3), prefix=(8, 8))
+    rejected = 0
+    for variant in range(3):
+        inp = synth.generate(w, variant, with_attention=False)
+        z = inp.target_logits.astype(np.float64) / inp.temperature[:, None, None].astype(np.float64)
+        p = np.exp(z - z.max(-1, keepdims=True))
+        wobble = 1.0 + 3e-7 * np.random.default_rng(variant).choice([-1.0, 1.0], size=p.shape)
+        inp.draft_probs[...] = (p / p.sum(-1, keepdims=True) * wobble).astype(np.float32)
+        # uniforms just below one: r * q < p now fails wherever q lies above p, so rejections do occur
+        keep = inp.uniforms[:, -1].copy()
+        inp.uniforms[...] = np.nextafter(np.float32(1), np.float32(0))
+        inp.uniforms[:, -1] = keep
+        _assert_parity(inp, allow_near=w.batch)
+        r = oracle.tree_accept(inp.target_logits, inp.draft_probs, inp.draft_tokens, inp.parent,
+                               inp.temperature, inp.uniforms)
+        rejected += int((~np.isnan(r["trace_rq"])).sum() - (r["n_accepted"] - 1).sum())
+    assert rejected > 0
+
+
 def test_zero_mass_and_minus_inf_logits():
     w = synth.scaled(W["llama3_8b_2k"], batch=4, vocab=512, n_nodes=16, depth=4, branch=3,
                      temperatures=(1.0,) * 4, prefix=(8, 8))
