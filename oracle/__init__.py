@@ -106,3 +106,21 @@ def kv_compact(cache: np.ndarray, accepted_path, n_accepted, prefix_len):
     if rc != 0:
         raise RuntimeError("oracle_kv_compact failed: %d" % rc)
     return new_len
+
+
+def tree_build(cand_parent, cand_token, cand_logp, root_token, n_nodes: int):
+    """Final stage of the dynamic token tree: keep the n_nodes - 1 most probable candidates and
+    flatten them breadth-first behind the root.  Arrays [B][C]; returns parent, token, cand [B][N]
+    and n_out [B]; `valid` is False when the joint probabilities were not monotone along a path."""
+    cand_parent = np.ascontiguousarray(cand_parent, np.int32)
+    B, C = cand_parent.shape
+    parent = np.empty((B, n_nodes), np.int32)
+    token = np.empty((B, n_nodes), np.int32)
+    cand = np.empty((B, n_nodes), np.int32)
+    n_out = np.empty(B, np.int32)
+    rc = lib().oracle_tree_build(_p(cand_parent, np.int32), _p(cand_token, np.int32), _p(cand_logp, np.float32),
+                                 _p(root_token, np.int32), B, C, n_nodes, _p(parent, np.int32),
+                                 _p(token, np.int32), _p(cand, np.int32), _p(n_out, np.int32))
+    if rc not in (0, -3):
+        raise RuntimeError("oracle_tree_build failed: %d" % rc)
+    return {"parent": parent, "token": token, "cand": cand, "n_out": n_out, "valid": rc == 0}

@@ -14,7 +14,9 @@
  * Parity pins (tests/test_oracle_*.py): chain tree == dense causal
  * attention, per-path brute force, greedy == naive per-path comparison,
  * exact emitted-token distribution of the rejection sampler at vocab 8,
- * hand-worked decision traces, brute-force compaction.
+ * hand-worked decision traces, brute-force compaction; tree builder
+ * (tests/test_oracle_tree_build.py): hand-worked cases, stable library sort,
+ * brute force over ancestor-closed subsets, flattened-tree invariants.
  *
  * The only parallelism is an OpenMP loop over independent units (heads,
  * node rows, cache slices); each unit runs the plain definition.
@@ -319,4 +321,74 @@ int oracle_kv_compact(uint16_t *cache, const int32_t *accepted_path, const int32
     if (new_len)
         for (int b = 0; b < B; ++b) new_len[b] = prefix_len[b] + n_accepted[b];
     return bad ? -2 : 0;
+}
+
+/* -------------------------------------------------------------------------
+ * O5  Dynamic token tree, final stage (paper, Section "Preliminaries", last
+ * paragraph: every draft step is truncated to its top-k, each token carries
+ * the joint probability of its path, and one top-k over all tokens after the
+ * draft phase yields a valid tree of bounded size; Section "Performance on
+ * Fewer Candidate Tokens" halves both budgets).
+ *
+ * Input: C candidates per sequence, listed level by level, so that the parent
+ * of a candidate has a lower index; cand_parent = -1 for the children of the
+ * root; cand_logp = joint log-probability of the path, never larger than the
+ * parent's.  The N - 1 candidates with the largest joint probability are kept
+ * (equal values: the lower index first, which keeps parents before children).
+ * Because the joint probability cannot grow along a path the kept set is
+ * closed under "parent of"; an input that violates this is reported (-3).
+ * Output: the flattened tree the verification step takes.  Node 0 is the root
+ * (root_token); the kept candidates follow ordered by depth and, inside a
+ * depth, by candidate index (breadth-first numbering, so parent[i] < i).
+ *   parent_out, token_out, cand_out [B][N] (cand_out[0] = -1; entries at and
+ *   beyond n_out[b] are -1), n_out[b] = 1 + min(N - 1, C).
+ * Plain selection: one pass per kept node over all candidates.
+ * ---------------------------------------------------------------------- */
+int oracle_tree_build(const int32_t *cand_parent, const int32_t *cand_token, const float *cand_logp,
+                      const int32_t *root_token, int B, int C, int N, int32_t *parent_out,
+                      int32_t *token_out, int32_t *cand_out, int32_t *n_out)
+{
+    int rc = 0;
+    for (int b = 0; b < B; ++b) {
+        const int32_t *cp = cand_parent + (size_t)b * C, *ct = cand_token + (size_t)b * C;
+        const float *lp = cand_logp + (size_t)b * C;
+        int32_t *po = parent_out + (size_t)b * N, *to = token_out + (size_t)b * N, *co = cand_out + (size_t)b * N;
+        char *kept = (char *)calloc((size_t)(C > 0 ? C : 1), 1);
+        int *depth = (int *)calloc((size_t)(C > 0 ? C : 1), sizeof(int));
+        int *node_of = (int *)malloc(sizeof(int) * (size_t)(C > 0 ? C : 1));
+        if (!kept || !depth || !node_of) { free(kept); free(depth); free(node_of); return -2; }
+        for (int i = 0; i < N; ++i) { po[i] = -1; to[i] = -1; co[i] = -1; }
+        const int want = (N - 1 < C) ? N - 1 : C;
+        /* selection: repeatedly take the best candidate not yet kept */
+        for (int s = 0; s < want; ++s) {
+            int best = -1;
+            for (int c = 0; c < C; ++c) {
+                if (kept[c]) continue;
+                if (best < 0 || lp[c] > lp[best]) best = c;   /* strict: equal values keep the lower index */
+            }
+            kept[best] = 1;
+        }
+        /* closure and depths (parents precede children) */
+        for (int c = 0; c < C; ++c) {
+            node_of[c] = -1;
+            if (cp[c] < -1 || cp[c] >= c) { rc = -3; continue; }
+            depth[c] = (cp[c] < 0) ? 1 : depth[cp[c]] + 1;
+            if (kept[c] && cp[c] >= 0 && !kept[cp[c]]) rc = -3;
+        }
+        /* breadth-first numbering: by depth, then by candidate index */
+        po[0] = -1; to[0] = root_token[b]; co[0] = -1;
+        int n = 1;
+        for (int d = 1; n < want + 1 && d <= C; ++d)
+            for (int c = 0; c < C; ++c)
+                if (kept[c] && depth[c] == d) {
+                    node_of[c] = n;
+                    co[n] = c;
+                    to[n] = ct[c];
+                    po[n] = (cp[c] < 0) ? 0 : node_of[cp[c]];
+                    ++n;
+                }
+        n_out[b] = n;
+        free(kept); free(depth); free(node_of);
+    }
+    return rc;
 }

@@ -345,3 +345,52 @@ def random_path(rng: np.random.Generator, parent: np.ndarray) -> np.ndarray:
         c = ch[path[-1]]
         path.append(int(c[int(rng.integers(len(c)))]))
     return np.asarray(path, dtype=np.int32)
+
+
+# --------------------------------------------------------------------------
+# candidate lists for the tree builder
+# --------------------------------------------------------------------------
+def tree_candidates(seed: int, batch: int, levels: int = 5, width: int = 10, branch: int = 10,
+                    vocab: int = 32000, step: float = 0.0):
+    """Candidate tokens as a top-k draft phase leaves them behind, listed level by level.
+
+    Level 1: `branch` children of the root.  Every later level: `width` candidates of the previous
+    level (drawn at random, not by score - choosing them is the builder's business) get `branch`
+    children each.  A candidate's joint log-probability is its parent's plus log U(0,1), so it
+    never grows along a path; with `step` > 0 the values are rounded down to multiples of `step`,
+    which produces many ties, including children equal to their parent.  With the paper's sizes
+    (levels 5, width 10, branch 10) a sequence has 10 + 4 * 100 = 410 candidates; a level never
+    expands more parents than the previous level has.
+    Returns cand_parent, cand_token [B][C] int32, cand_logp [B][C] float32, root_token [B] int32.
+    """
+    rng = np.random.default_rng([SEED_BASE % (2 ** 32), 7, seed])
+    sizes = [branch]                            # candidates per level
+    for _ in range(levels - 1):
+        sizes.append(min(width, sizes[-1]) * branch)
+    C = sum(sizes)
+    cand_parent = np.empty((batch, C), np.int32)
+    cand_token = rng.integers(0, vocab, size=(batch, C), dtype=np.int32)
+    cand_logp = np.empty((batch, C), np.float32)
+    for b in range(batch):
+        lo, hi = 0, branch                      # index range of the previous level
+        cand_parent[b, :branch] = -1
+        cand_logp[b, :branch] = np.log(rng.random(branch))
+        at = branch
+        for _ in range(levels - 1):
+            parents = rng.choice(np.arange(lo, hi), size=min(width, hi - lo), replace=False)
+            parents.sort()
+            for p in parents:
+                cand_parent[b, at:at + branch] = p
+                cand_logp[b, at:at + branch] = cand_logp[b, p] + np.log(rng.random(branch))
+                at += branch
+            lo, hi = hi, at
+        assert at == C
+    if step > 0:
+        cand_logp = (np.floor(cand_logp / step) * step).astype(np.float32)
+        for b in range(batch):                  # flooring keeps order; make sure of it in fp32
+            for c in range(C):
+                p = cand_parent[b, c]
+                if p >= 0 and cand_logp[b, c] > cand_logp[b, p]:
+                    cand_logp[b, c] = cand_logp[b, p]
+    root_token = rng.integers(0, vocab, size=batch, dtype=np.int32)
+    return cand_parent, cand_token, cand_logp.astype(np.float32), root_token
