@@ -12,6 +12,8 @@
  *                      sampling at temperature > 0; Section "Experiments"
  *                      evaluates T = 0 and T = 1 with unrelaxed acceptance)
  *   fspad_kv_compact   keep the accepted path's K/V rows, contiguous in the cache
+ * and, one step earlier in the pipeline,
+ *   fspad_tree_build   the draft phase's candidates -> the flattened token tree
  *
  * Conventions (shared by every call)
  *   - A tree has N <= 64 nodes in topological order: parent[0] = -1 (node 0 is
@@ -191,6 +193,40 @@ int fspad_accept_stats(fspad_ctx *ctx, const float *logits, const float *tempera
 int fspad_accept_stats_noalloc(const float *logits, const float *temperature, int rows,
                                int rows_per_seq, int vocab, float *row_max, double *row_sum,
                                int32_t *row_arg, void *stream);
+
+/*
+ * Dynamic token tree, final stage ("Preliminaries", last paragraph: each draft
+ * step is truncated to its top-k, every token carries the joint probability of
+ * its path, and one top-k over all tokens after the draft phase gives a valid
+ * tree of bounded size; "Performance on Fewer Candidate Tokens" halves both
+ * budgets).  Turns the candidates a draft phase left behind into the flattened
+ * tree that fspad_tree_attn / fspad_tree_accept take.
+ *
+ *   cand_parent [batch][n_cand] int32, device: index of the candidate's parent
+ *               candidate, -1 for a child of the root.  Candidates are listed
+ *               level by level: a parent has a lower index than its children.
+ *   cand_token  [batch][n_cand] int32, device.
+ *   cand_logp   [batch][n_cand] float, device: joint log-probability of the path
+ *               from the root; never larger than the parent's; -inf allowed, NaN
+ *               not.
+ *   root_token  [batch] int32, device: token of node 0.
+ *   n_cand      1 .. 1024;  n_nodes 1 .. max_nodes of the context.
+ *
+ * Kept: the n_nodes - 1 candidates with the largest joint probability; among
+ * equal values the lower index first (so a parent is never displaced by a child
+ * of equal probability).  Output, all [batch][n_nodes] int32, device, written
+ * by the call: node 0 is the root (parent -1, token root_token, candidate -1);
+ * the kept candidates follow ordered by depth and, inside a depth, by candidate
+ * index, so parent_out[i] < i.  cand_out[i] is the candidate a node came from.
+ * n_out[b] = 1 + min(n_nodes - 1, n_cand); entries from n_out[b] on are -1.
+ * Nothing is allocated; the caller owns every array.  A parent index out of
+ * order, or joint probabilities that grow along a path (a kept candidate whose
+ * parent was not kept), set FSPAD_ERR_BAD_TREE in the status word; all writes
+ * stay in bounds.
+ */
+int fspad_tree_build(fspad_ctx *ctx, const int32_t *cand_parent, const int32_t *cand_token,
+                     const float *cand_logp, const int32_t *root_token, int n_cand, int n_nodes, int batch,
+                     int32_t *parent_out, int32_t *token_out, int32_t *cand_out, int32_t *n_out, void *stream);
 
 /*
  * Accepted-path KV compaction ("Preliminaries": the discarded tokens leave the

@@ -19,7 +19,7 @@ _lib = None
 
 EXPORTS = ["fspad_create", "fspad_destroy", "fspad_status", "fspad_strerror", "fspad_launch_count",
            "fspad_tree_attn", "fspad_tree_accept", "fspad_accept_stats", "fspad_kv_compact",
-           "fspad_verify_step_host", "fspad_accept_stats_noalloc"]
+           "fspad_verify_step_host", "fspad_accept_stats_noalloc", "fspad_tree_build"]
 
 
 class FspadConfig(ctypes.Structure):
@@ -58,6 +58,7 @@ def load():
     lib.fspad_kv_compact.argtypes = [vp, vp, vp, vp, vp, ci, vp, vp]
     lib.fspad_accept_stats_noalloc.argtypes = [vp, vp, ci, ci, ci, vp, vp, vp, vp]
     lib.fspad_verify_step_host.argtypes = [vp] * 12 + [ci, ci] + [vp] * 6
+    lib.fspad_tree_build.argtypes = [vp] * 5 + [ci, ci, ci] + [vp] * 5
     _lib = lib
     return lib
 
@@ -181,6 +182,23 @@ class Context:
         if rc != 0:
             raise FspadError(rc, "fspad_kv_compact")
         return new_len
+
+    def tree_build(self, cand_parent, cand_token, cand_logp, root_token, n_nodes, out=None, stream=None):
+        """Candidates [B][C] (device) -> (parent, token, cand) [B][n_nodes] and n_out [B]."""
+        B, C = cand_parent.shape
+        i32 = torch.int32
+        if out is None:
+            dev = cand_parent.device
+            out = tuple(torch.empty((B, n_nodes), dtype=i32, device=dev) for _ in range(3)) + \
+                (torch.empty((B,), dtype=i32, device=dev),)
+        parent, token, cand, n_out = out
+        rc = load().fspad_tree_build(self._h, _ptr(cand_parent, i32), _ptr(cand_token, i32),
+                                     _ptr(cand_logp, torch.float32), _ptr(root_token, i32), C, n_nodes, B,
+                                     _ptr(parent, i32), _ptr(token, i32), _ptr(cand, i32), _ptr(n_out, i32),
+                                     _stream(stream))
+        if rc != 0:
+            raise FspadError(rc, "fspad_tree_build")
+        return parent, token, cand, n_out
 
     def verify_step_host(self, cache, q, tree_k, tree_v, parent, prefix_len, target_logits, draft_probs,
                          draft_tokens, temperature, uniforms, attn_out, accepted_path, n_accepted,

@@ -9,6 +9,7 @@
 #include "fspad.h"
 
 #define FSPAD_MAX_NODES 64
+#define FSPAD_MAX_CANDIDATES 1024
 #define FSPAD_HEAD_DIM 128
 
 // Scratch and bookkeeping owned by a context (all device pointers unless noted).
@@ -237,6 +238,10 @@ cudaError_t fspad_launch_accept_walk(fspad_ctx *ctx, const float *logits, const 
 cudaError_t fspad_launch_stats_partials(fspad_ctx *ctx, const float *logits, const float *temperature,
                                         int rows, int rows_per_seq, int V, FspadStatsGeom *geom,
                                         cudaStream_t st);
+cudaError_t fspad_launch_tree_build(fspad_ctx *ctx, const int *cand_parent, const int *cand_token,
+                                    const float *cand_logp, const int *root_token, int n_cand, int n_nodes,
+                                    int B, int *parent_out, int *token_out, int *cand_out, int *n_out,
+                                    cudaStream_t st);
 cudaError_t fspad_launch_kv_compact(fspad_ctx *ctx, fspad_bf16 *cache, const int *path,
                                     const int *n_acc, const int *prefix_len, int B, int *new_len,
                                     cudaStream_t st);
