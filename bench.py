@@ -288,12 +288,20 @@ def main():
         cur.wait_stream(side)
 
     two_us = timed(step_two_streams, args.steps)
+    # the step before the verify step (not part of `value`): candidates of a top-10, five-level draft
+    # phase -> the flattened tree of N nodes; verified against the oracle, oracle timed beside it
+    cpa, cta, lpa, rta = synth.tree_candidates(w.cfg, B)
+    dcand = [torch.from_numpy(np.ascontiguousarray(a)).cuda() for a in (cpa, cta, lpa, rta)]
+    tb_out = tuple(torch.empty((B, N), dtype=torch.int32, device="cuda") for _ in range(3)) + \
+        (torch.empty((B,), dtype=torch.int32, device="cuda"),)
+    tree_build_us = timed(lambda i: ctx.tree_build(*dcand, N, out=tb_out), args.steps)
     clocks = sampler.stop()
     ctx.check()
 
     # ---- correctness of what was timed: compare the last step with the oracle on rank 0 ----
     n_acc_host = n_acc.cpu().numpy()
     verified = None
+    tree_build_ok, tree_build_cpu_us = None, None
     if rank == 0 and not args.no_verify and B <= 2:
         import oracle
         step(0)
@@ -305,6 +313,11 @@ def main():
                   and all(np.array_equal(path[b_, :k[b_]].cpu().numpy(), ref["accepted_path"][b_, :k[b_]]) for b_ in range(B)))
         ref_o = oracle.tree_attn(inp.q, inp.k_cache, inp.v_cache, inp.tree_k, inp.tree_v, inp.parent, inp.prefix_len)
         err = np.abs(out.float().cpu().numpy() - ref_o)
+        t0 = time.perf_counter()
+        tb_ref = oracle.tree_build(cpa, cta, lpa, rta, N)
+        tree_build_cpu_us = (time.perf_counter() - t0) * 1e6
+        tree_build_ok = all(np.array_equal(tb_out[j].cpu().numpy(), tb_ref[k_])
+                            for j, k_ in enumerate(("parent", "token", "cand", "n_out")))
         verified = {"accept_bit_exact": bool(ok_acc), "attn_max_abs_err": float(err.max()),
                     "attn_mean_abs_err": float(err.mean()),
                     "ok": bool(ok_acc and err.max() <= 1e-2 and err.mean() <= 1e-3)}
@@ -374,6 +387,10 @@ def main():
                          "frac": achieved / peak, "traffic": 30800128 if (w.name == "llama3_8b_2k") else None,
                          "traffic_note": "dram__bytes_read+write per launch, ncu capture in profiles/accept_stats_kernel_llama3_8b_2k.md", "algorithmic_bytes_per_launch": stats_bytes},
             "tree_attn_call": attention_report(w, L_mean, attn_us, bytes_real["attention"], peak),
+            "tree_build_call": {"us": tree_build_us, "candidates_per_sequence": int(cpa.shape[1]), "n_nodes": N,
+                                "batch": B, "bit_exact_vs_oracle": tree_build_ok,
+                                "oracle_us_one_thread": tree_build_cpu_us,
+                                "note": "step before the verify step; not part of value"},
             "e2e": {"value": e2e_us, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "steps": e2e_steps, "note": "fspad_verify_step_host: pinned host inputs, device-resident KV cache"},
             "gpu_launches": int(launches),

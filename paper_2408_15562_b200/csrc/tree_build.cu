@@ -6,9 +6,11 @@
 //
 // One CTA per sequence.  The candidates (at most 1024, level by level, joint
 // log-probabilities that never grow along a path) are sorted in shared memory by
-// a bitonic network over 64-bit composites (order-preserving image of the float
-// in the high word, complemented candidate index in the low word), so equal
-// probabilities keep the lower index and parents stay ahead of their children.
+// a 1024-entry bitonic network over 64-bit composites (order-preserving image of
+// the float in the high word, complemented candidate index in the low word; four
+// entries per thread in registers, exchanges by shuffle inside a warp and through
+// shared memory only for the three widest distances), so equal probabilities
+// keep the lower index and parents stay ahead of their children.
 // The first N - 1 entries are the kept set; one thread per kept candidate walks
 // its parent chain (depth, and that every ancestor was kept), takes its
 // breadth-first position by counting the kept candidates that come before it in
@@ -19,6 +21,7 @@
 namespace {
 
 constexpr int kThreads = 256;
+constexpr int kPerThread = FSPAD_MAX_CANDIDATES / kThreads;   // 4 entries of the sorting network per thread
 
 // order-preserving map float -> uint32 (larger float, larger integer); -0.0 < +0.0 is harmless here
 __device__ __forceinline__ uint32_t orderable(float f)
@@ -29,11 +32,11 @@ __device__ __forceinline__ uint32_t orderable(float f)
 
 __global__ void __launch_bounds__(kThreads)
 tree_build_kernel(const int *__restrict__ cand_parent, const int *__restrict__ cand_token,
-                  const float *__restrict__ cand_logp, const int *__restrict__ root_token, int C, int P, int N,
+                  const float *__restrict__ cand_logp, const int *__restrict__ root_token, int C, int N,
                   int *__restrict__ parent_out, int *__restrict__ token_out, int *__restrict__ cand_out,
                   int *__restrict__ n_out, int *__restrict__ status)
 {
-    __shared__ unsigned long long s_key[FSPAD_MAX_CANDIDATES];   // sorted composites
+    __shared__ unsigned long long s_key[FSPAD_MAX_CANDIDATES];   // exchange buffer, then the sorted composites
     __shared__ short s_par[FSPAD_MAX_CANDIDATES];                // parent candidate (-1: child of the root)
     __shared__ short s_node[FSPAD_MAX_CANDIDATES];               // node number of a kept candidate, else -1
     __shared__ short s_kc[FSPAD_MAX_NODES], s_kd[FSPAD_MAX_NODES];   // kept candidates and their depths
@@ -43,7 +46,11 @@ tree_build_kernel(const int *__restrict__ cand_parent, const int *__restrict__ c
     const int *cp = cand_parent + (size_t)b * C;
     const float *lp = cand_logp + (size_t)b * C;
     bool bad = false;
-    for (int c = tid; c < P; c += kThreads) {
+    // thread t holds entries 4 t .. 4 t + 3 of the 1024-entry network in registers
+    unsigned long long v[kPerThread];
+#pragma unroll
+    for (int r = 0; r < kPerThread; ++r) {
+        const int c = kPerThread * tid + r;
         unsigned long long key = 0ull;                           // padding sorts behind every candidate
         int p = -1;
         if (c < C) {
@@ -51,25 +58,51 @@ tree_build_kernel(const int *__restrict__ cand_parent, const int *__restrict__ c
             p = cp[c];
             if (p < -1 || p >= c) { bad = true; p = -1; }
         }
-        s_key[c] = key;
+        v[r] = key;
         s_par[c] = (short)p;
         s_node[c] = -1;
     }
-    __syncthreads();
-    // bitonic sort, descending
-    for (int k = 2; k <= P; k <<= 1) {
+    // bitonic network, descending.  Partners 1 or 2 apart sit in the same thread, up to 64 apart in
+    // the same warp (shuffles); only the three widest distances go through shared memory.
+    for (int k = 2; k <= FSPAD_MAX_CANDIDATES; k <<= 1) {
         for (int j = k >> 1; j > 0; j >>= 1) {
-            for (int i = tid; i < P; i += kThreads) {
-                const int l = i ^ j;
-                if (l > i) {
-                    const unsigned long long x = s_key[i], y = s_key[l];
-                    const bool desc = (i & k) == 0;
-                    if (desc ? (x < y) : (x > y)) { s_key[i] = y; s_key[l] = x; }
+            if (j < kPerThread) {
+#pragma unroll
+                for (int r = 0; r < kPerThread; ++r) {
+                    const int l = r ^ j;
+                    if (l > r) {
+                        const bool desc = ((kPerThread * tid + r) & k) == 0;
+                        const unsigned long long x = v[r], y = v[l];
+                        if (desc ? (x < y) : (x > y)) { v[r] = y; v[l] = x; }
+                    }
                 }
+            } else {
+                unsigned long long o[kPerThread];
+                if (j < kPerThread * 32) {
+#pragma unroll
+                    for (int r = 0; r < kPerThread; ++r) o[r] = __shfl_xor_sync(0xffffffffu, v[r], j / kPerThread);
+                } else {
+                    __syncthreads();                             // the buffer's previous readers are done
+#pragma unroll
+                    for (int r = 0; r < kPerThread; ++r) s_key[kPerThread * tid + r] = v[r];
+                    __syncthreads();
+                    const int pt = tid ^ (j / kPerThread);
+#pragma unroll
+                    for (int r = 0; r < kPerThread; ++r) o[r] = s_key[kPerThread * pt + r];
+                }
+                const int i0 = kPerThread * tid;
+                const bool lower = (i0 & j) == 0, desc = (i0 & k) == 0;   // same for the thread's four entries
+                const bool take_max = lower == desc;
+#pragma unroll
+                for (int r = 0; r < kPerThread; ++r)
+                    v[r] = take_max ? (v[r] > o[r] ? v[r] : o[r]) : (v[r] < o[r] ? v[r] : o[r]);
             }
-            __syncthreads();
         }
     }
+    __syncthreads();
+#pragma unroll
+    for (int r = 0; r < kPerThread; ++r) s_key[kPerThread * tid + r] = v[r];
+    __syncthreads();
     const int want = min(N - 1, C);
     if (tid < want) s_node[0xffffffffu - (uint32_t)(s_key[tid] & 0xffffffffull)] = 0;   // kept (number follows)
     __syncthreads();
@@ -114,9 +147,7 @@ cudaError_t fspad_launch_tree_build(fspad_ctx *ctx, const int *cand_parent, cons
                                     cudaStream_t st)
 {
     if (B == 0) return cudaSuccess;
-    int P = 2;                                                   // sorting network size: a power of two
-    while (P < n_cand) P <<= 1;
     ctx->launches++;
     return fspad_launch(tree_build_kernel, dim3(B), dim3(kThreads), 0, st, 0, cand_parent, cand_token, cand_logp,
-                        root_token, n_cand, P, n_nodes, parent_out, token_out, cand_out, n_out, ctx->d_status);
+                        root_token, n_cand, n_nodes, parent_out, token_out, cand_out, n_out, ctx->d_status);
 }
