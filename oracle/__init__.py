@@ -118,9 +118,10 @@ def tree_build(cand_parent, cand_token, cand_logp, root_token, n_nodes: int):
     token = np.empty((B, n_nodes), np.int32)
     cand = np.empty((B, n_nodes), np.int32)
     n_out = np.empty(B, np.int32)
+    anc = np.empty((B, n_nodes), np.uint64)
     rc = lib().oracle_tree_build(_p(cand_parent, np.int32), _p(cand_token, np.int32), _p(cand_logp, np.float32),
                                  _p(root_token, np.int32), B, C, n_nodes, _p(parent, np.int32),
-                                 _p(token, np.int32), _p(cand, np.int32), _p(n_out, np.int32))
+                                 _p(token, np.int32), _p(cand, np.int32), _p(anc, np.uint64), _p(n_out, np.int32))
     if rc not in (0, -3):
         raise RuntimeError("oracle_tree_build failed: %d" % rc)
-    return {"parent": parent, "token": token, "cand": cand, "n_out": n_out, "valid": rc == 0}
+    return {"parent": parent, "token": token, "cand": cand, "anc": anc, "n_out": n_out, "valid": rc == 0}

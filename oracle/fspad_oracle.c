@@ -341,12 +341,15 @@ int oracle_kv_compact(uint16_t *cache, const int32_t *accepted_path, const int32
  * (root_token); the kept candidates follow ordered by depth and, inside a
  * depth, by candidate index (breadth-first numbering, so parent[i] < i).
  *   parent_out, token_out, cand_out [B][N] (cand_out[0] = -1; entries at and
- *   beyond n_out[b] are -1), n_out[b] = 1 + min(N - 1, C).
+ *   beyond n_out[b] are -1), n_out[b] = 1 + min(N - 1, C); anc_out [B][N]
+ *   (optional): bit j of anc_out[i] set iff node j is node i or one of its
+ *   ancestors - the mask under which the target verifies the tree
+ *   ("Preliminaries": the mask is updated from the token tree); 0 beyond n_out.
  * Plain selection: one pass per kept node over all candidates.
  * ---------------------------------------------------------------------- */
 int oracle_tree_build(const int32_t *cand_parent, const int32_t *cand_token, const float *cand_logp,
                       const int32_t *root_token, int B, int C, int N, int32_t *parent_out,
-                      int32_t *token_out, int32_t *cand_out, int32_t *n_out)
+                      int32_t *token_out, int32_t *cand_out, uint64_t *anc_out, int32_t *n_out)
 {
     int rc = 0;
     for (int b = 0; b < B; ++b) {
@@ -388,6 +391,12 @@ int oracle_tree_build(const int32_t *cand_parent, const int32_t *cand_token, con
                     ++n;
                 }
         n_out[b] = n;
+        /* attention mask of the flattened tree: node i sees itself and its ancestors */
+        if (anc_out) {
+            uint64_t *ao = anc_out + (size_t)b * N;
+            for (int i = 0; i < N; ++i) ao[i] = 0;
+            for (int i = 0; i < n; ++i) ao[i] = ((i > 0) ? ao[po[i]] : 0) | ((uint64_t)1 << i);
+        }
         free(kept); free(depth); free(node_of);
     }
     return rc;

@@ -28,6 +28,8 @@ def test_hand_worked_cases():
         assert r["n_out"] == case["n_out"], case["name"]
         for key in ("parent", "token", "cand"):
             assert r[key].tolist() == case[key], (case["name"], key, r[key].tolist())
+        if "anc" in case:
+            assert [int(v) for v in r["anc"]] == case["anc"], (case["name"], "anc")
 
 
 @pytest.mark.parametrize("step", [0.0, 0.5])
@@ -79,6 +81,13 @@ def test_flattened_tree_invariants_and_path_preservation():
                 assert tok[i] == ct[b, cand[i]]
                 # the node's parent is the node of the candidate's parent (the root for level 1)
                 assert (par[i] == 0 and cp[b, cand[i]] == -1) or cand[par[i]] == cp[b, cand[i]]
+            # mask: exactly the nodes on the path to the root (brute force by walking up)
+            for i in range(n):
+                path, j = set(), i
+                while j >= 0:
+                    path.add(j)
+                    j = par[j]
+                assert int(r["anc"][b, i]) == sum(1 << int(j) for j in path)
             keys = [(depth[i], cand[i]) for i in range(1, n)]
             assert keys == sorted(keys)                                # breadth-first, index order inside a level
             dropped = np.setdiff1d(np.arange(cp.shape[1]), cand[1:n])
