@@ -219,6 +219,10 @@ int fspad_accept_stats_noalloc(const float *logits, const float *temperature, in
  * the kept candidates follow ordered by depth and, inside a depth, by candidate
  * index, so parent_out[i] < i.  cand_out[i] is the candidate a node came from.
  * n_out[b] = 1 + min(n_nodes - 1, n_cand); entries from n_out[b] on are -1.
+ * anc_out [batch][n_nodes] uint64, device, may be NULL: bit j of anc_out[i] is
+ * set iff node j is node i or one of its ancestors - the attention mask the
+ * target verifies the tree under ("Preliminaries": the mask is updated from the
+ * token tree); 0 from n_out[b] on.
  * Nothing is allocated; the caller owns every array.  A parent index out of
  * order, or joint probabilities that grow along a path (a kept candidate whose
  * parent was not kept), set FSPAD_ERR_BAD_TREE in the status word; all writes
@@ -226,7 +230,8 @@ int fspad_accept_stats_noalloc(const float *logits, const float *temperature, in
  */
 int fspad_tree_build(fspad_ctx *ctx, const int32_t *cand_parent, const int32_t *cand_token,
                      const float *cand_logp, const int32_t *root_token, int n_cand, int n_nodes, int batch,
-                     int32_t *parent_out, int32_t *token_out, int32_t *cand_out, int32_t *n_out, void *stream);
+                     int32_t *parent_out, int32_t *token_out, int32_t *cand_out, uint64_t *anc_out,
+                     int32_t *n_out, void *stream);
 
 /*
  * Accepted-path KV compaction ("Preliminaries": the discarded tokens leave the

@@ -58,7 +58,7 @@ def load():
     lib.fspad_kv_compact.argtypes = [vp, vp, vp, vp, vp, ci, vp, vp]
     lib.fspad_accept_stats_noalloc.argtypes = [vp, vp, ci, ci, ci, vp, vp, vp, vp]
     lib.fspad_verify_step_host.argtypes = [vp] * 12 + [ci, ci] + [vp] * 6
-    lib.fspad_tree_build.argtypes = [vp] * 5 + [ci, ci, ci] + [vp] * 5
+    lib.fspad_tree_build.argtypes = [vp] * 5 + [ci, ci, ci] + [vp] * 6
     _lib = lib
     return lib
 
@@ -183,8 +183,9 @@ class Context:
             raise FspadError(rc, "fspad_kv_compact")
         return new_len
 
-    def tree_build(self, cand_parent, cand_token, cand_logp, root_token, n_nodes, out=None, stream=None):
-        """Candidates [B][C] (device) -> (parent, token, cand) [B][n_nodes] and n_out [B]."""
+    def tree_build(self, cand_parent, cand_token, cand_logp, root_token, n_nodes, out=None, anc=None, stream=None):
+        """Candidates [B][C] (device) -> (parent, token, cand) [B][n_nodes] and n_out [B]; `anc`, if given,
+        is an int64 tensor [B][n_nodes] that receives the ancestor masks (bit patterns of uint64)."""
         B, C = cand_parent.shape
         i32 = torch.int32
         if out is None:
@@ -194,7 +195,8 @@ class Context:
         parent, token, cand, n_out = out
         rc = load().fspad_tree_build(self._h, _ptr(cand_parent, i32), _ptr(cand_token, i32),
                                      _ptr(cand_logp, torch.float32), _ptr(root_token, i32), C, n_nodes, B,
-                                     _ptr(parent, i32), _ptr(token, i32), _ptr(cand, i32), _ptr(n_out, i32),
+                                     _ptr(parent, i32), _ptr(token, i32), _ptr(cand, i32),
+                                     _ptr(anc, torch.int64) if anc is not None else None, _ptr(n_out, i32),
                                      _stream(stream))
         if rc != 0:
             raise FspadError(rc, "fspad_tree_build")

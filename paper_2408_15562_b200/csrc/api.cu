@@ -218,7 +218,8 @@ int fspad_kv_compact(fspad_ctx *ctx, fspad_bf16 *cache, const int32_t *accepted_
 
 int fspad_tree_build(fspad_ctx *ctx, const int32_t *cand_parent, const int32_t *cand_token,
                      const float *cand_logp, const int32_t *root_token, int n_cand, int n_nodes, int batch,
-                     int32_t *parent_out, int32_t *token_out, int32_t *cand_out, int32_t *n_out, void *stream)
+                     int32_t *parent_out, int32_t *token_out, int32_t *cand_out, uint64_t *anc_out,
+                     int32_t *n_out, void *stream)
 {
     int rc = check_common(ctx, n_nodes, batch);
     if (rc) return rc;
@@ -227,7 +228,8 @@ int fspad_tree_build(fspad_ctx *ctx, const int32_t *cand_parent, const int32_t *
     if (n_cand < 1 || n_cand > FSPAD_MAX_CANDIDATES) return FSPAD_ERR_SHAPE;
     if (batch == 0) return FSPAD_OK;
     cudaError_t e = fspad_launch_tree_build(ctx, cand_parent, cand_token, cand_logp, root_token, n_cand, n_nodes,
-                                            batch, parent_out, token_out, cand_out, n_out, fspad_stream(stream));
+                                            batch, parent_out, token_out, cand_out,
+                                            reinterpret_cast<unsigned long long *>(anc_out), n_out, fspad_stream(stream));
     return e == cudaSuccess ? FSPAD_OK : FSPAD_ERR_CUDA;
 }
 

@@ -240,8 +240,8 @@ cudaError_t fspad_launch_stats_partials(fspad_ctx *ctx, const float *logits, con
                                         cudaStream_t st);
 cudaError_t fspad_launch_tree_build(fspad_ctx *ctx, const int *cand_parent, const int *cand_token,
                                     const float *cand_logp, const int *root_token, int n_cand, int n_nodes,
-                                    int B, int *parent_out, int *token_out, int *cand_out, int *n_out,
-                                    cudaStream_t st);
+                                    int B, int *parent_out, int *token_out, int *cand_out,
+                                    unsigned long long *anc_out, int *n_out, cudaStream_t st);
 cudaError_t fspad_launch_kv_compact(fspad_ctx *ctx, fspad_bf16 *cache, const int *path,
                                     const int *n_acc, const int *prefix_len, int B, int *new_len,
                                     cudaStream_t st);

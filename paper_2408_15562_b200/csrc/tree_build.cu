@@ -15,7 +15,7 @@
 // its parent chain (depth, and that every ancestor was kept), takes its
 // breadth-first position by counting the kept candidates that come before it in
 // (depth, index) order, and writes the flattened tree the verification step
-// consumes.  Integer work throughout; no arithmetic on the probabilities.
+// consumes, with (optionally) each node's ancestor-or-self mask.  Integer work throughout; no arithmetic on the probabilities.
 #include "common.cuh"
 
 namespace {
@@ -34,7 +34,7 @@ __global__ void __launch_bounds__(kThreads)
 tree_build_kernel(const int *__restrict__ cand_parent, const int *__restrict__ cand_token,
                   const float *__restrict__ cand_logp, const int *__restrict__ root_token, int C, int N,
                   int *__restrict__ parent_out, int *__restrict__ token_out, int *__restrict__ cand_out,
-                  int *__restrict__ n_out, int *__restrict__ status)
+                  unsigned long long *__restrict__ anc_out, int *__restrict__ n_out, int *__restrict__ status)
 {
     __shared__ unsigned long long s_key[FSPAD_MAX_CANDIDATES];   // exchange buffer, then the sorted composites
     __shared__ short s_par[FSPAD_MAX_CANDIDATES];                // parent candidate (-1: child of the root)
@@ -133,9 +133,20 @@ tree_build_kernel(const int *__restrict__ cand_parent, const int *__restrict__ c
         po[pos] = (p < 0) ? 0 : (int)s_node[p];
         to[pos] = cand_token[(size_t)b * C + my_c];
         co[pos] = my_c;
+        if (anc_out) {                                           // the node, its ancestors and the root
+            unsigned long long mask = 1ull;
+            for (int a = my_c; a >= 0; a = s_par[a]) mask |= 1ull << s_node[a];
+            anc_out[(size_t)b * N + pos] = mask;
+        }
     }
-    if (tid == 0) { po[0] = -1; to[0] = root_token[b]; co[0] = -1; n_out[b] = want + 1; }
-    for (int i = want + 1 + tid; i < N; i += kThreads) { po[i] = -1; to[i] = -1; co[i] = -1; }
+    if (tid == 0) {
+        po[0] = -1; to[0] = root_token[b]; co[0] = -1; n_out[b] = want + 1;
+        if (anc_out) anc_out[(size_t)b * N] = 1ull;
+    }
+    for (int i = want + 1 + tid; i < N; i += kThreads) {
+        po[i] = -1; to[i] = -1; co[i] = -1;
+        if (anc_out) anc_out[(size_t)b * N + i] = 0ull;
+    }
     if (bad) fspad_report(status, FSPAD_ERR_BAD_TREE);
 }
 
@@ -143,11 +154,11 @@ tree_build_kernel(const int *__restrict__ cand_parent, const int *__restrict__ c
 
 cudaError_t fspad_launch_tree_build(fspad_ctx *ctx, const int *cand_parent, const int *cand_token,
                                     const float *cand_logp, const int *root_token, int n_cand, int n_nodes,
-                                    int B, int *parent_out, int *token_out, int *cand_out, int *n_out,
-                                    cudaStream_t st)
+                                    int B, int *parent_out, int *token_out, int *cand_out,
+                                    unsigned long long *anc_out, int *n_out, cudaStream_t st)
 {
     if (B == 0) return cudaSuccess;
     ctx->launches++;
     return fspad_launch(tree_build_kernel, dim3(B), dim3(kThreads), 0, st, 0, cand_parent, cand_token, cand_logp,
-                        root_token, n_cand, n_nodes, parent_out, token_out, cand_out, n_out, ctx->d_status);
+                        root_token, n_cand, n_nodes, parent_out, token_out, cand_out, anc_out, n_out, ctx->d_status);
 }

@@ -15,15 +15,17 @@ def _ctx(max_nodes=64, max_batch=16):
 
 def _run(ctx, cp, ct, lp, rt, n):
     dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
-    parent, token, cand, n_out = ctx.tree_build(dev(cp), dev(ct), dev(lp), dev(rt), n)
-    return [t.cpu().numpy() for t in (parent, token, cand, n_out)]
+    anc = torch.empty((cp.shape[0], n), dtype=torch.int64, device="cuda")
+    parent, token, cand, n_out = ctx.tree_build(dev(cp), dev(ct), dev(lp), dev(rt), n, anc=anc)
+    return [t.cpu().numpy() for t in (parent, token, cand, n_out)] + [anc.cpu().numpy().view(np.uint64)]
 
 
 def _assert_equal(ctx, cp, ct, lp, rt, n):
     ref = oracle.tree_build(cp, ct, lp, rt, n)
     assert ref["valid"]
-    parent, token, cand, n_out = _run(ctx, cp, ct, lp, rt, n)
+    parent, token, cand, n_out, anc = _run(ctx, cp, ct, lp, rt, n)
     ctx.check()
+    assert np.array_equal(anc, ref["anc"])
     assert np.array_equal(n_out, ref["n_out"])
     assert np.array_equal(parent, ref["parent"])
     assert np.array_equal(token, ref["token"])
