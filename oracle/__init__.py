@@ -125,3 +125,22 @@ def tree_build(cand_parent, cand_token, cand_logp, root_token, n_nodes: int):
     if rc not in (0, -3):
         raise RuntimeError("oracle_tree_build failed: %d" % rc)
     return {"parent": parent, "token": token, "cand": cand, "anc": anc, "n_out": n_out, "valid": rc == 0}
+
+
+def draft_expand(logprobs, frontier_logp, frontier_cand, top_k: int, width: int, base: int,
+                 cand_parent, cand_token, cand_logp):
+    """One draft step of the dynamic tree: per-row top-k, joint log-probabilities, next frontier.
+    logprobs [B][F][V]; the candidate arrays [B][cap] are updated in place at base .. base + F*top_k - 1.
+    Returns (next_cand [B][width], next_logp [B][width])."""
+    logprobs = np.ascontiguousarray(logprobs, np.float32)
+    B, F, V = logprobs.shape
+    cap = cand_parent.shape[1]
+    next_cand = np.empty((B, width), np.int32)
+    next_logp = np.empty((B, width), np.float32)
+    rc = lib().oracle_draft_expand(_p(logprobs, np.float32), _p(np.ascontiguousarray(frontier_logp, np.float32), np.float32),
+                                   _p(np.ascontiguousarray(frontier_cand, np.int32), np.int32), B, F, V, top_k, width,
+                                   base, cap, _p(cand_parent, np.int32), _p(cand_token, np.int32),
+                                   _p(cand_logp, np.float32), _p(next_cand, np.int32), _p(next_logp, np.float32))
+    if rc != 0:
+        raise RuntimeError("oracle_draft_expand failed: %d" % rc)
+    return next_cand, next_logp

@@ -16,7 +16,9 @@
  * exact emitted-token distribution of the rejection sampler at vocab 8,
  * hand-worked decision traces, brute-force compaction; tree builder
  * (tests/test_oracle_tree_build.py): hand-worked cases, stable library sort,
- * brute force over ancestor-closed subsets, flattened-tree invariants.
+ * brute force over ancestor-closed subsets, flattened-tree invariants; draft
+ * step: hand-worked cases, library sorts plus numpy's own fp32 addition,
+ * levels chained into the builder.
  *
  * The only parallelism is an OpenMP loop over independent units (heads,
  * node rows, cache slices); each unit runs the plain definition.
@@ -400,4 +402,69 @@ int oracle_tree_build(const int32_t *cand_parent, const int32_t *cand_token, con
         free(kept); free(depth); free(node_of);
     }
     return rc;
+}
+
+/* -------------------------------------------------------------------------
+ * O6  Dynamic token tree, one draft step (paper, Section "Preliminaries", last
+ * paragraph: "the output of each step can be truncated by selecting the
+ * top-k" and "the computation of joint probabilities for each token").
+ *
+ * For every frontier node f of sequence b the row logprobs[b][f][.] holds the
+ * draft model's log-probabilities of the next token.  Its top_k entries
+ * (largest value; equal values: the lower token first) become new candidates,
+ * numbered base + f * top_k + r with r = 0 for the most probable, with parent
+ * frontier_cand[b][f] and joint log-probability frontier_logp[b][f] + value,
+ * formed by ONE single-precision addition (so that the order of the joint
+ * values is the same on every implementation).  The `width` new candidates
+ * with the largest joint value (equal values: the lower candidate index first)
+ * form the next frontier, returned in that order.
+ *   logprobs [B][F][V] float; frontier_logp [B][F] float; frontier_cand [B][F]
+ *   cand_parent, cand_token, cand_logp [B][cap]: entries base .. base + F*top_k - 1 written
+ *   next_cand [B][width] int32, next_logp [B][width] float
+ * Plain selection loops.
+ * ---------------------------------------------------------------------- */
+int oracle_draft_expand(const float *logprobs, const float *frontier_logp, const int32_t *frontier_cand,
+                        int B, int F, int V, int top_k, int width, int base, int cap,
+                        int32_t *cand_parent, int32_t *cand_token, float *cand_logp, int32_t *next_cand,
+                        float *next_logp)
+{
+    if (top_k < 1 || top_k > V || width < 1 || width > F * top_k || base < 0 || base + F * top_k > cap) return -1;
+    for (int b = 0; b < B; ++b) {
+        int32_t *cp = cand_parent + (size_t)b * cap, *ct = cand_token + (size_t)b * cap;
+        float *cl = cand_logp + (size_t)b * cap;
+        for (int f = 0; f < F; ++f) {
+            const float *row = logprobs + ((size_t)b * F + f) * V;
+            char *taken = (char *)calloc((size_t)V, 1);
+            if (!taken) return -2;
+            for (int r = 0; r < top_k; ++r) {
+                int best = -1;
+                for (int j = 0; j < V; ++j) {
+                    if (taken[j]) continue;
+                    if (best < 0 || row[j] > row[best]) best = j;      /* strict: the lower token wins a tie */
+                }
+                taken[best] = 1;
+                const int c = base + f * top_k + r;
+                cp[c] = frontier_cand[(size_t)b * F + f];
+                ct[c] = best;
+                const volatile float joint = frontier_logp[(size_t)b * F + f] + row[best];   /* one fp32 addition */
+                cl[c] = joint;
+            }
+            free(taken);
+        }
+        const int n_new = F * top_k;
+        char *used = (char *)calloc((size_t)n_new, 1);
+        if (!used) return -2;
+        for (int w = 0; w < width; ++w) {
+            int best = -1;
+            for (int i = 0; i < n_new; ++i) {
+                if (used[i]) continue;
+                if (best < 0 || cl[base + i] > cl[base + best]) best = i;
+            }
+            used[best] = 1;
+            next_cand[(size_t)b * width + w] = base + best;
+            next_logp[(size_t)b * width + w] = cl[base + best];
+        }
+        free(used);
+    }
+    return 0;
 }

@@ -394,3 +394,16 @@ def tree_candidates(seed: int, batch: int, levels: int = 5, width: int = 10, bra
                     cand_logp[b, c] = cand_logp[b, p]
     root_token = rng.integers(0, vocab, size=batch, dtype=np.int32)
     return cand_parent, cand_token, cand_logp.astype(np.float32), root_token
+
+
+def draft_logprob_rows(seed: int, batch: int, n_frontier: int, vocab: int, sigma: float = 3.0, step: float = 0.0):
+    """Stand-in output of one draft step: log-probabilities [B][F][V] float32 (log-softmax of
+    N(0, sigma^2) logits, taken in float64).  With `step` > 0 the values are rounded down to multiples
+    of `step`, which puts many equal values into every row (ties between tokens)."""
+    rng = np.random.default_rng([SEED_BASE % (2 ** 32), 8, seed])
+    z = rng.standard_normal((batch, n_frontier, vocab)) * sigma
+    z -= z.max(-1, keepdims=True)
+    lp = z - np.log(np.exp(z).sum(-1, keepdims=True))
+    if step > 0:
+        lp = np.floor(lp / step) * step
+    return lp.astype(np.float32)

@@ -105,3 +105,79 @@ def test_chain_of_candidates_gives_a_chain():
 def test_growing_probability_along_a_path_is_reported():
     r = _one([-1, 0, -1], [1, 2, 3], np.log([0.1, 0.5, 0.3]), 0, 3)   # child more probable than its parent
     assert not r["valid"]
+
+
+# ---------------------------------------------------------------------------
+# one draft step: per-row top-k, joint log-probability, next frontier
+# ---------------------------------------------------------------------------
+def _expand(lp, flp, fc, k, width, base, cap):
+    B = lp.shape[0]
+    cp = np.full((B, cap), -7, np.int32)
+    ct = np.full((B, cap), -7, np.int32)
+    cl = np.full((B, cap), np.nan, np.float32)
+    nc, nl = oracle.draft_expand(lp, flp, fc, k, width, base, cp, ct, cl)
+    return cp, ct, cl, nc, nl
+
+
+def test_expand_hand_worked_cases():
+    for case in json.load(open(GOLDEN))["expand_cases"]:
+        lp = np.log(np.asarray([case["row_prob"]], np.float64)).astype(np.float32)
+        flp = np.log(np.asarray([case["frontier_prob"]], np.float64)).astype(np.float32)
+        k, base = case["top_k"], case["base"]
+        n_new = len(case["frontier_cand"]) * k
+        cp, ct, cl, nc, nl = _expand(lp, flp, np.asarray([case["frontier_cand"]], np.int32), k, case["width"], base,
+                                     base + n_new + 2)
+        assert cp[0, base:base + n_new].tolist() == case["cand_parent"], case["name"]
+        assert ct[0, base:base + n_new].tolist() == case["cand_token"], case["name"]
+        assert np.allclose(np.exp(cl[0, base:base + n_new].astype(np.float64)), case["cand_prob"], rtol=1e-6)
+        assert nc[0].tolist() == case["next_cand"], case["name"]
+        assert (cp[0, :base] == -7).all() and (cp[0, base + n_new:] == -7).all()      # nothing else written
+
+
+@pytest.mark.parametrize("step", [0.0, 0.5])
+def test_expand_equals_library_sorts_and_one_float_addition(step):
+    for seed in range(4):
+        B, F, V, k, width, base = 3, 5, 777, 7, 6, 11
+        lp = synth.draft_logprob_rows(seed, B, F, V, step=step)
+        rng = np.random.default_rng(seed)
+        flp = (-rng.random((B, F)) * 5).astype(np.float32)
+        fc = rng.integers(-1, base, size=(B, F)).astype(np.int32)
+        cp, ct, cl, nc, nl = _expand(lp, flp, fc, k, width, base, base + F * k)
+        for b in range(B):
+            joint = []
+            for f in range(F):
+                top = np.argsort(-lp[b, f].astype(np.float64), kind="stable")[:k]
+                sl = slice(base + f * k, base + (f + 1) * k)
+                assert ct[b, sl].tolist() == top.tolist()
+                assert (cp[b, sl] == fc[b, f]).all()
+                want = (np.float32(flp[b, f]) + lp[b, f, top]).astype(np.float32)     # numpy's own fp32 addition
+                assert np.array_equal(cl[b, sl], want)
+                joint.extend(want.tolist())
+            order = np.argsort(-np.asarray(joint, np.float64), kind="stable")[:width]
+            assert nc[b].tolist() == (base + order).tolist()
+            assert np.array_equal(nl[b], np.asarray(joint, np.float32)[order])
+
+
+def test_levels_chained_into_the_builder_keep_path_sums():
+    """Expand level by level, then build: every node's joint value is the fp32 sum along its path,
+    and the joint values never grow along a path (log-probabilities are <= 0)."""
+    B, V, k, width, levels, N = 2, 500, 4, 3, 4, 20
+    cap = k + (levels - 1) * width * k
+    cp = np.full((B, cap), -7, np.int32)
+    ct = np.full((B, cap), -7, np.int32)
+    cl = np.full((B, cap), np.nan, np.float32)
+    fc = np.full((B, 1), -1, np.int32)
+    flp = np.zeros((B, 1), np.float32)
+    base = 0
+    for lvl in range(levels):
+        F = fc.shape[1]
+        lp = synth.draft_logprob_rows(50 + lvl, B, F, V)
+        fc, flp = oracle.draft_expand(lp, flp, fc, k, min(width, F * k), base, cp, ct, cl)
+        base += F * k
+    assert base == cap
+    r = oracle.tree_build(cp, ct, cl, np.zeros(B, np.int32), N)
+    assert r["valid"]
+    for b in range(B):
+        for c in range(cap):
+            if cp[b, c] >= 0:
+                assert cl[b, c] <= cl[b, cp[b, c]]
