@@ -13,6 +13,7 @@
  *                      evaluates T = 0 and T = 1 with unrelaxed acceptance)
  *   fspad_kv_compact   keep the accepted path's K/V rows, contiguous in the cache
  * and, one step earlier in the pipeline,
+ *   fspad_draft_expand one draft step: per-row top-k, joint probabilities, next frontier
  *   fspad_tree_build   the draft phase's candidates -> the flattened token tree
  *
  * Conventions (shared by every call)
@@ -193,6 +194,42 @@ int fspad_accept_stats(fspad_ctx *ctx, const float *logits, const float *tempera
 int fspad_accept_stats_noalloc(const float *logits, const float *temperature, int rows,
                                int rows_per_seq, int vocab, float *row_max, double *row_sum,
                                int32_t *row_arg, void *stream);
+
+/*
+ * Dynamic token tree, one draft step ("Preliminaries", last paragraph: the
+ * output of each draft step is truncated to its top-k, and every token carries
+ * the joint probability of its path).  Called once per level of the draft
+ * phase; fspad_tree_build then turns the accumulated candidates into the tree.
+ *
+ *   logprobs      [batch][n_frontier][vocab] float, device: the draft model's
+ *                 log-probabilities of the next token after each frontier node
+ *                 (vocab is the context's); NaN not allowed.
+ *   frontier_logp [batch][n_frontier] float, device: joint log-probability of
+ *                 each frontier node (0 for the root at the first level).
+ *   frontier_cand [batch][n_frontier] int32, device: candidate index of each
+ *                 frontier node (-1 for the root).
+ *   n_frontier, top_k: 1 .. 16 (top_k <= vocab); width: 1 .. n_frontier * top_k.
+ *   base, n_cand_cap: the new candidates get the indices base .. base +
+ *                 n_frontier * top_k - 1 of arrays that hold n_cand_cap entries
+ *                 per sequence; the caller advances base from level to level.
+ *
+ * For frontier node f the top_k largest entries of its row (equal values: the
+ * lower token first) become the candidates base + f * top_k + r, r = 0 for the
+ * most probable: cand_parent = frontier_cand[f], cand_token = the token,
+ * cand_logp = frontier_logp[f] + value (one single-precision addition).  The
+ * `width` new candidates with the largest joint value (equal values: the lower
+ * candidate index first) are returned, in that order, as next_cand / next_logp
+ * [batch][width]: the frontier of the next level.  cand_* are [batch][n_cand_cap],
+ * device, owned by the caller; only the new entries are written.  Per-piece
+ * lists live in the context's scratch (allocated by fspad_create): one call per
+ * context at a time.  Asynchronous on `stream`.  Errors: FSPAD_ERR_SHAPE for
+ * sizes outside the ranges above, FSPAD_ERR_TOO_LARGE when ceil(vocab / 4096) *
+ * top_k exceeds 1024.
+ */
+int fspad_draft_expand(fspad_ctx *ctx, const float *logprobs, const float *frontier_logp,
+                       const int32_t *frontier_cand, int n_frontier, int top_k, int width, int base, int n_cand_cap,
+                       int batch, int32_t *cand_parent, int32_t *cand_token, float *cand_logp, int32_t *next_cand,
+                       float *next_logp, void *stream);
 
 /*
  * Dynamic token tree, final stage ("Preliminaries", last paragraph: each draft

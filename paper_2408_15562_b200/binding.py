@@ -19,7 +19,7 @@ _lib = None
 
 EXPORTS = ["fspad_create", "fspad_destroy", "fspad_status", "fspad_strerror", "fspad_launch_count",
            "fspad_tree_attn", "fspad_tree_accept", "fspad_accept_stats", "fspad_kv_compact",
-           "fspad_verify_step_host", "fspad_accept_stats_noalloc", "fspad_tree_build"]
+           "fspad_verify_step_host", "fspad_accept_stats_noalloc", "fspad_tree_build", "fspad_draft_expand"]
 
 
 class FspadConfig(ctypes.Structure):
@@ -59,6 +59,7 @@ def load():
     lib.fspad_accept_stats_noalloc.argtypes = [vp, vp, ci, ci, ci, vp, vp, vp, vp]
     lib.fspad_verify_step_host.argtypes = [vp] * 12 + [ci, ci] + [vp] * 6
     lib.fspad_tree_build.argtypes = [vp] * 5 + [ci, ci, ci] + [vp] * 6
+    lib.fspad_draft_expand.argtypes = [vp] * 4 + [ci] * 6 + [vp] * 6
     _lib = lib
     return lib
 
@@ -201,6 +202,25 @@ class Context:
         if rc != 0:
             raise FspadError(rc, "fspad_tree_build")
         return parent, token, cand, n_out
+
+    def draft_expand(self, logprobs, frontier_logp, frontier_cand, top_k, width, base, cand_parent, cand_token,
+                     cand_logp, next_cand=None, next_logp=None, stream=None):
+        """One draft step: logprobs [B][F][V] (device) -> new candidates written into cand_* [B][cap] at
+        base .. base + F*top_k - 1; returns (next_cand, next_logp) [B][width]."""
+        B, F, V = logprobs.shape
+        assert V == self.cfg.vocab
+        i32, f32 = torch.int32, torch.float32
+        if next_cand is None:
+            next_cand = torch.empty((B, width), dtype=i32, device=logprobs.device)
+        if next_logp is None:
+            next_logp = torch.empty((B, width), dtype=f32, device=logprobs.device)
+        rc = load().fspad_draft_expand(self._h, _ptr(logprobs, f32), _ptr(frontier_logp, f32), _ptr(frontier_cand, i32),
+                                       F, top_k, width, base, cand_parent.shape[1], B, _ptr(cand_parent, i32),
+                                       _ptr(cand_token, i32), _ptr(cand_logp, f32), _ptr(next_cand, i32),
+                                       _ptr(next_logp, f32), _stream(stream))
+        if rc != 0:
+            raise FspadError(rc, "fspad_draft_expand")
+        return next_cand, next_logp
 
     def verify_step_host(self, cache, q, tree_k, tree_v, parent, prefix_len, target_logits, draft_probs,
                          draft_tokens, temperature, uniforms, attn_out, accepted_path, n_accepted,

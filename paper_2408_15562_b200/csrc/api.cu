@@ -97,6 +97,11 @@ int fspad_create(const fspad_config *cfg, fspad_ctx **out)
     ok = ok && dev_alloc(&ctx->row_max, rows);
     ok = ok && dev_alloc(&ctx->row_sum, rows);
     ok = ok && dev_alloc(&ctx->row_arg, rows);
+    {
+        uint2 *dx = nullptr;
+        ok = ok && dev_alloc(&dx, B * FSPAD_MAX_FRONTIER * (size_t)fspad_draft_expand_pieces(cfg->vocab) * FSPAD_MAX_FRONTIER);
+        ctx->dx_part = dx;
+    }
     if (ok) {
         ok = cudaMemset(ctx->d_status, 0, sizeof(int)) == cudaSuccess && cudaDeviceSynchronize() == cudaSuccess;
     }
@@ -112,7 +117,7 @@ void fspad_destroy(fspad_ctx *ctx)
 {
     if (!ctx) return;
     cudaDeviceSynchronize();
-    void *ptrs[] = {ctx->d_status, ctx->part_o, ctx->part_ml, ctx->st_part, ctx->row_max, ctx->row_sum, ctx->row_arg, ctx->h_q, ctx->h_tk,
+    void *ptrs[] = {ctx->dx_part, ctx->d_status, ctx->part_o, ctx->part_ml, ctx->st_part, ctx->row_max, ctx->row_sum, ctx->row_arg, ctx->h_q, ctx->h_tk,
                     ctx->h_tv, ctx->h_out, ctx->h_parent, ctx->h_prefix, ctx->h_tokens, ctx->h_path,
                     ctx->h_nacc, ctx->h_bonus, ctx->h_newlen, ctx->h_logits, ctx->h_draft, ctx->h_temp,
                     ctx->h_unif};
@@ -230,6 +235,29 @@ int fspad_tree_build(fspad_ctx *ctx, const int32_t *cand_parent, const int32_t *
     cudaError_t e = fspad_launch_tree_build(ctx, cand_parent, cand_token, cand_logp, root_token, n_cand, n_nodes,
                                             batch, parent_out, token_out, cand_out,
                                             reinterpret_cast<unsigned long long *>(anc_out), n_out, fspad_stream(stream));
+    return e == cudaSuccess ? FSPAD_OK : FSPAD_ERR_CUDA;
+}
+
+int fspad_draft_expand(fspad_ctx *ctx, const float *logprobs, const float *frontier_logp,
+                       const int32_t *frontier_cand, int n_frontier, int top_k, int width, int base, int n_cand_cap,
+                       int batch, int32_t *cand_parent, int32_t *cand_token, float *cand_logp, int32_t *next_cand,
+                       float *next_logp, void *stream)
+{
+    if (!ctx) return FSPAD_ERR_NULL;
+    if (!logprobs || !frontier_logp || !frontier_cand || !cand_parent || !cand_token || !cand_logp || !next_cand ||
+        !next_logp)
+        return FSPAD_ERR_NULL;
+    if (batch < 0 || batch > ctx->cfg.max_batch) return FSPAD_ERR_SHAPE;
+    if (n_frontier < 1 || n_frontier > FSPAD_MAX_FRONTIER || top_k < 1 || top_k > FSPAD_MAX_FRONTIER ||
+        top_k > ctx->cfg.vocab)
+        return FSPAD_ERR_SHAPE;
+    if (width < 1 || width > n_frontier * top_k || base < 0 || base + n_frontier * top_k > n_cand_cap)
+        return FSPAD_ERR_SHAPE;
+    if ((long long)fspad_draft_expand_pieces(ctx->cfg.vocab) * top_k > FSPAD_MAX_CANDIDATES) return FSPAD_ERR_TOO_LARGE;
+    if (batch == 0) return FSPAD_OK;
+    cudaError_t e = fspad_launch_draft_expand(ctx, logprobs, frontier_logp, frontier_cand, n_frontier, top_k, width,
+                                              base, n_cand_cap, batch, cand_parent, cand_token, cand_logp, next_cand,
+                                              next_logp, fspad_stream(stream));
     return e == cudaSuccess ? FSPAD_OK : FSPAD_ERR_CUDA;
 }
 

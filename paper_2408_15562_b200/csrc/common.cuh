@@ -10,6 +10,7 @@
 
 #define FSPAD_MAX_NODES 64
 #define FSPAD_MAX_CANDIDATES 1024
+#define FSPAD_MAX_FRONTIER 16      /* frontier nodes per sequence, and top-k per row, of a draft step */
 #define FSPAD_HEAD_DIM 128
 
 // Scratch and bookkeeping owned by a context (all device pointers unless noted).
@@ -40,6 +41,8 @@ struct fspad_ctx {
     double *row_sum;
     int *row_arg;
     int walk_cluster;         // cluster size used by the sampling walk (0 = not probed yet)
+
+    void *dx_part;            // draft step: per-piece top-k lists [max_batch * 16 rows][pieces][16] (value, token)
 
     // device staging for the host entry point
     fspad_bf16 *h_q, *h_tk, *h_tv, *h_out;
@@ -242,6 +245,11 @@ cudaError_t fspad_launch_tree_build(fspad_ctx *ctx, const int *cand_parent, cons
                                     const float *cand_logp, const int *root_token, int n_cand, int n_nodes,
                                     int B, int *parent_out, int *token_out, int *cand_out,
                                     unsigned long long *anc_out, int *n_out, cudaStream_t st);
+int fspad_draft_expand_pieces(int V);
+cudaError_t fspad_launch_draft_expand(fspad_ctx *ctx, const float *logprobs, const float *frontier_logp,
+                                      const int *frontier_cand, int F, int k, int width, int base, int cap, int B,
+                                      int *cand_parent, int *cand_token, float *cand_logp, int *next_cand,
+                                      float *next_logp, cudaStream_t st);
 cudaError_t fspad_launch_kv_compact(fspad_ctx *ctx, fspad_bf16 *cache, const int *path,
                                     const int *n_acc, const int *prefix_len, int B, int *new_len,
                                     cudaStream_t st);

@@ -17,18 +17,13 @@
 // (depth, index) order, and writes the flattened tree the verification step
 // consumes, with (optionally) each node's ancestor-or-self mask.  Integer work throughout; no arithmetic on the probabilities.
 #include "common.cuh"
+#include "sort_network.cuh"
 
 namespace {
 
-constexpr int kThreads = 256;
-constexpr int kPerThread = FSPAD_MAX_CANDIDATES / kThreads;   // 4 entries of the sorting network per thread
-
-// order-preserving map float -> uint32 (larger float, larger integer); -0.0 < +0.0 is harmless here
-__device__ __forceinline__ uint32_t orderable(float f)
-{
-    const uint32_t u = __float_as_uint(f);
-    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
-}
+constexpr int kThreads = kSortThreads;
+constexpr int kPerThread = kSortPerThread;   // 4 entries of the sorting network per thread
+static_assert(FSPAD_MAX_CANDIDATES == kSortEntries, "the network is sized for the candidate limit");
 
 __global__ void __launch_bounds__(kThreads)
 tree_build_kernel(const int *__restrict__ cand_parent, const int *__restrict__ cand_token,
@@ -54,7 +49,7 @@ tree_build_kernel(const int *__restrict__ cand_parent, const int *__restrict__ c
         unsigned long long key = 0ull;                           // padding sorts behind every candidate
         int p = -1;
         if (c < C) {
-            key = ((unsigned long long)orderable(lp[c]) << 32) | (unsigned long long)(0xffffffffu - (uint32_t)c);
+            key = fspad_sort_key(lp[c], (uint32_t)c);
             p = cp[c];
             if (p < -1 || p >= c) { bad = true; p = -1; }
         }
@@ -62,53 +57,16 @@ tree_build_kernel(const int *__restrict__ cand_parent, const int *__restrict__ c
         s_par[c] = (short)p;
         s_node[c] = -1;
     }
-    // bitonic network, descending.  Partners 1 or 2 apart sit in the same thread, up to 64 apart in
-    // the same warp (shuffles); only the three widest distances go through shared memory.
-    for (int k = 2; k <= FSPAD_MAX_CANDIDATES; k <<= 1) {
-        for (int j = k >> 1; j > 0; j >>= 1) {
-            if (j < kPerThread) {
-#pragma unroll
-                for (int r = 0; r < kPerThread; ++r) {
-                    const int l = r ^ j;
-                    if (l > r) {
-                        const bool desc = ((kPerThread * tid + r) & k) == 0;
-                        const unsigned long long x = v[r], y = v[l];
-                        if (desc ? (x < y) : (x > y)) { v[r] = y; v[l] = x; }
-                    }
-                }
-            } else {
-                unsigned long long o[kPerThread];
-                if (j < kPerThread * 32) {
-#pragma unroll
-                    for (int r = 0; r < kPerThread; ++r) o[r] = __shfl_xor_sync(0xffffffffu, v[r], j / kPerThread);
-                } else {
-                    __syncthreads();                             // the buffer's previous readers are done
-#pragma unroll
-                    for (int r = 0; r < kPerThread; ++r) s_key[kPerThread * tid + r] = v[r];
-                    __syncthreads();
-                    const int pt = tid ^ (j / kPerThread);
-#pragma unroll
-                    for (int r = 0; r < kPerThread; ++r) o[r] = s_key[kPerThread * pt + r];
-                }
-                const int i0 = kPerThread * tid;
-                const bool lower = (i0 & j) == 0, desc = (i0 & k) == 0;   // same for the thread's four entries
-                const bool take_max = lower == desc;
-#pragma unroll
-                for (int r = 0; r < kPerThread; ++r)
-                    v[r] = take_max ? (v[r] > o[r] ? v[r] : o[r]) : (v[r] < o[r] ? v[r] : o[r]);
-            }
-        }
-    }
-    __syncthreads();
+    fspad_bitonic_sort_desc(v, s_key, tid);
 #pragma unroll
     for (int r = 0; r < kPerThread; ++r) s_key[kPerThread * tid + r] = v[r];
     __syncthreads();
     const int want = min(N - 1, C);
-    if (tid < want) s_node[0xffffffffu - (uint32_t)(s_key[tid] & 0xffffffffull)] = 0;   // kept (number follows)
+    if (tid < want) s_node[fspad_key_index(s_key[tid])] = 0;   // kept (number follows)
     __syncthreads();
     int my_c = -1, my_d = 0;
     if (tid < want) {
-        my_c = (int)(0xffffffffu - (uint32_t)(s_key[tid] & 0xffffffffull));
+        my_c = (int)fspad_key_index(s_key[tid]);
         for (int a = my_c; a >= 0; a = s_par[a]) {               // indices strictly decrease: the walk ends
             if (s_node[a] < 0) bad = true;                       // an ancestor was not kept
             ++my_d;
