@@ -295,6 +295,17 @@ def main():
     tb_out = tuple(torch.empty((B, N), dtype=torch.int32, device="cuda") for _ in range(3)) + \
         (torch.empty((B,), dtype=torch.int32, device="cuda"),)
     tree_build_us = timed(lambda i: ctx.tree_build(*dcand, N, out=tb_out), args.steps)
+    # one draft step of that phase: ten frontier rows of log-probabilities -> top-10 each, joint values, next frontier
+    DF, DK = 10, 10
+    dlp_host = synth.draft_logprob_rows(w.cfg, B, DF, w.vocab)
+    dlp = [torch.from_numpy(dlp_host).cuda() for _ in range(max(2, min(R, 1 + int(3e8 // dlp_host.nbytes))))]
+    dfl = torch.zeros((B, DF), dtype=torch.float32, device="cuda")
+    dfc = torch.full((B, DF), -1, dtype=torch.int32, device="cuda")
+    dx_arr = (torch.zeros((B, DF * DK), dtype=torch.int32, device="cuda"), torch.zeros((B, DF * DK), dtype=torch.int32, device="cuda"),
+              torch.zeros((B, DF * DK), dtype=torch.float32, device="cuda"))
+    dx_next = (torch.empty((B, DK), dtype=torch.int32, device="cuda"), torch.empty((B, DK), dtype=torch.float32, device="cuda"))
+    draft_expand_us = timed(lambda i: ctx.draft_expand(dlp[i % len(dlp)], dfl, dfc, DK, DK, 0, *dx_arr, next_cand=dx_next[0],
+                                                       next_logp=dx_next[1]), args.steps)
     clocks = sampler.stop()
     ctx.check()
 
@@ -302,6 +313,7 @@ def main():
     n_acc_host = n_acc.cpu().numpy()
     verified = None
     tree_build_ok, tree_build_cpu_us = None, None
+    draft_expand_ok, draft_expand_cpu_us = None, None
     if rank == 0 and not args.no_verify and B <= 2:
         import oracle
         step(0)
@@ -318,6 +330,13 @@ def main():
         tree_build_cpu_us = (time.perf_counter() - t0) * 1e6
         tree_build_ok = all(np.array_equal(tb_out[j].cpu().numpy(), tb_ref[k_])
                             for j, k_ in enumerate(("parent", "token", "cand", "n_out")))
+        dx_ref = [np.zeros((B, DF * DK), np.int32), np.zeros((B, DF * DK), np.int32), np.zeros((B, DF * DK), np.float32)]
+        t0 = time.perf_counter()
+        nc_ref, nl_ref = oracle.draft_expand(dlp_host, np.zeros((B, DF), np.float32), np.full((B, DF), -1, np.int32), DK, DK, 0,
+                                             *dx_ref)
+        draft_expand_cpu_us = (time.perf_counter() - t0) * 1e6
+        draft_expand_ok = (all(np.array_equal(dx_arr[j].cpu().numpy(), dx_ref[j]) for j in range(3))
+                           and np.array_equal(dx_next[0].cpu().numpy(), nc_ref) and np.array_equal(dx_next[1].cpu().numpy(), nl_ref))
         verified = {"accept_bit_exact": bool(ok_acc), "attn_max_abs_err": float(err.max()),
                     "attn_mean_abs_err": float(err.mean()),
                     "ok": bool(ok_acc and err.max() <= 1e-2 and err.mean() <= 1e-3)}
@@ -391,6 +410,12 @@ def main():
                                 "batch": B, "bit_exact_vs_oracle": tree_build_ok,
                                 "oracle_us_one_thread": tree_build_cpu_us,
                                 "note": "step before the verify step; not part of value"},
+            "draft_expand_call": {"us": draft_expand_us, "rows": B * DF, "top_k": DK, "width": DK,
+                                  "algorithmic_bytes": int(dlp_host.nbytes),
+                                  "gbs": dlp_host.nbytes / (draft_expand_us * 1e-6) / 1e9,
+                                  "frac_of_hbm_peak": dlp_host.nbytes / (draft_expand_us * 1e-6) / 1e9 / peak,
+                                  "bit_exact_vs_oracle": draft_expand_ok, "oracle_us_one_thread": draft_expand_cpu_us,
+                                  "note": "one level of the draft phase (three kernels); not part of value"},
             "e2e": {"value": e2e_us, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "steps": e2e_steps, "note": "fspad_verify_step_host: pinned host inputs, device-resident KV cache"},
             "gpu_launches": int(launches),

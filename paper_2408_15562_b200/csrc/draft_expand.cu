@@ -3,9 +3,10 @@
 // token carries the joint probability of its path).
 //
 // Three small kernels per call:
-//   1. draft_topk_partial_kernel - grid (pieces of 4096 tokens, rows): the top-k of
-//      the piece by k rounds of a block-wide arg-max (value, then lower token), the
-//      16 values of a thread staying in registers; the one HBM pass over the rows.
+//   1. draft_topk_partial_kernel - grid (pieces of 4096 tokens, rows): the top-k of the
+//      piece from one pass: a lower bound of the k-th largest key from the half-warp
+//      maxima, the few keys at or above it listed in shared memory and ranked by
+//      counting; the one HBM pass over the rows.
 //   2. draft_topk_row_kernel - one CTA per row: the pieces' lists (at most 1024
 //      entries) through the sorting network; the first k become candidates
 //      base + f k + r with the frontier node as parent and the joint
@@ -22,26 +23,32 @@ constexpr int kThreads = kSortThreads;                 // 256
 constexpr int kPerThread = 16;                         // tokens per thread in the partial kernel
 constexpr int kPiece = kThreads * kPerThread;          // 4096 tokens per CTA
 
-struct Best {
-    float v;
-    int i;
-};
-__device__ __forceinline__ bool better(float v, int i, float bv, int bi) { return v > bv || (v == bv && i < bi); }
-
+// The top-k of one piece of one row.  Tokens become 64-bit keys (order-preserving image of the value,
+// complemented token index: larger key = larger value, or equal value and lower token; all keys of
+// a piece are distinct).  The k-th largest of the 16 half-warp maxima is a lower bound of the
+// piece's k-th largest key, because k keys at least that large exist; every key at or above the
+// bound goes to a shared list (a few dozen entries on ordinary data, the whole piece at worst) and
+// the list's members are ranked by counting.  One pass over the data, no per-round rescans.
 __global__ void __launch_bounds__(kThreads)
 draft_topk_partial_kernel(const float *__restrict__ logprobs, int V, int k, int pieces, uint2 *__restrict__ part)
 {
-    __shared__ Best s_w[kThreads / 32];
-    __shared__ Best s_win;
+    __shared__ unsigned long long s_list[kPiece];               // candidates at or above the bound
+    __shared__ unsigned long long s_hmax[kThreads / 16];
+    __shared__ unsigned long long s_bound;
+    __shared__ int s_cnt;
     fspad_pdl_trigger();
     fspad_pdl_wait();
-    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    const int tid = threadIdx.x, lane = tid & 31;
     const int piece = blockIdx.x, row = blockIdx.y;
     const float *x = logprobs + (size_t)row * V;
     const int e0 = piece * kPiece;
     const bool vec = (V % 4 == 0) && ((reinterpret_cast<uintptr_t>(logprobs) & 15) == 0);
+    if (tid == 0) s_cnt = 0;
+    // The values stay floats; a key is built only for the thread's maximum and for listed tokens.
+    // Scanning in token order with a strict comparison keeps the lowest token among equal values.
     float val[kPerThread];
-    // element (i, c) of thread t is token e0 + 4 (i 256 + t) + c: increasing with (i, c)
+    float bv = 0.f;
+    int bu = -1;                                                 // slot of the thread's maximum, -1: no token
 #pragma unroll
     for (int i = 0; i < kPerThread / 4; ++i) {
         const int e = e0 + 4 * (i * kThreads + tid);
@@ -50,48 +57,54 @@ draft_topk_partial_kernel(const float *__restrict__ logprobs, int V, int k, int 
             val[4 * i] = t4.x; val[4 * i + 1] = t4.y; val[4 * i + 2] = t4.z; val[4 * i + 3] = t4.w;
         } else {
 #pragma unroll
-            for (int c = 0; c < 4; ++c) val[4 * i + c] = (e + c < V) ? x[e + c] : -INFINITY;
+            for (int c = 0; c < 4; ++c) val[4 * i + c] = (e + c < V) ? x[e + c] : 0.f;
         }
-    }
-    unsigned taken = 0u;
-#pragma unroll
-    for (int i = 0; i < kPerThread / 4; ++i)            // tokens past the row's end never compete
 #pragma unroll
         for (int c = 0; c < 4; ++c)
-            if (e0 + 4 * (i * kThreads + tid) + c >= V) taken |= 1u << (4 * i + c);
-    uint2 *out = part + ((size_t)row * pieces + piece) * k;
-    for (int r = 0; r < k; ++r) {
-        Best b{-INFINITY, 0x7fffffff};
-        int slot = -1;
-#pragma unroll
-        for (int u = 0; u < kPerThread; ++u) {
-            const int idx = e0 + 4 * ((u >> 2) * kThreads + tid) + (u & 3);
-            if (!((taken >> u) & 1u) && (slot < 0 || val[u] > b.v)) { b.v = val[u]; b.i = idx; slot = u; }
-        }
-        Best w = b;
-#pragma unroll
-        for (int off = 16; off > 0; off >>= 1) {
-            const float ov = __shfl_xor_sync(0xffffffffu, w.v, off);
-            const int oi = __shfl_xor_sync(0xffffffffu, w.i, off);
-            if (better(ov, oi, w.v, w.i)) { w.v = ov; w.i = oi; }
-        }
-        if (lane == 0) s_w[wid] = w;
-        __syncthreads();
-        if (wid == 0) {
-            Best q = (lane < kThreads / 32) ? s_w[lane] : Best{-INFINITY, 0x7fffffff};
-#pragma unroll
-            for (int off = 4; off > 0; off >>= 1) {
-                const float ov = __shfl_xor_sync(0xffffffffu, q.v, off);
-                const int oi = __shfl_xor_sync(0xffffffffu, q.i, off);
-                if (better(ov, oi, q.v, q.i)) { q.v = ov; q.i = oi; }
-            }
-            if (lane == 0) s_win = q;
-        }
-        __syncthreads();
-        const Best win = s_win;
-        if (slot >= 0 && win.i == b.i) taken |= 1u << slot;      // the owner retires the winner
-        if (tid == 0) out[r] = make_uint2(__float_as_uint(win.v), (unsigned)win.i);
+            if (e + c < V && (bu < 0 || val[4 * i + c] > bv)) { bv = val[4 * i + c]; bu = 4 * i + c; }
     }
+    auto token_of = [&](int u) { return e0 + 4 * ((u >> 2) * kThreads + tid) + (u & 3); };
+    unsigned long long best = (bu >= 0) ? fspad_sort_key(bv, (uint32_t)token_of(bu)) : 0ull;   // 0: "no token"
+    // maxima of the 16 half-warps
+#pragma unroll
+    for (int off = 8; off > 0; off >>= 1) {
+        const unsigned long long o = __shfl_xor_sync(0xffffffffu, best, off);
+        best = o > best ? o : best;
+    }
+    if ((lane & 15) == 0) s_hmax[tid >> 4] = best;
+    __syncthreads();
+    if (tid < kThreads / 16) {
+        const unsigned long long me = s_hmax[tid];
+        int rank = 0;
+#pragma unroll
+        for (int o = 0; o < kThreads / 16; ++o) {
+            const unsigned long long ot = s_hmax[o];
+            rank += (ot > me || (ot == me && o < tid)) ? 1 : 0;  // equal only for empty half-warps (key 0)
+        }
+        if (rank == k - 1) s_bound = me;                         // k <= 16: exactly one thread
+    }
+    __syncthreads();
+    const unsigned long long bound = s_bound;
+    // key >= bound  <=>  value above the bound's, or equal to it with a token not after the bound's
+    // (bound == 0: fewer than k half-warps hold a token at all - a short last piece - list every token)
+    const float bound_v = (bound != 0ull) ? fspad_key_value(bound) : -INFINITY;
+    const int bound_i = (bound != 0ull) ? (int)fspad_key_index(bound) : 0x7fffffff;
+#pragma unroll
+    for (int u = 0; u < kPerThread; ++u) {
+        const int tok = token_of(u);
+        if (tok < V && (val[u] > bound_v || (val[u] == bound_v && tok <= bound_i)))
+            s_list[atomicAdd(&s_cnt, 1)] = fspad_sort_key(val[u], (uint32_t)tok);
+    }
+    __syncthreads();
+    const int n = s_cnt;
+    uint2 *out = part + ((size_t)row * pieces + piece) * k;
+    for (int i = tid; i < n; i += kThreads) {
+        const unsigned long long me = s_list[i];
+        int rank = 0;
+        for (int o = 0; o < n; ++o) rank += (s_list[o] > me) ? 1 : 0;
+        if (rank < k) out[rank] = make_uint2(__float_as_uint(fspad_key_value(me)), fspad_key_index(me));
+    }
+    for (int r = n + tid; r < k; r += kThreads) out[r] = make_uint2(__float_as_uint(-INFINITY), 0x7fffffffu);   // empty slots
 }
 
 // one row: partial lists -> top-k -> candidates
