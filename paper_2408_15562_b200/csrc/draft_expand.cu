@@ -4,8 +4,8 @@
 //
 // Three small kernels per call:
 //   1. draft_topk_partial_kernel - grid (pieces of 4096 tokens, rows): the top-k of the
-//      piece from one pass: a lower bound of the k-th largest key from the half-warp
-//      maxima, the few keys at or above it listed in shared memory and ranked by
+//      piece from one pass: a lower bound of the k-th largest value from the half-warp
+//      maxima, the few tokens that reach it listed in shared memory and ranked by
 //      counting; the one HBM pass over the rows.
 //   2. draft_topk_row_kernel - one CTA per row: the pieces' lists (at most 1024
 //      entries) through the sorting network; the first k become candidates
@@ -23,18 +23,18 @@ constexpr int kThreads = kSortThreads;                 // 256
 constexpr int kPerThread = 16;                         // tokens per thread in the partial kernel
 constexpr int kPiece = kThreads * kPerThread;          // 4096 tokens per CTA
 
-// The top-k of one piece of one row.  Tokens become 64-bit keys (order-preserving image of the value,
-// complemented token index: larger key = larger value, or equal value and lower token; all keys of
-// a piece are distinct).  The k-th largest of the 16 half-warp maxima is a lower bound of the
-// piece's k-th largest key, because k keys at least that large exist; every key at or above the
-// bound goes to a shared list (a few dozen entries on ordinary data, the whole piece at worst) and
-// the list's members are ranked by counting.  One pass over the data, no per-round rescans.
+// The top-k of one piece of one row.  The k-th largest of the 16 half-warp maxima is a lower bound of
+// the piece's k-th largest value, because k tokens at least that large exist; every token whose value
+// reaches the bound goes to a shared list (a few dozen entries on ordinary data, the whole piece at
+// worst) as a 64-bit key (order-preserving image of the value, complemented token index: larger key
+// = larger value, or equal value and lower token), and the list's members are ranked by counting.
+// One pass over the data: per token one maximum and one comparison.
 __global__ void __launch_bounds__(kThreads)
 draft_topk_partial_kernel(const float *__restrict__ logprobs, int V, int k, int pieces, uint2 *__restrict__ part)
 {
-    __shared__ unsigned long long s_list[kPiece];               // candidates at or above the bound
-    __shared__ unsigned long long s_hmax[kThreads / 16];
-    __shared__ unsigned long long s_bound;
+    __shared__ unsigned long long s_list[kPiece];               // tokens whose value reaches the bound
+    __shared__ float s_hmax[kThreads / 16];
+    __shared__ float s_bound;
     __shared__ int s_cnt;
     fspad_pdl_trigger();
     fspad_pdl_wait();
@@ -44,11 +44,8 @@ draft_topk_partial_kernel(const float *__restrict__ logprobs, int V, int k, int 
     const int e0 = piece * kPiece;
     const bool vec = (V % 4 == 0) && ((reinterpret_cast<uintptr_t>(logprobs) & 15) == 0);
     if (tid == 0) s_cnt = 0;
-    // The values stay floats; a key is built only for the thread's maximum and for listed tokens.
-    // Scanning in token order with a strict comparison keeps the lowest token among equal values.
-    float val[kPerThread];
-    float bv = 0.f;
-    int bu = -1;                                                 // slot of the thread's maximum, -1: no token
+    float val[kPerThread];                                       // positions past the row's end hold -inf
+    float bv = -INFINITY;
 #pragma unroll
     for (int i = 0; i < kPerThread / 4; ++i) {
         const int e = e0 + 4 * (i * kThreads + tid);
@@ -57,43 +54,35 @@ draft_topk_partial_kernel(const float *__restrict__ logprobs, int V, int k, int 
             val[4 * i] = t4.x; val[4 * i + 1] = t4.y; val[4 * i + 2] = t4.z; val[4 * i + 3] = t4.w;
         } else {
 #pragma unroll
-            for (int c = 0; c < 4; ++c) val[4 * i + c] = (e + c < V) ? x[e + c] : 0.f;
+            for (int c = 0; c < 4; ++c) val[4 * i + c] = (e + c < V) ? x[e + c] : -INFINITY;
         }
 #pragma unroll
-        for (int c = 0; c < 4; ++c)
-            if (e + c < V && (bu < 0 || val[4 * i + c] > bv)) { bv = val[4 * i + c]; bu = 4 * i + c; }
+        for (int c = 0; c < 4; ++c) bv = fmaxf(bv, val[4 * i + c]);
     }
-    auto token_of = [&](int u) { return e0 + 4 * ((u >> 2) * kThreads + tid) + (u & 3); };
-    unsigned long long best = (bu >= 0) ? fspad_sort_key(bv, (uint32_t)token_of(bu)) : 0ull;   // 0: "no token"
-    // maxima of the 16 half-warps
+    // maxima of the 16 half-warps (a half-warp without any token reports -inf, which can only lower
+    // the bound and so lengthen the list, never lose a token)
 #pragma unroll
-    for (int off = 8; off > 0; off >>= 1) {
-        const unsigned long long o = __shfl_xor_sync(0xffffffffu, best, off);
-        best = o > best ? o : best;
-    }
-    if ((lane & 15) == 0) s_hmax[tid >> 4] = best;
+    for (int off = 8; off > 0; off >>= 1) bv = fmaxf(bv, __shfl_xor_sync(0xffffffffu, bv, off));
+    if ((lane & 15) == 0) s_hmax[tid >> 4] = bv;
     __syncthreads();
     if (tid < kThreads / 16) {
-        const unsigned long long me = s_hmax[tid];
+        const float me = s_hmax[tid];
         int rank = 0;
 #pragma unroll
         for (int o = 0; o < kThreads / 16; ++o) {
-            const unsigned long long ot = s_hmax[o];
-            rank += (ot > me || (ot == me && o < tid)) ? 1 : 0;  // equal only for empty half-warps (key 0)
+            const float ot = s_hmax[o];
+            rank += (ot > me || (ot == me && o < tid)) ? 1 : 0;
         }
         if (rank == k - 1) s_bound = me;                         // k <= 16: exactly one thread
     }
     __syncthreads();
-    const unsigned long long bound = s_bound;
-    // key >= bound  <=>  value above the bound's, or equal to it with a token not after the bound's
-    // (bound == 0: fewer than k half-warps hold a token at all - a short last piece - list every token)
-    const float bound_v = (bound != 0ull) ? fspad_key_value(bound) : -INFINITY;
-    const int bound_i = (bound != 0ull) ? (int)fspad_key_index(bound) : 0x7fffffff;
+    const float bound = s_bound;
 #pragma unroll
     for (int u = 0; u < kPerThread; ++u) {
-        const int tok = token_of(u);
-        if (tok < V && (val[u] > bound_v || (val[u] == bound_v && tok <= bound_i)))
-            s_list[atomicAdd(&s_cnt, 1)] = fspad_sort_key(val[u], (uint32_t)tok);
+        if (val[u] >= bound) {
+            const int tok = e0 + 4 * ((u >> 2) * kThreads + tid) + (u & 3);
+            if (tok < V) s_list[atomicAdd(&s_cnt, 1)] = fspad_sort_key(val[u], (uint32_t)tok);
+        }
     }
     __syncthreads();
     const int n = s_cnt;
