@@ -3,13 +3,18 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
 
-A step is one pass of the whole hot path over one synthetic input set.  The
-input sets are rotated over enough copies to exceed twice the L2 capacity, so
-every step reads its inputs from HBM.  Prints ONE JSON line (rank 0).
+A step is one pass of the whole hot path over one synthetic input set, made
+through the library's one-call form (attention beside acceptance, then
+compaction).  The input sets are rotated over enough copies that the bytes each
+timed function touches before it returns to a set exceed twice the L2 capacity,
+and L2 is flushed between replays, so every step reads its inputs from HBM.
+Every quantity is timed as several replays of a CUDA graph holding K calls;
+median and minimum are reported.  Prints ONE JSON line (rank 0).
 """
 from __future__ import annotations
 
 import argparse
+import hashlib
 import json
 import os
 import statistics
@@ -28,6 +33,30 @@ from paper_2408_15562_b200 import synth  # noqa: E402
 METRIC = "tree_verify_step_latency"
 UNIT = "us/step"
 L2_BYTES = 126 * 1024 * 1024
+REPLAYS = 10                       # timed graph replays per quantity (median and minimum are reported)
+SET_MEMORY_CAP = 40e9              # bytes of device memory the rotated input sets may take
+
+
+def workload_config(w: synth.Workload, n_layers: int, L_mean: float):
+    """What both arms print as `config` (the workload, nothing about how it was run)."""
+    return {"workload": w.name, "batch": w.batch, "n_nodes": w.n_nodes, "prefix_len_mean": L_mean, "vocab": w.vocab,
+            "q_heads": w.n_q_heads, "kv_heads": w.n_kv_heads, "layers_compacted": n_layers,
+            "temperatures": sorted(set(float(t) for t in w.temperatures))}
+
+
+def recorded_traffic(kernel: str, workload: str):
+    """DRAM bytes per launch of `kernel` from the ncu capture recorded under profiles/, or None when there
+    is no record or a source file of the kernel has changed since the counters were taken."""
+    path = os.path.join(ROOT, "profiles", "%s_%s.json" % (kernel, workload))
+    if not os.path.exists(path):
+        return None, "no ncu record for this kernel and workload"
+    with open(path) as f:
+        rec = json.load(f)
+    for rel, digest in rec.get("source_sha256", {}).items():
+        src = os.path.join(ROOT, rel)
+        if not os.path.exists(src) or hashlib.sha256(open(src, "rb").read()).hexdigest() != digest:
+            return None, "kernel source changed since the ncu capture in profiles/%s" % os.path.basename(path)
+    return int(rec["dram_bytes_read"]) + int(rec["dram_bytes_write"]), "dram__bytes_read+write per launch, profiles/%s" % os.path.basename(path)
 
 
 def algorithmic_bytes(w: synth.Workload, L_mean: float, n_acc_rows: float):
@@ -105,12 +134,14 @@ class ClockSampler:
                 "reasons": reasons, "samples": len(sm)}
 
 
-def time_oracle(inp: synth.VerifyInputs, steps: int):
-    """The CPU oracle as it stands, timed on whole verify steps of this workload."""
+def time_oracle(inp: synth.VerifyInputs, steps: int, threads=None):
+    """The CPU oracle as it stands, timed on whole verify steps of this workload, on `threads`
+    OpenMP threads (default: every host core)."""
     import oracle
     oracle.build()
     cache = synth.make_cache(inp, 1)
-    threads = os.cpu_count() or 1
+    threads = threads or (os.cpu_count() or 1)
+    oracle.set_threads(threads)
     times = []
     for _ in range(steps):
         c = cache.copy()
@@ -132,13 +163,15 @@ def run_reference(args, w):
     for _ in range(min(args.warmup, 1)):
         time_oracle(inp, 1)
     us, threads = time_oracle(inp, steps)
+    us1, _ = time_oracle(inp, 1, threads=1)
     line = {"impl": "reference", "metric": METRIC, "value": us, "unit": UNIT, "n_gpus": args.gpus,
             "steps": steps, "warmup": min(args.warmup, 1), "ms_per_step": us / 1e3, "higher_is_better": False,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": w.name, "batch": w.batch, "n_nodes": w.n_nodes, "vocab": w.vocab,
-                       "layers_compacted": 1},
+            "config": workload_config(w, w.n_layers, float(inp.prefix_len.mean())),
             "cpu_baseline": {"value": us, "unit": UNIT, "cores": threads, "kind": "oracle",
-                             "sample": "%d whole verify steps of %s (layer-0 cache only)" % (steps, w.name)},
+                             "value_one_thread": us1,
+                             "sample": "%d whole verify steps of %s (layer-0 cache only; a bounded sample: the oracle is capped "
+                                       "at 5 steps whatever --steps says)" % (steps, w.name)},
             "e2e": {"value": us, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line), flush=True)
@@ -176,12 +209,19 @@ def main():
     L_mean = float(inp.prefix_len.mean())
     n_layers = w.n_layers
     step_bytes = algorithmic_bytes(w, L_mean, 0)
-    one_set = step_bytes["attention"] + step_bytes["accept_all_rows"]
-    R = max(2, int(np.ceil(2 * L2_BYTES / one_set)))
+    # Bytes each timed function is sure to read per call (the walk reads only the draft rows of the realised
+    # path, so draft rows are not counted): the rotation is sized for the function that touches the least.
+    touched = {"step": step_bytes["attention"] + step_bytes["accept_logits"], "tree_attn": step_bytes["attention"],
+               "tree_accept": step_bytes["accept_logits"], "accept_stats_kernel": step_bytes["accept_logits"]}
+    cache_host = synth.make_cache(inp, n_layers)
+    set_bytes = cache_host.nbytes + 2 * inp.q.nbytes + 2 * inp.tree_k.nbytes + inp.target_logits.nbytes * \
+        (2 if inp.draft_probs is not None else 1)
+    R = max(2, int(np.ceil(2 * L2_BYTES / min(touched.values()))))
+    R = max(2, min(R, int(SET_MEMORY_CAP // set_bytes)))
     bf = binding.bf16_tensor
     dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()  # noqa: E731
     sets = []
-    cache0 = bf(synth.make_cache(inp, n_layers))       # [layers][2][B][Hkv][max_len][d]
+    cache0 = bf(cache_host)                            # [layers][2][B][Hkv][max_len][d]
     for r in range(R):
         s = {"cache": cache0.clone(), "q": bf(inp.q).clone(), "tree_k": bf(inp.tree_k), "tree_v": bf(inp.tree_v),
              "logits": dev(inp.target_logits), "draft": dev(inp.draft_probs) if inp.draft_probs is not None else None}
@@ -196,6 +236,7 @@ def main():
     n_acc = torch.empty((B,), dtype=torch.int32, device="cuda")
     bonus = torch.empty((B,), dtype=torch.int32, device="cuda")
     new_len = torch.empty((B,), dtype=torch.int32, device="cuda")
+    flush_buf = torch.empty(3 * L2_BYTES, dtype=torch.uint8, device="cuda")
 
     def attn(s):
         ctx.tree_attn(s["q"], s["cache"][0, 0], s["cache"][0, 1], s["tree_k"], s["tree_v"], parent, prefix, out=out)
@@ -207,6 +248,12 @@ def main():
         ctx.kv_compact(s["cache"], path, n_acc, prefix, new_len)
 
     def step(i):
+        """The verify step as a user makes it: one call of the library."""
+        s = sets[i % R]
+        ctx.verify_step(s["cache"], s["q"], s["tree_k"], s["tree_v"], parent, prefix, s["logits"], s["draft"], tokens,
+                        temp, unif, out, path, n_acc, bonus, new_len)
+
+    def step_three_calls(i):
         s = sets[i % R]
         attn(s)
         accept(s)
@@ -227,6 +274,7 @@ def main():
             for b in range(B):
                 Lb = int(inp.prefix_len[b])
                 s["cache"][:, :, b, :, Lb:Lb + N] = t[b]
+        flush_buf.fill_(1)                               # nothing of the inputs is left in L2
         torch.cuda.synchronize()
 
     for i in range(args.warmup):
@@ -234,10 +282,11 @@ def main():
     barrier()
     ctx.check()
 
-    def timed(fn, steps, graph=True):
-        """us per call of fn over `steps` calls.  The calls are captured once into a CUDA graph
-        (the library only enqueues kernels on the given stream), replayed once untimed, and the
-        timed region is exactly one replay = `steps` calls, bracketed by events on that stream."""
+    def timed(fn, steps, graph=True, replays=REPLAYS):
+        """(median, minimum) us per call of fn.  `steps` calls are captured once into a CUDA graph (the
+        library only enqueues kernels and events on the given stream), replayed once untimed, and then
+        timed `replays` times: each timed region is exactly one replay = `steps` calls, bracketed by
+        events on that stream, after the tree rows were restored and L2 was flushed."""
         restore()
         g = None
         if graph:
@@ -246,55 +295,45 @@ def main():
                 for i in range(steps):
                     fn(i)
             g.replay()
+        samples = []
+        for _ in range(replays):
             restore()
-        barrier()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        if g is not None:
-            g.replay()
-        else:
-            for i in range(steps):
-                fn(i)
-        e1.record()
-        barrier()
-        return e0.elapsed_time(e1) * 1e3 / steps          # us per call
+            barrier()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            if g is not None:
+                g.replay()
+            else:
+                for i in range(steps):
+                    fn(i)
+            e1.record()
+            barrier()
+            samples.append(e0.elapsed_time(e1) * 1e3 / steps)          # us per call
+        return statistics.median(samples), min(samples)
 
     sampler = ClockSampler(local)
     sampler.start()
     launches0 = ctx.launch_count()
-    step_us = timed(step, args.steps)
+    step_us, step_min = timed(step, args.steps)
     launches = (ctx.launch_count() - launches0)          # kernels enqueued into the graph = kernels per replay
     # per-call breakdown and the dominant kernel alone (same rotated inputs, same stream)
-    attn_us = timed(lambda i: attn(sets[i % R]), args.steps)
-    accept_us = timed(lambda i: accept(sets[i % R]), args.steps)
-    compact_us = timed(lambda i: compact(sets[i % R]), args.steps)
+    three_us, three_min = timed(step_three_calls, args.steps)
+    attn_us, attn_min = timed(lambda i: attn(sets[i % R]), args.steps)
+    accept_us, accept_min = timed(lambda i: accept(sets[i % R]), args.steps)
+    compact_us, _ = timed(lambda i: compact(sets[i % R]), args.steps)
     lg2d = [s["logits"].view(B * N, w.vocab) for s in sets]
     st_out = (torch.empty(B * N, dtype=torch.float32, device="cuda"), torch.empty(B * N, dtype=torch.float64, device="cuda"),
               torch.empty(B * N, dtype=torch.int32, device="cuda"))
-    stats_us = timed(lambda i: ctx.accept_stats(lg2d[i % R], temp, N, out="scan_only"), args.steps)
-    stats_merge_us = timed(lambda i: ctx.accept_stats(lg2d[i % R], temp, N, out=st_out), args.steps)
-    eager_us = timed(step, args.steps, graph=False)
-    # attention and acceptance use disjoint scratch, so a caller may queue them on two streams
-    side = torch.cuda.Stream()
-
-    def step_two_streams(i):
-        s = sets[i % R]
-        cur = torch.cuda.current_stream()
-        side.wait_stream(cur)
-        with torch.cuda.stream(side):
-            attn(s)
-        accept(s)
-        compact(s)
-        cur.wait_stream(side)
-
-    two_us = timed(step_two_streams, args.steps)
+    stats_us, stats_min = timed(lambda i: ctx.accept_stats(lg2d[i % R], temp, N, out="scan_only"), args.steps)
+    stats_merge_us, _ = timed(lambda i: ctx.accept_stats(lg2d[i % R], temp, N, out=st_out), args.steps)
+    eager_us, _ = timed(step, args.steps, graph=False, replays=3)
     # the step before the verify step (not part of `value`): candidates of a top-10, five-level draft
     # phase -> the flattened tree of N nodes; verified against the oracle, oracle timed beside it
     cpa, cta, lpa, rta = synth.tree_candidates(w.cfg, B)
     dcand = [torch.from_numpy(np.ascontiguousarray(a)).cuda() for a in (cpa, cta, lpa, rta)]
     tb_out = tuple(torch.empty((B, N), dtype=torch.int32, device="cuda") for _ in range(3)) + \
         (torch.empty((B,), dtype=torch.int32, device="cuda"),)
-    tree_build_us = timed(lambda i: ctx.tree_build(*dcand, N, out=tb_out), args.steps)
+    tree_build_us, _ = timed(lambda i: ctx.tree_build(*dcand, N, out=tb_out), args.steps, replays=3)
     # one draft step of that phase: ten frontier rows of log-probabilities -> top-10 each, joint values, next frontier
     DF, DK = 10, 10
     dlp_host = synth.draft_logprob_rows(w.cfg, B, DF, w.vocab)
@@ -304,8 +343,8 @@ def main():
     dx_arr = (torch.zeros((B, DF * DK), dtype=torch.int32, device="cuda"), torch.zeros((B, DF * DK), dtype=torch.int32, device="cuda"),
               torch.zeros((B, DF * DK), dtype=torch.float32, device="cuda"))
     dx_next = (torch.empty((B, DK), dtype=torch.int32, device="cuda"), torch.empty((B, DK), dtype=torch.float32, device="cuda"))
-    draft_expand_us = timed(lambda i: ctx.draft_expand(dlp[i % len(dlp)], dfl, dfc, DK, DK, 0, *dx_arr, next_cand=dx_next[0],
-                                                       next_logp=dx_next[1]), args.steps)
+    draft_expand_us, _ = timed(lambda i: ctx.draft_expand(dlp[i % len(dlp)], dfl, dfc, DK, DK, 0, *dx_arr, next_cand=dx_next[0],
+                                                          next_logp=dx_next[1]), args.steps, replays=3)
     clocks = sampler.stop()
     ctx.check()
 
@@ -314,8 +353,9 @@ def main():
     verified = None
     tree_build_ok, tree_build_cpu_us = None, None
     draft_expand_ok, draft_expand_cpu_us = None, None
-    if rank == 0 and not args.no_verify and B <= 2:
+    if rank == 0 and not args.no_verify:
         import oracle
+        restore()
         step(0)
         torch.cuda.synchronize()
         ref = oracle.tree_accept(inp.target_logits, inp.draft_probs, inp.draft_tokens, inp.parent, inp.temperature,
@@ -372,8 +412,10 @@ def main():
     d2h = sum(t.numel() * t.element_size() for t in (hout, hpath, hn, hb, hl))
 
     # max over ranks
-    step_us, attn_us, accept_us, compact_us, stats_us, e2e_us, eager_us, two_us, stats_merge_us = dist_util.max_over_ranks(
-        [step_us, attn_us, accept_us, compact_us, stats_us, e2e_us, eager_us, two_us, stats_merge_us], device="cuda")
+    (step_us, step_min, three_us, three_min, attn_us, attn_min, accept_us, accept_min, compact_us, stats_us, stats_min, e2e_us,
+     eager_us, stats_merge_us) = dist_util.max_over_ranks(
+        [step_us, step_min, three_us, three_min, attn_us, attn_min, accept_us, accept_min, compact_us, stats_us, stats_min,
+         e2e_us, eager_us, stats_merge_us], device="cuda")
 
     if rank == 0:
         peak, peak_kind = peaks()
@@ -381,30 +423,37 @@ def main():
         stats_bytes = bytes_real["accept_logits"]
         step_all = bytes_real["attention"] + bytes_real["accept_all_rows"] + bytes_real["compaction"]
         achieved = stats_bytes / (stats_us * 1e-6) / 1e9
+        traffic, traffic_note = recorded_traffic("accept_stats_kernel", w.name)
+        cfg = workload_config(w, n_layers, L_mean)
+        cfg.update({"launch": "K calls of fspad_verify_step captured in one CUDA graph; %d replays timed one by one, "
+                              "value = median" % REPLAYS,
+                    "l2": "inputs rotated over %d sets; bytes touched before a set is reused: step %.0f MB, tree_attn %.0f MB, "
+                          "tree_accept and the scan kernel alone %.0f MB (L2: %.0f MB); L2 flushed between replays"
+                          % (R, R * touched["step"] / 1e6, R * touched["tree_attn"] / 1e6,
+                             R * touched["tree_accept"] / 1e6, L2_BYTES / 1e6),
+                    "multi_gpu": "independent replicas, no collective"})
         line = {
-            "metric": METRIC, "value": step_us, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "metric": METRIC, "value": step_us, "value_median": step_us, "value_min": step_min, "replays": REPLAYS,
+            "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": step_us / 1e3, "higher_is_better": False, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": w.name, "batch": B, "n_nodes": N, "prefix_len_mean": L_mean, "vocab": w.vocab,
-                       "q_heads": w.n_q_heads, "kv_heads": w.n_kv_heads, "layers_compacted": n_layers,
-                       "temperatures": sorted(set(float(t) for t in w.temperatures)),
-                       "launch": "K steps captured in one CUDA graph, one replay timed",
-                       "l2": "inputs rotated over %d copies (%.0f MB per copy, > 2x L2 in total)" % (R, one_set / 1e6),
-                       "multi_gpu": "independent replicas, no collective"},
+            "config": cfg,
             "steps_per_s_all_gpus": dist_util.aggregate_replicas(step_us, world),
             "step_hbm_gbs_all_rows_definition": step_all / (step_us * 1e-6) / 1e9,
             "step_frac_of_hbm_peak": step_all / (step_us * 1e-6) / 1e9 / peak,
             "step_algorithmic_bytes": step_all,
-            "breakdown_us": {"tree_attn": attn_us, "tree_accept": accept_us, "kv_compact": compact_us,
-                             "accept_stats_kernel_alone": stats_us, "accept_stats_with_merge": stats_merge_us,
-                             "whole_step_eager_python_launches": eager_us,
-                             "whole_step_two_streams_attn_overlapping_accept": two_us},
+            "breakdown_us": {"three_calls_on_one_stream": three_us, "three_calls_on_one_stream_min": three_min,
+                             "tree_attn": attn_us, "tree_attn_min": attn_min, "tree_accept": accept_us,
+                             "tree_accept_min": accept_min, "kv_compact_warm_l2": compact_us,
+                             "accept_stats_kernel_alone": stats_us, "accept_stats_kernel_alone_min": stats_min,
+                             "accept_stats_with_merge": stats_merge_us,
+                             "whole_step_eager_python_launches": eager_us},
             "verified_against_oracle": verified,
             "mean_accepted_len": float(n_acc_host.mean()),
             "roofline": {"kernel": "accept_stats_kernel", "bound": "hbm", "achieved": achieved, "peak": peak,
                          "peak_kind": "%s copy bandwidth (burst, kernel timed alone)" % peak_kind, "unit": "GB/s",
-                         "frac": achieved / peak, "traffic": 30800128 if (w.name == "llama3_8b_2k") else None,
-                         "traffic_note": "dram__bytes_read+write per launch, ncu capture in profiles/accept_stats_kernel_llama3_8b_2k.md", "algorithmic_bytes_per_launch": stats_bytes},
+                         "frac": achieved / peak, "traffic": traffic, "traffic_note": traffic_note,
+                         "algorithmic_bytes_per_launch": stats_bytes, "launch_us_median": stats_us, "launch_us_min": stats_min},
             "tree_attn_call": attention_report(w, L_mean, attn_us, bytes_real["attention"], peak),
             "tree_build_call": {"us": tree_build_us, "candidates_per_sequence": int(cpa.shape[1]), "n_nodes": N,
                                 "batch": B, "bit_exact_vs_oracle": tree_build_ok,
@@ -423,8 +472,11 @@ def main():
         }
         if not args.no_cpu_baseline and world == 1:
             us, threads = time_oracle(inp, 3)
+            us1, _ = time_oracle(inp, 1, threads=1)
             line["cpu_baseline"] = {"value": us, "unit": UNIT, "cores": threads, "kind": "oracle",
-                                    "sample": "3 whole verify steps of %s (layer-0 cache only), median" % w.name}
+                                    "value_one_thread": us1,
+                                    "sample": "3 whole verify steps of %s (layer-0 cache only) on all cores, median; "
+                                              "one step on one thread" % w.name}
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()

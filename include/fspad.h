@@ -73,8 +73,10 @@ typedef struct {
 } fspad_config;
 
 /* Create a context on the CURRENT device: allocates the scratch buffers every
- * call needs (split-KV partials, per-node statistics, staging for the host
- * entry point), sized from `cfg`.  Synchronous.  *out is NULL on failure. */
+ * call needs (split-KV partials, per-node statistics), the second stream and
+ * the events of fspad_verify_step, sized from `cfg`.  Synchronous.  *out is
+ * NULL on failure.  (The device staging of fspad_verify_step_host is allocated
+ * by that entry point's first call.) */
 int fspad_create(const fspad_config *cfg, fspad_ctx **out);
 
 /* Free everything the context owns.  Synchronises the device first. */
@@ -90,6 +92,16 @@ const char *fspad_strerror(int err);
 /* Number of kernels the library has launched through this context so far
  * (host counter; lets a caller verify that work ran on the device). */
 long long fspad_launch_count(const fspad_ctx *ctx);
+
+/*
+ * Self-test of the library's bounded device-side waits (error handling of the
+ * library; no passage of the paper).  Every wait of a kernel on a barrier has
+ * a poll limit; when it runs out the kernel records FSPAD_ERR_TIMEOUT in the
+ * status word and returns.  This call queues one warp that waits, with a limit
+ * of `polls` polls (1 .. 4096), on a barrier nothing ever arrives on: after it
+ * fspad_status() returns FSPAD_ERR_TIMEOUT, and the context stays usable.
+ */
+int fspad_selftest_wait_timeout(fspad_ctx *ctx, int polls, void *stream);
 
 /*
  * Tree-masked verify attention of one layer ("Preliminaries": the flattened
@@ -286,9 +298,38 @@ int fspad_kv_compact(fspad_ctx *ctx, fspad_bf16 *cache, const int32_t *accepted_
                      int32_t *new_len, void *stream);
 
 /*
+ * One whole verify step on DEVICE buffers ("Preliminaries": the target's single
+ * forward over the flattened tree, the strict comparison of its results with the
+ * tree, and the removal of the rejected tokens are one step of the decoding
+ * loop).  Equivalent to fspad_tree_attn (over the K and V planes of layer
+ * `attn_layer` of `cache`), fspad_tree_accept and fspad_kv_compact queued one
+ * after the other on `stream`, with the same arguments, outputs and errors, but
+ * the attention runs on a second stream owned by the context, forked from and
+ * joined back into `stream` with events: attention and acceptance share no
+ * data, so their kernels overlap on the device.  Compaction follows the
+ * acceptance directly when tree_k / tree_v are given (attention then never
+ * reads the cache rows compaction rewrites); when they are NULL (tree rows
+ * taken from cache rows L_b ..) compaction waits for the attention as well.
+ * Work queued on `stream` after the call sees every output.  The call only
+ * enqueues work and records / waits on events, so it may be captured into a
+ * CUDA graph.  One call per context at a time.
+ *
+ *   cache  [n_layers][2][batch][Hkv][max_len][d] bf16, updated in place by the compaction
+ *   attn_layer  0 .. n_layers-1
+ *   every other argument as in the three calls it replaces
+ */
+int fspad_verify_step(fspad_ctx *ctx, fspad_bf16 *cache, int attn_layer, const fspad_bf16 *q,
+                      const fspad_bf16 *tree_k, const fspad_bf16 *tree_v, const int32_t *parent,
+                      const int32_t *prefix_len, const float *target_logits, const float *draft_probs,
+                      const int32_t *draft_tokens, const float *temperature, const float *uniforms,
+                      int n_nodes, int batch, fspad_bf16 *attn_out, int32_t *accepted_path,
+                      int32_t *n_accepted, int32_t *bonus_token, int32_t *new_len, void *stream);
+
+/*
  * One whole verify step from HOST buffers: copies the step's inputs to device
- * staging owned by the context, writes the tree rows into cache rows L_b.. of
- * layer 0, runs fspad_tree_attn, fspad_tree_accept and fspad_kv_compact on
+ * staging owned by the context (allocated by the first call, which therefore
+ * must not be made inside a stream capture), writes the tree rows into cache
+ * rows L_b.. of layer 0, runs fspad_verify_step (attention over layer 0) on
  * `stream`, copies the results back and synchronises the stream.  The KV cache
  * is device-resident state that persists between steps (the caller's device
  * pointer `cache`, layout as in fspad_kv_compact); everything else is host

@@ -44,7 +44,14 @@ def _p(a: Optional[np.ndarray], dtype):
 
 
 def set_threads(n: int) -> None:
+    """Number of OpenMP threads the oracle's parallel loops use from now on (timing only: the
+    loops run over independent units, results do not depend on it)."""
     os.environ["OMP_NUM_THREADS"] = str(n)
+    lib()                                             # the OpenMP runtime is in the process once the oracle is
+    try:
+        ctypes.CDLL("libgomp.so.1").omp_set_num_threads(int(n))
+    except OSError:
+        pass
 
 
 def tree_attn(q, k_cache, v_cache, tree_k, tree_v, parent, prefix_len, scale: Optional[float] = None):

@@ -19,7 +19,7 @@ _lib = None
 
 EXPORTS = ["fspad_create", "fspad_destroy", "fspad_status", "fspad_strerror", "fspad_launch_count",
            "fspad_tree_attn", "fspad_tree_accept", "fspad_accept_stats", "fspad_kv_compact",
-           "fspad_verify_step_host", "fspad_accept_stats_noalloc", "fspad_tree_build", "fspad_draft_expand"]
+           "fspad_verify_step", "fspad_verify_step_host", "fspad_selftest_wait_timeout", "fspad_accept_stats_noalloc", "fspad_tree_build", "fspad_draft_expand"]
 
 
 class FspadConfig(ctypes.Structure):
@@ -57,6 +57,8 @@ def load():
     lib.fspad_accept_stats.argtypes = [vp, vp, vp, ci, ci, vp, vp, vp, vp]
     lib.fspad_kv_compact.argtypes = [vp, vp, vp, vp, vp, ci, vp, vp]
     lib.fspad_accept_stats_noalloc.argtypes = [vp, vp, ci, ci, ci, vp, vp, vp, vp]
+    lib.fspad_selftest_wait_timeout.argtypes = [vp, ci, vp]
+    lib.fspad_verify_step.argtypes = [vp, vp, ci] + [vp] * 10 + [ci, ci] + [vp] * 6
     lib.fspad_verify_step_host.argtypes = [vp] * 12 + [ci, ci] + [vp] * 6
     lib.fspad_tree_build.argtypes = [vp] * 5 + [ci, ci, ci] + [vp] * 6
     lib.fspad_draft_expand.argtypes = [vp] * 4 + [ci] * 6 + [vp] * 6
@@ -121,6 +123,9 @@ class Context:
         rc = self.status(stream)
         if rc != 0:
             raise FspadError(rc, "device status")
+
+    def selftest_wait_timeout(self, polls: int = 64, stream=None) -> int:
+        return load().fspad_selftest_wait_timeout(self._h, polls, _stream(stream))
 
     # -- the three operations --------------------------------------------------
     def tree_attn(self, q, k_cache, v_cache, tree_k, tree_v, parent, prefix_len, out=None, stream=None):
@@ -221,6 +226,22 @@ class Context:
         if rc != 0:
             raise FspadError(rc, "fspad_draft_expand")
         return next_cand, next_logp
+
+    def verify_step(self, cache, q, tree_k, tree_v, parent, prefix_len, target_logits, draft_probs, draft_tokens,
+                    temperature, uniforms, attn_out, accepted_path, n_accepted, bonus_token, new_len, attn_layer=0,
+                    stream=None):
+        """The whole verify step on device tensors: attention (second stream of the context) beside
+        acceptance, then compaction; outputs are written in place."""
+        B, N = q.shape[0], q.shape[1]
+        bf, f32, i32 = torch.bfloat16, torch.float32, torch.int32
+        rc = load().fspad_verify_step(
+            self._h, _ptr(cache, bf), attn_layer, _ptr(q, bf), _ptr(tree_k, bf), _ptr(tree_v, bf), _ptr(parent, i32),
+            _ptr(prefix_len, i32), _ptr(target_logits, f32), _ptr(draft_probs, f32), _ptr(draft_tokens, i32),
+            _ptr(temperature, f32), _ptr(uniforms, f32), N, B, _ptr(attn_out, bf), _ptr(accepted_path, i32),
+            _ptr(n_accepted, i32), _ptr(bonus_token, i32), _ptr(new_len, i32), _stream(stream))
+        if rc != 0:
+            raise FspadError(rc, "fspad_verify_step")
+        return attn_out, accepted_path, n_accepted, bonus_token, new_len
 
     def verify_step_host(self, cache, q, tree_k, tree_v, parent, prefix_len, target_logits, draft_probs,
                          draft_tokens, temperature, uniforms, attn_out, accepted_path, n_accepted,

@@ -14,6 +14,8 @@
 // running sum once and adds the 16 exponentials: no per-element branch.  Partials are merged per
 // row by whoever needs them (the acceptance walk for the rows it visits, or
 // the small merge kernel behind fspad_accept_stats).
+#include <atomic>
+
 #include "common.cuh"
 
 namespace {
@@ -262,8 +264,8 @@ static __device__ __align__(256) unsigned char g_noalloc_scratch[kNaBytes];
 
 constexpr int kMaxDevices = 64;
 struct NoAllocDevice {
-    unsigned char *scratch;   // device address of g_noalloc_scratch on this device (NULL = not set up)
-    int sm_count;
+    std::atomic<unsigned char *> scratch;   // device address of g_noalloc_scratch on this device (NULL = not set up)
+    int sm_count;                            // written before `scratch` is published
 };
 NoAllocDevice g_na_dev[kMaxDevices];
 
@@ -280,19 +282,25 @@ extern "C" int fspad_accept_stats_noalloc(const float *logits, const float *temp
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return FSPAD_ERR_CUDA;
     NoAllocDevice &nd = g_na_dev[dev];
-    if (!nd.scratch) {
+    unsigned char *scratch = nd.scratch.load(std::memory_order_acquire);
+    if (!scratch) {
         // First call on this device: g_noalloc_scratch is only a host-side handle here, the
-        // kernels need the array's address in this device's memory.
+        // kernels need the array's address in this device's memory.  Host threads that race on
+        // this first call all compute the same two values; the address is published last, so a
+        // thread that sees it also sees the SM count.
         void *p = nullptr;
+        int sms = 0;
         if (cudaGetSymbolAddress(&p, g_noalloc_scratch) != cudaSuccess || !p) return FSPAD_ERR_CUDA;
-        if (cudaDeviceGetAttribute(&nd.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1)
             return FSPAD_ERR_CUDA;
-        nd.scratch = static_cast<unsigned char *>(p);
+        nd.sm_count = sms;
+        scratch = static_cast<unsigned char *>(p);
+        nd.scratch.store(scratch, std::memory_order_release);
     }
     cudaStream_t st = fspad_stream(stream);
     const bool vec = (vocab % 4 == 0) && ((reinterpret_cast<uintptr_t>(logits) & 15) == 0);
     const FspadStatsGeom g = fspad_stats_geom(nd.sm_count, rows, vocab, vec, kNoAllocSlots);
-    FspadStatsPart *parts = reinterpret_cast<FspadStatsPart *>(nd.scratch);
+    FspadStatsPart *parts = reinterpret_cast<FspadStatsPart *>(scratch);
     // every slot the merge reads is rewritten by this call's first kernel, so the contents an
     // earlier call left in the shared array never need clearing
     if (launch_partials(logits, temperature, rows_per_seq, g, parts, st) != cudaSuccess) return FSPAD_ERR_CUDA;

@@ -102,6 +102,9 @@ int fspad_create(const fspad_config *cfg, fspad_ctx **out)
         ok = ok && dev_alloc(&dx, B * FSPAD_MAX_FRONTIER * (size_t)fspad_draft_expand_pieces(cfg->vocab) * FSPAD_MAX_FRONTIER);
         ctx->dx_part = dx;
     }
+    ok = ok && cudaStreamCreateWithFlags(&ctx->side, cudaStreamNonBlocking) == cudaSuccess;
+    ok = ok && cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming) == cudaSuccess;
+    ok = ok && cudaEventCreateWithFlags(&ctx->ev_join, cudaEventDisableTiming) == cudaSuccess;
     if (ok) {
         ok = cudaMemset(ctx->d_status, 0, sizeof(int)) == cudaSuccess && cudaDeviceSynchronize() == cudaSuccess;
     }
@@ -123,6 +126,9 @@ void fspad_destroy(fspad_ctx *ctx)
                     ctx->h_unif};
     for (void *p : ptrs)
         if (p) cudaFree(p);
+    if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
+    if (ctx->ev_join) cudaEventDestroy(ctx->ev_join);
+    if (ctx->side) cudaStreamDestroy(ctx->side);
     delete ctx;
 }
 
@@ -143,6 +149,13 @@ int fspad_status(fspad_ctx *ctx, void *stream)
 }
 
 long long fspad_launch_count(const fspad_ctx *ctx) { return ctx ? ctx->launches : 0; }
+
+int fspad_selftest_wait_timeout(fspad_ctx *ctx, int polls, void *stream)
+{
+    if (!ctx) return FSPAD_ERR_NULL;
+    if (polls < 1 || polls > 4096) return FSPAD_ERR_RANGE;
+    return fspad_launch_wait_selftest(ctx, polls, fspad_stream(stream)) == cudaSuccess ? FSPAD_OK : FSPAD_ERR_CUDA;
+}
 
 int fspad_tree_attn(fspad_ctx *ctx, const fspad_bf16 *q, const fspad_bf16 *k_cache,
                     const fspad_bf16 *v_cache, const fspad_bf16 *tree_k, const fspad_bf16 *tree_v,
@@ -261,6 +274,55 @@ int fspad_draft_expand(fspad_ctx *ctx, const float *logprobs, const float *front
     return e == cudaSuccess ? FSPAD_OK : FSPAD_ERR_CUDA;
 }
 
+int fspad_verify_step(fspad_ctx *ctx, fspad_bf16 *cache, int attn_layer, const fspad_bf16 *q,
+                      const fspad_bf16 *tree_k, const fspad_bf16 *tree_v, const int32_t *parent,
+                      const int32_t *prefix_len, const float *target_logits, const float *draft_probs,
+                      const int32_t *draft_tokens, const float *temperature, const float *uniforms,
+                      int n_nodes, int batch, fspad_bf16 *attn_out, int32_t *accepted_path,
+                      int32_t *n_accepted, int32_t *bonus_token, int32_t *new_len, void *stream)
+{
+    int rc = check_common(ctx, n_nodes, batch);
+    if (rc) return rc;
+    if (!cache || !q || !parent || !prefix_len || !target_logits || !draft_tokens || !temperature || !attn_out ||
+        !accepted_path || !n_accepted || !bonus_token)
+        return FSPAD_ERR_NULL;
+    if ((tree_k == nullptr) != (tree_v == nullptr)) return FSPAD_ERR_NULL;
+    if ((draft_probs == nullptr) != (uniforms == nullptr)) return FSPAD_ERR_NULL;
+    if (misaligned(cache) || misaligned(q) || misaligned(tree_k) || misaligned(tree_v) || misaligned(attn_out) ||
+        misaligned(target_logits) || misaligned(draft_probs))
+        return FSPAD_ERR_ALIGN;
+    if (attn_layer < 0 || attn_layer >= ctx->cfg.n_layers) return FSPAD_ERR_SHAPE;
+    if (n_nodes > ctx->cfg.max_len) return FSPAD_ERR_RANGE;
+    if (batch == 0) return FSPAD_OK;
+    const fspad_config &c = ctx->cfg;
+    cudaStream_t st = fspad_stream(stream);
+    const size_t plane = (size_t)batch * c.n_kv_heads * (size_t)c.max_len * FSPAD_HEAD_DIM;
+    const fspad_bf16 *kc = cache + (size_t)attn_layer * 2 * plane, *vc = kc + plane;
+
+    // fork: the attention of this step on the context's second stream
+    if (cudaEventRecord(ctx->ev_fork, st) != cudaSuccess || cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0) != cudaSuccess)
+        return FSPAD_ERR_CUDA;
+    int rc_attn = fspad_tree_attn(ctx, q, kc, vc, tree_k, tree_v, parent, prefix_len, n_nodes, batch, attn_out, ctx->side);
+    // the join is queued whatever happened in between, so that a capture of `stream` never ends
+    // with the second stream left unjoined
+    const bool ev_ok = cudaEventRecord(ctx->ev_join, ctx->side) == cudaSuccess;
+    rc = fspad_tree_accept(ctx, target_logits, draft_probs, draft_tokens, parent, temperature, uniforms, n_nodes, batch,
+                           accepted_path, n_accepted, bonus_token, stream);
+    const bool aliased = tree_k == nullptr;      // attention reads the cache rows that compaction rewrites
+    bool joined = false;
+    if (aliased) joined = cudaStreamWaitEvent(st, ctx->ev_join, 0) == cudaSuccess;
+    if (rc == FSPAD_OK && rc_attn == FSPAD_OK) {
+        // behind a join the compaction has two predecessors, so it is launched as a plain dependent
+        cudaError_t e = fspad_launch_kv_compact(ctx, cache, accepted_path, n_accepted, prefix_len, batch, new_len, st,
+                                                !aliased);
+        if (e != cudaSuccess) rc = FSPAD_ERR_CUDA;
+    }
+    if (!aliased) joined = cudaStreamWaitEvent(st, ctx->ev_join, 0) == cudaSuccess;
+    if (rc_attn) return rc_attn;
+    if (rc) return rc;
+    return (ev_ok && joined) ? FSPAD_OK : FSPAD_ERR_CUDA;
+}
+
 int fspad_verify_step_host(fspad_ctx *ctx, fspad_bf16 *cache, const fspad_bf16 *q,
                            const fspad_bf16 *tree_k, const fspad_bf16 *tree_v, const int32_t *parent,
                            const int32_t *prefix_len, const float *target_logits,
@@ -280,8 +342,9 @@ int fspad_verify_step_host(fspad_ctx *ctx, fspad_bf16 *cache, const fspad_bf16 *
     const fspad_config &c = ctx->cfg;
     cudaStream_t st = fspad_stream(stream);
 
-    // staging buffers are created on first use, sized for the context's maxima
-    if (!ctx->h_q) {
+    // staging buffers are created by the first call, sized for the context's maxima; a failed
+    // attempt frees what it got, so that a later call starts over instead of using half a set
+    if (!ctx->h_ready) {
         const size_t B = (size_t)c.max_batch, N = (size_t)c.max_nodes;
         bool ok = dev_alloc(&ctx->h_q, B * N * c.n_q_heads * FSPAD_HEAD_DIM);
         ok = ok && dev_alloc(&ctx->h_out, B * N * c.n_q_heads * FSPAD_HEAD_DIM);
@@ -294,7 +357,20 @@ int fspad_verify_step_host(fspad_ctx *ctx, fspad_bf16 *cache, const fspad_bf16 *
         ok = ok && dev_alloc(&ctx->h_unif, B * (N + 1));
         ok = ok && dev_alloc(&ctx->h_logits, B * N * c.vocab);
         ok = ok && dev_alloc(&ctx->h_draft, B * N * c.vocab);
-        if (!ok) return FSPAD_ERR_NOMEM;
+        if (!ok) {
+            void **slots[] = {(void **)&ctx->h_q, (void **)&ctx->h_out, (void **)&ctx->h_tk, (void **)&ctx->h_tv,
+                              (void **)&ctx->h_parent, (void **)&ctx->h_tokens, (void **)&ctx->h_prefix,
+                              (void **)&ctx->h_nacc, (void **)&ctx->h_bonus, (void **)&ctx->h_newlen,
+                              (void **)&ctx->h_path, (void **)&ctx->h_temp, (void **)&ctx->h_unif,
+                              (void **)&ctx->h_logits, (void **)&ctx->h_draft};
+            for (void **sl : slots) {
+                if (*sl) cudaFree(*sl);
+                *sl = nullptr;
+            }
+            (void)cudaGetLastError();
+            return FSPAD_ERR_NOMEM;
+        }
+        ctx->h_ready = 1;
     }
     const size_t B = (size_t)batch, N = (size_t)n_nodes;
     const size_t q_bytes = B * N * c.n_q_heads * FSPAD_HEAD_DIM * sizeof(fspad_bf16);
@@ -321,19 +397,15 @@ int fspad_verify_step_host(fspad_ctx *ctx, fspad_bf16 *cache, const fspad_bf16 *
     }
     if (!ok) return FSPAD_ERR_CUDA;
 
-    // layer 0 of the cache: K at [0][0], V at [0][1]
-    const size_t plane = B * c.n_kv_heads * (size_t)c.max_len * FSPAD_HEAD_DIM;
+    // the tree rows go into cache rows L_b .. of layer 0 (K at [0][0], V at [0][1]); the step then
+    // takes them from there
     if (fspad_launch_tree_scatter(ctx, cache, ctx->h_tk, ctx->h_tv, ctx->h_prefix, n_nodes, batch, st) !=
         cudaSuccess)
         return FSPAD_ERR_CUDA;
-    rc = fspad_tree_attn(ctx, ctx->h_q, cache, cache + plane, nullptr, nullptr, ctx->h_parent, ctx->h_prefix,
-                         n_nodes, batch, ctx->h_out, stream);
-    if (rc) return rc;
-    rc = fspad_tree_accept(ctx, ctx->h_logits, draft_probs ? ctx->h_draft : nullptr, ctx->h_tokens,
-                           ctx->h_parent, ctx->h_temp, draft_probs ? ctx->h_unif : nullptr, n_nodes, batch,
-                           ctx->h_path, ctx->h_nacc, ctx->h_bonus, stream);
-    if (rc) return rc;
-    rc = fspad_kv_compact(ctx, cache, ctx->h_path, ctx->h_nacc, ctx->h_prefix, batch, ctx->h_newlen, stream);
+    rc = fspad_verify_step(ctx, cache, 0, ctx->h_q, nullptr, nullptr, ctx->h_parent, ctx->h_prefix, ctx->h_logits,
+                           draft_probs ? ctx->h_draft : nullptr, ctx->h_tokens, ctx->h_temp,
+                           draft_probs ? ctx->h_unif : nullptr, n_nodes, batch, ctx->h_out, ctx->h_path, ctx->h_nacc,
+                           ctx->h_bonus, ctx->h_newlen, stream);
     if (rc) return rc;
 
     d2h(attn_out, ctx->h_out, q_bytes);

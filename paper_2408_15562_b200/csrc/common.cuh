@@ -42,9 +42,14 @@ struct fspad_ctx {
     int *row_arg;
     int walk_cluster;         // cluster size used by the sampling walk (0 = not probed yet)
 
+    // whole-step entry point: attention runs on `side`, forked from and joined into the caller's stream
+    cudaStream_t side;
+    cudaEvent_t ev_fork, ev_join;
+
     void *dx_part;            // draft step: per-piece top-k lists [max_batch * 16 rows][pieces][16] (value, token)
 
-    // device staging for the host entry point
+    // device staging for the host entry point (h_ready: every buffer below is allocated)
+    int h_ready;
     fspad_bf16 *h_q, *h_tk, *h_tv, *h_out;
     int *h_parent, *h_prefix, *h_tokens, *h_path, *h_nacc, *h_bonus, *h_newlen;
     float *h_logits, *h_draft, *h_temp, *h_unif;
@@ -252,7 +257,7 @@ cudaError_t fspad_launch_draft_expand(fspad_ctx *ctx, const float *logprobs, con
                                       float *next_logp, cudaStream_t st);
 cudaError_t fspad_launch_kv_compact(fspad_ctx *ctx, fspad_bf16 *cache, const int *path,
                                     const int *n_acc, const int *prefix_len, int B, int *new_len,
-                                    cudaStream_t st);
+                                    cudaStream_t st, bool pdl = true);
 cudaError_t fspad_launch_tree_attn(fspad_ctx *ctx, const fspad_bf16 *q, const fspad_bf16 *kc,
                                    const fspad_bf16 *vc, const fspad_bf16 *tk, const fspad_bf16 *tv,
                                    const int *parent, const int *prefix_len, int N, int B,
@@ -261,6 +266,7 @@ cudaError_t fspad_launch_tree_scatter(fspad_ctx *ctx, fspad_bf16 *cache, const f
                                       const fspad_bf16 *tv, const int *prefix_len, int N, int B,
                                       cudaStream_t st);
 int fspad_attn_umma_splits(const fspad_ctx *ctx, int N, int B);
+cudaError_t fspad_launch_wait_selftest(fspad_ctx *ctx, int polls, cudaStream_t st);
 cudaError_t fspad_launch_attn_umma_split(fspad_ctx *ctx, const fspad_bf16 *q, const fspad_bf16 *kc,
                                          const fspad_bf16 *vc, const fspad_bf16 *tk, const fspad_bf16 *tv,
                                          const int *parent, const int *prefix_len, int N, int B, int n_splits,

@@ -60,6 +60,9 @@ kv_compact_kernel(uint4 *__restrict__ cache, const int *__restrict__ path, const
                 }
             }
         }
+        // the two half-warps own different rows and a destination of one may be a source of the
+        // other: every load of the batch is ordered before any of its stores
+        __syncwarp();
 #pragma unroll
         for (int u = 0; u < kBatchIters; ++u)
             if (dst[u] >= 0) base[(size_t)(L + dst[u]) * kChunks + chunk] = v[u];
@@ -95,14 +98,14 @@ tree_scatter_kernel(uint4 *__restrict__ cache, const uint4 *__restrict__ tk, con
 
 cudaError_t fspad_launch_kv_compact(fspad_ctx *ctx, fspad_bf16 *cache, const int *path,
                                     const int *n_acc, const int *prefix_len, int B, int *new_len,
-                                    cudaStream_t st)
+                                    cudaStream_t st, bool pdl)
 {
     if (B == 0) return cudaSuccess;
     const fspad_config &c = ctx->cfg;
     const long long slices = (long long)c.n_layers * 2 * B * c.n_kv_heads;
     const unsigned grid = (unsigned)((slices + kWarpsPerCta - 1) / kWarpsPerCta);
     ctx->launches++;
-    return fspad_launch(kv_compact_kernel, dim3(grid), dim3(kWarpsPerCta * 32), 0, st, 0,
+    return fspad_launch_opt(pdl, kv_compact_kernel, dim3(grid), dim3(kWarpsPerCta * 32), 0, st, 0,
                         reinterpret_cast<uint4 *>(cache), path, n_acc, prefix_len, c.n_layers, B, c.n_kv_heads,
                         c.max_len, c.max_nodes, c.max_nodes, new_len, ctx->d_status);
 }

@@ -79,12 +79,13 @@ __device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity)
 }
 // Bounded wait (non-blocking test + short sleep, about 20 ms in all); false if the cap ran out.
 // Lane 0 polls and the warp takes its verdict through a full-mask shuffle, so every lane leaves
-// together: the warp-collective tensor-memory instructions that follow need a converged warp.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
+// together with the same verdict: the warp-collective tensor-memory instructions that follow need
+// a converged warp, and the tensor-core warp's issue loop needs one `failed` flag for all lanes.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_t cap = WAIT_CAP)
 {
     int ok = 0;
     if ((threadIdx.x & 31) == 0) {
-        for (uint32_t i = 0; i < WAIT_CAP && !ok; ++i) {
+        for (uint32_t i = 0; i < cap && !ok; ++i) {
             ok = mbar_test(bar, parity) ? 1 : 0;
             if (!ok && i >= 64) __nanosleep(40);      // the first polls spin: hand-offs are short
         }
@@ -149,15 +150,6 @@ __device__ __forceinline__ void mma_f16_lo(uint32_t d_tmem, uint32_t a_lo, uint3
                  "@e tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, p;\n\t}\n"
                  :: "r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate), "r"(elect)
                  : "memory");
-}
-// single-thread bounded wait (the tensor-core thread polls alone; nothing warp-collective follows)
-__device__ __forceinline__ bool mbar_wait_one(uint32_t bar, uint32_t parity)
-{
-    for (uint32_t i = 0; i < WAIT_CAP; ++i) {
-        if (mbar_test(bar, parity)) return true;
-        if (i >= 64) __nanosleep(40);
-    }
-    return false;
 }
 __device__ __forceinline__ void mma_commit(uint32_t bar)
 {
@@ -266,7 +258,7 @@ __global__ void __launch_bounds__(NT, 1)
 tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV)
 {
     extern __shared__ unsigned char smem_raw[];
-    __shared__ __align__(8) unsigned long long s_bar[4 * NS + 12];
+    __shared__ __align__(8) unsigned long long s_bar[4 * NS + 13];
     __shared__ uint32_t s_tmem;
     __shared__ int s_fail;
     __shared__ int s_par[FSPAD_MAX_NODES];
@@ -313,12 +305,13 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
     auto sfull = [&](int par) { return bar0 + 8u * (uint32_t)(4 * NS + par); };
     auto pfull = [&](int grp2, int par) { return bar0 + 8u * (uint32_t)(4 * NS + 4 + 2 * grp2 + par); };
     auto odone = [&](int grp2, int par) { return bar0 + 8u * (uint32_t)(4 * NS + 8 + 2 * grp2 + par); };
+    const uint32_t drain = bar0 + 8u * (uint32_t)(4 * NS + 12);   // used only when a wait has run out
     const bool tma_ok = a.use_tma != 0;
     // The thread that issues the first TMA copies also initialises the barriers, so those copies
     // leave as soon as the prefix length is known, ahead of the CTA's first barrier.
     if (tid == 256) {
 #pragma unroll
-        for (int i = 0; i < 4 * NS + 12; ++i) mbar_init(bar0 + 8u * i, (i >= 4 * NS + 4 && i < 4 * NS + 8) ? 4 : 1);
+        for (int i = 0; i < 4 * NS + 13; ++i) mbar_init(bar0 + 8u * i, (i >= 4 * NS + 4 && i < 4 * NS + 8) ? 4 : 1);
         s_fail = 0;
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     }
@@ -408,6 +401,7 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
     const uint32_t idesc_s = make_idesc(false, 128), idesc_o = make_idesc(true, 128);
     const uint32_t tO = tmem + ((uint32_t)((warp & 3) * 32) << 16) + 256u + (uint32_t)grp * 128u;   // this group's O row
     bool failed = false;
+    int filled_k = min(n_ch, NS), filled_v = filled_k;   // copy warp: chunks whose K (V) fill has been started
 
     if (warp == 8) {
         // ================= copy warp: refills the K / V buffers =================
@@ -434,9 +428,9 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
         for (int i = 0; i + NS < n_ch; ++i) {
             // the K buffer of chunk i is free once S(i) has completed, its V buffer once O += P(i) V(i) has
             if (!failed && !mbar_wait(kfree(buf), ph)) failed = true;
-            if (!failed) fill(c0 + i + NS, buf, false);
+            if (!failed) { fill(c0 + i + NS, buf, false); ++filled_k; }
             if (!failed && !mbar_wait(vfree(buf), ph)) failed = true;
-            if (!failed) fill(c0 + i + NS, buf, true);
+            if (!failed) { fill(c0 + i + NS, buf, true); ++filled_v; }
             if (++buf == NS) { buf = 0; ph ^= 1u; }
         }
         if (failed) s_fail = 1;
@@ -454,7 +448,7 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
             // S(c) = Q K(c)^T into score buffer c & 1 (columns 0..63 of it belong to group 0, 64..127 to
             // group 1); K(c) sits in ring slot kbuf, which the second commit releases
             auto issue_s = [&](int c) {
-                if (!failed && !mbar_wait_one(kfull(kbuf), kph)) failed = true;
+                if (!failed && !mbar_wait(kfull(kbuf), kph)) failed = true;
                 if (!failed) {
                     tc_fence_after();
                     const uint32_t kb = k_lo + (uint32_t)kbuf * (TILE >> 4);
@@ -479,8 +473,8 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
                 for (int g2 = 0; g2 < 2; ++g2) {
                     // O[g2] += P_g2(c) V(c)[64 g2 .. 64 g2 + 63]: P from the four warps of group g2 (in tensor
                     // memory, over the scores it was computed from) and the V chunk
-                    if (!failed && !mbar_wait_one(pfull(g2, p), ph)) failed = true;
-                    if (g2 == 0 && !failed && !mbar_wait_one(vfull(vbuf), vph)) failed = true;
+                    if (!failed && !mbar_wait(pfull(g2, p), ph)) failed = true;
+                    if (g2 == 0 && !failed && !mbar_wait(vfull(vbuf), vph)) failed = true;
                     if (!failed) {
                         tc_fence_after();
                         const uint32_t a_t = tmem + (uint32_t)p * 128u + (uint32_t)g2 * 64u;
@@ -650,6 +644,22 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
     fspad_pdl_trigger();
     tc_fence_before();
     __syncthreads();
+    if (s_fail != 0) {
+        // A wait ran out somewhere in this CTA.  Before the shared and tensor memory go back to
+        // the SM, whatever was started asynchronously is given a bounded time to land: the copy warp
+        // waits for the last fill it started in every ring slot, the tensor-core warp for everything
+        // its thread has issued (one more commit on a barrier of its own).
+        if (warp == 8) {
+            for (int sl = 0; sl < NS; ++sl) {
+                const int nk = (filled_k - sl + NS - 1) / NS, nv = (filled_v - sl + NS - 1) / NS;   // fills of slot sl
+                if (nk > 0) (void)mbar_wait(kfull(sl), (uint32_t)(nk - 1) & 1u);
+                if (nv > 0) (void)mbar_wait(vfull(sl), (uint32_t)(nv - 1) & 1u);
+            }
+        } else {
+            mma_commit_if(drain, lane == 0);
+            (void)mbar_wait(drain, 0u);
+        }
+    }
     __syncthreads();
     if (warp != 9) return;
     tc_fence_after();
@@ -657,7 +667,29 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" :: "r"(tmem), "r"(TMEM_COLS) : "memory");
 }
 
+// Self-test of the bounded wait: one warp waits, with a small cap, on a barrier that nothing ever
+// arrives on; the wait must run out, the kernel records FSPAD_ERR_TIMEOUT and returns normally.
+__global__ void __launch_bounds__(32)
+wait_timeout_selftest_kernel(int *status, uint32_t cap)
+{
+    __shared__ __align__(8) unsigned long long bar;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bar), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+    }
+    __syncwarp();
+    const bool ok = mbar_wait(smem_u32(&bar), 0u, cap);
+    if (!ok && threadIdx.x == 0) fspad_report(status, FSPAD_ERR_TIMEOUT);
+}
+
 }  // namespace umma
+
+cudaError_t fspad_launch_wait_selftest(fspad_ctx *ctx, int polls, cudaStream_t st)
+{
+    ctx->launches++;
+    return fspad_launch_opt(false, umma::wait_timeout_selftest_kernel, dim3(1), dim3(32), 0, st, 0, ctx->d_status,
+                            (uint32_t)polls);
+}
 
 int fspad_attn_umma_splits(const fspad_ctx *ctx, int N, int B)
 {

@@ -120,11 +120,11 @@ def test_full_size_llama3_70b_8k_sampled_heads():
     _check(synth.generate(W["llama3_70b_8k"], 0, with_accept=False))
 
 
-def test_full_size_batch16_sampled_sequences():
+def test_full_size_batch16_every_sequence():
+    """The batched ragged workload in its full launch configuration; the oracle checks every
+    output of all sixteen sequences (about a minute of fp64 CPU work on all host cores)."""
     inp = synth.generate(W["batch16_ragged"], 0, with_accept=False)
-    shortest = int(np.argmin(inp.prefix_len))
-    longest = int(np.argmax(inp.prefix_len))
-    _check(inp, seqs=sorted({0, shortest, longest}))
+    _check(inp)
 
 
 def test_prefix_out_of_range_is_reported():

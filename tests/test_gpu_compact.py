@@ -66,6 +66,18 @@ def test_long_chain_path_uses_several_row_batches():
     _run_case(cache, paths, np.array([30, 64], np.int32), np.array([17, 100], np.int32), 2, N)
 
 
+@pytest.mark.parametrize("n", [3, 5, 7, 9, 15, 17, 31])
+def test_odd_lengths_where_one_half_warp_reads_what_the_other_writes(n):
+    """Paths [0, 2, 4, ...] and [0, 1, 3, 5, ...] of odd length: in every batch of eight moves the
+    destination row of one half-warp is the source row of the other."""
+    N = 64
+    cache = synth.hashed_u16((2, 2, 2, 3, 150, 128), n)
+    paths = np.full((2, N), -1, np.int32)
+    paths[0, :n] = np.arange(n) * 2
+    paths[1, :n] = np.concatenate([[0], np.arange(1, n) * 2 - 1])
+    _run_case(cache, paths, np.array([n, n], np.int32), np.array([11, 70], np.int32), 3, N)
+
+
 def test_full_size_batch16_32_layers_sampled_slices():
     """Configuration of the batched ragged workload: 32 layers x 16 sequences x 8 kv
     heads, max_len 4160.  The device cache is filled by a hash of the flat index;

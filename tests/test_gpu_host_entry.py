@@ -1,9 +1,11 @@
-"""The host-buffer entry point (`fspad_verify_step_host`) against the three device calls it wraps:
-same attention output, same acceptance result, same compacted cache, twice in a row."""
+"""The host-buffer entry point (`fspad_verify_step_host`) against the oracle (attention within the
+stated bound, acceptance and compacted cache bit-exact) and against the three device calls it
+stands for: same attention output, same acceptance result, same compacted cache, twice in a row."""
 import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2408_15562_b200 import binding, synth
 from tests import helpers
 
@@ -34,6 +36,12 @@ def test_host_entry_equals_device_calls(mode):
                                            d["temperature"], d["uniforms"])
     len_d = ctx.kv_compact(cache_d, path_d, n_d, prefix)
     ctx.check()
+    # --- the oracle on the same inputs ---
+    ref_o = oracle.tree_attn(inp.q, inp.k_cache, inp.v_cache, inp.tree_k, inp.tree_v, inp.parent, inp.prefix_len)
+    r = oracle.tree_accept(inp.target_logits, inp.draft_probs, inp.draft_tokens, inp.parent, inp.temperature,
+                           inp.uniforms if inp.draft_probs is not None else None)
+    want_cache = cache_host.copy()
+    want_len = oracle.kv_compact(want_cache, r["accepted_path"], r["n_accepted"], inp.prefix_len)
     # --- host entry, two calls in a row on fresh caches ---
     pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()   # noqa: E731
     hq = binding.bf16_tensor(inp.q, "cpu").pin_memory()
@@ -49,6 +57,14 @@ def test_host_entry_equals_device_calls(mode):
                              pin(inp.draft_probs) if sampling else None, pin(inp.draft_tokens), pin(inp.temperature),
                              pin(inp.uniforms) if sampling else None, hout, hpath, hn, hb, hl)
         torch.cuda.synchronize()
+        mx, mean = helpers.attn_errors(hout, ref_o)
+        assert mx <= 1e-2 and mean <= 1e-3, (mx, mean)
+        hard, near, msgs = helpers.compare_accept(inp, hpath.numpy(), hn.numpy(), hb.numpy())
+        assert hard == 0 and near == 0, msgs
+        np.testing.assert_array_equal(hl.numpy(), want_len)
+        got = binding.bf16_bits(cache_h)
+        for b in range(B):
+            np.testing.assert_array_equal(got[:, :, b, :, :int(want_len[b])], want_cache[:, :, b, :, :int(want_len[b])])
         assert torch.equal(hout.view(torch.int16), out_d.cpu().view(torch.int16))
         assert torch.equal(hn, n_d.cpu()) and torch.equal(hb, bonus_d.cpu()) and torch.equal(hl, len_d.cpu())
         for b in range(B):
