@@ -6,8 +6,8 @@
 // this kernel produces all of them in one HBM-bound sweep.
 //
 // Layout: logits [rows][V] fp32, viewed as one flat array that is cut into
-// equal contiguous ranges, one per CTA (four CTAs per SM, a single wave), so
-// the load is balanced whatever rows and V are.  A range may cross row
+// equal contiguous ranges, one per CTA (two 512-thread CTAs per SM, a single
+// wave), so the load is balanced whatever rows and V are.  A range may cross row
 // boundaries; each (row, CTA) piece yields one partial (max, argmax, sum).
 // A thread works in batches of four 128-bit loads, with the next batch already
 // in flight: it takes the maximum of the 16 values in registers, rescales its
@@ -20,7 +20,7 @@
 
 namespace {
 
-constexpr int kThreads = 256;
+constexpr int kThreads = FSPAD_STATS_THREADS;   // 512
 constexpr int kDeep = 4;                  // load units per batch per thread (two batches in flight)
 constexpr float kLog2e = 1.4426950408889634f;
 
@@ -74,7 +74,7 @@ template <> struct Unit<1> {
 };
 
 template <int UNIT>
-__global__ void __launch_bounds__(kThreads, 4)
+__global__ void __launch_bounds__(kThreads, 2)
 accept_stats_kernel(const float *__restrict__ logits, const float *__restrict__ temperature,
                     int rows_per_seq, const FspadStatsGeom g, FspadStatsPart *__restrict__ parts)
 {
@@ -85,8 +85,11 @@ accept_stats_kernel(const float *__restrict__ logits, const float *__restrict__ 
     __shared__ Acc wacc[kThreads / 32];
     __shared__ float s_bmax;
     __shared__ int s_barg;
-    fspad_pdl_trigger();
+    // Wait first, then let the successor start: a kernel that follows this one in the stream (the
+    // acceptance walk) can then rely on everything queued before the scan having completed, and may
+    // read the caller's arrays, which the scan never writes, while the scan is still running.
     fspad_pdl_wait();
+    fspad_pdl_trigger();
 
     long long seg_lo = lo;
     while (seg_lo < hi) {
@@ -153,7 +156,7 @@ accept_stats_kernel(const float *__restrict__ logits, const float *__restrict__ 
         if (wid == 0) {
             Acc q = (lane < kThreads / 32) ? wacc[lane] : Acc{-INFINITY, 0.f, 0};
 #pragma unroll
-            for (int o = 4; o > 0; o >>= 1) {
+            for (int o = kThreads / 64; o > 0; o >>= 1) {
                 const float om = __shfl_xor_sync(0xffffffffu, q.m, o);
                 const float os = __shfl_xor_sync(0xffffffffu, q.s, o);
                 acc_merge(q, om, os, k);
@@ -209,25 +212,25 @@ accept_stats_merge_kernel(const FspadStatsPart *__restrict__ parts, const FspadS
 }
 
 cudaError_t launch_partials(const float *logits, const float *temperature, int rows_per_seq,
-                            const FspadStatsGeom &g, FspadStatsPart *parts, cudaStream_t st)
+                            const FspadStatsGeom &g, FspadStatsPart *parts, cudaStream_t st, bool pdl = true)
 {
     if (g.unit == 4)
-        return fspad_launch(accept_stats_kernel<4>, dim3(g.n_cta), dim3(kThreads), 0, st, 0, logits, temperature,
+        return fspad_launch_opt(pdl, accept_stats_kernel<4>, dim3(g.n_cta), dim3(kThreads), 0, st, 0, logits, temperature,
                             rows_per_seq, g, parts);
-    return fspad_launch(accept_stats_kernel<1>, dim3(g.n_cta), dim3(kThreads), 0, st, 0, logits, temperature,
-                        rows_per_seq, g, parts);
+    return fspad_launch_opt(pdl, accept_stats_kernel<1>, dim3(g.n_cta), dim3(kThreads), 0, st, 0, logits, temperature,
+                            rows_per_seq, g, parts);
 }
 
 }  // namespace
 
 cudaError_t fspad_launch_stats_partials(fspad_ctx *ctx, const float *logits, const float *temperature,
                                         int rows, int rows_per_seq, int V, FspadStatsGeom *geom,
-                                        cudaStream_t st)
+                                        cudaStream_t st, bool pdl)
 {
     const bool vec = (V % 4 == 0) && ((reinterpret_cast<uintptr_t>(logits) & 15) == 0);
     *geom = fspad_stats_geom(ctx->sm_count, rows, V, vec, ctx->stats_slots);
     ctx->launches++;
-    return launch_partials(logits, temperature, rows_per_seq, *geom, ctx->st_part, st);
+    return launch_partials(logits, temperature, rows_per_seq, *geom, ctx->st_part, st, pdl);
 }
 
 cudaError_t fspad_launch_accept_stats(fspad_ctx *ctx, const float *logits, const float *temperature,

@@ -47,6 +47,8 @@ constexpr double kAmbiguous = 1e-4;
 constexpr double kScanRel = 1e-6;          // bound taken for the relative error of the scan's sum of exponentials
 constexpr double kFusedTol = 1e-9;         // relative error the fused first-rejection sweep may leave in the residual mass
 constexpr float kLog2eF = 1.4426950408889634f;
+constexpr int kPieceSlots = 16;            // pieces of a row whose scan sums are kept for the bonus draw
+enum { REQ_DONE = 0, REQ_EXP = 1, REQ_EXP_Q = 2, REQ_FUSED = 3, REQ_RESID = 4 };
 
 // 2^(i/64), i = 0..63, correctly rounded
 __constant__ double kExp2Tbl[64] = {
@@ -106,21 +108,32 @@ struct Shared {
     double tot[2];                  // cluster totals
     double warp5[kWarps][5], slot5[2][kMaxCluster][5], tot5[5];   // the same exchange for five values
     int fused_fallback;
-    double cta_total[kMaxCluster];  // bonus draw: every CTA's total, received from the peers
+    double cta_total[2][kMaxCluster];  // bonus draw: every CTA's total, received from the peers (by attempt)
+    int verdict[2];                    // bonus draw from one piece of the row: 1 = settled, 2 = the whole row must be swept
+    // serial walk -> sweeps: what thread 0 asks the CTA to do next
+    int req, req_child, req_last;
+    unsigned long long rem;            // children of the current node not tested yet
+    // approximate mass of every (row, CTA) piece of the vocabulary scan, relative to the row maximum;
+    // piece_cnt[row] = 0 when the row has more than kPieceSlots pieces (the draw then sweeps the whole row)
+    double piece_w[FSPAD_MAX_NODES][kPieceSlots];
+    int piece_cnt[FSPAD_MAX_NODES];
 };
 
 // exp(a) for a <= 0 in double precision: a = (64 n + i) ln2/64 + r, |r| <= ln2/128,
-// exp(a) = 2^n * 2^(i/64) * (1 + r + ... + r^5/120); relative error about 4e-16.
+// exp(a) = 2^n * 2^(i/64) * (1 + r + r^2/2 + r^3/6 + r^4/24); relative error below 5e-14
+// (truncation r^5/120 < 4e-14, one-step argument reduction < 3e-14 at the far end of the range).
+// Every operation is an fp64 multiply-add: the rounding to the nearest integer is done by adding
+// and subtracting 1.5 * 2^52 (the integer then sits in the low word of the sum), because the
+// conversions between integers and doubles cost as much as an fp64 operation each.
 __device__ __forceinline__ double exp_neg(double a, const double *tbl)
 {
     if (!(a > -700.0)) return 0.0;                        // also -inf and NaN
-    const double t = a * 92.33248261689366;               // 64 / ln 2
-    const int k = __double2int_rn(t);
-    const double kd = (double)k;
-    double r = fma(-kd, 0.010830424696249145, a);         // ln2/64, high part
-    r = fma(-kd, 3.623510646634843e-19, r);               // low part
-    double p = fma(r, 1.0 / 120.0, 1.0 / 24.0);
-    p = fma(p, r, 1.0 / 6.0);
+    const double magic = 6755399441055744.0;              // 1.5 * 2^52
+    const double tm = fma(a, 92.33248261689366, magic);   // a * 64 / ln 2, rounded to an integer
+    const int k = __double2loint(tm);
+    const double kd = tm - magic;
+    const double r = fma(-kd, 0.010830424696249145, a);   // ln2/64
+    double p = fma(r, 1.0 / 24.0, 1.0 / 6.0);
     p = fma(p, r, 0.5);
     p = fma(p, r, 1.0);
     p = fma(p, r, 1.0);
@@ -161,7 +174,8 @@ template <int MODE>
 __device__ Sweep sweep_chunk(const Shared &sh, const float *__restrict__ x, const float *__restrict__ q,
                              double *__restrict__ se, float *__restrict__ sq, int tid, int nthr, int lo, int hi,
                              bool vec, bool cache_ok, bool have_e, bool have_q, double c, int xnew,
-                             bool locate, double base, double run0, double target, int *found)
+                             bool locate, double base, double run0, double target, int *found,
+                             double *gap_below = nullptr, double *gap_above = nullptr)
 {
     const double m = sh.m, invT = sh.invT;
     const int nrem = sh.nrem;
@@ -175,6 +189,7 @@ __device__ Sweep sweep_chunk(const Shared &sh, const float *__restrict__ x, cons
         if (MODE == MODE_RESID) special |= (xnew >= lo && xnew < hi);
     }
     double a = 0.0, b = 0.0, run = run0;
+    double g_lo = -1.0, g_hi = -1.0;      // distances from the target to the located token's interval ends
     int last_pos = -1, hit = -1;
     for (int j = lo; j < hi; j += 4) {
         const int n = min(4, hi - j);
@@ -235,13 +250,22 @@ __device__ Sweep sweep_chunk(const Shared &sh, const float *__restrict__ x, cons
             if (MODE == MODE_RESID) {
                 if (q_counts) b += (double)qv[t];
             } else if (locate) {
+                const double before = base + run;
                 run += w;
                 if (w > 0.0) last_pos = j + t;
-                if (hit < 0 && base + run > target) hit = j + t;
+                if (hit < 0 && base + run > target) {
+                    hit = j + t;
+                    g_lo = target - before;
+                    g_hi = base + run - target;
+                }
             }
         }
     }
-    if (locate) *found = (hit >= 0) ? hit : last_pos;
+    if (locate) {
+        *found = (hit >= 0) ? hit : last_pos;
+        if (gap_below) *gap_below = g_lo;
+        if (gap_above) *gap_above = g_hi;
+    }
     return Sweep{a, b};
 }
 
@@ -293,7 +317,10 @@ __device__ Sweep5 fused_reject_sweep(const Shared &sh, const float *__restrict__
             r.v[0] += e;
             if (w > 0.0) { r.v[1] += e; r.v[2] += qd; }
             if (j + t != xnew) r.v[3] += qd;
-            if (pe > 0.0 && fabs(w) <= kScanRel * pe) r.v[4] += pe;
+            // |w| <= kScanRel * pe needs the binary exponent of w at least 19 below that of pe: an
+            // integer comparison sorts out all but a handful of tokens
+            if ((__double2hiint(w) & 0x7ff00000) <= (__double2hiint(pe) & 0x7ff00000) - (19 << 20))
+                if (pe > 0.0 && fabs(w) <= kScanRel * pe) r.v[4] += pe;
         }
     }
     return r;
@@ -314,8 +341,10 @@ accept_walk_kernel(const WalkArgs args)
 
     fspad_pdl_trigger();
     if (tid < 64) { sh.exp_tbl[tid] = kExp2Tbl[tid]; sh.child_mask[tid] = 0ull; }
-    fspad_pdl_wait();
-    // The prologue is a chain of dependent global loads; it is kept to two round trips.
+    // The vocabulary scan that precedes this kernel in the stream lets it start only after the scan's
+    // own predecessor has completed, and the scan writes nothing but its partial results.  So the
+    // caller's arrays may be read before the scan has finished: the prologue's two round trips of
+    // dependent loads run under the scan's tail.
     // Round trip 1: everything that depends on nothing - temperature, tree arrays, uniforms.
     float Tf = args.temperature[b];
     int p = -1, t = 0;
@@ -340,9 +369,7 @@ accept_walk_kernel(const WalkArgs args)
     const float kT = kLog2eF / (Tf > 0.0f ? Tf : 1.0f);
 
     // Round trip 2: thread c owns node c (tree arrays, the child bit of its parent and the scalars
-    // its accept test needs: target logit and draft probability of its token in its parent's row);
-    // half-warps merge the scan partials of the rows.  The gathered scalars stay in registers until
-    // the merge has issued its own loads.
+    // its accept test needs: target logit and draft probability of its token in its parent's row).
     float xv = 0.f, qv = 0.f;
     if (tid < N) {
         if (tid == 0) {
@@ -367,18 +394,33 @@ accept_walk_kernel(const WalkArgs args)
             }
         }
     }
+    // The root's draft row is the one most likely to be swept: ask for it now (a hint, no register
+    // is tied up and nothing waits for it).
+    const bool vec = (V % 4 == 0) && ((reinterpret_cast<uintptr_t>(args.logits) & 15) == 0) &&
+                     ((reinterpret_cast<uintptr_t>(args.draft) & 15) == 0);
+    // contiguous slice per CTA, contiguous chunk per thread (multiples of 4 tokens)
+    const int per_cta = (((V + C - 1) / C) + 3) & ~3;
+    const int per_thr = (((per_cta + nthr - 1) / nthr) + 3) & ~3;
+    const int cta_lo = rank * per_cta, cta_hi = min(V, cta_lo + per_cta);
+    const int lo = min(cta_hi, cta_lo + tid * per_thr), hi = min(cta_hi, lo + per_thr);
+    if (sampling && lo < hi)
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(dp + lo));
+    if (sampling && tid < N) {
+        if (tid >= 1) { sh.cx[tid] = xv; sh.cq[tid] = qv; sh.cu[tid] = uval; }
+        else sh.ubonus = uval;
+    }
+
+    fspad_pdl_wait();                            // from here on the scan's partial results may be read
     {
+        // half-warps merge the scan partials of the rows
         const int lane16 = tid & 15, n_half = nthr >> 4;
         for (int r0 = 0; r0 < N; r0 += n_half) {                 // whole warps iterate together
             const int row = r0 + (tid >> 4);
             float M; double S; int A;
-            fspad_stats_merge_half(args.parts, args.geom, b * N + row, row < N, kT, lane16, M, S, A);
+            fspad_stats_merge_half(args.parts, args.geom, b * N + row, row < N, kT, lane16, M, S, A,
+                                   sh.piece_w[row < N ? row : 0], &sh.piece_cnt[row < N ? row : 0]);
             if (lane16 == 0 && row < N) { sh.rowM[row] = M; sh.rowS[row] = S; sh.rowInvS[row] = 1.0 / S; sh.rowA[row] = A; }
         }
-    }
-    if (sampling && tid < N) {
-        if (tid >= 1) { sh.cx[tid] = xv; sh.cq[tid] = qv; sh.cu[tid] = uval; }
-        else sh.ubonus = uval;
     }
     __syncthreads();
     if (sampling && tid >= 1 && tid < N)
@@ -411,13 +453,6 @@ accept_walk_kernel(const WalkArgs args)
     }
 
     // ---- sampling ----
-    const bool vec = (V % 4 == 0) && ((reinterpret_cast<uintptr_t>(args.logits) & 15) == 0) &&
-                     ((reinterpret_cast<uintptr_t>(args.draft) & 15) == 0);
-    // contiguous slice per CTA, contiguous chunk per thread (multiples of 4 tokens)
-    const int per_cta = (((V + C - 1) / C) + 3) & ~3;
-    const int per_thr = (((per_cta + nthr - 1) / nthr) + 3) & ~3;
-    const int cta_lo = rank * per_cta, cta_hi = min(V, cta_lo + per_cta);
-    const int lo = min(cta_hi, cta_lo + tid * per_thr), hi = min(cta_hi, lo + per_thr);
     const bool cache_ok = args.cache_ok != 0;
     double *se = reinterpret_cast<double *>(dyn_smem);
     // the cache is laid out [k][thread] (k-th token of each thread's chunk): conflict-free
@@ -482,139 +517,144 @@ accept_walk_kernel(const WalkArgs args)
         if (wid == 0) {
 #pragma unroll
             for (int k = 0; k < 5; ++k) {
-                const double t = warp_sum((lane < C) ? sh.slot5[parity][lane][k] : 0.0);
-                if (lane == 0) sh.tot5[k] = t;
+                const double t5 = warp_sum((lane < C) ? sh.slot5[parity][lane][k] : 0.0);
+                if (lane == 0) sh.tot5[k] = t5;
             }
         }
         __syncthreads();
         parity ^= 1;
     };
 
-    if (tid == 0) { sh.cur = 0; sh.len = 1; sh.path[0] = 0; }
+    // Thread 0 of every CTA (all on identical data, so all take identical steps) walks ahead through
+    // every decision that needs nothing but scalars, and stops only to ask the CTA for a sweep of the
+    // current node's rows.  enter() makes a node the current one.
+    auto enter = [&](int node) {
+        sh.cur = node;
+        sh.m = (double)sh.rowM[node];
+        sh.S = sh.rowS[node];
+        sh.invS = sh.rowInvS[node];
+        sh.exact = 0; sh.have_e = 0; sh.have_q = 0;
+        sh.c = 0.0; sh.U = 1.0; sh.D = 1.0;
+        sh.nrem = 0;
+        sh.bonus_ok = 0;
+        sh.rem = sh.child_mask[node];
+    };
+    if (tid == 0) { sh.len = 1; sh.path[0] = 0; sh.invT = invT; enter(0); }
     double last_a = 0.0;                         // this thread's sum of weights in the latest residual sweep
-    __syncthreads();
 
-    for (;;) {   // one iteration per node on the path
+    for (;;) {
+        if (tid == 0) {
+            int req = REQ_DONE;
+            while (sh.rem != 0ull) {
+                const int ch = __ffsll((long long)sh.rem) - 1;
+                const int xt = sh.tok[ch];
+                const double r = (double)sh.cu[ch];
+                const double qx = (double)sh.cq[ch];
+                const double ex = sh.cex[ch];
+                int ridx = -1;
+                for (int k = 0; k < sh.nrem; ++k) if (sh.rem_tok[k] == xt) ridx = k;
+                // accept iff r * q_k(x) < p_k(x) with q_k = qx / D and p_k = u / U: compared as
+                // r * qx * U < u * D (both normalisers are positive), so no division is needed
+                const double u = (ridx >= 0) ? sh.rem_frozen[ridx] : weight(ex, qx, sh.invS, sh.c);
+                const double lhs = (ridx >= 0) ? 0.0 : r * qx * sh.U;
+                const double rhs = u * sh.D;
+                const bool acc = lhs < rhs;
+                if (!sh.exact) {
+                    // the scan's sum of exponentials is trusted only outside a margin around the boundary
+                    const double big = fmax(lhs, rhs);
+                    if (big > 0.0 && fabs(lhs - rhs) <= kAmbiguous * big) {
+                        req = acc ? REQ_EXP : REQ_EXP_Q;      // exact denominator first (and park the draft row if a rejection is likely)
+                        break;
+                    }
+                }
+                if (acc) {
+                    sh.path[sh.len++] = ch;
+                    enter(ch);
+                    continue;
+                }
+                // rejected: one sweep gives the new residual mass and the new draft mass
+                sh.ex = ex; sh.qx = qx; sh.ridx = ridx; sh.xnew = xt;
+                sh.cprime = sh.c + sh.U / sh.D;
+                req = sh.exact ? REQ_RESID : REQ_FUSED;       // first rejection at a node: exact denominator and residual in one sweep
+                break;
+            }
+            sh.req = req;
+            if (req != REQ_DONE) {
+                sh.req_child = __ffsll((long long)sh.rem) - 1;
+                sh.req_last = ((sh.rem & (sh.rem - 1)) == 0ull) ? 1 : 0;
+            }
+        }
+        __syncthreads();
+        const int req = sh.req;
+        if (req == REQ_DONE) break;                           // uniform
         const int cur = sh.cur;
         const float *x = lg + (size_t)cur * V;
         const float *q = dp + (size_t)cur * V;
-        if (tid == 0) {
-            sh.m = (double)sh.rowM[cur];
-            sh.S = sh.rowS[cur];
-            sh.invS = sh.rowInvS[cur];
-            sh.invT = invT;
-            sh.exact = 0; sh.have_e = 0; sh.have_q = 0;
-            sh.c = 0.0; sh.U = 1.0; sh.D = 1.0;
-            sh.nrem = 0;
-            sh.next = -1;
-            sh.bonus_ok = 0;
-        }
-        __syncthreads();
-
-        for (unsigned long long rem = sh.child_mask[cur]; rem; rem &= rem - 1) {   // uniform: shared data
-            const int ch = __ffsll((long long)rem) - 1;
-            const int xt = sh.tok[ch];
-            for (int attempt = 0; attempt < 2; ++attempt) {
-                if (tid == 0) {
-                    const double r = (double)sh.cu[ch];
-                    const double qx = (double)sh.cq[ch];
-                    const double ex = sh.cex[ch];
-                    int ridx = -1;
-                    for (int k = 0; k < sh.nrem; ++k) if (sh.rem_tok[k] == xt) ridx = k;
-                    // accept iff r * q_k(x) < p_k(x) with q_k = qx / D and p_k = u / U: compared as
-                    // r * qx * U < u * D (both normalisers are positive), so no division is needed
-                    const double u = (ridx >= 0) ? sh.rem_frozen[ridx] : weight(ex, qx, sh.invS, sh.c);
-                    const double lhs = (ridx >= 0) ? 0.0 : r * qx * sh.U;
-                    const double rhs = u * sh.D;
-                    int dec = (lhs < rhs) ? 1 : 0;
-                    sh.want_q = (dec == 0);
-                    if (!sh.exact) {
-                        const double big = fmax(lhs, rhs);
-                        if (big > 0.0 && fabs(lhs - rhs) <= kAmbiguous * big) dec = 2;
-                        else if (dec == 0) dec = 3;      // clear rejection: exact denominator and residual in one sweep
-                    }
-                    sh.decision = dec;
-                    sh.ex = ex; sh.qx = qx; sh.ridx = ridx; sh.xnew = xt;
-                }
-                __syncthreads();
-                if (sh.decision != 2) break;                  // 0, 1 or 3
-                // exact softmax denominator of this node (parks e_j in shared memory)
-                const bool with_q = sh.want_q != 0;
-                Sweep s = sweep_chunk<MODE_EXP>(sh, x, q, se, sq, tid, nthr, lo, hi, vec, cache_ok, false, false, 0.0,
-                                                with_q ? -2 : -1, false, 0, 0, 0, nullptr);
-                reduce_exchange(s.a, 0.0);
-                if (tid == 0) {
-                    sh.S = sh.tot[0]; sh.invS = 1.0 / sh.S; sh.exact = 1; sh.have_e = cache_ok;
-                    if (with_q) sh.have_q = cache_ok;
-                }
-                __syncthreads();
-            }
-            if (sh.decision == 1) {
-                if (tid == 0) sh.next = ch;
-                __syncthreads();
-                break;
-            }
-            // -- rejected: one sweep gives the new residual mass and the new draft mass
-            if (tid == 0) sh.cprime = sh.c + sh.U / sh.D;
-            __syncthreads();
-            const bool last_child = (rem & (rem - 1)) == 0;
-            bool fused_done = false;
-            if (sh.decision == 3) {
-                // first rejection at this node, nothing exact yet (c = 0, U = D = 1, nothing removed)
-                const double cp = sh.cprime;
-                const Sweep5 f = fused_reject_sweep(sh, x, q, se, sq, tid, nthr, lo, hi, vec, cache_ok, sh.invS, cp, xt);
-                reduce_exchange5(f);
-                if (tid == 0) {
-                    const double S = sh.tot5[0], invS = 1.0 / S;
-                    const double W = sh.tot5[1] * invS - cp * sh.tot5[2];
-                    sh.S = S; sh.invS = invS; sh.exact = 1; sh.have_e = cache_ok; sh.have_q = cache_ok;
-                    sh.fused_fallback = !(W > 0.0 && kScanRel * sh.tot5[4] <= kFusedTol * W);
-                    if (!sh.fused_fallback) {
-                        sh.tot[0] = W;
-                        sh.tot[1] = sh.tot5[3];
-                    }
-                }
-                __syncthreads();
-                fused_done = !sh.fused_fallback;
-                if (fused_done) last_a = f.v[1] * sh.invS - cp * f.v[2];
-            }
-            if (!fused_done) {
-                Sweep s = sweep_chunk<MODE_RESID>(sh, x, q, se, sq, tid, nthr, lo, hi, vec, cache_ok, sh.have_e != 0,
-                                                  sh.have_q != 0, sh.cprime, xt, false, 0, 0, 0, nullptr);
-                last_a = s.a;
-                reduce_exchange(s.a, s.b);
-            }
-            // When this was the node's last child, the weights just summed (residual at the new
-            // coefficient, the rejected tokens at their frozen values) are the ones the bonus token is
-            // drawn from, thread by thread in the same order: the draw reuses the sums (last_a).
+        if (req == REQ_EXP || req == REQ_EXP_Q) {
+            // exact softmax denominator of this node (parks e_j in shared memory)
+            const bool with_q = req == REQ_EXP_Q;
+            Sweep sw = sweep_chunk<MODE_EXP>(sh, x, q, se, sq, tid, nthr, lo, hi, vec, cache_ok, false, false, 0.0,
+                                             with_q ? -2 : -1, false, 0, 0, 0, nullptr);
+            reduce_exchange(sw.a, 0.0);
             if (tid == 0) {
-                const double W = sh.tot[0], Dn = sh.tot[1];
-                double frozen;
-                if (W > 0.0) {
-                    frozen = weight(sh.ex, sh.qx, sh.invS, sh.cprime);
-                    sh.c = sh.cprime;
-                    sh.U = W;
-                    sh.bonus_ok = last_child ? 1 : 0;
-                } else {
-                    frozen = weight(sh.ex, sh.qx, sh.invS, sh.c);   // residual vanished: p is kept
+                sh.S = sh.tot[0]; sh.invS = 1.0 / sh.S; sh.exact = 1; sh.have_e = cache_ok;
+                if (with_q) sh.have_q = cache_ok;
+            }
+            continue;                                         // thread 0 repeats the test with the exact sum
+        }
+        const int xt = sh.xnew;
+        bool fused_done = false;
+        if (req == REQ_FUSED) {
+            // first rejection at this node, nothing exact yet (c = 0, U = D = 1, nothing removed)
+            const double cp = sh.cprime;
+            const Sweep5 f = fused_reject_sweep(sh, x, q, se, sq, tid, nthr, lo, hi, vec, cache_ok, sh.invS, cp, xt);
+            reduce_exchange5(f);
+            if (tid == 0) {
+                const double S = sh.tot5[0], invS = 1.0 / S;
+                const double W = sh.tot5[1] * invS - cp * sh.tot5[2];
+                sh.S = S; sh.invS = invS; sh.exact = 1; sh.have_e = cache_ok; sh.have_q = cache_ok;
+                sh.fused_fallback = !(W > 0.0 && kScanRel * sh.tot5[4] <= kFusedTol * W);
+                if (!sh.fused_fallback) {
+                    sh.tot[0] = W;
+                    sh.tot[1] = sh.tot5[3];
                 }
-                if (sh.ridx < 0 && sh.nrem < FSPAD_MAX_NODES) {
-                    sh.rem_tok[sh.nrem] = xt;
-                    sh.rem_frozen[sh.nrem] = frozen;
-                    sh.nrem++;
-                }
-                if (Dn > 0.0) sh.D = Dn;
-                sh.have_q = cache_ok;
             }
             __syncthreads();
+            fused_done = !sh.fused_fallback;
+            // (the exact sum is taken from the exchange's result, which nothing rewrites before the next
+            // exchange; thread 0 may already be changing the walk's state)
+            if (fused_done) last_a = f.v[1] * (1.0 / sh.tot5[0]) - cp * f.v[2];
         }
-
-        if (sh.next < 0) break;                           // uniform
+        if (!fused_done) {
+            Sweep sw = sweep_chunk<MODE_RESID>(sh, x, q, se, sq, tid, nthr, lo, hi, vec, cache_ok, sh.have_e != 0,
+                                               sh.have_q != 0, sh.cprime, xt, false, 0, 0, 0, nullptr);
+            last_a = sw.a;
+            reduce_exchange(sw.a, sw.b);
+        }
+        // When this was the node's last child, the weights just summed (residual at the new
+        // coefficient, the rejected tokens at their frozen values) are the ones the bonus token is
+        // drawn from, thread by thread in the same order: the draw reuses the sums (last_a).
         if (tid == 0) {
-            sh.path[sh.len++] = sh.next;
-            sh.cur = sh.next;
+            const double W = sh.tot[0], Dn = sh.tot[1];
+            double frozen;
+            if (W > 0.0) {
+                frozen = weight(sh.ex, sh.qx, sh.invS, sh.cprime);
+                sh.c = sh.cprime;
+                sh.U = W;
+                sh.bonus_ok = sh.req_last;
+            } else {
+                frozen = weight(sh.ex, sh.qx, sh.invS, sh.c);   // residual vanished: p is kept
+            }
+            if (sh.ridx < 0 && sh.nrem < FSPAD_MAX_NODES) {
+                sh.rem_tok[sh.nrem] = xt;
+                sh.rem_frozen[sh.nrem] = frozen;
+                sh.nrem++;
+            }
+            if (Dn > 0.0) sh.D = Dn;
+            sh.have_q = cache_ok;
+            sh.rem &= sh.rem - 1;                               // this child is done
         }
-        __syncthreads();
+        // no barrier here: only thread 0 touches the walk's state until the next request is published
     }
 
     // ---- bonus token: inverse CDF of the current residual at the last node ----
@@ -624,86 +664,210 @@ accept_walk_kernel(const WalkArgs args)
         const float *q = dp + (size_t)cur * V;
         const double c = sh.c;
         const bool have_e = sh.have_e != 0, have_q = sh.have_q != 0;
-        // with nothing rejected at this node (c == 0) the weights are the e_j themselves and the
-        // denominator cancels, so no separate exact-sum sweep is needed
-        Sweep s{last_a, 0.0};
-        if (!sh.bonus_ok)
-            s = sweep_chunk<MODE_CDF>(sh, x, q, se, sq, tid, nthr, lo, hi, vec, cache_ok, have_e, have_q, c, -1, false, 0, 0,
-                                      0, nullptr);
-        // block-wide inclusive scan of the per-thread sums (index order)
-        double incl = s.a;
         const int lane = tid & 31, wid = tid >> 5;
-#pragma unroll
-        for (int off = 1; off < 32; off <<= 1) {
-            const double t = __shfl_up_sync(0xffffffffu, incl, off);
-            if (lane >= off) incl += t;
-        }
-        const double prev_incl = __shfl_up_sync(0xffffffffu, incl, 1);
-        if (lane == 31) sh.warp_a[wid] = incl;
-        __syncthreads();
-        if (wid == 0) {
-            // exclusive scan of the warp totals; the last inclusive value is the CTA total
-            const int nwarps = nthr >> 5;
-            const double v = (lane < nwarps) ? sh.warp_a[lane] : 0.0;
-            double sc = v;
+
+        // block-wide scan of one value per thread (index order): this thread's exclusive and inclusive
+        // prefix, the CTA total in sh.warp_a[kWarps - 1] ... returned through `total` (valid in every thread)
+        auto block_scan = [&](double v, double &excl_out, double &incl_out, double &total) {
+            double incl = v;
 #pragma unroll
             for (int off = 1; off < 32; off <<= 1) {
-                const double t = __shfl_up_sync(0xffffffffu, sc, off);
-                if (lane >= off) sc += t;
+                const double t2 = __shfl_up_sync(0xffffffffu, incl, off);
+                if (lane >= off) incl += t2;
             }
-            const double excl = __shfl_up_sync(0xffffffffu, sc, 1);
-            if (lane < nwarps) sh.warp_off[lane] = (lane == 0) ? 0.0 : excl;
-            // the CTA total goes to every CTA of the cluster (remote stores; read locally after the barrier)
-            const double total = __shfl_sync(0xffffffffu, sc, nwarps - 1);
-            if (lane < C) *cluster.map_shared_rank(&sh.cta_total[rank], lane) = total;
-        }
-        __syncthreads();
-        const double woff = sh.warp_off[wid];
-        const double P = woff + incl;
-        const double E = (lane == 0) ? woff : woff + prev_incl;
-        cluster.sync();
-        double Z = 0.0, base = 0.0;
-        for (int r = 0; r < C; ++r) {
-            if (r == rank) base = Z;
-            Z = Z + sh.cta_total[r];
-        }
-        const double target = (double)sh.ubonus * Z;
-        int owner = -1;
-        {
-            double cum = 0.0;
-            for (int r = 0; r < C; ++r) {
-                cum = cum + sh.cta_total[r];
-                if (cum > target) { owner = r; break; }
+            const double prev_incl = __shfl_up_sync(0xffffffffu, incl, 1);
+            if (lane == 31) sh.warp_a[wid] = incl;
+            __syncthreads();
+            if (wid == 0) {
+                // exclusive scan of the warp totals; the last inclusive value is the CTA total
+                const int nwarps = nthr >> 5;
+                const double wv = (lane < nwarps) ? sh.warp_a[lane] : 0.0;
+                double sc = wv;
+#pragma unroll
+                for (int off = 1; off < 32; off <<= 1) {
+                    const double t2 = __shfl_up_sync(0xffffffffu, sc, off);
+                    if (lane >= off) sc += t2;
+                }
+                const double excl = __shfl_up_sync(0xffffffffu, sc, 1);
+                if (lane < nwarps) sh.warp_off[lane] = (lane == 0) ? 0.0 : excl;
+                if (lane == nwarps - 1) sh.warp_b[0] = sc;
+            }
+            __syncthreads();
+            const double woff = sh.warp_off[wid];
+            incl_out = woff + incl;
+            excl_out = (lane == 0) ? woff : woff + prev_incl;
+            total = sh.warp_b[0];
+        };
+
+        // A draw at a node where nothing was rejected (a leaf, typically) is taken from the softmax
+        // of the row itself.  The scan left the mass of every piece of the row, accurate to kScanRel:
+        // enough to name the piece the target falls into and the mass in front of it.  That piece is
+        // then swept with single-precision exponentials - by every CTA on its own, all on the same
+        // data with the same arithmetic, so all reach the same verdict and nothing is exchanged - and
+        // the token is taken when the target clears both ends of its interval by more than the
+        // uncertainty of all the approximations together.  Otherwise, and for every other kind of
+        // draw, the cluster sweeps the whole row exactly.
+        bool settled = false;
+        const int n_piece = sh.piece_cnt[cur];
+        if (!sh.bonus_ok && c == 0.0 && sh.nrem == 0 && n_piece > 0) {
+            double Zs = 0.0;
+            for (int i = 0; i < n_piece; ++i) Zs += sh.piece_w[cur][i];
+            const double target = (double)sh.ubonus * Zs;
+            int pick = -1;
+            double pre = 0.0;
+            for (int i = 0; i < n_piece; ++i) {
+                const double nxt = pre + sh.piece_w[cur][i];
+                if (nxt > target) { pick = i; break; }
+                pre = nxt;
+            }
+            // error budget: the masses in front of the piece and the total (scan, kScanRel each, doubled
+            // for slack) and the single-precision sums inside the piece (argument rounding of the
+            // exponential 1.3e-7 per unit of |log2 e_j|, the approximation itself 2.4e-7, the partial sums)
+            const double tol = 4.0 * kScanRel * Zs + (pick >= 0 ? 4e-6 * sh.piece_w[cur][pick] : 0.0);
+            if (pick >= 0 && target - pre > tol && pre + sh.piece_w[cur][pick] - target > tol) {
+                // token range of that piece: CTA `first + pick` of the scan, clipped to the row
+                const FspadStatsGeom &g = args.geom;
+                const long long row_lo = (long long)(b * N + cur) * g.upr;
+                const long long first = row_lo / g.chunk;
+                const long long u_lo = max(row_lo, (first + pick) * g.chunk), u_hi = min(row_lo + g.upr, (first + pick + 1) * g.chunk);
+                const int p_lo = (int)(u_lo - row_lo) * g.unit, p_hi = (int)(u_hi - row_lo) * g.unit;
+                const int pt = ((((p_hi - p_lo) + nthr - 1) / nthr) + 3) & ~3;
+                const int t_lo = min(p_hi, p_lo + tid * pt), t_hi = min(p_hi, t_lo + pt);
+                const float Mf = sh.rowM[cur];
+                // weights relative to the row maximum, as the table's: e_j = exp2((x_j - max) * log2(e) / T)
+                auto e32 = [&](float xv2) {
+                    float y;
+                    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"((xv2 - Mf) * kT));
+                    return xv2 == -INFINITY ? 0.f : y;
+                };
+                double mine = 0.0;
+                for (int j = t_lo; j < t_hi; j += 4) {
+                    float xs[4];
+                    if (vec && j + 4 <= t_hi) {
+                        const float4 t4 = __ldg(reinterpret_cast<const float4 *>(x + j));
+                        xs[0] = t4.x; xs[1] = t4.y; xs[2] = t4.z; xs[3] = t4.w;
+                    } else {
+#pragma unroll
+                        for (int t2 = 0; t2 < 4; ++t2) xs[t2] = (j + t2 < t_hi) ? x[j + t2] : -INFINITY;
+                    }
+                    mine += (double)((e32(xs[0]) + e32(xs[1])) + (e32(xs[2]) + e32(xs[3])));
+                }
+                double E, P, total;
+                block_scan(mine, E, P, total);
+                const double tgt = target - pre;                  // within the piece
+                if (tid == 0) { sh.sel = 0x7fffffff; sh.verdict[0] = 2; }
+                __syncthreads();
+                if (P > tgt) atomicMin(&sh.sel, tid);
+                __syncthreads();
+                if (tid == sh.sel) {
+                    double run = E;
+                    for (int j = t_lo; j < t_hi; ++j) {
+                        const double before = run;
+                        run += (double)e32(x[j]);
+                        if (run > tgt) {
+                            if (tgt - before > tol && run - tgt > tol) {
+                                sh.verdict[0] = 1;
+                                if (rank == 0) args.bonus[b] = j;
+                            }
+                            break;
+                        }
+                    }
+                }
+                __syncthreads();
+                settled = sh.verdict[0] == 1;
             }
         }
-        if (owner == rank) {
-            // the first thread (index order) whose inclusive prefix passes the target owns the draw
-            if (tid == 0) sh.sel = 0x7fffffff;
-            __syncthreads();
-            if (base + P > target) atomicMin(&sh.sel, tid);
-            __syncthreads();
-            // rounding of the two-level prefix can leave no thread above the target although the
-            // CTA total is: the last non-empty chunk then takes the draw
-            if (tid == 0 && sh.sel == 0x7fffffff) sh.sel = max(0, (cta_hi - cta_lo - 1) / per_thr);
-            __syncthreads();
-            if (tid == sh.sel) {
-                int found = -1;
-                sweep_chunk<MODE_CDF>(sh, x, q, se, sq, tid, nthr, lo, hi, vec, false, cache_ok, cache_ok && (c != 0.0),
-                                      c, -1, true, base, E, target, &found);
-                if (found < 0) found = min(lo, V - 1);
-                args.bonus[b] = found;
-            }
-        }
-        if (owner < 0 && rank == 0 && tid == 0) args.bonus[b] = 0;   // no positive weight anywhere
         if (rank == 0) {
             if (tid == 0) args.n_acc[b] = sh.len;
             for (int i = tid; i < args.path_stride; i += nthr) out_path[i] = (i < sh.len) ? sh.path[i] : -1;
         }
-        // no CTA touches a peer's shared memory after the barrier above, so each may leave on its own
+        if (settled) return;                                // uniform over the cluster; no peer memory is touched after the walk's last exchange
+
+        // ---- exact draw over the whole row: every CTA a contiguous slice, every thread a contiguous chunk ----
+        {
+            // with nothing rejected at this node (c == 0) the weights are the e_j themselves and the
+            // denominator cancels, so no separate exact-sum sweep is needed
+            Sweep sw{last_a, 0.0};
+            if (!sh.bonus_ok)
+                sw = sweep_chunk<MODE_CDF>(sh, x, q, se, sq, tid, nthr, lo, hi, vec, cache_ok, have_e, have_q, c, -1, false, 0, 0,
+                                           0, nullptr);
+            double E, P, total;
+            block_scan(sw.a, E, P, total);
+            // the CTA total goes to every CTA of the cluster (remote stores; read locally after the barrier)
+            if (tid < C) *cluster.map_shared_rank(&sh.cta_total[0][rank], tid) = total;
+            cluster.sync();
+            double Z = 0.0, base = 0.0;
+            for (int r = 0; r < C; ++r) {
+                if (r == rank) base = Z;
+                Z = Z + sh.cta_total[0][r];
+            }
+            const double target = (double)sh.ubonus * Z;
+            int owner = -1;
+            {
+                double cum = 0.0;
+                for (int r = 0; r < C; ++r) {
+                    cum = cum + sh.cta_total[0][r];
+                    if (cum > target) { owner = r; break; }
+                }
+            }
+            if (owner == rank) {
+                // the first thread (index order) whose inclusive prefix passes the target owns the draw
+                if (tid == 0) sh.sel = 0x7fffffff;
+                __syncthreads();
+                if (base + P > target) atomicMin(&sh.sel, tid);
+                __syncthreads();
+                // rounding of the two-level prefix can leave no thread above the target although the
+                // CTA total is: the last non-empty chunk then takes the draw
+                if (tid == 0 && sh.sel == 0x7fffffff) sh.sel = max(0, (cta_hi - cta_lo - 1) / per_thr);
+                __syncthreads();
+                if (tid == sh.sel) {
+                    int found = -1;
+                    sweep_chunk<MODE_CDF>(sh, x, q, se, sq, tid, nthr, lo, hi, vec, false, cache_ok, cache_ok && (c != 0.0),
+                                          c, -1, true, base, E, target, &found);
+                    if (found < 0) found = min(lo, V - 1);
+                    args.bonus[b] = found;
+                }
+            }
+            if (owner < 0 && rank == 0 && tid == 0) args.bonus[b] = 0;   // no positive weight anywhere
+        }
+        // no CTA touches a peer's shared memory after the cluster barrier above, so each may leave on its own
     }
 }
 
 }  // namespace
+
+// Cluster size of the sampling walk.  Once per context: raise the dynamic shared-memory limit and find
+// the largest cluster the device can co-schedule for this kernel: 16 (opt-in), else 8.  Small
+// vocabularies do not need the whole cluster.  (Halving the clusters of a batch whose CTAs outnumber the
+// SMs was measured and not kept: on 16 sequences, half of them greedy and gone at once, the acceptance
+// took 186 us with clusters of 8 against 143 us with clusters of 16 in two waves.)
+static int walk_cluster_size(fspad_ctx *ctx, int B, int V)
+{
+    if (ctx->walk_cluster == 0) {
+        ctx->walk_cluster = 8;
+        cudaFuncSetAttribute(accept_walk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
+        if (cudaFuncSetAttribute(accept_walk_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) ==
+            cudaSuccess) {
+            cudaLaunchConfig_t probe = {};
+            probe.gridDim = dim3(kMaxCluster);
+            probe.blockDim = dim3(kWalkThreads);
+            probe.dynamicSmemBytes = kSmemBudget;
+            cudaLaunchAttribute at[1];
+            at[0].id = cudaLaunchAttributeClusterDimension;
+            at[0].val.clusterDim.x = kMaxCluster; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+            probe.attrs = at; probe.numAttrs = 1;
+            int n = 0;
+            if (cudaOccupancyMaxActiveClusters(&n, accept_walk_kernel, &probe) == cudaSuccess && n >= 1)
+                ctx->walk_cluster = kMaxCluster;
+        }
+        (void)cudaGetLastError();
+    }
+    int cluster = ctx->walk_cluster;
+    while (cluster > 1 && (V + cluster - 1) / cluster < 2048) cluster >>= 1;
+    return cluster;
+}
+
+int fspad_walk_ctas(fspad_ctx *ctx, int B, int V) { return B * walk_cluster_size(ctx, B, V); }
 
 cudaError_t fspad_launch_accept_walk(fspad_ctx *ctx, const float *logits, const float *draft,
                                      const int *tokens, const int *parent, const float *temperature,
@@ -723,30 +887,7 @@ cudaError_t fspad_launch_accept_walk(fspad_ctx *ctx, const float *logits, const 
     size_t smem = 0;
     if (sampling) {
         threads = kWalkThreads;
-        if (ctx->walk_cluster == 0) {
-            // once per context: raise the dynamic shared-memory limit and find the largest cluster
-            // the device can co-schedule for this kernel: 16 (opt-in), else 8
-            ctx->walk_cluster = 8;
-            cudaFuncSetAttribute(accept_walk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
-            if (cudaFuncSetAttribute(accept_walk_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) ==
-                cudaSuccess) {
-                cudaLaunchConfig_t probe = {};
-                probe.gridDim = dim3(kMaxCluster);
-                probe.blockDim = dim3(kWalkThreads);
-                probe.dynamicSmemBytes = kSmemBudget;
-                cudaLaunchAttribute at[1];
-                at[0].id = cudaLaunchAttributeClusterDimension;
-                at[0].val.clusterDim.x = kMaxCluster; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
-                probe.attrs = at; probe.numAttrs = 1;
-                int n = 0;
-                if (cudaOccupancyMaxActiveClusters(&n, accept_walk_kernel, &probe) == cudaSuccess && n >= 1)
-                    ctx->walk_cluster = kMaxCluster;
-            }
-            (void)cudaGetLastError();
-        }
-        cluster = ctx->walk_cluster;
-        // small vocabularies do not need the whole cluster
-        while (cluster > 1 && (V + cluster - 1) / cluster < 2048) cluster >>= 1;
+        cluster = walk_cluster_size(ctx, B, V);
         const size_t per_cta = (size_t)((((V + cluster - 1) / cluster) + 3) & ~3);
         const size_t per_thr = ((per_cta + kWalkThreads - 1) / kWalkThreads + 3) & ~(size_t)3;
         const size_t need = per_thr * kWalkThreads * (sizeof(double) + sizeof(float));

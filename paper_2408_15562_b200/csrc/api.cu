@@ -299,15 +299,50 @@ int fspad_verify_step(fspad_ctx *ctx, fspad_bf16 *cache, int attn_layer, const f
     const size_t plane = (size_t)batch * c.n_kv_heads * (size_t)c.max_len * FSPAD_HEAD_DIM;
     const fspad_bf16 *kc = cache + (size_t)attn_layer * 2 * plane, *vc = kc + plane;
 
+    // Which of the two goes first.  The acceptance is a streaming scan over every SM followed by a walk
+    // that one cluster per sampling sequence carries out; the attention is one CTA per SM.  When the
+    // attention's CTAs leave a good part of the SMs free, both start at once and the acceptance lives on
+    // the free SMs.  Otherwise the scan goes first on all SMs and the attention is forked behind it, sized
+    // to leave the walk's SMs alone, so that the walk (the longer chain) and the attention run side by side.
+    const int sms = ctx->sm_count;
+    const int G = c.n_q_heads / c.n_kv_heads;
+    const long long attn_ctas = (long long)batch * c.n_kv_heads * ((n_nodes * G + 127) / 128) *
+                                fspad_attn_umma_splits(ctx, n_nodes, batch);
+    const bool may_sample = draft_probs != nullptr;
+    const bool scan_first = may_sample && sms - attn_ctas < sms / 4;
+    int attn_sms = 0;
+    if (scan_first) {
+        const int walk = fspad_walk_ctas(ctx, batch, c.vocab);
+        attn_sms = sms - (walk < sms / 2 ? walk : sms / 2);
+    }
+    cudaError_t ce = cudaSuccess;
+    FspadStatsGeom geom;
+    const int rows = batch * n_nodes;
+    if (scan_first)
+        ce = fspad_launch_stats_partials(ctx, target_logits, temperature, rows, n_nodes, c.vocab, &geom, st);
     // fork: the attention of this step on the context's second stream
-    if (cudaEventRecord(ctx->ev_fork, st) != cudaSuccess || cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0) != cudaSuccess)
+    if (ce != cudaSuccess || cudaEventRecord(ctx->ev_fork, st) != cudaSuccess ||
+        cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0) != cudaSuccess)
         return FSPAD_ERR_CUDA;
-    int rc_attn = fspad_tree_attn(ctx, q, kc, vc, tree_k, tree_v, parent, prefix_len, n_nodes, batch, attn_out, ctx->side);
+    int rc_attn = FSPAD_OK;
+    if (!scan_first) {
+        rc_attn = fspad_launch_tree_attn(ctx, q, kc, vc, tree_k, tree_v, parent, prefix_len, n_nodes, batch, attn_out,
+                                         ctx->side, 0) == cudaSuccess ? FSPAD_OK : FSPAD_ERR_CUDA;
+        // Here the scan is launched as a plain dependent: as a programmatic dependent of the previous
+        // step's last kernel it was seen to hold the forked attention back behind the whole acceptance
+        // (steps replayed from one CUDA graph: 72.5 us per step against 48.8 on the 52-head shape).
+        ce = fspad_launch_stats_partials(ctx, target_logits, temperature, rows, n_nodes, c.vocab, &geom, st, false);
+    }
+    if (ce == cudaSuccess)
+        ce = fspad_launch_accept_walk(ctx, target_logits, draft_probs, draft_tokens, parent, temperature, uniforms, geom,
+                                      n_nodes, batch, c.vocab, accepted_path, n_accepted, bonus_token, st);
+    rc = ce == cudaSuccess ? FSPAD_OK : FSPAD_ERR_CUDA;
+    if (scan_first)
+        rc_attn = fspad_launch_tree_attn(ctx, q, kc, vc, tree_k, tree_v, parent, prefix_len, n_nodes, batch, attn_out,
+                                         ctx->side, attn_sms) == cudaSuccess ? FSPAD_OK : FSPAD_ERR_CUDA;
     // the join is queued whatever happened in between, so that a capture of `stream` never ends
     // with the second stream left unjoined
     const bool ev_ok = cudaEventRecord(ctx->ev_join, ctx->side) == cudaSuccess;
-    rc = fspad_tree_accept(ctx, target_logits, draft_probs, draft_tokens, parent, temperature, uniforms, n_nodes, batch,
-                           accepted_path, n_accepted, bonus_token, stream);
     const bool aliased = tree_k == nullptr;      // attention reads the cache rows that compaction rewrites
     bool joined = false;
     if (aliased) joined = cudaStreamWaitEvent(st, ctx->ev_join, 0) == cudaSuccess;

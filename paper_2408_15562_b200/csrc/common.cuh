@@ -12,6 +12,7 @@
 #define FSPAD_MAX_CANDIDATES 1024
 #define FSPAD_MAX_FRONTIER 16      /* frontier nodes per sequence, and top-k per row, of a draft step */
 #define FSPAD_HEAD_DIM 128
+#define FSPAD_STATS_THREADS 512     /* threads per CTA of the vocabulary scan */
 
 // Scratch and bookkeeping owned by a context (all device pointers unless noted).
 struct fspad_ctx {
@@ -80,8 +81,8 @@ static inline FspadStatsGeom fspad_stats_geom(int sm_count, int rows, int V, boo
     g.upr = V / g.unit;
     g.slots = slots;
     g.total = (long long)rows * g.upr;
-    long long n = (long long)sm_count * 4;                 // four 256-thread CTAs per SM, one wave
-    const long long by_size = (g.total + 255) / 256;       // at least one unit per thread
+    long long n = (long long)sm_count * 2;                 // two 512-thread CTAs per SM, one wave
+    const long long by_size = (g.total + FSPAD_STATS_THREADS - 1) / FSPAD_STATS_THREADS;   // at least one unit per thread
     if (n > by_size) n = by_size;
     if (n < 1) n = 1;
     g.chunk = (g.total + n - 1) / n;
@@ -136,10 +137,14 @@ __device__ __forceinline__ void fspad_stats_merge_warp(const FspadStatsPart *__r
 
 // The same merge by a half-warp (16 lanes, up to four slots per lane), so that one warp
 // serves two rows at once.  Both halves of the warp must call it together; `valid` is false
-// for a half that has no row (it only takes part in the shuffles).
+// for a half that has no row (it only takes part in the shuffles).  With `piece_w` given, the
+// mass of each of the row's pieces relative to the row maximum (what it adds to S) is stored
+// there, slot by slot, when the row has at most 16 pieces; *piece_cnt is the number of pieces,
+// or 0 when there are more than 16.
 __device__ __forceinline__ void fspad_stats_merge_half(const FspadStatsPart *__restrict__ parts,
                                                        const FspadStatsGeom &g, int row, bool valid, float k,
-                                                       int lane16, float &M, double &S, int &A)
+                                                       int lane16, float &M, double &S, int &A,
+                                                       double *piece_w = nullptr, int *piece_cnt = nullptr)
 {
     int cnt = 0;
     const FspadStatsPart *p = parts;
@@ -173,8 +178,12 @@ __device__ __forceinline__ void fspad_stats_merge_half(const FspadStatsPart *__r
     }
     double s = 0.0;
 #pragma unroll
-    for (int u = 0; u < 4; ++u)
-        if (mi[u] != -INFINITY) s += (double)si[u] * (double)exp2f((mi[u] - m) * k);
+    for (int u = 0; u < 4; ++u) {
+        const double w = (mi[u] != -INFINITY) ? (double)si[u] * (double)exp2f((mi[u] - m) * k) : 0.0;
+        s += w;
+        if (u == 0 && piece_w != nullptr && valid && lane16 < cnt && cnt <= 16) piece_w[lane16] = w;
+    }
+    if (piece_cnt != nullptr && valid && lane16 == 0) *piece_cnt = (cnt <= 16) ? cnt : 0;
 #pragma unroll
     for (int off = 8; off > 0; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off, 16);
     M = m;
@@ -243,9 +252,11 @@ cudaError_t fspad_launch_accept_walk(fspad_ctx *ctx, const float *logits, const 
                                      const int *tokens, const int *parent, const float *temperature,
                                      const float *uniforms, const FspadStatsGeom &geom, int N, int B, int V,
                                      int *path, int *n_acc, int *bonus, cudaStream_t st);
+// pdl = false: launched as a plain dependent of what precedes it in the stream (griddepcontrol.wait is
+// then a no-op; the guarantee its successor relies on holds either way)
 cudaError_t fspad_launch_stats_partials(fspad_ctx *ctx, const float *logits, const float *temperature,
                                         int rows, int rows_per_seq, int V, FspadStatsGeom *geom,
-                                        cudaStream_t st);
+                                        cudaStream_t st, bool pdl = true);
 cudaError_t fspad_launch_tree_build(fspad_ctx *ctx, const int *cand_parent, const int *cand_token,
                                     const float *cand_logp, const int *root_token, int n_cand, int n_nodes,
                                     int B, int *parent_out, int *token_out, int *cand_out,
@@ -258,14 +269,16 @@ cudaError_t fspad_launch_draft_expand(fspad_ctx *ctx, const float *logprobs, con
 cudaError_t fspad_launch_kv_compact(fspad_ctx *ctx, fspad_bf16 *cache, const int *path,
                                     const int *n_acc, const int *prefix_len, int B, int *new_len,
                                     cudaStream_t st, bool pdl = true);
+// sms: how many SMs the call may fill with CTAs (0 = all of them)
 cudaError_t fspad_launch_tree_attn(fspad_ctx *ctx, const fspad_bf16 *q, const fspad_bf16 *kc,
                                    const fspad_bf16 *vc, const fspad_bf16 *tk, const fspad_bf16 *tv,
                                    const int *parent, const int *prefix_len, int N, int B,
-                                   fspad_bf16 *out, cudaStream_t st);
+                                   fspad_bf16 *out, cudaStream_t st, int sms = 0);
 cudaError_t fspad_launch_tree_scatter(fspad_ctx *ctx, fspad_bf16 *cache, const fspad_bf16 *tk,
                                       const fspad_bf16 *tv, const int *prefix_len, int N, int B,
                                       cudaStream_t st);
-int fspad_attn_umma_splits(const fspad_ctx *ctx, int N, int B);
+int fspad_attn_umma_splits(const fspad_ctx *ctx, int N, int B, int sms = 0);
+int fspad_walk_ctas(fspad_ctx *ctx, int B, int V);   // CTAs of the sampling walk for B sequences
 cudaError_t fspad_launch_wait_selftest(fspad_ctx *ctx, int polls, cudaStream_t st);
 cudaError_t fspad_launch_attn_umma_split(fspad_ctx *ctx, const fspad_bf16 *q, const fspad_bf16 *kc,
                                          const fspad_bf16 *vc, const fspad_bf16 *tk, const fspad_bf16 *tv,

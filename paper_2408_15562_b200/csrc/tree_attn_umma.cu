@@ -691,12 +691,13 @@ cudaError_t fspad_launch_wait_selftest(fspad_ctx *ctx, int polls, cudaStream_t s
                             (uint32_t)polls);
 }
 
-int fspad_attn_umma_splits(const fspad_ctx *ctx, int N, int B)
+int fspad_attn_umma_splits(const fspad_ctx *ctx, int N, int B, int sms)
 {
+    if (sms <= 0 || sms > ctx->sm_count) sms = ctx->sm_count;
     const int G = ctx->cfg.n_q_heads / ctx->cfg.n_kv_heads;
     const int mtiles = (N * G + umma::BM - 1) / umma::BM;
     const long long base = (long long)B * ctx->cfg.n_kv_heads * mtiles;
-    long long s = ctx->sm_count / base;           // one CTA per SM, never a partial second wave
+    long long s = sms / base;                     // one CTA per SM, never a partial second wave
     const int max_chunks = (ctx->cfg.max_len + umma::BK - 1) / umma::BK;
     if (s > max_chunks) s = max_chunks;
     if (s > 64) s = 64;
