@@ -79,6 +79,25 @@ def row_stats(logits: np.ndarray, T: float = 1.0):
     return m, s, a
 
 
+def lm_head_stats(hidden, weight, T: float = 1.0, want_logits: bool = False):
+    """fp64 LM head (hidden [R][H] x weight [V][H]^T, bf16 bit patterns) followed by the row statistics of
+    its logits.  Returns a dict: max, sum, arg, gap (maximum minus runner-up) [R] and, on request, logits [R][V]."""
+    R, H = hidden.shape
+    V, H2 = weight.shape
+    assert H == H2
+    m = np.empty(R, np.float64)
+    s = np.empty(R, np.float64)
+    a = np.empty(R, np.int32)
+    gap = np.empty(R, np.float64)
+    z = np.empty((R, V), np.float64) if want_logits else None
+    rc = lib().oracle_lm_head_stats(_p(hidden, np.uint16), _p(weight, np.uint16), R, H, V, ctypes.c_double(T),
+                                    _p(z, np.float64), _p(m, np.float64), _p(s, np.float64), _p(a, np.int32),
+                                    _p(gap, np.float64))
+    if rc != 0:
+        raise RuntimeError("oracle_lm_head_stats failed: %d" % rc)
+    return {"max": m, "sum": s, "arg": a, "gap": gap, "logits": z}
+
+
 def tree_accept(target_logits, draft_probs, draft_tokens, parent, temperature, uniforms,
                 force: Optional[np.ndarray] = None):
     """Lossless tree acceptance. Returns a dict with accepted_path [B][N] (-1 padded),

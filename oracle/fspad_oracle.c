@@ -137,6 +137,59 @@ int oracle_row_stats(const float *logits, int R, int V, double T, double *row_ma
     return 0;
 }
 
+/* ------------------------------------------------------------------------
+ * Target LM head followed by the per-node vocabulary scan ("Preliminaries":
+ * the target's single forward over the flattened tree yields, for every tree
+ * node, the distribution the acceptance stage compares the tree with).  The
+ * last step of that forward is the product of the final hidden states with the
+ * vocabulary matrix; its rows are the logits the scan above is defined on:
+ *   z[r][v] = sum_h hidden[r][h] * weight[v][h]          (fp64, index order)
+ *   m = max_v z, a = its lowest index, S = sum_v exp((z - m) / T)
+ *   hidden [R][H], weight [V][H]: bf16 bit patterns
+ *   logits (may be NULL) [R][V] double ; row_max, row_sum double [R] ; row_arg int32 [R]
+ *   row_gap (may be NULL) double [R]: m minus the second largest value (ties: 0)
+ * ---------------------------------------------------------------------- */
+int oracle_lm_head_stats(const uint16_t *hidden, const uint16_t *weight, int R, int H, int V, double T,
+                         double *logits, double *row_max, double *row_sum, int32_t *row_arg, double *row_gap)
+{
+    const double Td = T > 0.0 ? T : 1.0;
+    int bad = 0;
+#pragma omp parallel for schedule(dynamic)
+    for (int r = 0; r < R; ++r) {
+        double *z = (double *)malloc((size_t)V * sizeof(double));
+        double *hr = (double *)malloc((size_t)H * sizeof(double));
+        if (!z || !hr) {
+            bad = 1;
+            free(z);
+            free(hr);
+            continue;
+        }
+        for (int h = 0; h < H; ++h) hr[h] = bf16_to_f64(hidden[(size_t)r * H + h]);
+        for (int v = 0; v < V; ++v) {
+            const uint16_t *wv = weight + (size_t)v * H;
+            double acc = 0.0;
+            for (int h = 0; h < H; ++h) acc += hr[h] * bf16_to_f64(wv[h]);
+            z[v] = acc;
+        }
+        double m = -INFINITY, second = -INFINITY;
+        int a = 0;
+        for (int v = 0; v < V; ++v) {
+            if (z[v] > m) { second = m; m = z[v]; a = v; }
+            else if (z[v] > second) second = z[v];
+        }
+        double S = 0.0;
+        for (int v = 0; v < V; ++v) S += exp((z[v] - m) / Td);
+        row_max[r] = m;
+        row_sum[r] = S;
+        row_arg[r] = a;
+        if (row_gap) row_gap[r] = m - second;
+        if (logits) memcpy(logits + (size_t)r * V, z, (size_t)V * sizeof(double));
+        free(z);
+        free(hr);
+    }
+    return bad ? -1 : 0;
+}
+
 /* Inverse-CDF draw: weights w_j >= 0 summed in index order to Z; the token is
  * the smallest j whose running sum exceeds u*Z; if rounding leaves none, the
  * largest j with w_j > 0.  info (may be NULL) receives

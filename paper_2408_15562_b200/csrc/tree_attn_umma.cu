@@ -273,7 +273,22 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
     const int b = blockIdx.z;
     const int N = a.N, G = a.G, M = a.M;
 
+    // The prologue's global loads are independent of one another: the prefix length, this thread's
+    // parent entry and the Q tile are all requested before anything waits for the first of them.
     int L = a.prefix_len[b];
+    const int my_par = (tid < N) ? a.parent[(size_t)b * N + tid] : 0;
+    // 1024-byte aligned tiles: Q | K[NS] | V[NS]
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t sQ = base, sK = base + TILE, sV = base + (1 + NS) * TILE;
+    for (int i = tid; i < BM * 16; i += NT) {
+        const int r = i >> 4, c = i & 15;
+        const int grr = blockIdx.y % a.mtiles * BM + r;
+        const bool ok = grr < M;
+        const int nd = ok ? grr / G : 0, hh = ok ? grr % G : 0;
+        const fspad_bf16 *src = a.q + (((size_t)b * N + nd) * a.Hq + g * G + hh) * D + c * 8;
+        cp_async16(sQ + tile_off(r, c), src, ok);
+    }
+    cp_async_commit();
     if (L < 0 || L + N > a.max_len) {
         if (tid == 0) fspad_report(a.status, FSPAD_ERR_RANGE);
         L = max(0, min(L, a.max_len - N));
@@ -291,12 +306,10 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
 
     if (c0 >= c1) {                               // nothing to do for this split: empty partial
         if (row_ok && grp == 0) { float *ml = a.part_ml + (prow * M + gr) * 2; ml[0] = -INFINITY; ml[1] = 0.f; }
+        cp_async_wait<0>();                       // the Q copies land before the shared memory is given back
         return;
     }
 
-    // 1024-byte aligned tiles: Q | K[NS] | V[NS]
-    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    const uint32_t sQ = base, sK = base + TILE, sV = base + (1 + NS) * TILE;
     const uint32_t bar0 = smem_u32(&s_bar[0]);
     auto kfull = [&](int buf) { return bar0 + 8u * (uint32_t)buf; };
     auto vfull = [&](int buf) { return bar0 + 8u * (uint32_t)(NS + buf); };
@@ -361,23 +374,17 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
             gather(c0 + u, u, true, tid, NT);
         }
     }
-    for (int i = tid; i < BM * 16; i += NT) {
-        const int r = i >> 4, c = i & 15;
-        const int grr = mt * BM + r;
-        const bool ok = grr < M;
-        const int nd = ok ? grr / G : 0, hh = ok ? grr % G : 0;
-        const fspad_bf16 *src = a.q + (((size_t)b * N + nd) * a.Hq + g * G + hh) * D + c * 8;
-        cp_async16(sQ + tile_off(r, c), src, ok);
-    }
-    cp_async_commit();
-    if (tid < N) s_par[tid] = a.parent[(size_t)b * N + tid];
-    __syncthreads();                              // barriers initialised, parents staged
+    cp_async_commit();                            // (gathered chunks, if any)
+    if (tid < N) s_par[tid] = my_par;
     if (warp == 9) {
+        // tensor memory is allocated while the other warps are still issuing copies
         __syncwarp();
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n"
                      :: "r"(smem_u32(&s_tmem)), "r"(TMEM_COLS) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
-    } else if (tid < N) {
+    }
+    __syncthreads();                              // barriers initialised, parents staged
+    if (warp != 9 && tid < N) {
         // tree -> ancestor-or-self masks (parents were staged in shared memory above)
         unsigned long long mask = 0ull;
         int cur = tid;

@@ -407,3 +407,18 @@ def draft_logprob_rows(seed: int, batch: int, n_frontier: int, vocab: int, sigma
     if step > 0:
         lp = np.floor(lp / step) * step
     return lp.astype(np.float32)
+
+
+# --------------------------------------------------------------------------
+# LM-head inputs (final hidden states of the tree nodes, vocabulary matrix)
+# --------------------------------------------------------------------------
+def lm_head_inputs(seed: int, rows: int, hidden: int, vocab: int, sigma_logit: float = 3.0):
+    """Stand-in for the target's final hidden states [rows][hidden] and LM-head matrix [vocab][hidden],
+    both bf16 bit patterns: hidden ~ N(0, 1), weights ~ N(0, sigma_logit^2 / hidden), so that the logits
+    hidden . weight^T are ~ N(0, sigma_logit^2) like the logits of the verify workloads."""
+    rng = np.random.default_rng(24081556200 + 7919 * seed + 13)
+    h = normal_bf16(rng, (rows, hidden))
+    w = f32_to_bf16_bits((rng.standard_normal((vocab, hidden), dtype=np.float32) *
+                          np.float32(sigma_logit / np.sqrt(hidden))))
+    return h, w
+
