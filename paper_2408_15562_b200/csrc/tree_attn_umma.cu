@@ -273,22 +273,7 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
     const int b = blockIdx.z;
     const int N = a.N, G = a.G, M = a.M;
 
-    // The prologue's global loads are independent of one another: the prefix length, this thread's
-    // parent entry and the Q tile are all requested before anything waits for the first of them.
     int L = a.prefix_len[b];
-    const int my_par = (tid < N) ? a.parent[(size_t)b * N + tid] : 0;
-    // 1024-byte aligned tiles: Q | K[NS] | V[NS]
-    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    const uint32_t sQ = base, sK = base + TILE, sV = base + (1 + NS) * TILE;
-    for (int i = tid; i < BM * 16; i += NT) {
-        const int r = i >> 4, c = i & 15;
-        const int grr = blockIdx.y % a.mtiles * BM + r;
-        const bool ok = grr < M;
-        const int nd = ok ? grr / G : 0, hh = ok ? grr % G : 0;
-        const fspad_bf16 *src = a.q + (((size_t)b * N + nd) * a.Hq + g * G + hh) * D + c * 8;
-        cp_async16(sQ + tile_off(r, c), src, ok);
-    }
-    cp_async_commit();
     if (L < 0 || L + N > a.max_len) {
         if (tid == 0) fspad_report(a.status, FSPAD_ERR_RANGE);
         L = max(0, min(L, a.max_len - N));
@@ -306,10 +291,12 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
 
     if (c0 >= c1) {                               // nothing to do for this split: empty partial
         if (row_ok && grp == 0) { float *ml = a.part_ml + (prow * M + gr) * 2; ml[0] = -INFINITY; ml[1] = 0.f; }
-        cp_async_wait<0>();                       // the Q copies land before the shared memory is given back
         return;
     }
 
+    // 1024-byte aligned tiles: Q | K[NS] | V[NS]
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t sQ = base, sK = base + TILE, sV = base + (1 + NS) * TILE;
     const uint32_t bar0 = smem_u32(&s_bar[0]);
     auto kfull = [&](int buf) { return bar0 + 8u * (uint32_t)buf; };
     auto vfull = [&](int buf) { return bar0 + 8u * (uint32_t)(NS + buf); };
@@ -374,17 +361,23 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
             gather(c0 + u, u, true, tid, NT);
         }
     }
-    cp_async_commit();                            // (gathered chunks, if any)
-    if (tid < N) s_par[tid] = my_par;
+    for (int i = tid; i < BM * 16; i += NT) {
+        const int r = i >> 4, c = i & 15;
+        const int grr = mt * BM + r;
+        const bool ok = grr < M;
+        const int nd = ok ? grr / G : 0, hh = ok ? grr % G : 0;
+        const fspad_bf16 *src = a.q + (((size_t)b * N + nd) * a.Hq + g * G + hh) * D + c * 8;
+        cp_async16(sQ + tile_off(r, c), src, ok);
+    }
+    cp_async_commit();
+    if (tid < N) s_par[tid] = a.parent[(size_t)b * N + tid];
+    __syncthreads();                              // barriers initialised, parents staged
     if (warp == 9) {
-        // tensor memory is allocated while the other warps are still issuing copies
         __syncwarp();
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n"
                      :: "r"(smem_u32(&s_tmem)), "r"(TMEM_COLS) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
-    }
-    __syncthreads();                              // barriers initialised, parents staged
-    if (warp != 9 && tid < N) {
+    } else if (tid < N) {
         // tree -> ancestor-or-self masks (parents were staged in shared memory above)
         unsigned long long mask = 0ull;
         int cur = tid;
@@ -622,7 +615,12 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
         const float m_all = fmaxf(ml0.x, ml1.x);
         const float m_fin = (m_all == -INFINITY) ? 0.f : m_all;
         const float f0 = ex2f(ml0.x - m_fin), f1 = ex2f(ml1.x - m_fin);     // exp2(-inf) = 0 for a fully masked half
-        float *po = a.part_o + (prow * M + (row_ok ? gr : 0)) * D + grp * 64;
+        // The merged rows go through shared memory (the K ring is idle by now), so that the global
+        // stores are whole 512-byte rows per warp instead of 32 row-strided pieces per instruction
+        // (every such piece is a transaction of its own: the direct stores cost 3 us per CTA).
+        constexpr int SROW = D + 4;                   // floats per staged row; the pad keeps 16-byte stores conflict-free
+        float *stg = reinterpret_cast<float *>(smem_raw + (base - smem_u32(smem_raw)) + TILE);
+        float *ps = stg + row * SROW + grp * 64;
         const uint32_t tO0 = tmem + lanes + 256u + (uint32_t)grp * 64u, tO1 = tO0 + 128u;
 #pragma unroll
         for (int q2 = 0; q2 < 2; ++q2) {
@@ -631,16 +629,23 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
             tmem_ld32(tO1 + q2 * 32, o1);
 #pragma unroll
             for (int j = 0; j < 32; ++j) o[j] = fmaf(o1[j], f1, o[j] * f0);
-            if (store) {
 #pragma unroll
-                for (int j = 0; j < 32; j += 4)
-                    *reinterpret_cast<float4 *>(po + q2 * 32 + j) = make_float4(o[j], o[j + 1], o[j + 2], o[j + 3]);
-            }
+            for (int j = 0; j < 32; j += 4)
+                *reinterpret_cast<float4 *>(ps + q2 * 32 + j) = make_float4(o[j], o[j + 1], o[j + 2], o[j + 3]);
         }
         if (store && grp == 0) {
             float *ml = a.part_ml + (prow * M + gr) * 2;
             ml[0] = m_all;
             ml[1] = ml0.y * f0 + ml1.y * f1;
+        }
+        asm volatile("bar.sync 1, 256;\n" ::: "memory");   // the eight softmax warps
+        if (!any_fail) {
+            for (int r = warp; r < BM; r += 8) {
+                const int grr = mt * BM + r;
+                if (grr < M)
+                    *reinterpret_cast<float4 *>(a.part_o + (prow * M + grr) * D + lane * 4) =
+                        *reinterpret_cast<const float4 *>(stg + r * SROW + lane * 4);
+            }
         }
         tc_fence_before();
         __syncthreads();
