@@ -208,6 +208,49 @@ int fspad_accept_stats_noalloc(const float *logits, const float *temperature, in
                                int32_t *row_arg, void *stream);
 
 /*
+ * Target LM head with the per-node scan as its epilogue ("Preliminaries": the
+ * target's one forward over the flattened tree yields, for every tree node, the
+ * distribution the tree is compared with; the last step of that forward is the
+ * product of the nodes' final hidden states with the vocabulary matrix).
+ *
+ *   logits[r][v] = sum_h hidden[r][h] * lm_head[v][h]     bf16 inputs, fp32 accumulation
+ *   row_max / row_arg / row_sum of every row of logits as in fspad_accept_stats
+ *
+ * The tiles of the product are reduced to (maximum, lowest index, sum of
+ * exponentials) as they leave the tensor cores; the logits themselves are
+ * written only if logits_out is given.
+ *
+ *   hidden     [rows][hidden_dim] bf16        lm_head [vocab][hidden_dim] bf16 (vocab is the context's)
+ *   hidden_dim a multiple of 8;  rows <= max_batch * max_nodes of the context
+ *   temperature [rows / rows_per_seq] fp32 or NULL (0 -> 1), as in fspad_accept_stats
+ *   logits_out [rows][vocab] fp32 or NULL;  row_max fp32, row_sum fp64, row_arg int32: [rows]
+ * All pointers are device pointers, 16-byte aligned.  Rows are processed in slabs of 128; every slab
+ * streams the vocabulary matrix once.  Accuracy: the products are exact, the fp32 accumulation over
+ * hidden_dim terms leaves an absolute error of about 1e-5 (bounded by hidden_dim / 16 roundings of the
+ * running sum) in every logit, so row_arg is the exact argmax wherever the maximum leads the runner-up
+ * by more than that.
+ */
+int fspad_lm_head_stats(fspad_ctx *ctx, const fspad_bf16 *hidden, const fspad_bf16 *lm_head, int hidden_dim, int rows,
+                        int rows_per_seq, const float *temperature, float *logits_out, float *row_max, double *row_sum,
+                        int32_t *row_arg, void *stream);
+
+/*
+ * fspad_tree_accept fed by the LM head directly ("Preliminaries": forward, then strict comparison):
+ * the logits of fspad_tree_accept are hidden . lm_head^T as in fspad_lm_head_stats, their scan happens
+ * in the product's epilogue, and the acceptance walk follows.  Every other argument, the outputs and
+ * the acceptance rule are those of fspad_tree_accept.
+ *
+ *   hidden [batch][n_nodes][hidden_dim] bf16;  lm_head [vocab][hidden_dim] bf16
+ *   logits [batch][n_nodes][vocab] fp32, written by the call: required when draft_probs is given (the
+ *          sampling walk reads the rows on its path), may be NULL when every temperature is 0, in
+ *          which case no logit is ever written to memory.
+ */
+int fspad_lm_head_accept(fspad_ctx *ctx, const fspad_bf16 *hidden, const fspad_bf16 *lm_head, int hidden_dim,
+                         const float *draft_probs, const int32_t *draft_tokens, const int32_t *parent,
+                         const float *temperature, const float *uniforms, int n_nodes, int batch, float *logits,
+                         int32_t *accepted_path, int32_t *n_accepted, int32_t *bonus_token, void *stream);
+
+/*
  * Dynamic token tree, one draft step ("Preliminaries", last paragraph: the
  * output of each draft step is truncated to its top-k, and every token carries
  * the joint probability of its path).  Called once per level of the draft

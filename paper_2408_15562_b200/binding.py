@@ -19,7 +19,7 @@ _lib = None
 
 EXPORTS = ["fspad_create", "fspad_destroy", "fspad_status", "fspad_strerror", "fspad_launch_count",
            "fspad_tree_attn", "fspad_tree_accept", "fspad_accept_stats", "fspad_kv_compact",
-           "fspad_verify_step", "fspad_verify_step_host", "fspad_selftest_wait_timeout", "fspad_accept_stats_noalloc", "fspad_tree_build", "fspad_draft_expand"]
+           "fspad_lm_head_stats", "fspad_lm_head_accept", "fspad_verify_step", "fspad_verify_step_host", "fspad_selftest_wait_timeout", "fspad_accept_stats_noalloc", "fspad_tree_build", "fspad_draft_expand"]
 
 
 class FspadConfig(ctypes.Structure):
@@ -57,6 +57,8 @@ def load():
     lib.fspad_accept_stats.argtypes = [vp, vp, vp, ci, ci, vp, vp, vp, vp]
     lib.fspad_kv_compact.argtypes = [vp, vp, vp, vp, vp, ci, vp, vp]
     lib.fspad_accept_stats_noalloc.argtypes = [vp, vp, ci, ci, ci, vp, vp, vp, vp]
+    lib.fspad_lm_head_stats.argtypes = [vp, vp, vp, ci, ci, ci, vp, vp, vp, vp, vp, vp]
+    lib.fspad_lm_head_accept.argtypes = [vp, vp, vp, ci, vp, vp, vp, vp, vp, ci, ci, vp, vp, vp, vp, vp]
     lib.fspad_selftest_wait_timeout.argtypes = [vp, ci, vp]
     lib.fspad_verify_step.argtypes = [vp, vp, ci] + [vp] * 10 + [ci, ci] + [vp] * 6
     lib.fspad_verify_step_host.argtypes = [vp] * 12 + [ci, ci] + [vp] * 6
@@ -176,6 +178,43 @@ class Context:
         if rc != 0:
             raise FspadError(rc, "fspad_accept_stats")
         return row_max, row_sum, row_arg
+
+    def lm_head_stats(self, hidden, lm_head, temperature, rows_per_seq, logits_out=None, out=None, stream=None):
+        """hidden [rows][H], lm_head [V][H] (bf16, device) -> (row_max, row_sum, row_arg); logits_out, if given,
+        receives the fp32 logits [rows][V]."""
+        rows, H = hidden.shape
+        dev = hidden.device
+        if out is None:
+            out = (torch.empty((rows,), dtype=torch.float32, device=dev), torch.empty((rows,), dtype=torch.float64, device=dev),
+                   torch.empty((rows,), dtype=torch.int32, device=dev))
+        bf = torch.bfloat16
+        rc = load().fspad_lm_head_stats(self._h, _ptr(hidden, bf), _ptr(lm_head, bf), H, rows, rows_per_seq,
+                                        _ptr(temperature, torch.float32), _ptr(logits_out, torch.float32),
+                                        _ptr(out[0], torch.float32), _ptr(out[1], torch.float64), _ptr(out[2], torch.int32),
+                                        _stream(stream))
+        if rc != 0:
+            raise FspadError(rc, "fspad_lm_head_stats")
+        return out
+
+    def lm_head_accept(self, hidden, lm_head, draft_probs, draft_tokens, parent, temperature, uniforms, logits=None,
+                       accepted_path=None, n_accepted=None, bonus_token=None, stream=None):
+        """hidden [B][N][H] -> acceptance result, the logits' scan fused behind the LM-head product."""
+        B, N, H = hidden.shape
+        dev = hidden.device
+        i32, f32, bf = torch.int32, torch.float32, torch.bfloat16
+        if accepted_path is None:
+            accepted_path = torch.empty((B, self.cfg.max_nodes), dtype=i32, device=dev)
+        if n_accepted is None:
+            n_accepted = torch.empty((B,), dtype=i32, device=dev)
+        if bonus_token is None:
+            bonus_token = torch.empty((B,), dtype=i32, device=dev)
+        rc = load().fspad_lm_head_accept(self._h, _ptr(hidden, bf), _ptr(lm_head, bf), H, _ptr(draft_probs, f32),
+                                         _ptr(draft_tokens, i32), _ptr(parent, i32), _ptr(temperature, f32),
+                                         _ptr(uniforms, f32), N, B, _ptr(logits, f32), _ptr(accepted_path, i32),
+                                         _ptr(n_accepted, i32), _ptr(bonus_token, i32), _stream(stream))
+        if rc != 0:
+            raise FspadError(rc, "fspad_lm_head_accept")
+        return accepted_path, n_accepted, bonus_token
 
     def kv_compact(self, cache, accepted_path, n_accepted, prefix_len, new_len=None, stream=None):
         B = prefix_len.shape[0]

@@ -102,6 +102,7 @@ int fspad_create(const fspad_config *cfg, fspad_ctx **out)
         ok = ok && dev_alloc(&dx, B * FSPAD_MAX_FRONTIER * (size_t)fspad_draft_expand_pieces(cfg->vocab) * FSPAD_MAX_FRONTIER);
         ctx->dx_part = dx;
     }
+    ok = ok && dev_alloc(&ctx->lm_parts, (size_t)128 * fspad_lm_head_tiles(cfg->vocab));
     ok = ok && cudaStreamCreateWithFlags(&ctx->side, cudaStreamNonBlocking) == cudaSuccess;
     ok = ok && cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming) == cudaSuccess;
     ok = ok && cudaEventCreateWithFlags(&ctx->ev_join, cudaEventDisableTiming) == cudaSuccess;
@@ -120,7 +121,7 @@ void fspad_destroy(fspad_ctx *ctx)
 {
     if (!ctx) return;
     cudaDeviceSynchronize();
-    void *ptrs[] = {ctx->dx_part, ctx->d_status, ctx->part_o, ctx->part_ml, ctx->st_part, ctx->row_max, ctx->row_sum, ctx->row_arg, ctx->h_q, ctx->h_tk,
+    void *ptrs[] = {ctx->lm_parts, ctx->dx_part, ctx->d_status, ctx->part_o, ctx->part_ml, ctx->st_part, ctx->row_max, ctx->row_sum, ctx->row_arg, ctx->h_q, ctx->h_tk,
                     ctx->h_tv, ctx->h_out, ctx->h_parent, ctx->h_prefix, ctx->h_tokens, ctx->h_path,
                     ctx->h_nacc, ctx->h_bonus, ctx->h_newlen, ctx->h_logits, ctx->h_draft, ctx->h_temp,
                     ctx->h_unif};
@@ -218,6 +219,48 @@ int fspad_tree_accept(fspad_ctx *ctx, const float *target_logits, const float *d
                                  uniforms, geom, n_nodes, batch, ctx->cfg.vocab, accepted_path, n_accepted,
                                  bonus_token, st);
     return e == cudaSuccess ? FSPAD_OK : FSPAD_ERR_CUDA;
+}
+
+int fspad_lm_head_stats(fspad_ctx *ctx, const fspad_bf16 *hidden, const fspad_bf16 *lm_head, int hidden_dim, int rows,
+                        int rows_per_seq, const float *temperature, float *logits_out, float *row_max, double *row_sum,
+                        int32_t *row_arg, void *stream)
+{
+    if (!ctx) return FSPAD_ERR_NULL;
+    if (!hidden || !lm_head || !row_max || !row_sum || !row_arg) return FSPAD_ERR_NULL;
+    if (misaligned(hidden) || misaligned(lm_head) || misaligned(logits_out)) return FSPAD_ERR_ALIGN;
+    if (hidden_dim < 8 || hidden_dim % 8 != 0 || rows < 0 || rows_per_seq < 1 ||
+        rows > ctx->cfg.max_batch * ctx->cfg.max_nodes)
+        return FSPAD_ERR_SHAPE;
+    if (rows == 0) return FSPAD_OK;
+    return fspad_launch_lm_head(ctx, hidden, lm_head, hidden_dim, rows, rows_per_seq, temperature, logits_out, nullptr,
+                                row_max, row_sum, row_arg, fspad_stream(stream)) == cudaSuccess ? FSPAD_OK : FSPAD_ERR_CUDA;
+}
+
+int fspad_lm_head_accept(fspad_ctx *ctx, const fspad_bf16 *hidden, const fspad_bf16 *lm_head, int hidden_dim,
+                         const float *draft_probs, const int32_t *draft_tokens, const int32_t *parent,
+                         const float *temperature, const float *uniforms, int n_nodes, int batch, float *logits,
+                         int32_t *accepted_path, int32_t *n_accepted, int32_t *bonus_token, void *stream)
+{
+    int rc = check_common(ctx, n_nodes, batch);
+    if (rc) return rc;
+    if (!hidden || !lm_head || !draft_tokens || !parent || !temperature || !accepted_path || !n_accepted || !bonus_token)
+        return FSPAD_ERR_NULL;
+    if ((draft_probs == nullptr) != (uniforms == nullptr)) return FSPAD_ERR_NULL;
+    if (draft_probs != nullptr && logits == nullptr) return FSPAD_ERR_NULL;     // the sampling walk reads logits rows
+    if (misaligned(hidden) || misaligned(lm_head) || misaligned(logits) || misaligned(draft_probs)) return FSPAD_ERR_ALIGN;
+    if (hidden_dim < 8 || hidden_dim % 8 != 0) return FSPAD_ERR_SHAPE;
+    if (batch == 0) return FSPAD_OK;
+    cudaStream_t st = fspad_stream(stream);
+    const int V = ctx->cfg.vocab, rows = batch * n_nodes;
+    const bool vec = (V % 4 == 0);          // logits and draft rows are 16-byte aligned (checked above)
+    const FspadStatsGeom geom = fspad_lm_head_geom(rows, V, vec, ctx->stats_slots);
+    if (fspad_launch_lm_head(ctx, hidden, lm_head, hidden_dim, rows, n_nodes, temperature, logits, &geom, nullptr, nullptr,
+                             nullptr, st) != cudaSuccess)
+        return FSPAD_ERR_CUDA;
+    // a greedy walk needs only the partials; logits may be NULL then, and the walk never reads them
+    return fspad_launch_accept_walk(ctx, logits, draft_probs, draft_tokens, parent, temperature, uniforms, geom, n_nodes,
+                                    batch, V, accepted_path, n_accepted, bonus_token, st) == cudaSuccess
+               ? FSPAD_OK : FSPAD_ERR_CUDA;
 }
 
 int fspad_kv_compact(fspad_ctx *ctx, fspad_bf16 *cache, const int32_t *accepted_path,

@@ -47,6 +47,10 @@ struct fspad_ctx {
     cudaStream_t side;
     cudaEvent_t ev_fork, ev_join;
 
+    // LM head: per-(row, vocabulary tile) partials of one slab of 128 rows, [128][tiles]
+    struct FspadStatsPart *lm_parts;
+    int lm_attr_done;
+
     void *dx_part;            // draft step: per-piece top-k lists [max_batch * 16 rows][pieces][16] (value, token)
 
     // device staging for the host entry point (h_ready: every buffer below is allocated)
@@ -278,6 +282,13 @@ cudaError_t fspad_launch_tree_scatter(fspad_ctx *ctx, fspad_bf16 *cache, const f
                                       const fspad_bf16 *tv, const int *prefix_len, int N, int B,
                                       cudaStream_t st);
 int fspad_attn_umma_splits(const fspad_ctx *ctx, int N, int B, int sms = 0);
+int fspad_lm_head_tiles(int V);
+FspadStatsGeom fspad_lm_head_geom(int rows, int V, bool vec, int slots);
+// LM head over R rows; with walk_geom the merged partials go to the context's scan scratch in that
+// geometry (for the acceptance walk), otherwise to row_max / row_sum / row_arg
+cudaError_t fspad_launch_lm_head(fspad_ctx *ctx, const fspad_bf16 *hidden, const fspad_bf16 *weight, int H, int R,
+                                 int rows_per_seq, const float *temperature, float *logits, const FspadStatsGeom *walk_geom,
+                                 float *row_max, double *row_sum, int *row_arg, cudaStream_t st);
 int fspad_walk_ctas(fspad_ctx *ctx, int B, int V);   // CTAs of the sampling walk for B sequences
 cudaError_t fspad_launch_wait_selftest(fspad_ctx *ctx, int polls, cudaStream_t st);
 cudaError_t fspad_launch_attn_umma_split(fspad_ctx *ctx, const fspad_bf16 *q, const fspad_bf16 *kc,
