@@ -186,6 +186,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-verify", action="store_true", help="skip the oracle check of the timed step")
+    ap.add_argument("--no-lm-head", action="store_true", help="skip the LM-head leg (a vocabulary matrix of 2*H*V bytes)")
     args = ap.parse_args()
     w = synth.WORKLOADS[args.workload]
     if args.impl == "reference":
@@ -345,6 +346,24 @@ def main():
     dx_next = (torch.empty((B, DK), dtype=torch.int32, device="cuda"), torch.empty((B, DK), dtype=torch.float32, device="cuda"))
     draft_expand_us, _ = timed(lambda i: ctx.draft_expand(dlp[i % len(dlp)], dfl, dfc, DK, DK, 0, *dx_arr, next_cand=dx_next[0],
                                                           next_logp=dx_next[1]), args.steps, replays=3)
+    # the step in front of the acceptance (not part of `value`): the LM-head product with the scan as its
+    # epilogue, alone and with the acceptance walk behind it; the vocabulary matrix is far larger than L2
+    lm_H = w.n_q_heads * w.head_dim
+    lm = None
+    if not args.no_lm_head:
+        hid_host, wgt_host = synth.lm_head_inputs(w.cfg, B * N, lm_H, w.vocab)
+        d_hid, d_wgt = bf(hid_host).view(B, N, lm_H), bf(wgt_host)
+        lm_logits = torch.empty((B, N, w.vocab), dtype=torch.float32, device="cuda") if inp.draft_probs is not None else None
+        lm_out = (torch.empty(B * N, dtype=torch.float32, device="cuda"), torch.empty(B * N, dtype=torch.float64, device="cuda"),
+                  torch.empty(B * N, dtype=torch.int32, device="cuda"))
+        lm_path, lm_nacc, lm_bonus = torch.empty_like(path), torch.empty_like(n_acc), torch.empty_like(bonus)
+        lm_steps = max(2, min(args.steps, 10))
+        lm_stats_us, lm_stats_min = timed(lambda i: ctx.lm_head_stats(d_hid.view(B * N, lm_H), d_wgt, temp, N, out=lm_out),
+                                          lm_steps, replays=5)
+        lm_accept_us, lm_accept_min = timed(
+            lambda i: ctx.lm_head_accept(d_hid, d_wgt, sets[i % R]["draft"], tokens, parent, temp, unif, logits=lm_logits,
+                                         accepted_path=lm_path, n_accepted=lm_nacc, bonus_token=lm_bonus), lm_steps, replays=5)
+        lm = {"stats_us": lm_stats_us, "stats_us_min": lm_stats_min, "accept_us": lm_accept_us, "accept_us_min": lm_accept_min}
     clocks = sampler.stop()
     ctx.check()
 
@@ -377,6 +396,19 @@ def main():
         draft_expand_cpu_us = (time.perf_counter() - t0) * 1e6
         draft_expand_ok = (all(np.array_equal(dx_arr[j].cpu().numpy(), dx_ref[j]) for j in range(3))
                            and np.array_equal(dx_next[0].cpu().numpy(), nc_ref) and np.array_equal(dx_next[1].cpu().numpy(), nl_ref))
+        if lm is not None:
+            # two rows of the LM-head statistics against the fp64 product over the whole vocabulary
+            pick = sorted({0, B * N - 1})
+            ctx.lm_head_stats(d_hid.view(B * N, lm_H), d_wgt, temp, N, out=lm_out)
+            torch.cuda.synchronize()
+            lm_ok = True
+            for i_ in pick:
+                T_ = float(inp.temperature[i_ // N]) or 1.0
+                r_ = oracle.lm_head_stats(np.ascontiguousarray(hid_host[i_:i_ + 1]), wgt_host, T_)
+                lm_ok &= abs(float(lm_out[0][i_]) - r_["max"][0]) <= 1e-3 and abs(float(lm_out[1][i_]) / r_["sum"][0] - 1) <= 3e-3 \
+                    and (r_["gap"][0] <= 2e-3 or int(lm_out[2][i_]) == int(r_["arg"][0]))
+            lm["rows_checked_against_oracle"] = pick
+            lm["ok"] = bool(lm_ok)
         verified = {"accept_bit_exact": bool(ok_acc), "attn_max_abs_err": float(err.max()),
                     "attn_mean_abs_err": float(err.mean()),
                     "ok": bool(ok_acc and err.max() <= 1e-2 and err.mean() <= 1e-3)}
@@ -465,6 +497,13 @@ def main():
                                   "frac_of_hbm_peak": dlp_host.nbytes / (draft_expand_us * 1e-6) / 1e9 / peak,
                                   "bit_exact_vs_oracle": draft_expand_ok, "oracle_us_one_thread": draft_expand_cpu_us,
                                   "note": "one level of the draft phase (three kernels); not part of value"},
+            "lm_head_call": None if lm is None else dict(lm, **{
+                "rows": B * N, "hidden": lm_H, "vocab": w.vocab, "weight_bytes": 2.0 * lm_H * w.vocab,
+                "slabs_of_128_rows": (B * N + 127) // 128,
+                "stats_gbs": 2.0 * lm_H * w.vocab * ((B * N + 127) // 128) / (lm["stats_us"] * 1e-6) / 1e9,
+                "stats_frac_of_hbm_peak": 2.0 * lm_H * w.vocab * ((B * N + 127) // 128) / (lm["stats_us"] * 1e-6) / 1e9 / peak,
+                "note": "LM head with the scan as its epilogue (stats) and with the walk behind it (accept); weights are "
+                        "streamed once per slab; not part of value"}),
             "e2e": {"value": e2e_us, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "steps": e2e_steps, "note": "fspad_verify_step_host: pinned host inputs, device-resident KV cache"},
             "gpu_launches": int(launches),
