@@ -98,6 +98,21 @@ def lm_head_stats(hidden, weight, T: float = 1.0, want_logits: bool = False):
     return {"max": m, "sum": s, "arg": a, "gap": gap, "logits": z}
 
 
+def feature_sampler(f, e, wup, wgate, wdown, want_inter: bool = False):
+    """fp64 Feature Sampler forward: eta = Wdown (silu(Wgate e) * (Wup f)) + f.  f, e [R][H]; wup, wgate [I][H];
+    wdown [H][I] (bf16 bit patterns).  Returns eta [R][H] float64 (and the intermediate [R][I] on request)."""
+    R, H = f.shape
+    I = wup.shape[0]
+    assert e.shape == (R, H) and wup.shape == (I, H) and wgate.shape == (I, H) and wdown.shape == (H, I)
+    eta = np.empty((R, H), np.float64)
+    inter = np.empty((R, I), np.float64) if want_inter else None
+    rc = lib().oracle_feature_sampler(_p(f, np.uint16), _p(e, np.uint16), _p(wup, np.uint16), _p(wgate, np.uint16),
+                                      _p(wdown, np.uint16), R, H, I, _p(eta, np.float64), _p(inter, np.float64))
+    if rc != 0:
+        raise RuntimeError("oracle_feature_sampler failed: %d" % rc)
+    return (eta, inter) if want_inter else eta
+
+
 def tree_accept(target_logits, draft_probs, draft_tokens, parent, temperature, uniforms,
                 force: Optional[np.ndarray] = None):
     """Lossless tree acceptance. Returns a dict with accepted_path [B][N] (-1 padded),

@@ -190,6 +190,54 @@ int oracle_lm_head_stats(const uint16_t *hidden, const uint16_t *weight, int R, 
     return bad ? -1 : 0;
 }
 
+/* ------------------------------------------------------------------------
+ * Feature Sampler forward ("Feature Sampling": three projectors and a sampling
+ * operation in the intermediate space).  The Up projector maps the feature f and
+ * the Gate projector the token embedding e to intermediate size; the embedding's
+ * image is activated by SiLU and multiplied element by element with the
+ * feature's image; the Down projector maps the result back to hidden size, where
+ * the residual connection the section mentions adds the input feature:
+ *   u = Wup f,  g = Wgate e,  s = silu(g) * u,  eta = Wdown s + f      (fp64)
+ *   f, e [R][H]; Wup, Wgate [I][H]; Wdown [H][I]: bf16 bit patterns; eta [R][H] double
+ *   inter (may be NULL) [R][I] double receives s.
+ * ---------------------------------------------------------------------- */
+int oracle_feature_sampler(const uint16_t *f, const uint16_t *e, const uint16_t *wup, const uint16_t *wgate,
+                           const uint16_t *wdown, int R, int H, int I, double *eta, double *inter)
+{
+    int bad = 0;
+#pragma omp parallel for schedule(dynamic)
+    for (int r = 0; r < R; ++r) {
+        double *fr = (double *)malloc((size_t)H * sizeof(double));
+        double *er = (double *)malloc((size_t)H * sizeof(double));
+        double *s = (double *)malloc((size_t)I * sizeof(double));
+        if (!fr || !er || !s) {
+            bad = 1;
+            free(fr); free(er); free(s);
+            continue;
+        }
+        for (int h = 0; h < H; ++h) {
+            fr[h] = bf16_to_f64(f[(size_t)r * H + h]);
+            er[h] = bf16_to_f64(e[(size_t)r * H + h]);
+        }
+        for (int i = 0; i < I; ++i) {
+            double u = 0.0, g = 0.0;
+            for (int h = 0; h < H; ++h) {
+                u += bf16_to_f64(wup[(size_t)i * H + h]) * fr[h];
+                g += bf16_to_f64(wgate[(size_t)i * H + h]) * er[h];
+            }
+            s[i] = g / (1.0 + exp(-g)) * u;
+        }
+        for (int h = 0; h < H; ++h) {
+            double acc = 0.0;
+            for (int i = 0; i < I; ++i) acc += bf16_to_f64(wdown[(size_t)h * I + i]) * s[i];
+            eta[(size_t)r * H + h] = acc + fr[h];
+        }
+        if (inter) memcpy(inter + (size_t)r * I, s, (size_t)I * sizeof(double));
+        free(fr); free(er); free(s);
+    }
+    return bad ? -1 : 0;
+}
+
 /* Inverse-CDF draw: weights w_j >= 0 summed in index order to Z; the token is
  * the smallest j whose running sum exceeds u*Z; if rounding leaves none, the
  * largest j with w_j > 0.  info (may be NULL) receives

@@ -422,3 +422,17 @@ def lm_head_inputs(seed: int, rows: int, hidden: int, vocab: int, sigma_logit: f
                           np.float32(sigma_logit / np.sqrt(hidden))))
     return h, w
 
+
+def feature_sampler_inputs(seed: int, rows: int, hidden: int, inter: int):
+    """Stand-in inputs of the Feature Sampler (bf16 bit patterns): features f and token embeddings e [rows][hidden]
+    ~ N(0, 1); Up and Gate projectors [inter][hidden] ~ N(0, 1/hidden); Down projector [hidden][inter] ~ N(0, 1/inter),
+    so that every projection keeps values of order one."""
+    rng = np.random.default_rng(24081556200 + 104729 * seed + 29)
+    f = normal_bf16(rng, (rows, hidden))
+    e = normal_bf16(rng, (rows, hidden))
+    sc = np.float32(1.0 / np.sqrt(hidden))
+    wup = f32_to_bf16_bits(rng.standard_normal((inter, hidden), dtype=np.float32) * sc)
+    wgate = f32_to_bf16_bits(rng.standard_normal((inter, hidden), dtype=np.float32) * sc)
+    wdown = f32_to_bf16_bits(rng.standard_normal((hidden, inter), dtype=np.float32) * np.float32(1.0 / np.sqrt(inter)))
+    return f, e, wup, wgate, wdown
+
