@@ -251,6 +251,32 @@ int fspad_lm_head_accept(fspad_ctx *ctx, const fspad_bf16 *hidden, const fspad_b
                          int32_t *accepted_path, int32_t *n_accepted, int32_t *bonus_token, void *stream);
 
 /*
+ * Feature Sampler forward ("Feature Sampling": the Up projector maps the feature f and the Gate projector
+ * the token embedding e to intermediate size; the embedding's image is activated by SiLU and multiplied,
+ * element by element, with the feature's image; the Down projector maps the result back to hidden size,
+ * where the residual connection adds the input feature):
+ *
+ *   eta[r] = W_down ( silu(W_gate e[r]) * (W_up f[r]) ) + f[r]
+ *
+ * bf16 inputs and weights, fp32 accumulation; the gated product is rounded to bf16 (it is the Down
+ * projector's tensor-core operand) and so is eta.  This is the draft model's input synthesis, run once per
+ * draft step on the frontier rows; no positional or normalisation step is applied here.
+ *
+ *   f, e     [rows][hidden_dim] bf16          rows <= 128
+ *   w_up, w_gate [inter_dim][hidden_dim] bf16 w_down [hidden_dim][inter_dim] bf16
+ *   inter    [rows][inter_dim] bf16, written: the gated product (kept: it is the second product's operand)
+ *   eta      [rows][hidden_dim] bf16, written
+ *   workspace  device memory of at least fspad_feature_sampler_workspace_bytes(rows, hidden_dim, inter_dim)
+ *            bytes, owned by the caller (fp32 partial sums of the split products); contents are scratch
+ * hidden_dim and inter_dim multiples of 8; all pointers device, 16-byte aligned.  Errors: FSPAD_ERR_SHAPE
+ * for sizes outside these ranges, FSPAD_ERR_RANGE for a workspace that is too small.
+ */
+size_t fspad_feature_sampler_workspace_bytes(int rows, int hidden_dim, int inter_dim);
+int fspad_feature_sampler(fspad_ctx *ctx, const fspad_bf16 *f, const fspad_bf16 *e, const fspad_bf16 *w_up,
+                          const fspad_bf16 *w_gate, const fspad_bf16 *w_down, int rows, int hidden_dim, int inter_dim,
+                          fspad_bf16 *inter, fspad_bf16 *eta, void *workspace, size_t workspace_bytes, void *stream);
+
+/*
  * Dynamic token tree, one draft step ("Preliminaries", last paragraph: the
  * output of each draft step is truncated to its top-k, and every token carries
  * the joint probability of its path).  Called once per level of the draft

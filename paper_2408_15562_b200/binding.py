@@ -19,7 +19,7 @@ _lib = None
 
 EXPORTS = ["fspad_create", "fspad_destroy", "fspad_status", "fspad_strerror", "fspad_launch_count",
            "fspad_tree_attn", "fspad_tree_accept", "fspad_accept_stats", "fspad_kv_compact",
-           "fspad_lm_head_stats", "fspad_lm_head_accept", "fspad_verify_step", "fspad_verify_step_host", "fspad_selftest_wait_timeout", "fspad_accept_stats_noalloc", "fspad_tree_build", "fspad_draft_expand"]
+           "fspad_lm_head_stats", "fspad_lm_head_accept", "fspad_feature_sampler", "fspad_feature_sampler_workspace_bytes", "fspad_verify_step", "fspad_verify_step_host", "fspad_selftest_wait_timeout", "fspad_accept_stats_noalloc", "fspad_tree_build", "fspad_draft_expand"]
 
 
 class FspadConfig(ctypes.Structure):
@@ -59,6 +59,9 @@ def load():
     lib.fspad_accept_stats_noalloc.argtypes = [vp, vp, ci, ci, ci, vp, vp, vp, vp]
     lib.fspad_lm_head_stats.argtypes = [vp, vp, vp, ci, ci, ci, vp, vp, vp, vp, vp, vp]
     lib.fspad_lm_head_accept.argtypes = [vp, vp, vp, ci, vp, vp, vp, vp, vp, ci, ci, vp, vp, vp, vp, vp]
+    lib.fspad_feature_sampler_workspace_bytes.argtypes = [ci, ci, ci]
+    lib.fspad_feature_sampler_workspace_bytes.restype = ctypes.c_size_t
+    lib.fspad_feature_sampler.argtypes = [vp] * 6 + [ci, ci, ci, vp, vp, vp, ctypes.c_size_t, vp]
     lib.fspad_selftest_wait_timeout.argtypes = [vp, ci, vp]
     lib.fspad_verify_step.argtypes = [vp, vp, ci] + [vp] * 10 + [ci, ci] + [vp] * 6
     lib.fspad_verify_step_host.argtypes = [vp] * 12 + [ci, ci] + [vp] * 6
@@ -215,6 +218,25 @@ class Context:
         if rc != 0:
             raise FspadError(rc, "fspad_lm_head_accept")
         return accepted_path, n_accepted, bonus_token
+
+    def feature_sampler(self, f, e, w_up, w_gate, w_down, inter=None, eta=None, workspace=None, stream=None):
+        """f, e [rows][H]; w_up, w_gate [I][H]; w_down [H][I] (bf16, device) -> (eta [rows][H], inter [rows][I])."""
+        rows, H = f.shape
+        I = w_up.shape[0]
+        bf = torch.bfloat16
+        if inter is None:
+            inter = torch.empty((rows, I), dtype=bf, device=f.device)
+        if eta is None:
+            eta = torch.empty((rows, H), dtype=bf, device=f.device)
+        need = load().fspad_feature_sampler_workspace_bytes(rows, H, I)
+        if workspace is None:
+            workspace = torch.empty((need,), dtype=torch.uint8, device=f.device)
+        rc = load().fspad_feature_sampler(self._h, _ptr(f, bf), _ptr(e, bf), _ptr(w_up, bf), _ptr(w_gate, bf), _ptr(w_down, bf),
+                                          rows, H, I, _ptr(inter, bf), _ptr(eta, bf), _ptr(workspace, torch.uint8),
+                                          workspace.numel(), _stream(stream))
+        if rc != 0:
+            raise FspadError(rc, "fspad_feature_sampler")
+        return eta, inter
 
     def kv_compact(self, cache, accepted_path, n_accepted, prefix_len, new_len=None, stream=None):
         B = prefix_len.shape[0]

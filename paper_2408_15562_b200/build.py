@@ -9,7 +9,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libfspad.so")
-SOURCES = ["api.cu", "accept_stats.cu", "accept_walk.cu", "kv_compact.cu", "tree_attn.cu", "tree_attn_umma.cu", "tree_build.cu", "draft_expand.cu", "lm_head.cu"]
+SOURCES = ["api.cu", "accept_stats.cu", "accept_walk.cu", "kv_compact.cu", "tree_attn.cu", "tree_attn_umma.cu", "tree_build.cu", "draft_expand.cu", "lm_head.cu", "feature_sampler.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-I" + os.path.join(ROOT, "include"), "-I" + CSRC]
 

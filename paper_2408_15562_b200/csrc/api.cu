@@ -263,6 +263,30 @@ int fspad_lm_head_accept(fspad_ctx *ctx, const fspad_bf16 *hidden, const fspad_b
                ? FSPAD_OK : FSPAD_ERR_CUDA;
 }
 
+size_t fspad_feature_sampler_workspace_bytes(int rows, int hidden_dim, int inter_dim)
+{
+    if (rows < 1 || hidden_dim < 1 || inter_dim < 1) return 0;
+    return fspad_feature_sampler_scratch_floats(rows, hidden_dim, inter_dim) * sizeof(float);
+}
+
+int fspad_feature_sampler(fspad_ctx *ctx, const fspad_bf16 *f, const fspad_bf16 *e, const fspad_bf16 *w_up,
+                          const fspad_bf16 *w_gate, const fspad_bf16 *w_down, int rows, int hidden_dim, int inter_dim,
+                          fspad_bf16 *inter, fspad_bf16 *eta, void *workspace, size_t workspace_bytes, void *stream)
+{
+    if (!ctx) return FSPAD_ERR_NULL;
+    if (!f || !e || !w_up || !w_gate || !w_down || !inter || !eta || !workspace) return FSPAD_ERR_NULL;
+    if (misaligned(f) || misaligned(e) || misaligned(w_up) || misaligned(w_gate) || misaligned(w_down) || misaligned(inter) ||
+        misaligned(eta) || misaligned(workspace))
+        return FSPAD_ERR_ALIGN;
+    if (rows < 0 || rows > 128 || hidden_dim < 8 || hidden_dim % 8 != 0 || inter_dim < 8 || inter_dim % 8 != 0)
+        return FSPAD_ERR_SHAPE;
+    if (rows == 0) return FSPAD_OK;
+    if (workspace_bytes < fspad_feature_sampler_workspace_bytes(rows, hidden_dim, inter_dim)) return FSPAD_ERR_RANGE;
+    return fspad_launch_feature_sampler(ctx, f, e, w_up, w_gate, w_down, rows, hidden_dim, inter_dim, inter, eta,
+                                        static_cast<float *>(workspace), fspad_stream(stream)) == cudaSuccess
+               ? FSPAD_OK : FSPAD_ERR_CUDA;
+}
+
 int fspad_kv_compact(fspad_ctx *ctx, fspad_bf16 *cache, const int32_t *accepted_path,
                      const int32_t *n_accepted, const int32_t *prefix_len, int batch,
                      int32_t *new_len, void *stream)

@@ -50,6 +50,7 @@ struct fspad_ctx {
     // LM head: per-(row, vocabulary tile) partials of one slab of 128 rows, [128][tiles]
     struct FspadStatsPart *lm_parts;
     int lm_attr_done;
+    int fs_attr_done;         // dynamic shared-memory limit raised for the Feature Sampler's product kernel
 
     void *dx_part;            // draft step: per-piece top-k lists [max_batch * 16 rows][pieces][16] (value, token)
 
@@ -283,6 +284,10 @@ cudaError_t fspad_launch_tree_scatter(fspad_ctx *ctx, fspad_bf16 *cache, const f
                                       cudaStream_t st);
 int fspad_attn_umma_splits(const fspad_ctx *ctx, int N, int B, int sms = 0);
 int fspad_lm_head_tiles(int V);
+size_t fspad_feature_sampler_scratch_floats(int rows, int H, int I);
+cudaError_t fspad_launch_feature_sampler(fspad_ctx *ctx, const fspad_bf16 *f, const fspad_bf16 *e, const fspad_bf16 *wup,
+                                         const fspad_bf16 *wgate, const fspad_bf16 *wdown, int R, int H, int I,
+                                         fspad_bf16 *inter, fspad_bf16 *eta, float *scratch, cudaStream_t st);
 FspadStatsGeom fspad_lm_head_geom(int rows, int V, bool vec, int slots);
 // LM head over R rows; with walk_geom the merged partials go to the context's scan scratch in that
 // geometry (for the acceptance walk), otherwise to row_max / row_sum / row_arg
