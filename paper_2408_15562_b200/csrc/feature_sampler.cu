@@ -5,9 +5,9 @@
 //     eta = Wdown (silu(Wgate e) * (Wup f)) + f
 // The draft model runs this on a handful of rows per step (the frontier of the draft tree), so the
 // three products are bound by streaming their matrices once (3 * 2 * H * I bytes).  One tcgen05
-// kernel serves all of them: a persistent CTA per SM takes work items (problem, tile of 128 output
+// kernel serves all of them: a persistent CTA per SM takes work items (problem, tile of 256 output
 // columns, range of the inner dimension), streams the matrix slab and the rows through a TMA ring
-// of 128-byte-swizzled [128][64] bf16 stages into 128 x 128 x 16 tensor-core instructions with two
+// of 128-byte-swizzled [128][64] / [256][64] bf16 stages into 128 x 256 x 16 tensor-core instructions with two
 // accumulators in tensor memory, and writes fp32 partial sums; the inner dimension is split so that
 // the items fill the SMs evenly.  Two small kernels add the partial sums: one applies SiLU and the
 // product (bf16 out, the Down projector's operand), one adds the residual (bf16 out).
@@ -20,16 +20,17 @@ namespace fsm {
 
 using namespace umma;
 
-constexpr int BM = 128, BN = 128, BKE = 64;
-constexpr int STAGE = 128 * 128;        // bytes of one [128][64] bf16 operand stage
-constexpr int NSTG = 6;
+constexpr int BM = 128, BN = 256, BKE = 64;
+constexpr int STAGE_A = BM * 128;       // bytes of one [128][64] bf16 stage of the rows
+constexpr int STAGE_B = BN * 128;       // bytes of one [256][64] bf16 stage of the matrix
+constexpr int NSTG = 4;
 constexpr int NT = 192;                 // warp 0: copies; warp 1: tensor cores; warps 2-5: epilogue
-constexpr int SMEM_BYTES = 2 * NSTG * STAGE + 1024;
-constexpr uint32_t TMEM_COLS = 256;
+constexpr int SMEM_BYTES = NSTG * (STAGE_A + STAGE_B) + 1024;
+constexpr uint32_t TMEM_COLS = 512;     // two fp32 accumulators of 256 columns
 
 struct Args {
     int R, K, N;                        // rows (<= 128), inner dimension, output columns
-    int n_tiles, splits, kps;           // tiles of 128 output columns; ranges of the inner dimension; stages per range
+    int n_tiles, splits, kps;           // tiles of 256 output columns; ranges of the inner dimension; stages per range
     int n_problems;                     // 1 or 2 products that share the shape (different operands)
     float *out[2];                      // [splits][R][N] fp32 partial sums of each problem
     int *status;
@@ -47,7 +48,7 @@ skinny_gemm_kernel(const Args a, const __grid_constant__ CUtensorMap tmA0, const
     fspad_pdl_wait();
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    const uint32_t sA = base, sB = base + NSTG * STAGE;
+    const uint32_t sA = base, sB = base + NSTG * STAGE_A;
     const uint32_t bar0 = smem_u32(&s_bar[0]);
     auto full = [&](int s) { return bar0 + 8u * (uint32_t)s; };
     auto empty = [&](int s) { return bar0 + 8u * (uint32_t)(NSTG + s); };
@@ -99,9 +100,9 @@ skinny_gemm_kernel(const Args a, const __grid_constant__ CUtensorMap tmA0, const
                 const uint32_t ph = (uint32_t)(it / NSTG) & 1u;
                 if (it >= NSTG && !failed && !mbar_wait(empty(s), ph ^ 1u)) failed = true;
                 if (!failed && lane == 0) {
-                    mbar_expect_tx(full(s), 2 * STAGE);
-                    tma_load_2d(sA + s * STAGE, mA, (k0 + k) * BKE, 0, full(s));
-                    tma_load_2d(sB + s * STAGE, mB, (k0 + k) * BKE, tile * BN, full(s));
+                    mbar_expect_tx(full(s), STAGE_A + STAGE_B);
+                    tma_load_2d(sA + s * STAGE_A, mA, (k0 + k) * BKE, 0, full(s));
+                    tma_load_2d(sB + s * STAGE_B, mB, (k0 + k) * BKE, tile * BN, full(s));
                 }
                 __syncwarp();
             }
@@ -127,10 +128,10 @@ skinny_gemm_kernel(const Args a, const __grid_constant__ CUtensorMap tmA0, const
                 if (!failed && !mbar_wait(full(s), ph)) failed = true;
                 if (!failed) {
                     tc_fence_after();
-                    const uint32_t so = (uint32_t)s * (STAGE >> 4);
+                    const uint32_t soa = (uint32_t)s * (STAGE_A >> 4), sob = (uint32_t)s * (STAGE_B >> 4);
 #pragma unroll
                     for (int ks = 0; ks < 4; ++ks)
-                        mma_f16_lo(tmem + (uint32_t)buf * BN, a_lo + so + ks * 2, hi, b_lo + so + ks * 2, hi, idesc,
+                        mma_f16_lo(tmem + (uint32_t)buf * BN, a_lo + soa + ks * 2, hi, b_lo + sob + ks * 2, hi, idesc,
                                    (k > 0) || (ks > 0), elect);
                     mma_commit_if(empty(s), elect);
                     if (k == nk - 1) mma_commit_if(accf(buf), elect);
