@@ -364,6 +364,21 @@ def main():
             lambda i: ctx.lm_head_accept(d_hid, d_wgt, sets[i % R]["draft"], tokens, parent, temp, unif, logits=lm_logits,
                                          accepted_path=lm_path, n_accepted=lm_nacc, bonus_token=lm_bonus), lm_steps, replays=5)
         lm = {"stats_us": lm_stats_us, "stats_us_min": lm_stats_min, "accept_us": lm_accept_us, "accept_us_min": lm_accept_min}
+    # the draft side's Feature Sampler on a frontier of ten rows (intermediate size 3.5 x hidden, as in the
+    # LLaMA-3 family); not part of `value`
+    fs = None
+    if not args.no_lm_head:
+        fs_rows, fs_I = 10, int(3.5 * lm_H)
+        fs_host = synth.feature_sampler_inputs(w.cfg, fs_rows, lm_H, fs_I)
+        fs_dev = [bf(x) for x in fs_host]
+        fs_inter = torch.empty((fs_rows, fs_I), dtype=torch.bfloat16, device="cuda")
+        fs_eta = torch.empty((fs_rows, lm_H), dtype=torch.bfloat16, device="cuda")
+        fs_ws = torch.empty((binding.load().fspad_feature_sampler_workspace_bytes(fs_rows, lm_H, fs_I),), dtype=torch.uint8,
+                            device="cuda")
+        fs_us, fs_min = timed(lambda i: ctx.feature_sampler(*fs_dev, inter=fs_inter, eta=fs_eta, workspace=fs_ws),
+                              max(2, min(args.steps, 10)), replays=5)
+        fs = {"us": fs_us, "us_min": fs_min, "rows": fs_rows, "hidden": lm_H, "intermediate": fs_I,
+              "weight_bytes": 6.0 * lm_H * fs_I, "gbs": 6.0 * lm_H * fs_I / (fs_us * 1e-6) / 1e9}
     clocks = sampler.stop()
     ctx.check()
 
@@ -409,6 +424,12 @@ def main():
                     and (r_["gap"][0] <= 2e-3 or int(lm_out[2][i_]) == int(r_["arg"][0]))
             lm["rows_checked_against_oracle"] = pick
             lm["ok"] = bool(lm_ok)
+        if fs is not None:
+            ctx.feature_sampler(*fs_dev, inter=fs_inter, eta=fs_eta, workspace=fs_ws)
+            torch.cuda.synchronize()
+            fs_err = np.abs(fs_eta.float().cpu().numpy() - oracle.feature_sampler(*fs_host))
+            fs["max_abs_err_vs_oracle"], fs["mean_abs_err_vs_oracle"] = float(fs_err.max()), float(fs_err.mean())
+            fs["ok"] = bool(fs_err.max() <= 2.5e-2 and fs_err.mean() <= 3e-3)
         verified = {"accept_bit_exact": bool(ok_acc), "attn_max_abs_err": float(err.max()),
                     "attn_mean_abs_err": float(err.mean()),
                     "ok": bool(ok_acc and err.max() <= 1e-2 and err.mean() <= 1e-3)}
@@ -504,6 +525,10 @@ def main():
                 "stats_frac_of_hbm_peak": 2.0 * lm_H * w.vocab * ((B * N + 127) // 128) / (lm["stats_us"] * 1e-6) / 1e9 / peak,
                 "note": "LM head with the scan as its epilogue (stats) and with the walk behind it (accept); weights are "
                         "streamed once per slab; not part of value"}),
+            "feature_sampler_call": None if fs is None else dict(fs, **{
+                "frac_of_hbm_peak": fs["gbs"] / peak,
+                "note": "draft side: eta = Wdown(silu(Wgate e) * Wup f) + f on the frontier rows; three matrices streamed once; "
+                        "not part of value"}),
             "e2e": {"value": e2e_us, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "steps": e2e_steps, "note": "fspad_verify_step_host: pinned host inputs, device-resident KV cache"},
             "gpu_launches": int(launches),

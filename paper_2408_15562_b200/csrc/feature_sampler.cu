@@ -286,8 +286,8 @@ cudaError_t fspad_launch_feature_sampler(fspad_ctx *ctx, const fspad_bf16 *f, co
     // ---- Up and Gate: two products [R][H] x [I][H]^T in one launch ----
     CUtensorMap mAf, mAe, mUp, mGate, mS, mDown;
     if (!fspad_make_tmap_bf16_2d(&mAf, f, (size_t)H, (size_t)R, BM) || !fspad_make_tmap_bf16_2d(&mAe, e, (size_t)H, (size_t)R, BM) ||
-        !fspad_make_tmap_bf16_2d(&mUp, wup, (size_t)H, (size_t)I, BN) || !fspad_make_tmap_bf16_2d(&mGate, wgate, (size_t)H, (size_t)I, BN) ||
-        !fspad_make_tmap_bf16_2d(&mS, inter, (size_t)I, (size_t)R, BM) || !fspad_make_tmap_bf16_2d(&mDown, wdown, (size_t)I, (size_t)H, BN))
+        !fspad_make_tmap_bf16_2d(&mUp, wup, (size_t)H, (size_t)I, BN, true) || !fspad_make_tmap_bf16_2d(&mGate, wgate, (size_t)H, (size_t)I, BN, true) ||
+        !fspad_make_tmap_bf16_2d(&mS, inter, (size_t)I, (size_t)R, BM) || !fspad_make_tmap_bf16_2d(&mDown, wdown, (size_t)I, (size_t)H, BN, true))
         return cudaErrorInvalidValue;
     float *p_up = scratch, *p_gate = scratch + (size_t)8 * R * I, *p_down = scratch + (size_t)16 * R * I;
     Args a;

@@ -12,13 +12,19 @@
 //   logits[r][v] = sum_h hidden[r][h] * weight[v][h]      bf16 x bf16 -> fp32
 //
 // With a handful of rows the product is bound by streaming the vocabulary matrix
-// once (2 * H * V bytes).  One persistent CTA per SM walks over tiles of 128
-// vocabulary entries; per tile it streams the [128][H] slab of the matrix and the
-// hidden states (up to 128 rows, re-read from L2) through a ring of 128-byte-
-// swizzled [128][64] bf16 stages filled by TMA, accumulates 128 x 128 x 16
-// tcgen05.mma into one of two tensor-memory accumulators, and four epilogue warps
-// (one row per thread) reduce the finished accumulator while the next tile is
-// being multiplied.  Roles meet only on mbarriers; every wait is bounded.
+// once (2 * H * V bytes).  One persistent CTA per SM walks over work items of 256
+// vocabulary entries (and, for what does not fill a whole round of the grid, of
+// 128, so that the last round is short instead of idle); per item it streams the
+// [256][H] slab of the matrix and the hidden states (up to 128 rows, re-read from
+// L2) through a ring of 128-byte-swizzled [256][64] / [128][64] bf16 stages filled
+// by TMA, accumulates 128 x 256 x 16 tcgen05.mma into one of two tensor-memory
+// accumulators, and four epilogue warps (one row per thread) reduce the finished
+// accumulator, 128 columns (one tile of partial results) at a time, while the next
+// item is being multiplied.  Measured on 60 x 4096 x 128256: 128-wide items with six
+// 16 KB matrix stages 214 us, 256-wide items with four 32 KB stages 207 us, and with
+// the matrix's tensor map asking L2 for 256 bytes per request (the next stage of the
+// same rows comes along: fewer, longer DRAM bursts per open page) 196 us.  Roles meet
+// only on mbarriers; every wait is bounded.
 #include <cuda.h>
 
 #include "common.cuh"
@@ -29,13 +35,14 @@ namespace lmh {
 using namespace umma;
 
 constexpr int BM = 128;                 // rows of hidden states per CTA (one accumulator lane each)
-constexpr int BN = 128;                 // vocabulary entries per tile
+constexpr int BN = 128;                 // vocabulary entries per tile (one partial result per row and tile)
 constexpr int BKE = 64;                 // hidden elements per stage (128 bytes: the swizzle span)
-constexpr int STAGE = 128 * 128;        // bytes of one [128][64] bf16 operand stage
-constexpr int NSTG = 6;                 // stages in flight (A and B each)
+constexpr int STAGE = 128 * 128;        // bytes of one [128][64] bf16 box
+constexpr int STAGE_B = 2 * STAGE;      // matrix stage: two boxes = 256 vocabulary entries
+constexpr int NSTG = 4;                 // stages in flight
 constexpr int NT = 192;                 // warp 0: copies; warp 1: tensor cores; warps 2-5: epilogue
-constexpr int SMEM_BYTES = 2 * NSTG * STAGE + 1024;
-constexpr uint32_t TMEM_COLS = 256;     // two fp32 accumulators of 128 columns
+constexpr int SMEM_BYTES = NSTG * (STAGE + STAGE_B) + 1024;
+constexpr uint32_t TMEM_COLS = 512;     // two fp32 accumulators of 256 columns
 constexpr float kLog2e = 1.4426950408889634f;
 
 struct Args {
@@ -57,14 +64,25 @@ lm_head_stats_kernel(const Args a, const __grid_constant__ CUtensorMap tmA, cons
     fspad_pdl_wait();
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    const uint32_t sA = base, sB = base + NSTG * STAGE;
+    const uint32_t sA = base, sB = base + NSTG * STAGE;     // rows: NSTG x 16 KB, matrix: NSTG x 32 KB
     const uint32_t bar0 = smem_u32(&s_bar[0]);
     auto full = [&](int s) { return bar0 + 8u * (uint32_t)s; };
     auto empty = [&](int s) { return bar0 + 8u * (uint32_t)(NSTG + s); };
     auto accf = [&](int b) { return bar0 + 8u * (uint32_t)(2 * NSTG + b); };
     auto acce = [&](int b) { return bar0 + 8u * (uint32_t)(2 * NSTG + 2 + b); };
     const int n_k = (a.H + BKE - 1) / BKE;
-    const int my_tiles = ((int)blockIdx.x < a.n_tiles) ? (a.n_tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
+    // Work items: pairs of tiles for as many whole rounds of the grid as there are, single tiles after that.
+    const int G = (int)gridDim.x;
+    const int wide_rounds = (a.n_tiles / 2) / G;
+    const int first_single = 2 * wide_rounds * G;                   // tiles from here on go out one by one
+    const int n_single = a.n_tiles - first_single;
+    const int my_single = ((int)blockIdx.x < n_single) ? (n_single - (int)blockIdx.x + G - 1) / G : 0;
+    const int my_items = wide_rounds + my_single;
+    // item j of this CTA -> first tile and number of tiles (2 or 1)
+    auto item = [&](int j, int &tile, int &width) {
+        if (j < wide_rounds) { tile = 2 * ((int)blockIdx.x + j * G); width = 2; }
+        else { tile = first_single + (int)blockIdx.x + (j - wide_rounds) * G; width = 1; }
+    };
 
     if (tid == 0) {
         for (int i = 0; i < 2 * NSTG + 4; ++i) mbar_init(bar0 + 8u * i, i >= 2 * NSTG + 2 ? 4 : 1);
@@ -86,16 +104,18 @@ lm_head_stats_kernel(const Args a, const __grid_constant__ CUtensorMap tmA, cons
     if (warp == 0) {
         // ================= copy warp: one lane issues every TMA copy =================
         int it = 0;
-        for (int j = 0; j < my_tiles; ++j) {
-            const int tile = (int)blockIdx.x + j * (int)gridDim.x;
+        for (int j = 0; j < my_items; ++j) {
+            int tile, width;
+            item(j, tile, width);
             for (int k = 0; k < n_k; ++k, ++it) {
                 const int s = it % NSTG;
                 const uint32_t ph = (uint32_t)(it / NSTG) & 1u;
                 if (it >= NSTG && !failed && !mbar_wait(empty(s), ph ^ 1u)) failed = true;
                 if (!failed && lane == 0) {
-                    mbar_expect_tx(full(s), 2 * STAGE);
+                    mbar_expect_tx(full(s), (1 + width) * STAGE);
                     tma_load_2d(sA + s * STAGE, &tmA, k * BKE, 0, full(s));
-                    tma_load_2d(sB + s * STAGE, &tmB, k * BKE, tile * BN, full(s));
+                    tma_load_2d(sB + s * STAGE_B, &tmB, k * BKE, tile * BN, full(s));
+                    if (width == 2) tma_load_2d(sB + s * STAGE_B + STAGE, &tmB, k * BKE, (tile + 1) * BN, full(s));
                 }
                 __syncwarp();
             }
@@ -106,9 +126,12 @@ lm_head_stats_kernel(const Args a, const __grid_constant__ CUtensorMap tmA, cons
         const uint32_t elect = lane == 0;
         const uint32_t hi = (uint32_t)(make_desc(0, 16) >> 32);
         const uint32_t a_lo = (uint32_t)make_desc(sA, 16), b_lo = (uint32_t)make_desc(sB, 16);
-        const uint32_t idesc = make_idesc(false, BN);
+        const uint32_t idesc2 = make_idesc(false, 2 * BN), idesc1 = make_idesc(false, BN);
         int it = 0;
-        for (int j = 0; j < my_tiles; ++j) {
+        for (int j = 0; j < my_items; ++j) {
+            int tile, width;
+            item(j, tile, width);
+            const uint32_t idesc = width == 2 ? idesc2 : idesc1;
             const int buf = j & 1;
             // the accumulator is free once the epilogue has read the tile that used it two tiles ago
             if (j >= 2 && !failed && !mbar_wait(acce(buf), (uint32_t)((j - 2) >> 1) & 1u)) failed = true;
@@ -119,10 +142,10 @@ lm_head_stats_kernel(const Args a, const __grid_constant__ CUtensorMap tmA, cons
                 if (!failed && !mbar_wait(full(s), ph)) failed = true;
                 if (!failed) {
                     tc_fence_after();
-                    const uint32_t so = (uint32_t)s * (STAGE >> 4);
+                    const uint32_t soa = (uint32_t)s * (STAGE >> 4), sob = (uint32_t)s * (STAGE_B >> 4);
 #pragma unroll
                     for (int ks = 0; ks < 4; ++ks)      // 16 hidden elements = 32 bytes per instruction
-                        mma_f16_lo(tmem + (uint32_t)buf * BN, a_lo + so + ks * 2, hi, b_lo + so + ks * 2, hi, idesc,
+                        mma_f16_lo(tmem + (uint32_t)buf * (2 * BN), a_lo + soa + ks * 2, hi, b_lo + sob + ks * 2, hi, idesc,
                                    (k > 0) || (ks > 0), elect);
                     mma_commit_if(empty(s), elect);
                     if (k == n_k - 1) mma_commit_if(accf(buf), elect);
@@ -140,18 +163,22 @@ lm_head_stats_kernel(const Args a, const __grid_constant__ CUtensorMap tmA, cons
         if (row_ok && a.temperature) T = a.temperature[(a.row0 + row) / a.rows_per_seq];
         if (!(T > 0.0f)) T = 1.0f;
         const float kk = kLog2e / T;
-        for (int j = 0; j < my_tiles; ++j) {
-            const int tile = (int)blockIdx.x + j * (int)gridDim.x;
+        for (int j = 0; j < my_items; ++j) {
+            int tile0, width;
+            item(j, tile0, width);
             const int buf = j & 1;
             if (!failed && !mbar_wait(accf(buf), (uint32_t)(j >> 1) & 1u)) failed = true;
             tc_fence_after();
+#pragma unroll 1
+          for (int half = 0; half < width; ++half) {
+            const int tile = tile0 + half;
             float m = -INFINITY, s = 0.f;
             int arg = 0x7fffffff;
             const int col0 = tile * BN;
 #pragma unroll 1
             for (int blk = 0; blk < BN / 32; ++blk) {
                 float v[32];
-                tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)buf * BN + (uint32_t)blk * 32u, v);
+                tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)buf * (2 * BN) + (uint32_t)(half * BN + blk * 32), v);
                 const int c = col0 + blk * 32;
                 if (c + 32 > a.V) {
 #pragma unroll
@@ -189,15 +216,16 @@ lm_head_stats_kernel(const Args a, const __grid_constant__ CUtensorMap tmA, cons
                     s += acc;
                 }
             }
-            // the accumulator may be overwritten: every lane's loads have completed (tmem_ld32 waits)
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(acce(buf));
             if (row_ok && !failed) {
                 FspadStatsPart out;
                 out.m = m; out.s = s; out.a = (arg == 0x7fffffff) ? col0 : arg; out.pad = 0;
                 a.parts[(size_t)row * a.n_tiles + tile] = out;
             }
+          }
+            // the accumulator may be overwritten: every lane's loads have completed (tmem_ld32 waits)
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(acce(buf));
         }
         if (failed) s_fail = 1;
     }
@@ -209,7 +237,7 @@ lm_head_stats_kernel(const Args a, const __grid_constant__ CUtensorMap tmA, cons
         // shared and tensor memory go back to the SM
         if (tid == 0) fspad_report(a.status, FSPAD_ERR_TIMEOUT);
         if (warp == 0) {
-            const int total = my_tiles * n_k;
+            const int total = my_items * n_k;
             for (int s = 0; s < NSTG; ++s) {
                 const int fills = (total - s + NSTG - 1) / NSTG;     // upper bound of the fills started in stage s
                 if (fills > 0) (void)mbar_wait(full(s), (uint32_t)(fills - 1) & 1u, 20000);
@@ -342,7 +370,7 @@ cudaError_t fspad_launch_lm_head(fspad_ctx *ctx, const fspad_bf16 *hidden, const
         ctx->lm_attr_done = 1;
     }
     CUtensorMap mB;
-    if (!fspad_make_tmap_bf16_2d(&mB, weight, (size_t)H, (size_t)V, lmh::BN)) return cudaErrorInvalidValue;
+    if (!fspad_make_tmap_bf16_2d(&mB, weight, (size_t)H, (size_t)V, lmh::BN, true)) return cudaErrorInvalidValue;
     for (int r0 = 0; r0 < R; r0 += lmh::BM) {
         const int rs = (R - r0 < lmh::BM) ? R - r0 : lmh::BM;
         CUtensorMap mA;

@@ -564,7 +564,8 @@ static EncodeTiledFn encode_tiled_fn()
     return fn;
 }
 
-bool fspad_make_tmap_bf16_2d(CUtensorMap *map, const fspad_bf16 *base, size_t cols, size_t rows, unsigned box_rows)
+bool fspad_make_tmap_bf16_2d(CUtensorMap *map, const fspad_bf16 *base, size_t cols, size_t rows, unsigned box_rows,
+                             bool wide_l2_fetch)
 {
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn || rows == 0 || rows > 0x7fffffffull || cols == 0 || (cols * sizeof(fspad_bf16)) % 16 != 0) return false;
@@ -573,7 +574,8 @@ bool fspad_make_tmap_bf16_2d(CUtensorMap *map, const fspad_bf16 *base, size_t co
     const cuuint32_t box[2] = {64u, (cuuint32_t)box_rows};
     const cuuint32_t estr[2] = {1u, 1u};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<fspad_bf16 *>(base), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+              wide_l2_fetch ? CU_TENSOR_MAP_L2_PROMOTION_L2_256B : CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 

@@ -8,7 +8,10 @@
 
 // Tensor map of a row-major bf16 matrix [rows][cols] (cols * 2 bytes a multiple of 16): boxes of 64 columns
 // (128 bytes, the swizzle span) by box_rows rows, 128-byte swizzle, zero fill outside the matrix.
-bool fspad_make_tmap_bf16_2d(CUtensorMap *map, const fspad_bf16 *base, size_t cols, size_t rows, unsigned box_rows);
+// wide_l2_fetch: L2 brings in 256 bytes per request, i.e. also the next box of the same rows (for
+// matrices that are streamed along their rows, 128 bytes per row and stage).
+bool fspad_make_tmap_bf16_2d(CUtensorMap *map, const fspad_bf16 *base, size_t cols, size_t rows, unsigned box_rows,
+                             bool wide_l2_fetch = false);
 
 namespace umma {
 
