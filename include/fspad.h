@@ -367,6 +367,30 @@ int fspad_kv_compact(fspad_ctx *ctx, fspad_bf16 *cache, const int32_t *accepted_
                      int32_t *new_len, void *stream);
 
 /*
+ * The same two operations on a cache that is not contiguous (the paper's remark on practical frameworks in
+ * "Performance on Fewer Candidate Tokens" is the only place it touches deployment; serving systems keep the
+ * cache in fixed-size blocks).  The cache is a pool of blocks of 128 rows and a per-sequence block table:
+ * cache row r of sequence b is row r % 128 of block block_table[b][r / 128].
+ *
+ *   k_pool, v_pool [n_blocks][Hkv][128][d] bf16          (fspad_tree_attn_paged: one layer's K and V pools)
+ *   pool   [n_layers][2][n_blocks][Hkv][128][d] bf16     (fspad_kv_compact_paged: all layers, updated in place)
+ *   block_table [batch][blocks_per_seq] int32, entries in [0, n_blocks); the blocks of the rows a call touches
+ *               (rows 0 .. L_b + n_nodes - 1) must be distinct within a sequence and not shared between sequences
+ * Everything else - the other arguments, the results, the error reporting - is as in fspad_tree_attn and
+ * fspad_kv_compact with max_len = 128 * blocks_per_seq; a table entry out of range is reported as
+ * FSPAD_ERR_RANGE (device-checked, accesses stay inside the pool).  FSPAD_ERR_TOO_LARGE: more than 128
+ * blocks would fall to one CTA (blocks_per_seq above 128 times the number of key ranges the call uses).
+ * Trees stay limited to 64 nodes in these calls as in all others.
+ */
+int fspad_tree_attn_paged(fspad_ctx *ctx, const fspad_bf16 *q, const fspad_bf16 *k_pool, const fspad_bf16 *v_pool,
+                          const int32_t *block_table, int blocks_per_seq, int n_blocks, const fspad_bf16 *tree_k,
+                          const fspad_bf16 *tree_v, const int32_t *parent, const int32_t *prefix_len, int n_nodes,
+                          int batch, fspad_bf16 *out, void *stream);
+int fspad_kv_compact_paged(fspad_ctx *ctx, fspad_bf16 *pool, const int32_t *block_table, int blocks_per_seq, int n_blocks,
+                           const int32_t *accepted_path, const int32_t *n_accepted, const int32_t *prefix_len, int batch,
+                           int32_t *new_len, void *stream);
+
+/*
  * One whole verify step on DEVICE buffers ("Preliminaries": the target's single
  * forward over the flattened tree, the strict comparison of its results with the
  * tree, and the removal of the rejected tokens are one step of the decoding

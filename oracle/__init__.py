@@ -149,6 +149,28 @@ def kv_compact(cache: np.ndarray, accepted_path, n_accepted, prefix_len):
     return new_len
 
 
+def paged_to_contiguous(pool: np.ndarray, table: np.ndarray) -> np.ndarray:
+    """What a paged cache means: pool [..., n_blocks, Hkv, 128, d] and table [B][blocks] -> the contiguous cache
+    [..., B, Hkv, blocks * 128, d] in which row r of sequence b is row r % 128 of block table[b][r // 128]."""
+    B, nb = table.shape
+    lead = pool.shape[:-4]
+    _, Hkv, bs, d = pool.shape[-4:]
+    out = np.empty(lead + (B, Hkv, nb * bs, d), dtype=pool.dtype)
+    for b in range(B):
+        for i in range(nb):
+            out[..., b, :, i * bs:(i + 1) * bs, :] = pool[..., int(table[b, i]), :, :, :]
+    return out
+
+
+def contiguous_to_paged(cache: np.ndarray, table: np.ndarray, pool: np.ndarray) -> None:
+    """The inverse: writes the rows of the contiguous cache [..., B, Hkv, blocks * 128, d] into their blocks of pool."""
+    B, nb = table.shape
+    bs = pool.shape[-2]
+    for b in range(B):
+        for i in range(nb):
+            pool[..., int(table[b, i]), :, :, :] = cache[..., b, :, i * bs:(i + 1) * bs, :]
+
+
 def tree_build(cand_parent, cand_token, cand_logp, root_token, n_nodes: int):
     """Final stage of the dynamic token tree: keep the n_nodes - 1 most probable candidates and
     flatten them breadth-first behind the root.  Arrays [B][C]; returns parent, token, cand [B][N]

@@ -19,7 +19,7 @@ _lib = None
 
 EXPORTS = ["fspad_create", "fspad_destroy", "fspad_status", "fspad_strerror", "fspad_launch_count",
            "fspad_tree_attn", "fspad_tree_accept", "fspad_accept_stats", "fspad_kv_compact",
-           "fspad_lm_head_stats", "fspad_lm_head_accept", "fspad_feature_sampler", "fspad_feature_sampler_workspace_bytes", "fspad_verify_step", "fspad_verify_step_host", "fspad_selftest_wait_timeout", "fspad_accept_stats_noalloc", "fspad_tree_build", "fspad_draft_expand"]
+           "fspad_tree_attn_paged", "fspad_kv_compact_paged", "fspad_lm_head_stats", "fspad_lm_head_accept", "fspad_feature_sampler", "fspad_feature_sampler_workspace_bytes", "fspad_verify_step", "fspad_verify_step_host", "fspad_selftest_wait_timeout", "fspad_accept_stats_noalloc", "fspad_tree_build", "fspad_draft_expand"]
 
 
 class FspadConfig(ctypes.Structure):
@@ -62,6 +62,8 @@ def load():
     lib.fspad_feature_sampler_workspace_bytes.argtypes = [ci, ci, ci]
     lib.fspad_feature_sampler_workspace_bytes.restype = ctypes.c_size_t
     lib.fspad_feature_sampler.argtypes = [vp] * 6 + [ci, ci, ci, vp, vp, vp, ctypes.c_size_t, vp]
+    lib.fspad_tree_attn_paged.argtypes = [vp, vp, vp, vp, vp, ci, ci, vp, vp, vp, vp, ci, ci, vp, vp]
+    lib.fspad_kv_compact_paged.argtypes = [vp, vp, vp, ci, ci, vp, vp, vp, ci, vp, vp]
     lib.fspad_selftest_wait_timeout.argtypes = [vp, ci, vp]
     lib.fspad_verify_step.argtypes = [vp, vp, ci] + [vp] * 10 + [ci, ci] + [vp] * 6
     lib.fspad_verify_step_host.argtypes = [vp] * 12 + [ci, ci] + [vp] * 6
@@ -181,6 +183,32 @@ class Context:
         if rc != 0:
             raise FspadError(rc, "fspad_accept_stats")
         return row_max, row_sum, row_arg
+
+    def tree_attn_paged(self, q, k_pool, v_pool, block_table, tree_k, tree_v, parent, prefix_len, out=None, stream=None):
+        """Attention over a cache kept as pools of 128-row blocks [n_blocks][Hkv][128][d] and a block table [B][blocks]."""
+        B, N = q.shape[0], q.shape[1]
+        if out is None:
+            out = torch.empty_like(q)
+        bf, i32 = torch.bfloat16, torch.int32
+        rc = load().fspad_tree_attn_paged(self._h, _ptr(q, bf), _ptr(k_pool, bf), _ptr(v_pool, bf), _ptr(block_table, i32),
+                                          block_table.shape[1], k_pool.shape[0], _ptr(tree_k, bf), _ptr(tree_v, bf),
+                                          _ptr(parent, i32), _ptr(prefix_len, i32), N, B, _ptr(out, bf), _stream(stream))
+        if rc != 0:
+            raise FspadError(rc, "fspad_tree_attn_paged")
+        return out
+
+    def kv_compact_paged(self, pool, block_table, accepted_path, n_accepted, prefix_len, new_len=None, stream=None):
+        """Compaction on a pool [layers][2][n_blocks][Hkv][128][d] addressed through block_table [B][blocks]."""
+        B = prefix_len.shape[0]
+        i32 = torch.int32
+        if new_len is None:
+            new_len = torch.empty((B,), dtype=i32, device=pool.device)
+        rc = load().fspad_kv_compact_paged(self._h, _ptr(pool, torch.bfloat16), _ptr(block_table, i32), block_table.shape[1],
+                                           pool.shape[2], _ptr(accepted_path, i32), _ptr(n_accepted, i32), _ptr(prefix_len, i32),
+                                           B, _ptr(new_len, i32), _stream(stream))
+        if rc != 0:
+            raise FspadError(rc, "fspad_kv_compact_paged")
+        return new_len
 
     def lm_head_stats(self, hidden, lm_head, temperature, rows_per_seq, logits_out=None, out=None, stream=None):
         """hidden [rows][H], lm_head [V][H] (bf16, device) -> (row_max, row_sum, row_arg); logits_out, if given,

@@ -287,6 +287,41 @@ int fspad_feature_sampler(fspad_ctx *ctx, const fspad_bf16 *f, const fspad_bf16 
                ? FSPAD_OK : FSPAD_ERR_CUDA;
 }
 
+int fspad_tree_attn_paged(fspad_ctx *ctx, const fspad_bf16 *q, const fspad_bf16 *k_pool, const fspad_bf16 *v_pool,
+                          const int32_t *block_table, int blocks_per_seq, int n_blocks, const fspad_bf16 *tree_k,
+                          const fspad_bf16 *tree_v, const int32_t *parent, const int32_t *prefix_len, int n_nodes,
+                          int batch, fspad_bf16 *out, void *stream)
+{
+    int rc = check_common(ctx, n_nodes, batch);
+    if (rc) return rc;
+    if (!q || !k_pool || !v_pool || !block_table || !parent || !prefix_len || !out) return FSPAD_ERR_NULL;
+    if ((tree_k == nullptr) != (tree_v == nullptr)) return FSPAD_ERR_NULL;
+    if (misaligned(q) || misaligned(k_pool) || misaligned(v_pool) || misaligned(tree_k) || misaligned(tree_v) || misaligned(out))
+        return FSPAD_ERR_ALIGN;
+    if (blocks_per_seq < 1 || n_blocks < 1 || (long long)blocks_per_seq * 128 < n_nodes) return FSPAD_ERR_SHAPE;
+    if (batch == 0) return FSPAD_OK;
+    // a CTA keeps the blocks of its chunks in shared memory: at most 128 of them
+    const int splits = fspad_attn_umma_splits(ctx, n_nodes, batch);
+    if ((blocks_per_seq + splits - 1) / splits > 128) return FSPAD_ERR_TOO_LARGE;
+    const FspadPaged pg{block_table, blocks_per_seq, n_blocks};
+    return fspad_launch_tree_attn(ctx, q, k_pool, v_pool, tree_k, tree_v, parent, prefix_len, n_nodes, batch, out,
+                                  fspad_stream(stream), 0, pg) == cudaSuccess ? FSPAD_OK : FSPAD_ERR_CUDA;
+}
+
+int fspad_kv_compact_paged(fspad_ctx *ctx, fspad_bf16 *pool, const int32_t *block_table, int blocks_per_seq, int n_blocks,
+                           const int32_t *accepted_path, const int32_t *n_accepted, const int32_t *prefix_len, int batch,
+                           int32_t *new_len, void *stream)
+{
+    if (!ctx) return FSPAD_ERR_NULL;
+    if (!pool || !block_table || !accepted_path || !n_accepted || !prefix_len) return FSPAD_ERR_NULL;
+    if (misaligned(pool)) return FSPAD_ERR_ALIGN;
+    if (batch < 0 || batch > ctx->cfg.max_batch || blocks_per_seq < 1 || n_blocks < 1) return FSPAD_ERR_SHAPE;
+    if (batch == 0) return FSPAD_OK;
+    const FspadPaged pg{block_table, blocks_per_seq, n_blocks};
+    return fspad_launch_kv_compact_paged(ctx, pool, pg, accepted_path, n_accepted, prefix_len, batch, new_len,
+                                         fspad_stream(stream)) == cudaSuccess ? FSPAD_OK : FSPAD_ERR_CUDA;
+}
+
 int fspad_kv_compact(fspad_ctx *ctx, fspad_bf16 *cache, const int32_t *accepted_path,
                      const int32_t *n_accepted, const int32_t *prefix_len, int batch,
                      int32_t *new_len, void *stream)

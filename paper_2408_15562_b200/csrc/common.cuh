@@ -31,7 +31,8 @@ struct fspad_ctx {
     alignas(64) unsigned char attn_tmap_k[128];
     alignas(64) unsigned char attn_tmap_v[128];
     const void *attn_tmap_kptr, *attn_tmap_vptr;
-    int attn_tmap_batch, attn_tmap_ok;
+    size_t attn_tmap_rows;
+    int attn_tmap_ok;
     float *part_o;            // [batch][Hkv][splits][M][d]
     float *part_ml;           // [batch][Hkv][splits][M][2]  (running max in log2 units, sum)
 
@@ -274,11 +275,17 @@ cudaError_t fspad_launch_draft_expand(fspad_ctx *ctx, const float *logprobs, con
 cudaError_t fspad_launch_kv_compact(fspad_ctx *ctx, fspad_bf16 *cache, const int *path,
                                     const int *n_acc, const int *prefix_len, int B, int *new_len,
                                     cudaStream_t st, bool pdl = true);
+// A cache kept as a pool of 128-row blocks: table[b * stride + i] is the block with rows 128 i .. 128 i + 127
+// of sequence b (table == NULL: contiguous cache).
+struct FspadPaged {
+    const int *table;
+    int stride, n_blocks;
+};
 // sms: how many SMs the call may fill with CTAs (0 = all of them)
 cudaError_t fspad_launch_tree_attn(fspad_ctx *ctx, const fspad_bf16 *q, const fspad_bf16 *kc,
                                    const fspad_bf16 *vc, const fspad_bf16 *tk, const fspad_bf16 *tv,
                                    const int *parent, const int *prefix_len, int N, int B,
-                                   fspad_bf16 *out, cudaStream_t st, int sms = 0);
+                                   fspad_bf16 *out, cudaStream_t st, int sms = 0, FspadPaged paged = FspadPaged{nullptr, 0, 0});
 cudaError_t fspad_launch_tree_scatter(fspad_ctx *ctx, fspad_bf16 *cache, const fspad_bf16 *tk,
                                       const fspad_bf16 *tv, const int *prefix_len, int N, int B,
                                       cudaStream_t st);
@@ -299,4 +306,6 @@ cudaError_t fspad_launch_wait_selftest(fspad_ctx *ctx, int polls, cudaStream_t s
 cudaError_t fspad_launch_attn_umma_split(fspad_ctx *ctx, const fspad_bf16 *q, const fspad_bf16 *kc,
                                          const fspad_bf16 *vc, const fspad_bf16 *tk, const fspad_bf16 *tv,
                                          const int *parent, const int *prefix_len, int N, int B, int n_splits,
-                                         float scale_log2, cudaStream_t st);
+                                         float scale_log2, cudaStream_t st, FspadPaged paged);
+cudaError_t fspad_launch_kv_compact_paged(fspad_ctx *ctx, fspad_bf16 *pool, FspadPaged paged, const int *path,
+                                          const int *n_acc, const int *prefix_len, int B, int *new_len, cudaStream_t st);

@@ -70,6 +70,65 @@ kv_compact_kernel(uint4 *__restrict__ cache, const int *__restrict__ path, const
     if (bad) fspad_report(status, FSPAD_ERR_RANGE);
 }
 
+// The same moves on a cache kept as a pool of 128-row blocks, [layers][2][n_blocks][Hkv][128][d]: cache row r
+// of sequence b lives in block table[b * stride + r / 128] at offset r % 128.  One warp per (layer, K/V,
+// sequence, head); blocks are looked up per row (a handful of rows per slice).
+__global__ void __launch_bounds__(kWarpsPerCta * 32)
+kv_compact_paged_kernel(uint4 *__restrict__ pool, const int *__restrict__ table, int table_stride, int n_blocks,
+                        const int *__restrict__ path, const int *__restrict__ n_acc, const int *__restrict__ prefix_len,
+                        int n_layers, int B, int Hkv, int path_stride, int n_tree_max, int *__restrict__ new_len,
+                        int *__restrict__ status)
+{
+    fspad_pdl_trigger();
+    fspad_pdl_wait();
+    const int lane = threadIdx.x & 31;
+    const long long slice = (long long)blockIdx.x * kWarpsPerCta + (threadIdx.x >> 5);
+    const long long n_slices = (long long)n_layers * 2 * B * Hkv;
+    if (slice >= n_slices) return;
+    const int h = (int)(slice % Hkv);
+    const int b = (int)((slice / Hkv) % B);
+    const long long lk = slice / ((long long)Hkv * B);              // layer * 2 + (K or V)
+    const int max_len = table_stride * 128;
+    int L = prefix_len[b], n = n_acc[b];
+    const int *pth = path + (size_t)b * path_stride;
+    bool bad = false;
+    if (n < 0 || n > path_stride || n > n_tree_max) { bad = true; n = 0; }
+    if (L < 0 || L + n > max_len) { bad = true; n = 0; }
+    if (new_len && lane == 0 && lk == 0 && h == 0) new_len[b] = L + n;
+    // first 16-byte chunk of cache row r of this slice
+    auto row_ptr = [&](int r) -> uint4 * {
+        int blk = table[(size_t)b * table_stride + (r >> 7)];
+        if (blk < 0 || blk >= n_blocks) { bad = true; blk = 0; }
+        return pool + ((((size_t)lk * n_blocks + blk) * Hkv + h) * 128 + (r & 127)) * kChunks;
+    };
+    const int chunk = lane & 15, half = lane >> 4;
+    for (int j0 = 0; j0 < n; j0 += 2 * kBatchIters) {
+        uint4 v[kBatchIters];
+        int dst[kBatchIters];
+#pragma unroll
+        for (int u = 0; u < kBatchIters; ++u) {
+            const int j = j0 + 2 * u + half;
+            dst[u] = -1;
+            if (j < n) {
+                const int src = pth[j];
+                if (src < j || src >= n_tree_max || L + src >= max_len || (j > 0 && src <= pth[j - 1])) {
+                    bad = true;
+                    continue;
+                }
+                if (src != j) {
+                    v[u] = row_ptr(L + src)[chunk];
+                    dst[u] = j;
+                }
+            }
+        }
+        __syncwarp();      // every load of the batch before any of its stores (the half-warps own different rows)
+#pragma unroll
+        for (int u = 0; u < kBatchIters; ++u)
+            if (dst[u] >= 0) row_ptr(L + dst[u])[chunk] = v[u];
+    }
+    if (bad) fspad_report(status, FSPAD_ERR_RANGE);
+}
+
 // cache[layer 0][K|V][b][h][L_b + j][:] = tree_{k|v}[b][h][j][:]
 __global__ void __launch_bounds__(256)
 tree_scatter_kernel(uint4 *__restrict__ cache, const uint4 *__restrict__ tk, const uint4 *__restrict__ tv,
@@ -123,4 +182,17 @@ cudaError_t fspad_launch_tree_scatter(fspad_ctx *ctx, fspad_bf16 *cache, const f
     return fspad_launch(tree_scatter_kernel, dim3(grid), dim3(256), 0, st, 0, reinterpret_cast<uint4 *>(cache),
                         reinterpret_cast<const uint4 *>(tk), reinterpret_cast<const uint4 *>(tv), prefix_len, N, B,
                         c.n_kv_heads, c.max_len, ctx->d_status);
+}
+
+cudaError_t fspad_launch_kv_compact_paged(fspad_ctx *ctx, fspad_bf16 *pool, FspadPaged paged, const int *path,
+                                          const int *n_acc, const int *prefix_len, int B, int *new_len, cudaStream_t st)
+{
+    if (B == 0) return cudaSuccess;
+    const fspad_config &c = ctx->cfg;
+    const long long slices = (long long)c.n_layers * 2 * B * c.n_kv_heads;
+    const unsigned grid = (unsigned)((slices + kWarpsPerCta - 1) / kWarpsPerCta);
+    ctx->launches++;
+    return fspad_launch(kv_compact_paged_kernel, dim3(grid), dim3(kWarpsPerCta * 32), 0, st, 0,
+                        reinterpret_cast<uint4 *>(pool), paged.table, paged.stride, paged.n_blocks, path, n_acc, prefix_len,
+                        c.n_layers, B, c.n_kv_heads, c.max_nodes, c.max_nodes, new_len, ctx->d_status);
 }

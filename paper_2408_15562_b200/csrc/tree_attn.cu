@@ -99,20 +99,20 @@ tree_attn_combine_kernel(const AttnArgs a, int B)
 cudaError_t fspad_launch_tree_attn(fspad_ctx *ctx, const fspad_bf16 *q, const fspad_bf16 *kc,
                                    const fspad_bf16 *vc, const fspad_bf16 *tk, const fspad_bf16 *tv,
                                    const int *parent, const int *prefix_len, int N, int B,
-                                   fspad_bf16 *out, cudaStream_t st, int sms)
+                                   fspad_bf16 *out, cudaStream_t st, int sms, FspadPaged paged)
 {
     if (B == 0 || N == 0) return cudaSuccess;
     const fspad_config &c = ctx->cfg;
     AttnArgs a;
     a.q = q; a.kc = kc; a.vc = vc; a.tk = tk; a.tv = tv; a.parent = parent; a.prefix_len = prefix_len;
     a.N = N; a.Hq = c.n_q_heads; a.Hkv = c.n_kv_heads; a.G = c.n_q_heads / c.n_kv_heads;
-    a.M = N * a.G; a.max_len = c.max_len;
+    a.M = N * a.G; a.max_len = paged.table ? paged.stride * 128 : c.max_len;
     a.n_splits = fspad_attn_umma_splits(ctx, N, B, sms);
     a.mtiles = (a.M + 127) / 128;
     a.scale_log2 = ctx->scale * kLog2e;
     a.part_o = ctx->part_o; a.part_ml = ctx->part_ml; a.out = out; a.status = ctx->d_status;
     cudaError_t e = fspad_launch_attn_umma_split(ctx, q, kc, vc, tk, tv, parent, prefix_len, N, B, a.n_splits,
-                                                 a.scale_log2, st);
+                                                 a.scale_log2, st, paged);
     if (e != cudaSuccess) return e;
     const long long rows = (long long)B * c.n_kv_heads * a.M;
     ctx->launches++;

@@ -37,11 +37,16 @@ constexpr int TILE = 2 * HALF;         // bytes of one [128][128] bf16 tile
 constexpr int NS = 3;                  // K / V chunks in flight per CTA
 constexpr int SMEM_BYTES = (1 + 2 * NS) * TILE + 1024;   // Q, K[NS], V[NS] + alignment slack
 constexpr uint32_t TMEM_COLS = 512;    // S/P of group 0, of group 1: columns 0..255; O of group 0, of group 1: 256..511
+constexpr int kMaxBlocksPerCta = 128;  // paged cache: chunks (= blocks) one CTA may be given
 constexpr float kLazyLog2 = 8.f;        // a row's reference maximum may lag its true maximum by this much (log2)
 struct Args {
     const fspad_bf16 *q, *kc, *vc, *tk, *tv;
     const int *parent, *prefix_len;
     int N, Hq, Hkv, G, M, max_len, n_splits, mtiles, use_tma;
+    // paged cache: the planes are pools of 128-row blocks [n_blocks][Hkv][128][d] and block_table[b][i] names
+    // the block that holds rows 128 i .. 128 i + 127 of sequence b (NULL: contiguous planes)
+    const int *block_table;
+    int table_stride, n_blocks;
     float scale_log2;
     float *part_o, *part_ml;
     int *status;
@@ -86,6 +91,7 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
     __shared__ uint32_t s_tmem;
     __shared__ int s_fail;
     __shared__ int s_par[FSPAD_MAX_NODES];
+    __shared__ int s_blk[kMaxBlocksPerCta];       // paged cache: blocks of this CTA's chunks
     __shared__ unsigned long long s_anc[FSPAD_MAX_NODES];
 
     fspad_pdl_wait();
@@ -140,11 +146,27 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     }
 
-    const fspad_bf16 *kcb = a.kc + ((size_t)b * a.Hkv + g) * (size_t)a.max_len * D;
-    const fspad_bf16 *vcb = a.vc + ((size_t)b * a.Hkv + g) * (size_t)a.max_len * D;
-    const fspad_bf16 *tkb = a.tk ? a.tk + ((size_t)b * a.Hkv + g) * (size_t)N * D : kcb + (size_t)L * D;
-    const fspad_bf16 *tvb = a.tv ? a.tv + ((size_t)b * a.Hkv + g) * (size_t)N * D : vcb + (size_t)L * D;
-    const int plane_row0 = (b * a.Hkv + g) * a.max_len;   // first row of this kv head in the cache planes
+    const bool paged = a.block_table != nullptr;
+    if (paged) {
+        // the blocks of this CTA's chunks (a chunk is one block); an entry out of range is reported and replaced
+        if (n_ch > kMaxBlocksPerCta && tid == 0) fspad_report(a.status, FSPAD_ERR_SHAPE);
+        for (int i = tid; i < n_ch && i < kMaxBlocksPerCta; i += NT) {
+            int blk = a.block_table[(size_t)b * a.table_stride + c0 + i];
+            if (blk < 0 || blk >= a.n_blocks) { fspad_report(a.status, FSPAD_ERR_RANGE); blk = 0; }
+            s_blk[i] = blk;
+        }
+        __syncthreads();
+    }
+    const int plane_row0 = (b * a.Hkv + g) * a.max_len;   // contiguous planes: first row of this kv head
+    // row of the plane matrix [rows][128] that holds cache row `key` of this sequence and kv head
+    // (key inside this CTA's chunks)
+    auto phys_row = [&](int key) -> size_t {
+        if (!paged) return (size_t)plane_row0 + (size_t)key;
+        const int i = min((key >> 7) - c0, kMaxBlocksPerCta - 1);
+        return ((size_t)s_blk[i] * a.Hkv + g) * 128 + (size_t)(key & 127);
+    };
+    const fspad_bf16 *tkb = a.tk ? a.tk + ((size_t)b * a.Hkv + g) * (size_t)N * D : nullptr;
+    const fspad_bf16 *tvb = a.tv ? a.tv + ((size_t)b * a.Hkv + g) * (size_t)N * D : nullptr;
     auto is_tma = [&](int ch) { return tma_ok && (ch + 1) * BK <= L; };
 
     // Start the fill of an operand buffer with chunk `ch`.  A chunk inside the cached prefix comes
@@ -154,13 +176,14 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
     // whole CTA in the prologue, the producer warp alone inside the loop).
     auto gather = [&](int ch, int buf, bool is_v, int t0, int nt) {
         const uint32_t dst = (is_v ? sV : sK) + buf * TILE;
-        const fspad_bf16 *cb = is_v ? vcb : kcb, *tb = is_v ? tvb : tkb;
+        const fspad_bf16 *cb = is_v ? a.vc : a.kc, *tb = is_v ? tvb : tkb;
         for (int i = t0; i < BK * 16; i += nt) {
             const int r = i >> 4, c = i & 15;
             const int key = ch * BK + r;
             const bool ok = key < Ltot;
             const fspad_bf16 *src = cb;
-            if (ok) src = (key < L) ? cb + (size_t)key * D + c * 8 : tb + (size_t)(key - L) * D + c * 8;
+            // prefix rows, and tree rows that live in the cache, come from the planes; explicit tree rows from their array
+            if (ok) src = (key < L || tb == nullptr) ? cb + phys_row(key) * D + c * 8 : tb + (size_t)(key - L) * D + c * 8;
             cp_async16(dst + tile_off(r, c), src, ok);
         }
     };
@@ -169,7 +192,7 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
         const uint32_t bar = is_v ? vfull(buf) : kfull(buf);
         const CUtensorMap *map = is_v ? &tmV : &tmK;
         mbar_expect_tx(bar, TILE);
-        const int y = plane_row0 + ch * BK;
+        const int y = (int)phys_row(ch * BK);
         tma_load_2d(dst, map, 0, y, bar);
         tma_load_2d(dst + HALF, map, 64, y, bar);
     };
@@ -587,13 +610,14 @@ static bool make_plane_map(CUtensorMap *map, const fspad_bf16 *plane, size_t row
 cudaError_t fspad_launch_attn_umma_split(fspad_ctx *ctx, const fspad_bf16 *q, const fspad_bf16 *kc,
                                          const fspad_bf16 *vc, const fspad_bf16 *tk, const fspad_bf16 *tv,
                                          const int *parent, const int *prefix_len, int N, int B, int n_splits,
-                                         float scale_log2, cudaStream_t st)
+                                         float scale_log2, cudaStream_t st, FspadPaged paged)
 {
     const fspad_config &c = ctx->cfg;
     umma::Args a;
     a.q = q; a.kc = kc; a.vc = vc; a.tk = tk; a.tv = tv; a.parent = parent; a.prefix_len = prefix_len;
     a.N = N; a.Hq = c.n_q_heads; a.Hkv = c.n_kv_heads; a.G = c.n_q_heads / c.n_kv_heads;
-    a.M = N * a.G; a.max_len = c.max_len; a.n_splits = n_splits;
+    a.M = N * a.G; a.max_len = paged.table ? paged.stride * umma::BK : c.max_len; a.n_splits = n_splits;
+    a.block_table = paged.table; a.table_stride = paged.stride; a.n_blocks = paged.n_blocks;
     a.mtiles = (a.M + umma::BM - 1) / umma::BM;
     a.scale_log2 = scale_log2;
     a.part_o = ctx->part_o; a.part_ml = ctx->part_ml; a.status = ctx->d_status;
@@ -607,10 +631,11 @@ cudaError_t fspad_launch_attn_umma_split(fspad_ctx *ctx, const fspad_bf16 *q, co
     static_assert(sizeof(CUtensorMap) <= sizeof(ctx->attn_tmap_k), "tensor map storage");
     CUtensorMap *mk = reinterpret_cast<CUtensorMap *>(ctx->attn_tmap_k);
     CUtensorMap *mv = reinterpret_cast<CUtensorMap *>(ctx->attn_tmap_v);
-    if (ctx->attn_tmap_kptr != kc || ctx->attn_tmap_vptr != vc || ctx->attn_tmap_batch != B) {
-        const size_t rows = (size_t)B * c.n_kv_heads * c.max_len;
+    // rows of the plane matrix: every sequence's cache, or the whole pool of blocks
+    const size_t rows = paged.table ? (size_t)paged.n_blocks * c.n_kv_heads * umma::BK : (size_t)B * c.n_kv_heads * c.max_len;
+    if (ctx->attn_tmap_kptr != kc || ctx->attn_tmap_vptr != vc || ctx->attn_tmap_rows != rows) {
         ctx->attn_tmap_ok = make_plane_map(mk, kc, rows) && make_plane_map(mv, vc, rows);
-        ctx->attn_tmap_kptr = kc; ctx->attn_tmap_vptr = vc; ctx->attn_tmap_batch = B;
+        ctx->attn_tmap_kptr = kc; ctx->attn_tmap_vptr = vc; ctx->attn_tmap_rows = rows;
     }
     a.use_tma = ctx->attn_tmap_ok ? 1 : 0;
     dim3 grid(n_splits, c.n_kv_heads * a.mtiles, B);
