@@ -17,7 +17,7 @@
  *   fspad_tree_build   the draft phase's candidates -> the flattened token tree
  *
  * Conventions (shared by every call)
- *   - A tree has N <= 64 nodes in topological order: parent[0] = -1 (node 0 is
+ *   - A tree has N <= 256 nodes (N <= 64 for fspad_tree_build) in topological order: parent[0] = -1 (node 0 is
  *     the root = the last token already emitted; it is always accepted) and
  *     0 <= parent[i] < i.  Children of a node are visited in increasing index.
  *   - "bf16" is a 16-bit brain-float bit pattern (typedef below).
@@ -51,7 +51,7 @@ typedef enum {
     FSPAD_ERR_NULL = -1,           /* a required pointer is NULL                       */
     FSPAD_ERR_ALIGN = -2,          /* a pointer is not 16-byte aligned                 */
     FSPAD_ERR_SHAPE = -3,          /* sizes inconsistent with the context              */
-    FSPAD_ERR_TREE_TOO_LARGE = -4, /* n_nodes > 64 or > max_nodes                      */
+    FSPAD_ERR_TREE_TOO_LARGE = -4, /* n_nodes > 256 (tree builder: 64) or > max_nodes    */
     FSPAD_ERR_RANGE = -5,          /* prefix_len + n_nodes > max_len, T < 0 or NaN     */
     FSPAD_ERR_CUDA = -6,           /* a CUDA runtime call or launch failed             */
     FSPAD_ERR_TIMEOUT = -7,        /* a bounded device-side wait ran out               */
@@ -64,7 +64,7 @@ typedef struct {
     int n_q_heads;        /* Hq                                                     */
     int n_kv_heads;       /* Hkv, divides Hq; query head h uses kv head h/(Hq/Hkv)   */
     int head_dim;         /* d, must be 128                                         */
-    int max_nodes;        /* largest N any call will pass, 1..64                    */
+    int max_nodes;        /* largest N any call will pass, 1..256                   */
     int vocab;            /* V                                                      */
     int n_layers;         /* layers in the cache handed to fspad_kv_compact          */
     int max_len;          /* rows per (sequence, kv head) of the cache               */
@@ -328,7 +328,7 @@ int fspad_draft_expand(fspad_ctx *ctx, const float *logprobs, const float *front
  *               from the root; never larger than the parent's; -inf allowed, NaN
  *               not.
  *   root_token  [batch] int32, device: token of node 0.
- *   n_cand      1 .. 1024;  n_nodes 1 .. max_nodes of the context.
+ *   n_cand      1 .. 1024;  n_nodes 1 .. min(64, max_nodes of the context).
  *
  * Kept: the n_nodes - 1 candidates with the largest joint probability; among
  * equal values the lower index first (so a parent is never displaced by a child
@@ -380,7 +380,7 @@ int fspad_kv_compact(fspad_ctx *ctx, fspad_bf16 *cache, const int32_t *accepted_
  * fspad_kv_compact with max_len = 128 * blocks_per_seq; a table entry out of range is reported as
  * FSPAD_ERR_RANGE (device-checked, accesses stay inside the pool).  FSPAD_ERR_TOO_LARGE: more than 128
  * blocks would fall to one CTA (blocks_per_seq above 128 times the number of key ranges the call uses).
- * Trees stay limited to 64 nodes in these calls as in all others.
+ * Trees of up to 256 nodes, as in the contiguous calls.
  */
 int fspad_tree_attn_paged(fspad_ctx *ctx, const fspad_bf16 *q, const fspad_bf16 *k_pool, const fspad_bf16 *v_pool,
                           const int32_t *block_table, int blocks_per_seq, int n_blocks, const fspad_bf16 *tree_k,

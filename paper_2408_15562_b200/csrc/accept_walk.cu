@@ -43,6 +43,7 @@ constexpr int kMaxCluster = 16;
 constexpr int kWalkThreads = 1024;
 constexpr int kWarps = kWalkThreads / 32;
 constexpr int kSmemBudget = 200 * 1024;   // dynamic shared memory for the per-node cache
+constexpr int kSmemBudgetWide = 188 * 1024;   // the same for the instance with room for 256 nodes (its static part is larger)
 constexpr double kAmbiguous = 1e-4;
 constexpr double kScanRel = 1e-6;          // bound taken for the relative error of the scan's sum of exponentials
 constexpr double kFusedTol = 1e-9;         // relative error the fused first-rejection sweep may leave in the residual mass
@@ -79,26 +80,61 @@ struct WalkArgs {
     int *path, *n_acc, *bonus, *status;
 };
 
-struct Shared {
+// A set of tree nodes as a bit mask of W 64-bit words (W = 1: trees of up to 64 nodes, the common case;
+// W = 4: up to 256).
+template <int W> struct NodeSet {
+    unsigned long long w[W];
+    __device__ __forceinline__ bool any() const
+    {
+        unsigned long long o = 0ull;
+#pragma unroll
+        for (int i = 0; i < W; ++i) o |= w[i];
+        return o != 0ull;
+    }
+    __device__ __forceinline__ int first() const          // lowest member (the set is not empty)
+    {
+#pragma unroll
+        for (int i = 0; i < W; ++i)
+            if (w[i]) return i * 64 + __ffsll((long long)w[i]) - 1;
+        return -1;
+    }
+    __device__ __forceinline__ void drop_first()
+    {
+#pragma unroll
+        for (int i = 0; i < W; ++i)
+            if (w[i]) { w[i] &= w[i] - 1; return; }
+    }
+    __device__ __forceinline__ bool single() const        // exactly one member
+    {
+        NodeSet t = *this;
+        t.drop_first();
+        return any() && !t.any();
+    }
+};
+
+// MAXN: capacity in tree nodes of this instance of the kernel (64 or FSPAD_MAX_NODES_WIDE)
+template <int MAXN> struct SharedT {
+    static constexpr int W = MAXN / 64;
+    static constexpr int kPieceRows = (MAXN == 64) ? 64 : 1;   // the per-piece masses are kept only by the 64-node instance
     double exp_tbl[64];             // 2^(i/64)
-    int parent[FSPAD_MAX_NODES];
-    int tok[FSPAD_MAX_NODES];
-    int path[FSPAD_MAX_NODES];
+    int parent[MAXN];
+    int tok[MAXN];
+    int path[MAXN];
     // state of the current node (written by thread 0, read by all after a barrier)
     double S, invS, c, U, D, m, invT;
-    unsigned long long child_mask[FSPAD_MAX_NODES];   // bit c set in child_mask[i] iff parent[c] == i
+    NodeSet<W> child_mask[MAXN];    // c in child_mask[i] iff parent[c] == i
     int exact, nrem, decision, xnew, ridx, next, len, cur, have_e, have_q, sel;
     double cprime, ex, qx;
-    int rem_tok[FSPAD_MAX_NODES];
-    double rem_frozen[FSPAD_MAX_NODES];
+    int rem_tok[MAXN];
+    double rem_frozen[MAXN];
     // gathered once, in parallel, before the walk: the scan result of every row and, for
     // every node, its parent's logit and draft probability at the node's token and its uniform
-    float rowM[FSPAD_MAX_NODES];
-    double rowS[FSPAD_MAX_NODES];
-    double rowInvS[FSPAD_MAX_NODES];   // 1 / rowS, so that no division sits on the serial path
-    int rowA[FSPAD_MAX_NODES];
-    float cx[FSPAD_MAX_NODES], cq[FSPAD_MAX_NODES], cu[FSPAD_MAX_NODES];
-    double cex[FSPAD_MAX_NODES];    // exp((logit - row max)/T) of each node's token in its parent's row
+    float rowM[MAXN];
+    double rowS[MAXN];
+    double rowInvS[MAXN];   // 1 / rowS, so that no division sits on the serial path
+    int rowA[MAXN];
+    float cx[MAXN], cq[MAXN], cu[MAXN];
+    double cex[MAXN];    // exp((logit - row max)/T) of each node's token in its parent's row
     float ubonus;
     int want_q;
     int bonus_ok;                   // the last residual sweep already holds the bonus draw's per-thread sums
@@ -112,11 +148,11 @@ struct Shared {
     int verdict[2];                    // bonus draw from one piece of the row: 1 = settled, 2 = the whole row must be swept
     // serial walk -> sweeps: what thread 0 asks the CTA to do next
     int req, req_child, req_last;
-    unsigned long long rem;            // children of the current node not tested yet
+    NodeSet<W> rem;                    // children of the current node not tested yet
     // approximate mass of every (row, CTA) piece of the vocabulary scan, relative to the row maximum;
     // piece_cnt[row] = 0 when the row has more than kPieceSlots pieces (the draw then sweeps the whole row)
-    double piece_w[FSPAD_MAX_NODES][kPieceSlots];
-    int piece_cnt[FSPAD_MAX_NODES];
+    double piece_w[kPieceRows][kPieceSlots];
+    int piece_cnt[kPieceRows];
 };
 
 // exp(a) for a <= 0 in double precision: a = (64 n + i) ln2/64 + r, |r| <= ln2/128,
@@ -170,7 +206,7 @@ struct Sweep {
 //               (nothing rejected at this node: the e_j themselves)
 // With `locate` the running sum starts at run0 and *found receives the first
 // token where base + run exceeds target (else the last positive-weight token).
-template <int MODE>
+template <int MODE, class Shared>
 __device__ Sweep sweep_chunk(const Shared &sh, const float *__restrict__ x, const float *__restrict__ q,
                              double *__restrict__ se, float *__restrict__ sq, int tid, int nthr, int lo, int hi,
                              bool vec, bool cache_ok, bool have_e, bool have_q, double c, int xnew,
@@ -282,6 +318,7 @@ __device__ Sweep sweep_chunk(const Shared &sh, const float *__restrict__ x, cons
 struct Sweep5 {
     double v[5];
 };
+template <class Shared>
 __device__ Sweep5 fused_reject_sweep(const Shared &sh, const float *__restrict__ x, const float *__restrict__ q,
                                      double *__restrict__ se, float *__restrict__ sq, int tid, int nthr, int lo, int hi,
                                      bool vec, bool cache_ok, double inv_s_scan, double c, int xnew)
@@ -326,9 +363,12 @@ __device__ Sweep5 fused_reject_sweep(const Shared &sh, const float *__restrict__
     return r;
 }
 
+template <int MAXN>
 __global__ void __launch_bounds__(kWalkThreads, 1)
 accept_walk_kernel(const WalkArgs args)
 {
+    typedef SharedT<MAXN> Shared;
+    constexpr int W = Shared::W;
     cg::cluster_group cluster = cg::this_cluster();
     const int C = (int)cluster.num_blocks();
     const int rank = (int)cluster.block_rank();
@@ -340,7 +380,11 @@ accept_walk_kernel(const WalkArgs args)
     extern __shared__ __align__(16) unsigned char dyn_smem[];
 
     fspad_pdl_trigger();
-    if (tid < 64) { sh.exp_tbl[tid] = kExp2Tbl[tid]; sh.child_mask[tid] = 0ull; }
+    if (tid < 64) sh.exp_tbl[tid] = kExp2Tbl[tid];
+    if (tid < MAXN) {
+#pragma unroll
+        for (int i = 0; i < W; ++i) sh.child_mask[tid].w[i] = 0ull;
+    }
     // The vocabulary scan that precedes this kernel in the stream lets it start only after the scan's
     // own predecessor has completed, and the scan writes nothing but its partial results.  So the
     // caller's arrays may be read before the scan has finished: the prologue's two round trips of
@@ -386,7 +430,7 @@ accept_walk_kernel(const WalkArgs args)
         sh.parent[tid] = p;
         sh.tok[tid] = t;
         if (tid >= 1) {
-            atomicOr(&sh.child_mask[p], 1ull << tid);
+            atomicOr(&sh.child_mask[p].w[tid >> 6], 1ull << (tid & 63));
             if (sampling) {
                 const size_t at = (size_t)p * V + t;
                 xv = lg[at];
@@ -417,8 +461,11 @@ accept_walk_kernel(const WalkArgs args)
         for (int r0 = 0; r0 < N; r0 += n_half) {                 // whole warps iterate together
             const int row = r0 + (tid >> 4);
             float M; double S; int A;
-            fspad_stats_merge_half(args.parts, args.geom, b * N + row, row < N, kT, lane16, M, S, A,
-                                   sh.piece_w[row < N ? row : 0], &sh.piece_cnt[row < N ? row : 0]);
+            if (MAXN == 64)
+                fspad_stats_merge_half(args.parts, args.geom, b * N + row, row < N, kT, lane16, M, S, A,
+                                       sh.piece_w[row < N ? row : 0], &sh.piece_cnt[row < N ? row : 0]);
+            else
+                fspad_stats_merge_half(args.parts, args.geom, b * N + row, row < N, kT, lane16, M, S, A);
             if (lane16 == 0 && row < N) { sh.rowM[row] = M; sh.rowS[row] = S; sh.rowInvS[row] = 1.0 / S; sh.rowA[row] = A; }
         }
     }
@@ -435,8 +482,8 @@ accept_walk_kernel(const WalkArgs args)
             for (;;) {
                 const int want = sh.rowA[cur];
                 int next = -1;
-                for (unsigned long long rem = sh.child_mask[cur]; rem; rem &= rem - 1) {
-                    const int c = __ffsll((long long)rem) - 1;
+                for (NodeSet<W> rem = sh.child_mask[cur]; rem.any(); rem.drop_first()) {
+                    const int c = rem.first();
                     if (sh.tok[c] == want) { next = c; break; }
                 }
                 if (next < 0) { args.bonus[b] = want; break; }
@@ -545,8 +592,8 @@ accept_walk_kernel(const WalkArgs args)
     for (;;) {
         if (tid == 0) {
             int req = REQ_DONE;
-            while (sh.rem != 0ull) {
-                const int ch = __ffsll((long long)sh.rem) - 1;
+            while (sh.rem.any()) {
+                const int ch = sh.rem.first();
                 const int xt = sh.tok[ch];
                 const double r = (double)sh.cu[ch];
                 const double qx = (double)sh.cq[ch];
@@ -580,8 +627,8 @@ accept_walk_kernel(const WalkArgs args)
             }
             sh.req = req;
             if (req != REQ_DONE) {
-                sh.req_child = __ffsll((long long)sh.rem) - 1;
-                sh.req_last = ((sh.rem & (sh.rem - 1)) == 0ull) ? 1 : 0;
+                sh.req_child = sh.rem.first();
+                sh.req_last = sh.rem.single() ? 1 : 0;
             }
         }
         __syncthreads();
@@ -645,14 +692,14 @@ accept_walk_kernel(const WalkArgs args)
             } else {
                 frozen = weight(sh.ex, sh.qx, sh.invS, sh.c);   // residual vanished: p is kept
             }
-            if (sh.ridx < 0 && sh.nrem < FSPAD_MAX_NODES) {
+            if (sh.ridx < 0 && sh.nrem < MAXN) {
                 sh.rem_tok[sh.nrem] = xt;
                 sh.rem_frozen[sh.nrem] = frozen;
                 sh.nrem++;
             }
             if (Dn > 0.0) sh.D = Dn;
             sh.have_q = cache_ok;
-            sh.rem &= sh.rem - 1;                               // this child is done
+            sh.rem.drop_first();                                // this child is done
         }
         // no barrier here: only thread 0 touches the walk's state until the next request is published
     }
@@ -708,23 +755,23 @@ accept_walk_kernel(const WalkArgs args)
         // uncertainty of all the approximations together.  Otherwise, and for every other kind of
         // draw, the cluster sweeps the whole row exactly.
         bool settled = false;
-        const int n_piece = sh.piece_cnt[cur];
+        const int n_piece = (MAXN == 64) ? sh.piece_cnt[MAXN == 64 ? cur : 0] : 0;
         if (!sh.bonus_ok && c == 0.0 && sh.nrem == 0 && n_piece > 0) {
             double Zs = 0.0;
-            for (int i = 0; i < n_piece; ++i) Zs += sh.piece_w[cur][i];
+            for (int i = 0; i < n_piece; ++i) Zs += sh.piece_w[MAXN == 64 ? cur : 0][i];
             const double target = (double)sh.ubonus * Zs;
             int pick = -1;
             double pre = 0.0;
             for (int i = 0; i < n_piece; ++i) {
-                const double nxt = pre + sh.piece_w[cur][i];
+                const double nxt = pre + sh.piece_w[MAXN == 64 ? cur : 0][i];
                 if (nxt > target) { pick = i; break; }
                 pre = nxt;
             }
             // error budget: the masses in front of the piece and the total (scan, kScanRel each, doubled
             // for slack) and the single-precision sums inside the piece (argument rounding of the
             // exponential 1.3e-7 per unit of |log2 e_j|, the approximation itself 2.4e-7, the partial sums)
-            const double tol = 4.0 * kScanRel * Zs + (pick >= 0 ? 4e-6 * sh.piece_w[cur][pick] : 0.0);
-            if (pick >= 0 && target - pre > tol && pre + sh.piece_w[cur][pick] - target > tol) {
+            const double tol = 4.0 * kScanRel * Zs + (pick >= 0 ? 4e-6 * sh.piece_w[MAXN == 64 ? cur : 0][pick] : 0.0);
+            if (pick >= 0 && target - pre > tol && pre + sh.piece_w[MAXN == 64 ? cur : 0][pick] - target > tol) {
                 // token range of that piece: CTA `first + pick` of the scan, clipped to the row
                 const FspadStatsGeom &g = args.geom;
                 const long long row_lo = (long long)(b * N + cur) * g.upr;
@@ -845,9 +892,11 @@ static int walk_cluster_size(fspad_ctx *ctx, int B, int V)
 {
     if (ctx->walk_cluster == 0) {
         ctx->walk_cluster = 8;
-        cudaFuncSetAttribute(accept_walk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
-        if (cudaFuncSetAttribute(accept_walk_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) ==
-            cudaSuccess) {
+        cudaFuncSetAttribute(accept_walk_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
+        cudaFuncSetAttribute(accept_walk_kernel<FSPAD_MAX_NODES_WIDE>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudgetWide);
+        if (cudaFuncSetAttribute(accept_walk_kernel<64>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess &&
+            cudaFuncSetAttribute(accept_walk_kernel<FSPAD_MAX_NODES_WIDE>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) ==
+                cudaSuccess) {
             cudaLaunchConfig_t probe = {};
             probe.gridDim = dim3(kMaxCluster);
             probe.blockDim = dim3(kWalkThreads);
@@ -857,7 +906,11 @@ static int walk_cluster_size(fspad_ctx *ctx, int B, int V)
             at[0].val.clusterDim.x = kMaxCluster; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
             probe.attrs = at; probe.numAttrs = 1;
             int n = 0;
-            if (cudaOccupancyMaxActiveClusters(&n, accept_walk_kernel, &probe) == cudaSuccess && n >= 1)
+            int n2 = 0;
+            cudaLaunchConfig_t probe2 = probe;
+            probe2.dynamicSmemBytes = kSmemBudgetWide;
+            if (cudaOccupancyMaxActiveClusters(&n, accept_walk_kernel<64>, &probe) == cudaSuccess && n >= 1 &&
+                cudaOccupancyMaxActiveClusters(&n2, accept_walk_kernel<FSPAD_MAX_NODES_WIDE>, &probe2) == cudaSuccess && n2 >= 1)
                 ctx->walk_cluster = kMaxCluster;
         }
         (void)cudaGetLastError();
@@ -891,8 +944,13 @@ cudaError_t fspad_launch_accept_walk(fspad_ctx *ctx, const float *logits, const 
         const size_t per_cta = (size_t)((((V + cluster - 1) / cluster) + 3) & ~3);
         const size_t per_thr = ((per_cta + kWalkThreads - 1) / kWalkThreads + 3) & ~(size_t)3;
         const size_t need = per_thr * kWalkThreads * (sizeof(double) + sizeof(float));
-        if (need <= (size_t)kSmemBudget) { smem = need; a.cache_ok = 1; }
+        if (need <= (size_t)(N <= 64 ? kSmemBudget : kSmemBudgetWide)) { smem = need; a.cache_ok = 1; }
     }
     ctx->launches++;
-    return fspad_launch(accept_walk_kernel, dim3((unsigned)(B * cluster)), dim3(threads), smem, st, (unsigned)cluster, a);
+    // trees of up to 64 nodes (one mask word per node, per-piece masses kept for the bonus draw) and up to
+    // FSPAD_MAX_NODES_WIDE nodes are two instances of the kernel
+    if (N <= 64)
+        return fspad_launch(accept_walk_kernel<64>, dim3((unsigned)(B * cluster)), dim3(threads), smem, st, (unsigned)cluster, a);
+    return fspad_launch(accept_walk_kernel<FSPAD_MAX_NODES_WIDE>, dim3((unsigned)(B * cluster)), dim3(threads), smem, st,
+                        (unsigned)cluster, a);
 }

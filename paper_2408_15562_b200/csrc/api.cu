@@ -23,7 +23,7 @@ bool dev_alloc(T **p, size_t count)
 int check_common(const fspad_ctx *ctx, int n_nodes, int batch)
 {
     if (!ctx) return FSPAD_ERR_NULL;
-    if (n_nodes > FSPAD_MAX_NODES || n_nodes > ctx->cfg.max_nodes) return FSPAD_ERR_TREE_TOO_LARGE;
+    if (n_nodes > FSPAD_MAX_NODES_WIDE || n_nodes > ctx->cfg.max_nodes) return FSPAD_ERR_TREE_TOO_LARGE;
     if (n_nodes < 1 || batch < 0 || batch > ctx->cfg.max_batch) return FSPAD_ERR_SHAPE;
     return FSPAD_OK;
 }
@@ -59,7 +59,7 @@ int fspad_create(const fspad_config *cfg, fspad_ctx **out)
         cfg->n_q_heads % cfg->n_kv_heads != 0 || cfg->vocab < 1 || cfg->n_layers < 1 ||
         cfg->max_len < 1 || cfg->max_batch < 1 || cfg->max_nodes < 1)
         return FSPAD_ERR_SHAPE;
-    if (cfg->max_nodes > FSPAD_MAX_NODES) return FSPAD_ERR_TREE_TOO_LARGE;
+    if (cfg->max_nodes > FSPAD_MAX_NODES_WIDE) return FSPAD_ERR_TREE_TOO_LARGE;
     if (cfg->max_nodes > cfg->max_len) return FSPAD_ERR_RANGE;
     if (!(cfg->softmax_scale >= 0.0f)) return FSPAD_ERR_RANGE;
 
@@ -345,6 +345,7 @@ int fspad_tree_build(fspad_ctx *ctx, const int32_t *cand_parent, const int32_t *
     if (rc) return rc;
     if (!cand_parent || !cand_token || !cand_logp || !root_token || !parent_out || !token_out || !cand_out || !n_out)
         return FSPAD_ERR_NULL;
+    if (n_nodes > FSPAD_MAX_NODES) return FSPAD_ERR_TREE_TOO_LARGE;      // the builder's masks are one word per node
     if (n_cand < 1 || n_cand > FSPAD_MAX_CANDIDATES) return FSPAD_ERR_SHAPE;
     if (batch == 0) return FSPAD_OK;
     cudaError_t e = fspad_launch_tree_build(ctx, cand_parent, cand_token, cand_logp, root_token, n_cand, n_nodes,

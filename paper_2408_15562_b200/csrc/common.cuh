@@ -8,7 +8,8 @@
 
 #include "fspad.h"
 
-#define FSPAD_MAX_NODES 64
+#define FSPAD_MAX_NODES 64           /* nodes of a tree on the one-mask-word paths */
+#define FSPAD_MAX_NODES_WIDE 256     /* nodes of a tree, any call of the verify step */
 #define FSPAD_MAX_CANDIDATES 1024
 #define FSPAD_MAX_FRONTIER 16      /* frontier nodes per sequence, and top-k per row, of a draft step */
 #define FSPAD_HEAD_DIM 128

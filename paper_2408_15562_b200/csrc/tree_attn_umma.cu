@@ -83,6 +83,10 @@ __device__ __forceinline__ uint32_t tile_off(int r, int c)
 // A new phase of a barrier can only begin after every side that waits on it has seen the previous
 // one (a parity wait must never fall two phases behind).
 // Tensor-core order: S(0) S(1) | PV_0(0) PV_1(0) S(2) | PV_0(1) PV_1(1) S(3) | ...
+// NW: 64-bit words of a node's ancestor mask.  NW = 1 (trees of up to 64 nodes): the masks are built once per
+// CTA in shared memory.  NW = 4 (up to 256 nodes): there is no shared memory left for them, so every softmax
+// thread follows its own node's parent chain in global memory (a few cached loads) and keeps the mask in registers.
+template <int NW>
 __global__ void __launch_bounds__(NT, 1)
 tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV)
 {
@@ -90,9 +94,9 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
     __shared__ __align__(8) unsigned long long s_bar[4 * NS + 13];
     __shared__ uint32_t s_tmem;
     __shared__ int s_fail;
-    __shared__ int s_par[FSPAD_MAX_NODES];
+    __shared__ int s_par[NW == 1 ? FSPAD_MAX_NODES : 1];
     __shared__ int s_blk[kMaxBlocksPerCta];       // paged cache: blocks of this CTA's chunks
-    __shared__ unsigned long long s_anc[FSPAD_MAX_NODES];
+    __shared__ unsigned long long s_anc[NW == 1 ? FSPAD_MAX_NODES : 1];
 
     fspad_pdl_wait();
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -217,14 +221,14 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
         cp_async16(sQ + tile_off(r, c), src, ok);
     }
     cp_async_commit();
-    if (tid < N) s_par[tid] = a.parent[(size_t)b * N + tid];
+    if (NW == 1 && tid < N) s_par[tid] = a.parent[(size_t)b * N + tid];
     __syncthreads();                              // barriers initialised, parents staged
     if (warp == 9) {
         __syncwarp();
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n"
                      :: "r"(smem_u32(&s_tmem)), "r"(TMEM_COLS) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
-    } else if (tid < N) {
+    } else if (NW == 1 && tid < N) {
         // tree -> ancestor-or-self masks (parents were staged in shared memory above)
         unsigned long long mask = 0ull;
         int cur = tid;
@@ -345,7 +349,43 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
     } else {
         // ================= softmax warps =================
         const uint32_t lanes = (uint32_t)((warp & 3) * 32) << 16;
-        const unsigned long long anc = s_anc[node];
+        unsigned long long anc[NW];
+        if (NW == 1) {
+            anc[0] = s_anc[node];
+        } else {
+#pragma unroll
+            for (int w = 0; w < NW; ++w) anc[w] = 0ull;
+            if (row_ok) {
+                const int *par = a.parent + (size_t)b * N;
+                int cur = node;
+                bool bad = false;
+                for (int step = 0; step <= N && cur >= 0; ++step) {
+#pragma unroll
+                    for (int w = 0; w < NW; ++w) anc[w] |= ((cur >> 6) == w) ? (1ull << (cur & 63)) : 0ull;
+                    const int p = __ldg(par + cur);
+                    if (cur == 0) { bad |= (p != -1); break; }
+                    if (p < 0 || p >= cur) { bad = true; break; }
+                    cur = p;
+                }
+                if (bad) fspad_report(a.status, FSPAD_ERR_BAD_TREE);
+            }
+        }
+        // 32 bits of the mask from tree index `off` on (prefix keys, off < 0, count as set; bits beyond the mask are clear)
+        auto mask_word = [&](int off) -> uint32_t {
+            if (off >= 64 * NW) return 0u;
+            if (off <= -32) return ~0u;
+            if (off < 0) return ((1u << (-off)) - 1u) | (uint32_t)(anc[0] << (-off));
+            const int w = off >> 6, sft = off & 63;
+            unsigned long long lo = 0ull, hi = 0ull;
+#pragma unroll
+            for (int i = 0; i < NW; ++i) {
+                if (i == w) lo = anc[i];
+                if (i == w + 1) hi = anc[i];
+            }
+            unsigned long long v = lo >> sft;
+            if (sft > 32) v |= hi << (64 - sft);
+            return (uint32_t)v;
+        };
         const float scale = a.scale_log2;
         float m_run = -INFINITY, l_run = 0.f;
 
@@ -363,12 +403,7 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
 #pragma unroll
                 for (int blk = 0; blk < 2; ++blk) {
                     const int off = ch * BK + grp * 64 + blk * 32 - L;      // tree index of the word's first key
-                    uint32_t wv;
-                    if (off >= 64) wv = 0u;
-                    else if (off >= 0) wv = (uint32_t)(anc >> off);
-                    else if (off <= -32) wv = ~0u;
-                    else wv = ((1u << (-off)) - 1u) | (uint32_t)(anc << (-off));
-                    valid[blk] = wv;
+                    valid[blk] = mask_word(off);
                 }
             }
             // 32 scores of this thread's row, with the tree mask applied where it matters
@@ -622,8 +657,10 @@ cudaError_t fspad_launch_attn_umma_split(fspad_ctx *ctx, const fspad_bf16 *q, co
     a.scale_log2 = scale_log2;
     a.part_o = ctx->part_o; a.part_ml = ctx->part_ml; a.status = ctx->d_status;
     if (!ctx->attn_attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(umma::tree_attn_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaError_t e = cudaFuncSetAttribute(umma::tree_attn_umma_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              umma::SMEM_BYTES);
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(umma::tree_attn_umma_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, umma::SMEM_BYTES);
         if (e != cudaSuccess) return e;
         ctx->attn_attr_done = 1;
     }
@@ -640,5 +677,7 @@ cudaError_t fspad_launch_attn_umma_split(fspad_ctx *ctx, const fspad_bf16 *q, co
     a.use_tma = ctx->attn_tmap_ok ? 1 : 0;
     dim3 grid(n_splits, c.n_kv_heads * a.mtiles, B);
     ctx->launches++;
-    return fspad_launch_opt(false, umma::tree_attn_umma_kernel, grid, dim3(umma::NT), umma::SMEM_BYTES, st, 0, a, *mk, *mv);
+    if (N <= FSPAD_MAX_NODES)
+        return fspad_launch_opt(false, umma::tree_attn_umma_kernel<1>, grid, dim3(umma::NT), umma::SMEM_BYTES, st, 0, a, *mk, *mv);
+    return fspad_launch_opt(false, umma::tree_attn_umma_kernel<4>, grid, dim3(umma::NT), umma::SMEM_BYTES, st, 0, a, *mk, *mv);
 }

@@ -35,7 +35,7 @@ def test_host_side_validation_needs_no_device():
     h = ctypes.c_void_p()
     bad = binding.FspadConfig(32, 8, 64, 60, 1000, 1, 128, 1, 0.0)      # head_dim 64 is not supported
     assert lib.fspad_create(ctypes.byref(bad), ctypes.byref(h)) == -3 and not h.value
-    bad = binding.FspadConfig(32, 8, 128, 65, 1000, 1, 128, 1, 0.0)     # more than 64 nodes
+    bad = binding.FspadConfig(32, 8, 128, 257, 1000, 1, 512, 1, 0.0)    # more than 256 nodes
     assert lib.fspad_create(ctypes.byref(bad), ctypes.byref(h)) == -4 and not h.value
     bad = binding.FspadConfig(32, 5, 128, 60, 1000, 1, 128, 1, 0.0)     # Hkv does not divide Hq
     assert lib.fspad_create(ctypes.byref(bad), ctypes.byref(h)) == -3
