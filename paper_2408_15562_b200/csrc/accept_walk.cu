@@ -210,8 +210,7 @@ template <int MODE, class Shared>
 __device__ Sweep sweep_chunk(const Shared &sh, const float *__restrict__ x, const float *__restrict__ q,
                              double *__restrict__ se, float *__restrict__ sq, int tid, int nthr, int lo, int hi,
                              bool vec, bool cache_ok, bool have_e, bool have_q, double c, int xnew,
-                             bool locate, double base, double run0, double target, int *found,
-                             double *gap_below = nullptr, double *gap_above = nullptr)
+                             bool locate, double base, double run0, double target, int *found)
 {
     const double m = sh.m, invT = sh.invT;
     const int nrem = sh.nrem;
@@ -225,7 +224,6 @@ __device__ Sweep sweep_chunk(const Shared &sh, const float *__restrict__ x, cons
         if (MODE == MODE_RESID) special |= (xnew >= lo && xnew < hi);
     }
     double a = 0.0, b = 0.0, run = run0;
-    double g_lo = -1.0, g_hi = -1.0;      // distances from the target to the located token's interval ends
     int last_pos = -1, hit = -1;
     for (int j = lo; j < hi; j += 4) {
         const int n = min(4, hi - j);
@@ -286,22 +284,13 @@ __device__ Sweep sweep_chunk(const Shared &sh, const float *__restrict__ x, cons
             if (MODE == MODE_RESID) {
                 if (q_counts) b += (double)qv[t];
             } else if (locate) {
-                const double before = base + run;
                 run += w;
                 if (w > 0.0) last_pos = j + t;
-                if (hit < 0 && base + run > target) {
-                    hit = j + t;
-                    g_lo = target - before;
-                    g_hi = base + run - target;
-                }
+                if (hit < 0 && base + run > target) hit = j + t;
             }
         }
     }
-    if (locate) {
-        *found = (hit >= 0) ? hit : last_pos;
-        if (gap_below) *gap_below = g_lo;
-        if (gap_above) *gap_above = g_hi;
-    }
+    if (locate) *found = (hit >= 0) ? hit : last_pos;
     return Sweep{a, b};
 }
 
