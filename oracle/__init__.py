@@ -149,6 +149,21 @@ def kv_compact(cache: np.ndarray, accepted_path, n_accepted, prefix_len):
     return new_len
 
 
+def kv_append(cache: np.ndarray, tree_kv: np.ndarray, accepted_path, n_accepted, prefix_len):
+    """In place: the accepted path's rows of tree_kv [layers][2][B][Hkv][N][d] written behind the prefix of
+    cache [layers][2][B][Hkv][max_len][d] (both uint16); returns new_len."""
+    n_layers, two, B, Hkv, max_len, d = cache.shape
+    assert two == 2 and tree_kv.shape[:4] == cache.shape[:4] and tree_kv.shape[5] == d
+    N = tree_kv.shape[4]
+    new_len = np.empty(B, np.int32)
+    rc = lib().oracle_kv_append(_p(cache, np.uint16), _p(tree_kv, np.uint16), _p(accepted_path, np.int32),
+                                _p(n_accepted, np.int32), _p(prefix_len, np.int32), n_layers, B, Hkv, max_len,
+                                N, d, accepted_path.shape[1], _p(new_len, np.int32))
+    if rc != 0:
+        raise RuntimeError("oracle_kv_append failed: %d" % rc)
+    return new_len
+
+
 def paged_to_contiguous(pool: np.ndarray, table: np.ndarray) -> np.ndarray:
     """What a paged cache means: pool [..., n_blocks, Hkv, 128, d] and table [B][blocks] -> the contiguous cache
     [..., B, Hkv, blocks * 128, d] in which row r of sequence b is row r % 128 of block table[b][r // 128]."""

@@ -426,6 +426,45 @@ int oracle_kv_compact(uint16_t *cache, const int32_t *accepted_path, const int32
     return bad ? -2 : 0;
 }
 
+/* ------------------------------------------------------------------------
+ * Cache append of the accepted path ("Preliminaries": of the tree the target
+ * ran over, the accepted tokens continue the sequence and the rest is
+ * discarded).  The tree's K/V rows of every layer are held outside the cache;
+ * only the accepted ones are written, directly behind the prefix:
+ *   cache[l][kv][b][h][L_b + j][:] = tree_kv[l][kv][b][h][path[b][j]][:],  j < n_b
+ * Nothing else in the cache changes.  new_len[b] = L_b + n_b.
+ *   cache   [layers][2][B][Hkv][max_len][d] bf16 bits, in place
+ *   tree_kv [layers][2][B][Hkv][N][d] bf16 bits
+ * ---------------------------------------------------------------------- */
+int oracle_kv_append(uint16_t *cache, const uint16_t *tree_kv, const int32_t *accepted_path,
+                     const int32_t *n_accepted, const int32_t *prefix_len, int n_layers, int B, int Hkv,
+                     int max_len, int N, int d, int path_stride, int32_t *new_len)
+{
+    for (int b = 0; b < B; ++b) {
+        const int L = prefix_len[b], n = n_accepted[b];
+        if (n < 0 || n > N || L < 0 || L + n > max_len) return -1;
+        for (int j = 0; j < n; ++j) {
+            const int src = accepted_path[(size_t)b * path_stride + j];
+            if (src < 0 || src >= N) return -1;
+        }
+    }
+    for (int l = 0; l < n_layers; ++l)
+        for (int kv = 0; kv < 2; ++kv)
+            for (int b = 0; b < B; ++b)
+                for (int h = 0; h < Hkv; ++h) {
+                    const size_t slice = (((size_t)l * 2 + kv) * B + b) * Hkv + h;
+                    const int L = prefix_len[b], n = n_accepted[b];
+                    for (int j = 0; j < n; ++j) {
+                        const int src = accepted_path[(size_t)b * path_stride + j];
+                        memcpy(cache + (slice * max_len + (size_t)(L + j)) * d, tree_kv + (slice * N + (size_t)src) * d,
+                               sizeof(uint16_t) * d);
+                    }
+                }
+    if (new_len)
+        for (int b = 0; b < B; ++b) new_len[b] = prefix_len[b] + n_accepted[b];
+    return 0;
+}
+
 /* -------------------------------------------------------------------------
  * O5  Dynamic token tree, final stage (paper, Section "Preliminaries", last
  * paragraph: every draft step is truncated to its top-k, each token carries
