@@ -367,6 +367,25 @@ int fspad_kv_compact(fspad_ctx *ctx, fspad_bf16 *cache, const int32_t *accepted_
                      int32_t *new_len, void *stream);
 
 /*
+ * Cache append of the accepted path: compaction for a caller that keeps the tree's K/V rows of the verify
+ * forward outside the cache ("Preliminaries": the accepted tokens continue the sequence, the others and
+ * their descendants are discarded - here the discarded rows never reach the cache at all).  For every layer,
+ * K and V, sequence b and kv head:
+ *   cache[..][L_b + j][:] = tree_kv[..][accepted_path[b][j]][:],  j = 0 .. n_accepted[b]-1;
+ * nothing else in the cache changes.  new_len[b] = L_b + n_accepted[b] (may be NULL).
+ *
+ *   cache   [n_layers][2][batch][Hkv][max_len][d] bf16 (device), updated in place
+ *   tree_kv [n_layers][2][batch][Hkv][n_nodes][d] bf16 (device), read only; must not overlap cache
+ *   accepted_path [batch][max_nodes], n_accepted [batch], prefix_len [batch], new_len [batch]: int32 (device)
+ * Both arrays stay the caller's.  Errors: NULL / misaligned pointers and sizes beyond the context are
+ * refused on the host; a path entry outside [0, n_nodes), n_accepted outside [0, n_nodes] or
+ * L_b + n_accepted[b] > max_len set FSPAD_ERR_RANGE in the status word and the offending rows are skipped.
+ */
+int fspad_kv_append(fspad_ctx *ctx, fspad_bf16 *cache, const fspad_bf16 *tree_kv, const int32_t *accepted_path,
+                    const int32_t *n_accepted, const int32_t *prefix_len, int n_nodes, int batch, int32_t *new_len,
+                    void *stream);
+
+/*
  * The same two operations on a cache that is not contiguous (the paper's remark on practical frameworks in
  * "Performance on Fewer Candidate Tokens" is the only place it touches deployment; serving systems keep the
  * cache in fixed-size blocks).  The cache is a pool of blocks of 128 rows and a per-sequence block table:

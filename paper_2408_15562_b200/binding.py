@@ -19,7 +19,7 @@ _lib = None
 
 EXPORTS = ["fspad_create", "fspad_destroy", "fspad_status", "fspad_strerror", "fspad_launch_count",
            "fspad_tree_attn", "fspad_tree_accept", "fspad_accept_stats", "fspad_kv_compact",
-           "fspad_tree_attn_paged", "fspad_kv_compact_paged", "fspad_lm_head_stats", "fspad_lm_head_accept", "fspad_feature_sampler", "fspad_feature_sampler_workspace_bytes", "fspad_verify_step", "fspad_verify_step_host", "fspad_selftest_wait_timeout", "fspad_accept_stats_noalloc", "fspad_tree_build", "fspad_draft_expand"]
+           "fspad_tree_attn_paged", "fspad_kv_compact_paged", "fspad_kv_append", "fspad_lm_head_stats", "fspad_lm_head_accept", "fspad_feature_sampler", "fspad_feature_sampler_workspace_bytes", "fspad_verify_step", "fspad_verify_step_host", "fspad_selftest_wait_timeout", "fspad_accept_stats_noalloc", "fspad_tree_build", "fspad_draft_expand"]
 
 
 class FspadConfig(ctypes.Structure):
@@ -63,6 +63,7 @@ def load():
     lib.fspad_feature_sampler_workspace_bytes.restype = ctypes.c_size_t
     lib.fspad_feature_sampler.argtypes = [vp] * 6 + [ci, ci, ci, vp, vp, vp, ctypes.c_size_t, vp]
     lib.fspad_tree_attn_paged.argtypes = [vp, vp, vp, vp, vp, ci, ci, vp, vp, vp, vp, ci, ci, vp, vp]
+    lib.fspad_kv_append.argtypes = [vp, vp, vp, vp, vp, vp, ci, ci, vp, vp]
     lib.fspad_kv_compact_paged.argtypes = [vp, vp, vp, ci, ci, vp, vp, vp, ci, vp, vp]
     lib.fspad_selftest_wait_timeout.argtypes = [vp, ci, vp]
     lib.fspad_verify_step.argtypes = [vp, vp, ci] + [vp] * 10 + [ci, ci] + [vp] * 6
@@ -265,6 +266,19 @@ class Context:
         if rc != 0:
             raise FspadError(rc, "fspad_feature_sampler")
         return eta, inter
+
+    def kv_append(self, cache, tree_kv, accepted_path, n_accepted, prefix_len, new_len=None, stream=None):
+        """cache [layers][2][B][Hkv][max_len][d], tree_kv [layers][2][B][Hkv][N][d]: accepted rows written behind the prefix."""
+        B = prefix_len.shape[0]
+        i32 = torch.int32
+        if new_len is None:
+            new_len = torch.empty((B,), dtype=i32, device=cache.device)
+        rc = load().fspad_kv_append(self._h, _ptr(cache, torch.bfloat16), _ptr(tree_kv, torch.bfloat16), _ptr(accepted_path, i32),
+                                    _ptr(n_accepted, i32), _ptr(prefix_len, i32), tree_kv.shape[4], B, _ptr(new_len, i32),
+                                    _stream(stream))
+        if rc != 0:
+            raise FspadError(rc, "fspad_kv_append")
+        return new_len
 
     def kv_compact(self, cache, accepted_path, n_accepted, prefix_len, new_len=None, stream=None):
         B = prefix_len.shape[0]

@@ -336,6 +336,20 @@ int fspad_kv_compact(fspad_ctx *ctx, fspad_bf16 *cache, const int32_t *accepted_
     return e == cudaSuccess ? FSPAD_OK : FSPAD_ERR_CUDA;
 }
 
+int fspad_kv_append(fspad_ctx *ctx, fspad_bf16 *cache, const fspad_bf16 *tree_kv, const int32_t *accepted_path,
+                    const int32_t *n_accepted, const int32_t *prefix_len, int n_nodes, int batch, int32_t *new_len,
+                    void *stream)
+{
+    int rc = check_common(ctx, n_nodes, batch);
+    if (rc) return rc;
+    if (!cache || !tree_kv || !accepted_path || !n_accepted || !prefix_len) return FSPAD_ERR_NULL;
+    if (misaligned(cache) || misaligned(tree_kv)) return FSPAD_ERR_ALIGN;
+    if (batch == 0) return FSPAD_OK;
+    cudaError_t e = fspad_launch_kv_append(ctx, cache, tree_kv, accepted_path, n_accepted, prefix_len, n_nodes, batch,
+                                           new_len, fspad_stream(stream));
+    return e == cudaSuccess ? FSPAD_OK : FSPAD_ERR_CUDA;
+}
+
 int fspad_tree_build(fspad_ctx *ctx, const int32_t *cand_parent, const int32_t *cand_token,
                      const float *cand_logp, const int32_t *root_token, int n_cand, int n_nodes, int batch,
                      int32_t *parent_out, int32_t *token_out, int32_t *cand_out, uint64_t *anc_out,

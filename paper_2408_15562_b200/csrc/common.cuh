@@ -308,5 +308,7 @@ cudaError_t fspad_launch_attn_umma_split(fspad_ctx *ctx, const fspad_bf16 *q, co
                                          const fspad_bf16 *vc, const fspad_bf16 *tk, const fspad_bf16 *tv,
                                          const int *parent, const int *prefix_len, int N, int B, int n_splits,
                                          float scale_log2, cudaStream_t st, FspadPaged paged);
+cudaError_t fspad_launch_kv_append(fspad_ctx *ctx, fspad_bf16 *cache, const fspad_bf16 *tree_kv, const int *path,
+                                   const int *n_acc, const int *prefix_len, int N, int B, int *new_len, cudaStream_t st);
 cudaError_t fspad_launch_kv_compact_paged(fspad_ctx *ctx, fspad_bf16 *pool, FspadPaged paged, const int *path,
                                           const int *n_acc, const int *prefix_len, int B, int *new_len, cudaStream_t st);

@@ -1,4 +1,4 @@
-// Accepted-path KV compaction and the tree-row scatter used by the host entry.
+// Accepted-path KV compaction, the cache append of the accepted path, and the tree-row scatter used by the host entry.
 //
 // After verification the rejected tokens leave the sequence (paper, Section
 // "Preliminaries": differing tokens and their descendants are discarded), so
@@ -129,6 +129,54 @@ kv_compact_paged_kernel(uint4 *__restrict__ pool, const int *__restrict__ table,
     if (bad) fspad_report(status, FSPAD_ERR_RANGE);
 }
 
+// Cache append of the accepted path: the tree's K/V rows of every layer are held outside the cache,
+// [layers][2][B][Hkv][N][d], and only the accepted ones are written, directly behind the prefix:
+// cache[..][L + j][:] = tree_kv[..][path[j]][:].  The N - n rejected rows never reach the cache, so neither
+// the write of all N rows nor the later move of the accepted ones happens.  One warp per (layer, K/V,
+// sequence, head) slice, eight rows in flight; source and destination are different arrays, so there
+// is no ordering to keep.
+__global__ void __launch_bounds__(kWarpsPerCta * 32)
+kv_append_kernel(uint4 *__restrict__ cache, const uint4 *__restrict__ tree_kv, const int *__restrict__ path,
+                 const int *__restrict__ n_acc, const int *__restrict__ prefix_len, int n_layers, int B, int Hkv,
+                 int max_len, int N, int path_stride, int *__restrict__ new_len, int *__restrict__ status)
+{
+    fspad_pdl_trigger();
+    fspad_pdl_wait();
+    const int lane = threadIdx.x & 31;
+    const long long slice = (long long)blockIdx.x * kWarpsPerCta + (threadIdx.x >> 5);
+    const long long n_slices = (long long)n_layers * 2 * B * Hkv;
+    if (slice >= n_slices) return;
+    const int b = (int)((slice / Hkv) % B);
+    int L = prefix_len[b], n = n_acc[b];
+    const int *pth = path + (size_t)b * path_stride;
+    bool bad = false;
+    if (n < 0 || n > path_stride || n > N) { bad = true; n = 0; }
+    if (L < 0 || L + n > max_len) { bad = true; n = 0; }
+    if (new_len && lane == 0 && slice < (long long)B * Hkv && slice % Hkv == 0) new_len[b] = L + n;
+    uint4 *dst_base = cache + ((size_t)slice * max_len + L) * kChunks;
+    const uint4 *src_base = tree_kv + (size_t)slice * N * kChunks;
+    const int chunk = lane & 15, half = lane >> 4;
+    for (int j0 = 0; j0 < n; j0 += 2 * kBatchIters) {
+        uint4 v[kBatchIters];
+        int dst[kBatchIters];
+#pragma unroll
+        for (int u = 0; u < kBatchIters; ++u) {
+            const int j = j0 + 2 * u + half;
+            dst[u] = -1;
+            if (j < n) {
+                const int src = pth[j];
+                if (src < 0 || src >= N) { bad = true; continue; }
+                v[u] = __ldg(src_base + (size_t)src * kChunks + chunk);
+                dst[u] = j;
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < kBatchIters; ++u)
+            if (dst[u] >= 0) dst_base[(size_t)dst[u] * kChunks + chunk] = v[u];
+    }
+    if (bad) fspad_report(status, FSPAD_ERR_RANGE);
+}
+
 // cache[layer 0][K|V][b][h][L_b + j][:] = tree_{k|v}[b][h][j][:]
 __global__ void __launch_bounds__(256)
 tree_scatter_kernel(uint4 *__restrict__ cache, const uint4 *__restrict__ tk, const uint4 *__restrict__ tv,
@@ -167,6 +215,19 @@ cudaError_t fspad_launch_kv_compact(fspad_ctx *ctx, fspad_bf16 *cache, const int
     return fspad_launch_opt(pdl, kv_compact_kernel, dim3(grid), dim3(kWarpsPerCta * 32), 0, st, 0,
                         reinterpret_cast<uint4 *>(cache), path, n_acc, prefix_len, c.n_layers, B, c.n_kv_heads,
                         c.max_len, c.max_nodes, c.max_nodes, new_len, ctx->d_status);
+}
+
+cudaError_t fspad_launch_kv_append(fspad_ctx *ctx, fspad_bf16 *cache, const fspad_bf16 *tree_kv, const int *path,
+                                   const int *n_acc, const int *prefix_len, int N, int B, int *new_len, cudaStream_t st)
+{
+    if (B == 0) return cudaSuccess;
+    const fspad_config &c = ctx->cfg;
+    const long long slices = (long long)c.n_layers * 2 * B * c.n_kv_heads;
+    const unsigned grid = (unsigned)((slices + kWarpsPerCta - 1) / kWarpsPerCta);
+    ctx->launches++;
+    return fspad_launch(kv_append_kernel, dim3(grid), dim3(kWarpsPerCta * 32), 0, st, 0, reinterpret_cast<uint4 *>(cache),
+                        reinterpret_cast<const uint4 *>(tree_kv), path, n_acc, prefix_len, c.n_layers, B, c.n_kv_heads,
+                        c.max_len, N, c.max_nodes, new_len, ctx->d_status);
 }
 
 cudaError_t fspad_launch_tree_scatter(fspad_ctx *ctx, fspad_bf16 *cache, const fspad_bf16 *tk,
