@@ -322,6 +322,11 @@ def main():
     attn_us, attn_min = timed(lambda i: attn(sets[i % R]), args.steps)
     accept_us, accept_min = timed(lambda i: accept(sets[i % R]), args.steps)
     compact_us, _ = timed(lambda i: compact(sets[i % R]), args.steps)
+    # the same rows written from a tree K/V array held outside the cache (fspad_kv_append)
+    gen = torch.Generator(device="cuda").manual_seed(24081556200)
+    tree_kv = torch.randn((n_layers, 2, B, w.n_kv_heads, N, 128), dtype=torch.float32, device="cuda", generator=gen).to(torch.bfloat16)
+    append_us, _ = timed(lambda i: ctx.kv_append(sets[i % R]["cache"], tree_kv, path, n_acc, prefix, new_len), args.steps)
+    del tree_kv
     lg2d = [s["logits"].view(B * N, w.vocab) for s in sets]
     st_out = (torch.empty(B * N, dtype=torch.float32, device="cuda"), torch.empty(B * N, dtype=torch.float64, device="cuda"),
               torch.empty(B * N, dtype=torch.int32, device="cuda"))
@@ -497,7 +502,7 @@ def main():
             "step_algorithmic_bytes": step_all,
             "breakdown_us": {"three_calls_on_one_stream": three_us, "three_calls_on_one_stream_min": three_min,
                              "tree_attn": attn_us, "tree_attn_min": attn_min, "tree_accept": accept_us,
-                             "tree_accept_min": accept_min, "kv_compact_warm_l2": compact_us,
+                             "tree_accept_min": accept_min, "kv_compact_warm_l2": compact_us, "kv_append_warm_l2": append_us,
                              "accept_stats_kernel_alone": stats_us, "accept_stats_kernel_alone_min": stats_min,
                              "accept_stats_with_merge": stats_merge_us,
                              "whole_step_eager_python_launches": eager_us},

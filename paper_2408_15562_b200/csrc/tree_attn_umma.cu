@@ -43,6 +43,7 @@ struct Args {
     const fspad_bf16 *q, *kc, *vc, *tk, *tv;
     const int *parent, *prefix_len;
     int N, Hq, Hkv, G, M, max_len, n_splits, mtiles, use_tma;
+    int longest_first;                  // the launch needs several waves of CTAs: blockIdx.z counts the sequences from the longest down
     // paged cache: the planes are pools of 128-row blocks [n_blocks][Hkv][128][d] and block_table[b][i] names
     // the block that holds rows 128 i .. 128 i + 127 of sequence b (NULL: contiguous planes)
     const int *block_table;
@@ -94,6 +95,7 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
     __shared__ __align__(8) unsigned long long s_bar[4 * NS + 13];
     __shared__ uint32_t s_tmem;
     __shared__ int s_fail;
+    __shared__ int s_seq;
     __shared__ int s_par[NW == 1 ? FSPAD_MAX_NODES : 1];
     __shared__ int s_blk[kMaxBlocksPerCta];       // paged cache: blocks of this CTA's chunks
     __shared__ unsigned long long s_anc[NW == 1 ? FSPAD_MAX_NODES : 1];
@@ -104,7 +106,24 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
     const int row = tid & (BM - 1), grp = (tid >> 7) & 1;
     const int split = blockIdx.x;
     const int g = blockIdx.y / a.mtiles, mt = blockIdx.y % a.mtiles;
-    const int b = blockIdx.z;
+    int b = blockIdx.z;
+    if (a.longest_first) {
+        // CTAs are dispatched in index order as SMs come free, so with more CTAs than SMs the sequences
+        // handled last decide the tail: they should be the short ones.  Every CTA ranks the sequences by
+        // length (ties by index, so the ranks are a permutation) and takes the one whose rank is blockIdx.z.
+        const int nb = (int)gridDim.z;
+        for (int t = tid; t < nb; t += NT) {
+            const int Lt = a.prefix_len[t];
+            int rank = 0;
+            for (int u = 0; u < nb; ++u) {
+                const int Lu = a.prefix_len[u];
+                rank += (Lu > Lt || (Lu == Lt && u < t)) ? 1 : 0;
+            }
+            if (rank == (int)blockIdx.z) s_seq = t;
+        }
+        __syncthreads();
+        b = s_seq;
+    }
     const int N = a.N, G = a.G, M = a.M;
 
     int L = a.prefix_len[b];
@@ -654,6 +673,7 @@ cudaError_t fspad_launch_attn_umma_split(fspad_ctx *ctx, const fspad_bf16 *q, co
     a.M = N * a.G; a.max_len = paged.table ? paged.stride * umma::BK : c.max_len; a.n_splits = n_splits;
     a.block_table = paged.table; a.table_stride = paged.stride; a.n_blocks = paged.n_blocks;
     a.mtiles = (a.M + umma::BM - 1) / umma::BM;
+    a.longest_first = (B > 1 && (long long)B * c.n_kv_heads * a.mtiles * n_splits > ctx->sm_count) ? 1 : 0;
     a.scale_log2 = scale_log2;
     a.part_o = ctx->part_o; a.part_ml = ctx->part_ml; a.status = ctx->d_status;
     if (!ctx->attn_attr_done) {
