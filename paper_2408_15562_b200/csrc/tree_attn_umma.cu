@@ -306,8 +306,8 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
         if (failed) s_fail = 1;
     } else if (warp == 9) {
         // ================= tensor-core warp: one thread issues every tcgen05.mma =================
-        {
-            const uint32_t elect = lane == 0;     // every lane runs the loop, this one issues
+        if (lane == 0) {
+            const uint32_t elect = 1;             // the whole loop is this one thread's
             // low words of the shared-memory descriptors (start address and leading byte offset);
             // the high word (8-row group stride, version, swizzle mode) is the same for all
             const uint32_t hi = (uint32_t)(make_desc(0, 16) >> 32);
@@ -318,7 +318,7 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
             // S(c) = Q K(c)^T into score buffer c & 1 (columns 0..63 of it belong to group 0, 64..127 to
             // group 1); K(c) sits in ring slot kbuf, which the second commit releases
             auto issue_s = [&](int c) {
-                if (!failed && !mbar_wait(kfull(kbuf), kph)) failed = true;
+                if (!failed && !mbar_wait_thread(kfull(kbuf), kph)) failed = true;
                 if (!failed) {
                     tc_fence_after();
                     const uint32_t kb = k_lo + (uint32_t)kbuf * (TILE >> 4);
@@ -343,8 +343,8 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
                 for (int g2 = 0; g2 < 2; ++g2) {
                     // O[g2] += P_g2(c) V(c)[64 g2 .. 64 g2 + 63]: P from the four warps of group g2 (in tensor
                     // memory, over the scores it was computed from) and the V chunk
-                    if (!failed && !mbar_wait(pfull(g2, p), ph)) failed = true;
-                    if (g2 == 0 && !failed && !mbar_wait(vfull(vbuf), vph)) failed = true;
+                    if (!failed && !mbar_wait_thread(pfull(g2, p), ph)) failed = true;
+                    if (g2 == 0 && !failed && !mbar_wait_thread(vfull(vbuf), vph)) failed = true;
                     if (!failed) {
                         tc_fence_after();
                         const uint32_t a_t = tmem + (uint32_t)p * 128u + (uint32_t)g2 * 64u;

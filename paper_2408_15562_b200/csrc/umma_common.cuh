@@ -58,6 +58,16 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_
     return ok != 0;
 }
 
+// The same bounded wait for a thread on its own (no other lane of its warp takes part).
+__device__ __forceinline__ bool mbar_wait_thread(uint32_t bar, uint32_t parity, uint32_t cap = WAIT_CAP)
+{
+    for (uint32_t i = 0; i < cap; ++i) {
+        if (mbar_test(bar, parity)) return true;
+        if (i >= 64) __nanosleep(40);
+    }
+    return false;
+}
+
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
 {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(bytes) : "memory");
