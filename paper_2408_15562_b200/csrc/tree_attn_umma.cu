@@ -79,7 +79,8 @@ __device__ __forceinline__ uint32_t tile_off(int r, int c)
 //   kfull/vfull(b)  K / V ring slot b filled (TMA bytes, or one arrival)     tensor-core warp waits
 //   kfree/vfree(b)  both S (both P V) of the chunk in slot b complete        copy warp waits
 //   sfull(p)        S of a chunk of parity p complete (tcgen05.commit)       both groups wait
-//   pfull(g, p)     P_g written and O_g rescaled by the 4 warps of group g   tensor-core warp waits
+//   pfull(p)        P written and O rescaled by the 8 warps of both groups    tensor-core warp waits (one wait and
+//                                                                            one fence for both groups' products)
 //   odone(g, p)     O_g += P_g V of a chunk of parity p complete             group g waits (rescale, end)
 // A new phase of a barrier can only begin after every side that waits on it has seen the previous
 // one (a parity wait must never fall two phases behind).
@@ -156,7 +157,7 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
     auto kfree = [&](int buf) { return bar0 + 8u * (uint32_t)(2 * NS + buf); };
     auto vfree = [&](int buf) { return bar0 + 8u * (uint32_t)(3 * NS + buf); };
     auto sfull = [&](int par) { return bar0 + 8u * (uint32_t)(4 * NS + par); };
-    auto pfull = [&](int grp2, int par) { return bar0 + 8u * (uint32_t)(4 * NS + 4 + 2 * grp2 + par); };
+    auto pfull = [&](int par) { return bar0 + 8u * (uint32_t)(4 * NS + 4 + par); };
     auto odone = [&](int grp2, int par) { return bar0 + 8u * (uint32_t)(4 * NS + 8 + 2 * grp2 + par); };
     const uint32_t drain = bar0 + 8u * (uint32_t)(4 * NS + 12);   // used only when a wait has run out
     const bool tma_ok = a.use_tma != 0;
@@ -164,7 +165,7 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
     // leave as soon as the prefix length is known, ahead of the CTA's first barrier.
     if (tid == 256) {
 #pragma unroll
-        for (int i = 0; i < 4 * NS + 13; ++i) mbar_init(bar0 + 8u * i, (i >= 4 * NS + 4 && i < 4 * NS + 8) ? 4 : 1);
+        for (int i = 0; i < 4 * NS + 13; ++i) mbar_init(bar0 + 8u * i, (i >= 4 * NS + 4 && i < 4 * NS + 6) ? 8 : 1);
         s_fail = 0;
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     }
@@ -320,7 +321,9 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
             auto issue_s = [&](int c) {
                 if (!failed && !mbar_wait_thread(kfull(kbuf), kph)) failed = true;
                 if (!failed) {
-                    tc_fence_after();
+                    // no tcgen05 fence here: the K chunk comes through the barrier's own acquire, and the
+                    // score buffer's last readers and writers (softmax of chunk c - 2) were ordered before this
+                    // thread's instructions by the fence behind its pfull wait of that chunk
                     const uint32_t kb = k_lo + (uint32_t)kbuf * (TILE >> 4);
                     const uint32_t d = tmem + (uint32_t)(c & 1) * 128u;
 #pragma unroll
@@ -343,10 +346,10 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
                 for (int g2 = 0; g2 < 2; ++g2) {
                     // O[g2] += P_g2(c) V(c)[64 g2 .. 64 g2 + 63]: P from the four warps of group g2 (in tensor
                     // memory, over the scores it was computed from) and the V chunk
-                    if (!failed && !mbar_wait_thread(pfull(g2, p), ph)) failed = true;
+                    if (g2 == 0 && !failed && !mbar_wait_thread(pfull(p), ph)) failed = true;
                     if (g2 == 0 && !failed && !mbar_wait_thread(vfull(vbuf), vph)) failed = true;
                     if (!failed) {
-                        tc_fence_after();
+                        if (g2 == 0) tc_fence_after();
                         const uint32_t a_t = tmem + (uint32_t)p * 128u + (uint32_t)g2 * 64u;
 #pragma unroll
                         for (int ks = 0; ks < 4; ++ks) { // K = 16 keys per instruction = 8 columns of packed bf16 pairs
@@ -425,25 +428,28 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
                     valid[blk] = mask_word(off);
                 }
             }
-            // 32 scores of this thread's row, with the tree mask applied where it matters
-            auto load_scores = [&](int blk, float (&v)[32]) {
-                tmem_ld32(tS + (uint32_t)blk * 32u, v);
-                if (masked) {
-                    const uint32_t wv = valid[blk];
+            // ---- this row's 64 scores of the group, in registers after one trip to tensor memory, with the
+            // tree mask applied where it matters; the row maximum as four independent chains ----
+            float v[64];
+            {
+                uint32_t r0[32], r1[32];
+                __syncwarp();
+                tmem_ld32_issue(tS, r0);
+                tmem_ld32_issue(tS + 32u, r1);
+                tmem_ld_wait(r0);
+                tmem_ld_pin(r1);
 #pragma unroll
-                    for (int j = 0; j < 32; ++j)
-                        if (!((wv >> j) & 1u)) v[j] = -INFINITY;
-                }
-            };
-            // ---- pass 1: row maximum ----
-            float mx = -INFINITY;
-#pragma unroll
-            for (int blk = 0; blk < 2; ++blk) {
-                float v[32];
-                load_scores(blk, v);
-#pragma unroll
-                for (int j = 0; j < 32; ++j) mx = fmaxf(mx, v[j]);
+                for (int j = 0; j < 32; ++j) { v[j] = __uint_as_float(r0[j]); v[32 + j] = __uint_as_float(r1[j]); }
             }
+            if (masked) {
+#pragma unroll
+                for (int j = 0; j < 64; ++j)
+                    if (!((valid[j >> 5] >> (j & 31)) & 1u)) v[j] = -INFINITY;
+            }
+            float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+            for (int j = 0; j < 64; ++j) mx4[j & 3] = fmaxf(mx4[j & 3], v[j]);
+            const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
             // The reference value m of a row (P = exp2(s * scale - m), O and the sum are relative to it)
             // only has to bound the scores loosely: it follows the row maximum when some row of the warp
             // would otherwise see a P above 2^kLazyLog2, and stays put - no pass over O - when not.
@@ -467,29 +473,28 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
                     tmem_st32(tO + (uint32_t)blk * 32u, o);
                 }
             }
-            // ---- pass 2: P = exp2(s * scale - m) as bf16 pairs, written over the scores already consumed
-            // (block blk of P takes columns 16 blk .. 16 blk + 15, all below the 32 (blk + 1) columns read) ----
-            float rs = 0.f;
+            // ---- P = exp2(s * scale - m) as bf16 pairs, written over the group's score columns (every score
+            // is in registers by now); the row sum as four independent chains ----
+            float rs4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
             for (int blk = 0; blk < 2; ++blk) {
-                float v[32];
-                load_scores(blk, v);
                 uint32_t w[16];
 #pragma unroll
                 for (int e = 0; e < 16; ++e) {
-                    const float p0 = ex2f(fmaf(v[2 * e], scale, -m_safe));
-                    const float p1 = ex2f(fmaf(v[2 * e + 1], scale, -m_safe));
-                    rs += p0 + p1;
+                    const float p0 = ex2f(fmaf(v[blk * 32 + 2 * e], scale, -m_safe));
+                    const float p1 = ex2f(fmaf(v[blk * 32 + 2 * e + 1], scale, -m_safe));
+                    rs4[e & 3] += p0 + p1;
                     w[e] = pack_bf16(p0, p1);
                 }
                 tmem_st16(tS + (uint32_t)blk * 16u, w);
             }
+            const float rs = (rs4[0] + rs4[1]) + (rs4[2] + rs4[3]);
             l_run = l_run * alpha + rs;
             m_run = m_new;
             asm volatile("tcgen05.wait::st.sync.aligned;\n" ::: "memory");
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(pfull(grp, p));
+            if (lane == 0) mbar_arrive(pfull(p));
         }
         // ---- each group waits for its own last product (tensor-core work completes in order, so the
         // one before it is complete too); the CTA-wide barrier below then orders both accumulators
