@@ -678,7 +678,8 @@ cudaError_t fspad_launch_attn_umma_split(fspad_ctx *ctx, const fspad_bf16 *q, co
     a.M = N * a.G; a.max_len = paged.table ? paged.stride * umma::BK : c.max_len; a.n_splits = n_splits;
     a.block_table = paged.table; a.table_stride = paged.stride; a.n_blocks = paged.n_blocks;
     a.mtiles = (a.M + umma::BM - 1) / umma::BM;
-    a.longest_first = (B > 1 && (long long)B * c.n_kv_heads * a.mtiles * n_splits > ctx->sm_count) ? 1 : 0;
+    // (every CTA ranks all sequences itself, B loads each for B / 320 of its threads: kept to batches where that is small change)
+    a.longest_first = (B > 1 && B <= 128 && (long long)B * c.n_kv_heads * a.mtiles * n_splits > ctx->sm_count) ? 1 : 0;
     a.scale_log2 = scale_log2;
     a.part_o = ctx->part_o; a.part_ml = ctx->part_ml; a.status = ctx->d_status;
     if (!ctx->attn_attr_done) {
