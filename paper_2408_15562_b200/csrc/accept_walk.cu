@@ -78,6 +78,11 @@ struct WalkArgs {
     FspadStatsGeom geom;
     int N, V, path_stride, cache_ok;
     int *path, *n_acc, *bonus, *status;
+    // optional: the cluster that has walked a sequence also moves its accepted K/V rows up (NULL: not asked for)
+    uint4 *kv_cache;                    // [layers][2][B][Hkv][max_len][d] bf16 as 16-byte chunks
+    const int *kv_prefix;
+    int *kv_new_len;
+    int kv_layers, kv_B, kv_H, kv_max_len;
 };
 
 // A set of tree nodes as a bit mask of W 64-bit words (W = 1: trees of up to 64 nodes, the common case;
@@ -352,6 +357,51 @@ __device__ Sweep5 fused_reject_sweep(const Shared &sh, const float *__restrict__
     return r;
 }
 
+// Compaction of the accepted path by the CTAs that walked it (every CTA of the cluster holds the same path in
+// its shared memory): row L + path[j] -> row L + j of every (layer, K/V, head) slice of the sequence, one warp
+// per slice, eight rows in flight, every load of a batch before any of its stores (path[j] >= j and the path
+// is increasing, so moves in index order never overwrite a row that is still to be read).  The same moves as
+// the stand-alone compaction kernel makes; doing them here saves the step one dependent launch.
+template <typename Shared>
+__device__ __forceinline__ void compact_accepted(const WalkArgs &args, const Shared &sh, int b, int rank, int C, int tid, int nthr)
+{
+    if (args.kv_cache == nullptr) return;
+    const int lane = tid & 31, n_warps = nthr >> 5;
+    int n = sh.len;
+    const int L = args.kv_prefix[b];
+    if (L < 0 || n < 1 || L + sh.path[n - 1] >= args.kv_max_len) {
+        if (rank == 0 && tid == 0) fspad_report(args.status, FSPAD_ERR_RANGE);
+        n = 0;
+    }
+    if (rank == 0 && tid == 0 && args.kv_new_len) args.kv_new_len[b] = max(L, 0) + n;
+    const int per_seq = args.kv_layers * 2 * args.kv_H;
+    const int chunk = lane & 15, half = lane >> 4;
+    for (int s = rank * n_warps + (tid >> 5); s < per_seq; s += C * n_warps) {
+        const int lk = s / args.kv_H, h = s % args.kv_H;
+        uint4 *base = args.kv_cache + ((((size_t)lk * args.kv_B + b) * args.kv_H + h) * args.kv_max_len + L) * 16;
+        for (int j0 = 0; j0 < n; j0 += 8) {
+            uint4 v[4];
+            int dst[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int j = j0 + 2 * u + half;
+                dst[u] = -1;
+                if (j < n) {
+                    const int src = sh.path[j];
+                    if (src != j) {
+                        v[u] = base[(size_t)src * 16 + chunk];
+                        dst[u] = j;
+                    }
+                }
+            }
+            __syncwarp();
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                if (dst[u] >= 0) base[(size_t)dst[u] * 16 + chunk] = v[u];
+        }
+    }
+}
+
 template <int MAXN>
 __global__ void __launch_bounds__(kWalkThreads, 1)
 accept_walk_kernel(const WalkArgs args)
@@ -465,7 +515,7 @@ accept_walk_kernel(const WalkArgs args)
 
     if (!sampling) {
         // ---- greedy: strict token comparison against the target argmax ----
-        if (rank == 0 && tid == 0) {
+        if (tid == 0) {                               // every CTA of the cluster: same data, same path
             int cur = 0, len = 1;
             sh.path[0] = 0;
             for (;;) {
@@ -475,16 +525,17 @@ accept_walk_kernel(const WalkArgs args)
                     const int c = rem.first();
                     if (sh.tok[c] == want) { next = c; break; }
                 }
-                if (next < 0) { args.bonus[b] = want; break; }
+                if (next < 0) { if (rank == 0) args.bonus[b] = want; break; }
                 sh.path[len++] = next;
                 cur = next;
             }
-            args.n_acc[b] = len;
+            if (rank == 0) args.n_acc[b] = len;
             sh.len = len;
         }
         __syncthreads();
         if (rank == 0)
             for (int i = tid; i < args.path_stride; i += nthr) out_path[i] = (i < sh.len) ? sh.path[i] : -1;
+        compact_accepted(args, sh, b, rank, C, tid, nthr);
         return;   // the whole cluster takes this branch together; no peer memory is touched
     }
 
@@ -817,6 +868,7 @@ accept_walk_kernel(const WalkArgs args)
             if (tid == 0) args.n_acc[b] = sh.len;
             for (int i = tid; i < args.path_stride; i += nthr) out_path[i] = (i < sh.len) ? sh.path[i] : -1;
         }
+        compact_accepted(args, sh, b, rank, C, tid, nthr);   // the path is final; only the bonus token may still be open
         if (settled) return;                                // uniform over the cluster; no peer memory is touched after the walk's last exchange
 
         // ---- exact draw over the whole row: every CTA a contiguous slice, every thread a contiguous chunk ----
@@ -914,10 +966,12 @@ int fspad_walk_ctas(fspad_ctx *ctx, int B, int V) { return B * walk_cluster_size
 cudaError_t fspad_launch_accept_walk(fspad_ctx *ctx, const float *logits, const float *draft,
                                      const int *tokens, const int *parent, const float *temperature,
                                      const float *uniforms, const FspadStatsGeom &geom, int N, int B, int V,
-                                     int *path, int *n_acc, int *bonus, cudaStream_t st)
+                                     int *path, int *n_acc, int *bonus, cudaStream_t st, FspadWalkCompact kv)
 {
     if (B == 0) return cudaSuccess;
     WalkArgs a;
+    a.kv_cache = reinterpret_cast<uint4 *>(kv.cache); a.kv_prefix = kv.prefix_len; a.kv_new_len = kv.new_len;
+    a.kv_layers = ctx->cfg.n_layers; a.kv_B = B; a.kv_H = ctx->cfg.n_kv_heads; a.kv_max_len = ctx->cfg.max_len;
     a.logits = logits; a.draft = draft; a.temperature = temperature; a.uniforms = uniforms;
     a.tokens = tokens; a.parent = parent;
     a.parts = ctx->st_part; a.geom = geom;

@@ -450,9 +450,16 @@ int fspad_verify_step(fspad_ctx *ctx, fspad_bf16 *cache, int attn_layer, const f
         // (steps replayed from one CUDA graph: 72.5 us per step against 48.8 on the 52-head shape).
         ce = fspad_launch_stats_partials(ctx, target_logits, temperature, rows, n_nodes, c.vocab, &geom, st, false);
     }
+    // With the tree rows given apart from the cache the compaction depends on the walk alone, and when the
+    // sequence's slices are few (one warp each among the walk's own CTAs) the walk makes the moves itself
+    // at its end: one dependent launch less on the step's longest chain.
+    const bool aliased = tree_k == nullptr;      // attention reads the cache rows that compaction rewrites
+    const bool walk_compacts = !aliased && c.n_layers * 2 * c.n_kv_heads <= 64;
+    FspadWalkCompact kv;
+    if (walk_compacts) { kv.cache = cache; kv.prefix_len = prefix_len; kv.new_len = new_len; }
     if (ce == cudaSuccess)
         ce = fspad_launch_accept_walk(ctx, target_logits, draft_probs, draft_tokens, parent, temperature, uniforms, geom,
-                                      n_nodes, batch, c.vocab, accepted_path, n_accepted, bonus_token, st);
+                                      n_nodes, batch, c.vocab, accepted_path, n_accepted, bonus_token, st, kv);
     rc = ce == cudaSuccess ? FSPAD_OK : FSPAD_ERR_CUDA;
     if (scan_first)
         rc_attn = fspad_launch_tree_attn(ctx, q, kc, vc, tree_k, tree_v, parent, prefix_len, n_nodes, batch, attn_out,
@@ -460,10 +467,9 @@ int fspad_verify_step(fspad_ctx *ctx, fspad_bf16 *cache, int attn_layer, const f
     // the join is queued whatever happened in between, so that a capture of `stream` never ends
     // with the second stream left unjoined
     const bool ev_ok = cudaEventRecord(ctx->ev_join, ctx->side) == cudaSuccess;
-    const bool aliased = tree_k == nullptr;      // attention reads the cache rows that compaction rewrites
     bool joined = false;
     if (aliased) joined = cudaStreamWaitEvent(st, ctx->ev_join, 0) == cudaSuccess;
-    if (rc == FSPAD_OK && rc_attn == FSPAD_OK) {
+    if (rc == FSPAD_OK && rc_attn == FSPAD_OK && !walk_compacts) {
         // behind a join the compaction has two predecessors, so it is launched as a plain dependent
         cudaError_t e = fspad_launch_kv_compact(ctx, cache, accepted_path, n_accepted, prefix_len, batch, new_len, st,
                                                 !aliased);

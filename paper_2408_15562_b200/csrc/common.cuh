@@ -255,10 +255,17 @@ __device__ __forceinline__ void fspad_report(int *status, int err)
 cudaError_t fspad_launch_accept_stats(fspad_ctx *ctx, const float *logits, const float *temperature,
                                       int rows, int rows_per_seq, int V, float *row_max,
                                       double *row_sum, int *row_arg, cudaStream_t st);
+// cache != NULL: the walk also compacts the accepted path's rows of `cache` (all layers of the context) and
+// writes new_len; the caller then launches no compaction
+struct FspadWalkCompact {
+    fspad_bf16 *cache = nullptr;
+    const int *prefix_len = nullptr;
+    int *new_len = nullptr;
+};
 cudaError_t fspad_launch_accept_walk(fspad_ctx *ctx, const float *logits, const float *draft,
                                      const int *tokens, const int *parent, const float *temperature,
                                      const float *uniforms, const FspadStatsGeom &geom, int N, int B, int V,
-                                     int *path, int *n_acc, int *bonus, cudaStream_t st);
+                                     int *path, int *n_acc, int *bonus, cudaStream_t st, FspadWalkCompact kv = {});
 // pdl = false: launched as a plain dependent of what precedes it in the stream (griddepcontrol.wait is
 // then a no-op; the guarantee its successor relies on holds either way)
 cudaError_t fspad_launch_stats_partials(fspad_ctx *ctx, const float *logits, const float *temperature,
