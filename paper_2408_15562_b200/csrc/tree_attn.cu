@@ -117,6 +117,6 @@ cudaError_t fspad_launch_tree_attn(fspad_ctx *ctx, const fspad_bf16 *q, const fs
     const long long rows = (long long)B * c.n_kv_heads * a.M;
     ctx->launches++;
     const dim3 grid((unsigned)((rows + 3) / 4));
-    if (a.n_splits <= 4) return fspad_launch_opt(false, tree_attn_combine_kernel<4>, grid, dim3(128), 0, st, 0, a, B);
-    return fspad_launch_opt(false, tree_attn_combine_kernel<12>, grid, dim3(128), 0, st, 0, a, B);
+    if (a.n_splits <= 4) return fspad_launch_opt(true, tree_attn_combine_kernel<4>, grid, dim3(128), 0, st, 0, a, B);
+    return fspad_launch_opt(true, tree_attn_combine_kernel<12>, grid, dim3(128), 0, st, 0, a, B);
 }

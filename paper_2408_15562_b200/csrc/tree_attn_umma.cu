@@ -506,7 +506,6 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
         // carries the groups' (max, sum) exchange
         float2 *s_ml = reinterpret_cast<float2 *>(smem_raw + (base - smem_u32(smem_raw)));
         s_ml[grp * BM + row] = make_float2(m_run, l_run);
-        fspad_pdl_trigger();                      // the merge kernel may start launching
         tc_fence_before();
         __syncthreads();
         tc_fence_after();
@@ -553,13 +552,13 @@ tree_attn_umma_kernel(const Args a, const __grid_constant__ CUtensorMap tmK, con
                         *reinterpret_cast<const float4 *>(stg + r * SROW + lane * 4);
             }
         }
+        fspad_pdl_trigger();                      // partial written: the merge kernel may start launching
         tc_fence_before();
         __syncthreads();
         return;
     }
     // copy and tensor-core warps: meet the softmax warps at their two CTA-wide barriers; the warp
     // that allocated the tensor memory then frees it
-    fspad_pdl_trigger();
     tc_fence_before();
     __syncthreads();
     if (s_fail != 0) {
