@@ -94,6 +94,21 @@ def test_batched_ragged_small():
     _check(synth.generate(w, 0, with_accept=False))
 
 
+@pytest.mark.parametrize("lengths", ["equal", "pairs", "descending", "ascending"])
+def test_more_ctas_than_sms_sequences_taken_longest_first(lengths):
+    """24 sequences x 8 kv heads x 2 row tiles = 384 CTAs: more than the SMs, so the kernel hands the sequences
+    out longest first by a rank it computes from the lengths on the device.  Equal lengths (every rank decided by
+    the index), equal pairs, and lengths already in either order must all give every sequence its own output."""
+    B = 24
+    L = {"equal": np.full(B, 200), "pairs": 60 + 40 * (np.arange(B) // 2), "descending": 600 - 20 * np.arange(B),
+         "ascending": 50 + 20 * np.arange(B)}[lengths].astype(np.int32)
+    w = synth.scaled(W["batch16_ragged"], batch=B, prefix=(int(L.max()), int(L.max())), temperatures=(0.0,) * B,
+                     vocab=16, n_layers=1)
+    inp = synth.generate(w, 3, with_accept=False)
+    inp.prefix_len[:] = L                       # the cache is generated for the longest; shorter ones use its head
+    _check(inp)
+
+
 def test_equal_value_rows_reproduce_exactly():
     """All V rows equal to one bf16 row: the softmax weights sum to 1, so the output is that row."""
     w = synth.scaled(W["llama3_8b_2k"], prefix=(300, 300), vocab=16)
