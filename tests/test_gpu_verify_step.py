@@ -55,16 +55,17 @@ def _check(inp, outs, cache, ref_o, r, want, want_len):
         np.testing.assert_array_equal(got[:, :, b, :, :rows], want[:, :, b, :, :rows])
 
 
-@pytest.mark.parametrize("aliased", [False, True])
+@pytest.mark.parametrize("n_layers", [3, 5])      # 48 and 80 (layer, K/V, head) slices per sequence: up to 64 the walk's
+@pytest.mark.parametrize("aliased", [False, True])  # own CTAs compact the cache, above that the compaction kernel does
 @pytest.mark.parametrize("mode", ["sample", "greedy", "mixed"])
-def test_whole_step_against_oracle(mode, aliased):
+def test_whole_step_against_oracle(mode, aliased, n_layers):
     temps = {"sample": (1.0, 0.8, 1.0), "greedy": (0.0, 0.0, 0.0), "mixed": (0.0, 1.0, 0.0)}[mode]
     w = synth.scaled(W["llama3_8b_2k"], batch=3, prefix=(40, 300), n_nodes=24, depth=4, branch=4, vocab=3000,
                      temperatures=temps)
     inp = synth.generate(w, 11)
     B, N = inp.parent.shape
     layer = 1
-    cache_host = synth.make_cache(inp, 3)
+    cache_host = synth.make_cache(inp, n_layers)
     L = inp.prefix_len
     for b in range(B):          # the attention layer's planes are the workload's K/V; tree rows behind the prefix
         cache_host[layer, 0, b] = inp.k_cache[b]
@@ -72,7 +73,7 @@ def test_whole_step_against_oracle(mode, aliased):
         cache_host[layer, 0, b, :, L[b]:L[b] + N] = inp.tree_k[b]
         cache_host[layer, 1, b, :, L[b]:L[b] + N] = inp.tree_v[b]
     ref_o, r, want, want_len = _oracle_step(inp, cache_host, layer)
-    ctx = helpers.make_ctx(inp, n_layers=3)
+    ctx = helpers.make_ctx(inp, n_layers=n_layers)
     d, a, outs, cache = _device_inputs(inp, cache_host)
     _call(ctx, cache, a, d, outs, aliased, layer)
     ctx.check()
