@@ -443,18 +443,29 @@ int fspad_verify_step(fspad_ctx *ctx, fspad_bf16 *cache, int attn_layer, const f
         return FSPAD_ERR_CUDA;
     int rc_attn = FSPAD_OK;
     if (!scan_first) {
+        // An all-greedy acceptance is a scan and a one-CTA walk: beside an attention that holds most SMs the
+        // scan's CTAs only get going when the attention's leave.  Where the context is short enough for the
+        // attention to stay short on half the SMs (at most 8 chunks per CTA by the context's max_len), it
+        // gets half and the two really run side by side (17.2 against 20.5 us on the 26-node greedy workload).
+        int both_sms = 0;
+        if (!may_sample && attn_ctas > sms / 2) {
+            const int s_half = fspad_attn_umma_splits(ctx, n_nodes, batch, sms / 2);
+            const int max_chunks = (c.max_len + 127) / 128;
+            if ((max_chunks + s_half - 1) / s_half <= 8) both_sms = sms / 2;
+        }
         rc_attn = fspad_launch_tree_attn(ctx, q, kc, vc, tree_k, tree_v, parent, prefix_len, n_nodes, batch, attn_out,
-                                         ctx->side, 0) == cudaSuccess ? FSPAD_OK : FSPAD_ERR_CUDA;
+                                         ctx->side, both_sms) == cudaSuccess ? FSPAD_OK : FSPAD_ERR_CUDA;
         // Here the scan is launched as a plain dependent: as a programmatic dependent of the previous
         // step's last kernel it was seen to hold the forked attention back behind the whole acceptance
         // (steps replayed from one CUDA graph: 72.5 us per step against 48.8 on the 52-head shape).
         ce = fspad_launch_stats_partials(ctx, target_logits, temperature, rows, n_nodes, c.vocab, &geom, st, false);
     }
     // With the tree rows given apart from the cache the compaction depends on the walk alone, and when the
-    // sequence's slices are few (one warp each among the walk's own CTAs) the walk makes the moves itself
-    // at its end: one dependent launch less on the step's longest chain.
+    // sequence's slices are few (one warp each among the 16 x 32 warps of a sampling walk's cluster; an
+    // all-greedy walk is a single small CTA and keeps the kernel) the walk makes the moves itself at its
+    // end: one dependent launch less on the step's longest chain.
     const bool aliased = tree_k == nullptr;      // attention reads the cache rows that compaction rewrites
-    const bool walk_compacts = !aliased && c.n_layers * 2 * c.n_kv_heads <= 64;
+    const bool walk_compacts = !aliased && may_sample && c.n_layers * 2 * c.n_kv_heads <= 64;
     FspadWalkCompact kv;
     if (walk_compacts) { kv.cache = cache; kv.prefix_len = prefix_len; kv.new_len = new_len; }
     if (ce == cudaSuccess)
