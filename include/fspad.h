@@ -422,9 +422,10 @@ int fspad_kv_compact_paged(fspad_ctx *ctx, fspad_bf16 *pool, const int32_t *bloc
  * acceptance directly when tree_k / tree_v are given (attention then never
  * reads the cache rows compaction rewrites); when they are NULL (tree rows
  * taken from cache rows L_b ..) compaction waits for the attention as well.
- * In the first case, when a sequence has at most 64 (layer, K/V, kv head)
- * slices, the kernel that walks the tree makes the compaction's moves itself
- * (same result; an invalid prefix length is then reported by that kernel).
+ * In the first case, when draft_probs is given and a sequence has at most 64
+ * (layer, K/V, kv head) slices, the kernel that walks the tree makes the
+ * compaction's moves itself (same result; an invalid prefix length is then
+ * reported by that kernel).
  * Work queued on `stream` after the call sees every output.  The call only
  * enqueues work and records / waits on events, so it may be captured into a
  * CUDA graph.  One call per context at a time.
