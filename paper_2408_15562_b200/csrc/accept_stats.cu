@@ -225,10 +225,11 @@ cudaError_t launch_partials(const float *logits, const float *temperature, int r
 
 cudaError_t fspad_launch_stats_partials(fspad_ctx *ctx, const float *logits, const float *temperature,
                                         int rows, int rows_per_seq, int V, FspadStatsGeom *geom,
-                                        cudaStream_t st, bool pdl)
+                                        cudaStream_t st, bool pdl, int sms)
 {
     const bool vec = (V % 4 == 0) && ((reinterpret_cast<uintptr_t>(logits) & 15) == 0);
-    *geom = fspad_stats_geom(ctx->sm_count, rows, V, vec, ctx->stats_slots);
+    if (sms <= 0 || sms > ctx->sm_count) sms = ctx->sm_count;
+    *geom = fspad_stats_geom(sms, rows, V, vec, ctx->stats_slots);
     ctx->launches++;
     return launch_partials(logits, temperature, rows_per_seq, *geom, ctx->st_part, st, pdl);
 }

@@ -458,7 +458,21 @@ int fspad_verify_step(fspad_ctx *ctx, fspad_bf16 *cache, int attn_layer, const f
         // Here the scan is launched as a plain dependent: as a programmatic dependent of the previous
         // step's last kernel it was seen to hold the forked attention back behind the whole acceptance
         // (steps replayed from one CUDA graph: 72.5 us per step against 48.8 on the 52-head shape).
-        ce = fspad_launch_stats_partials(ctx, target_logits, temperature, rows, n_nodes, c.vocab, &geom, st, false);
+        // Where the acceptance is the longer chain (a sampling walk follows, or the attention is the short
+        // one above), the scan is cut for the SMs the attention leaves free - one wave of two CTAs per SM
+        // there: cut for the whole chip its CTAs queue for those few SMs in several waves, each with a
+        // launch's fixed cost (45.5 -> 41.2 us on the 52-head sampling workload, 17.1 -> 14.7 us on the
+        // 26-node greedy one).  Under a long attention with a greedy walk the short-lived CTAs of the
+        // full-size scan are the better neighbours (37.6 against 39.0 us): an attention CTA that finds
+        // its SM taken waits for a scan CTA's whole life.
+        int scan_sms = 0;
+        if (may_sample || both_sms > 0) {
+            const long long attn_now = (long long)batch * c.n_kv_heads * ((n_nodes * G + 127) / 128) *
+                                       fspad_attn_umma_splits(ctx, n_nodes, batch, both_sms);
+            scan_sms = sms - (int)(attn_now < sms ? attn_now : sms);
+            if (scan_sms < sms / 8) scan_sms = sms / 8;
+        }
+        ce = fspad_launch_stats_partials(ctx, target_logits, temperature, rows, n_nodes, c.vocab, &geom, st, false, scan_sms);
     }
     // With the tree rows given apart from the cache the compaction depends on the walk alone, and when the
     // sequence's slices are few (one warp each among the 16 x 32 warps of a sampling walk's cluster; an

@@ -270,7 +270,7 @@ cudaError_t fspad_launch_accept_walk(fspad_ctx *ctx, const float *logits, const 
 // then a no-op; the guarantee its successor relies on holds either way)
 cudaError_t fspad_launch_stats_partials(fspad_ctx *ctx, const float *logits, const float *temperature,
                                         int rows, int rows_per_seq, int V, FspadStatsGeom *geom,
-                                        cudaStream_t st, bool pdl = true);
+                                        cudaStream_t st, bool pdl = true, int sms = 0);   // sms > 0: one wave on that many SMs
 cudaError_t fspad_launch_tree_build(fspad_ctx *ctx, const int *cand_parent, const int *cand_token,
                                     const float *cand_logp, const int *root_token, int n_cand, int n_nodes,
                                     int B, int *parent_out, int *token_out, int *cand_out,
