@@ -486,9 +486,15 @@ int fspad_verify_step(fspad_ctx *ctx, fspad_bf16 *cache, int attn_layer, const f
         ce = fspad_launch_accept_walk(ctx, target_logits, draft_probs, draft_tokens, parent, temperature, uniforms, geom,
                                       n_nodes, batch, c.vocab, accepted_path, n_accepted, bonus_token, st, kv);
     rc = ce == cudaSuccess ? FSPAD_OK : FSPAD_ERR_CUDA;
-    if (scan_first)
+    if (scan_first) {
+        // When the walk's clusters need more than one wave, merge CTAs that sit resident waiting for the
+        // attention would keep the later clusters off their SMs (244 against 224 us on the ragged batch):
+        // the merge kernel is then a plain dependent.
+        const bool walk_one_wave = fspad_walk_ctas(ctx, batch, c.vocab) <= sms / 2;   // the attention was sized to leave that many free
         rc_attn = fspad_launch_tree_attn(ctx, q, kc, vc, tree_k, tree_v, parent, prefix_len, n_nodes, batch, attn_out,
-                                         ctx->side, attn_sms) == cudaSuccess ? FSPAD_OK : FSPAD_ERR_CUDA;
+                                         ctx->side, attn_sms, FspadPaged{nullptr, 0, 0}, walk_one_wave) == cudaSuccess
+                      ? FSPAD_OK : FSPAD_ERR_CUDA;
+    }
     // the join is queued whatever happened in between, so that a capture of `stream` never ends
     // with the second stream left unjoined
     const bool ev_ok = cudaEventRecord(ctx->ev_join, ctx->side) == cudaSuccess;

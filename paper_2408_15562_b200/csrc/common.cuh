@@ -289,11 +289,13 @@ struct FspadPaged {
     const int *table;
     int stride, n_blocks;
 };
-// sms: how many SMs the call may fill with CTAs (0 = all of them)
+// sms: how many SMs the call may fill with CTAs (0 = all of them).  merge_pdl: the merge kernel is a programmatic
+// dependent of the attention kernel (its CTAs become resident, waiting, as the attention's last CTAs finish).
 cudaError_t fspad_launch_tree_attn(fspad_ctx *ctx, const fspad_bf16 *q, const fspad_bf16 *kc,
                                    const fspad_bf16 *vc, const fspad_bf16 *tk, const fspad_bf16 *tv,
                                    const int *parent, const int *prefix_len, int N, int B,
-                                   fspad_bf16 *out, cudaStream_t st, int sms = 0, FspadPaged paged = FspadPaged{nullptr, 0, 0});
+                                   fspad_bf16 *out, cudaStream_t st, int sms = 0, FspadPaged paged = FspadPaged{nullptr, 0, 0},
+                                   bool merge_pdl = true);
 cudaError_t fspad_launch_tree_scatter(fspad_ctx *ctx, fspad_bf16 *cache, const fspad_bf16 *tk,
                                       const fspad_bf16 *tv, const int *prefix_len, int N, int B,
                                       cudaStream_t st);

@@ -99,7 +99,7 @@ tree_attn_combine_kernel(const AttnArgs a, int B)
 cudaError_t fspad_launch_tree_attn(fspad_ctx *ctx, const fspad_bf16 *q, const fspad_bf16 *kc,
                                    const fspad_bf16 *vc, const fspad_bf16 *tk, const fspad_bf16 *tv,
                                    const int *parent, const int *prefix_len, int N, int B,
-                                   fspad_bf16 *out, cudaStream_t st, int sms, FspadPaged paged)
+                                   fspad_bf16 *out, cudaStream_t st, int sms, FspadPaged paged, bool merge_pdl)
 {
     if (B == 0 || N == 0) return cudaSuccess;
     const fspad_config &c = ctx->cfg;
@@ -117,6 +117,6 @@ cudaError_t fspad_launch_tree_attn(fspad_ctx *ctx, const fspad_bf16 *q, const fs
     const long long rows = (long long)B * c.n_kv_heads * a.M;
     ctx->launches++;
     const dim3 grid((unsigned)((rows + 3) / 4));
-    if (a.n_splits <= 4) return fspad_launch_opt(true, tree_attn_combine_kernel<4>, grid, dim3(128), 0, st, 0, a, B);
-    return fspad_launch_opt(true, tree_attn_combine_kernel<12>, grid, dim3(128), 0, st, 0, a, B);
+    if (a.n_splits <= 4) return fspad_launch_opt(merge_pdl, tree_attn_combine_kernel<4>, grid, dim3(128), 0, st, 0, a, B);
+    return fspad_launch_opt(merge_pdl, tree_attn_combine_kernel<12>, grid, dim3(128), 0, st, 0, a, B);
 }
