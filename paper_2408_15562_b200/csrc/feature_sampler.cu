@@ -90,28 +90,32 @@ skinny_gemm_kernel(const Args a, const __grid_constant__ CUtensorMap tmA0, const
 
     if (warp == 0) {
         // ================= copy warp =================
+        // one thread's loop (its waits are plain polls; nothing is shuffled to the other lanes)
         int it = 0;
-        for (int j = 0; j < my_items; ++j) {
-            int prob, tile, k0, nk;
-            decode(j, prob, tile, k0, nk);
-            const CUtensorMap *mA = prob ? &tmA1 : &tmA0, *mB = prob ? &tmB1 : &tmB0;
-            for (int k = 0; k < nk; ++k, ++it) {
-                const int s = it % NSTG;
-                const uint32_t ph = (uint32_t)(it / NSTG) & 1u;
-                if (it >= NSTG && !failed && !mbar_wait(empty(s), ph ^ 1u)) failed = true;
-                if (!failed && lane == 0) {
-                    mbar_expect_tx(full(s), STAGE_A + STAGE_B);
-                    tma_load_2d(sA + s * STAGE_A, mA, (k0 + k) * BKE, 0, full(s));
-                    tma_load_2d(sB + s * STAGE_B, mB, (k0 + k) * BKE, tile * BN, full(s));
+        if (lane == 0) {
+            for (int j = 0; j < my_items; ++j) {
+                int prob, tile, k0, nk;
+                decode(j, prob, tile, k0, nk);
+                const CUtensorMap *mA = prob ? &tmA1 : &tmA0, *mB = prob ? &tmB1 : &tmB0;
+                for (int k = 0; k < nk; ++k, ++it) {
+                    const int s = it % NSTG;
+                    const uint32_t ph = (uint32_t)(it / NSTG) & 1u;
+                    if (it >= NSTG && !failed && !mbar_wait_thread(empty(s), ph ^ 1u)) failed = true;
+                    if (!failed) {
+                        mbar_expect_tx(full(s), STAGE_A + STAGE_B);
+                        tma_load_2d(sA + s * STAGE_A, mA, (k0 + k) * BKE, 0, full(s));
+                        tma_load_2d(sB + s * STAGE_B, mB, (k0 + k) * BKE, tile * BN, full(s));
+                    }
                 }
-                __syncwarp();
             }
+            if (failed) s_fail = 1;
         }
+        it = __shfl_sync(0xffffffffu, it, 0);
         total_stages = it;
-        if (failed) s_fail = 1;
     } else if (warp == 1) {
         // ================= tensor-core warp =================
-        const uint32_t elect = lane == 0;
+        if (lane == 0) {                              // one thread's loop, as the copy warp's
+        const uint32_t elect = 1;
         const uint32_t hi = (uint32_t)(make_desc(0, 16) >> 32);
         const uint32_t a_lo = (uint32_t)make_desc(sA, 16), b_lo = (uint32_t)make_desc(sB, 16);
         const uint32_t idesc = make_idesc(false, BN);
@@ -120,12 +124,12 @@ skinny_gemm_kernel(const Args a, const __grid_constant__ CUtensorMap tmA0, const
             int prob, tile, k0, nk;
             decode(j, prob, tile, k0, nk);
             const int buf = j & 1;
-            if (j >= 2 && !failed && !mbar_wait(acce(buf), (uint32_t)((j - 2) >> 1) & 1u)) failed = true;
+            if (j >= 2 && !failed && !mbar_wait_thread(acce(buf), (uint32_t)((j - 2) >> 1) & 1u)) failed = true;
             tc_fence_after();
             for (int k = 0; k < nk; ++k, ++it) {
                 const int s = it % NSTG;
                 const uint32_t ph = (uint32_t)(it / NSTG) & 1u;
-                if (!failed && !mbar_wait(full(s), ph)) failed = true;
+                if (!failed && !mbar_wait_thread(full(s), ph)) failed = true;
                 if (!failed) {
                     tc_fence_after();
                     const uint32_t soa = (uint32_t)s * (STAGE_A >> 4), sob = (uint32_t)s * (STAGE_B >> 4);
@@ -139,6 +143,7 @@ skinny_gemm_kernel(const Args a, const __grid_constant__ CUtensorMap tmA0, const
             }
         }
         if (failed) s_fail = 1;
+        }
         __syncwarp();
     } else {
         // ================= epilogue warps: one row per thread, fp32 partial sums out =================

@@ -102,28 +102,31 @@ lm_head_stats_kernel(const Args a, const __grid_constant__ CUtensorMap tmA, cons
     bool failed = false;
 
     if (warp == 0) {
-        // ================= copy warp: one lane issues every TMA copy =================
-        int it = 0;
-        for (int j = 0; j < my_items; ++j) {
-            int tile, width;
-            item(j, tile, width);
-            for (int k = 0; k < n_k; ++k, ++it) {
-                const int s = it % NSTG;
-                const uint32_t ph = (uint32_t)(it / NSTG) & 1u;
-                if (it >= NSTG && !failed && !mbar_wait(empty(s), ph ^ 1u)) failed = true;
-                if (!failed && lane == 0) {
-                    mbar_expect_tx(full(s), (1 + width) * STAGE);
-                    tma_load_2d(sA + s * STAGE, &tmA, k * BKE, 0, full(s));
-                    tma_load_2d(sB + s * STAGE_B, &tmB, k * BKE, tile * BN, full(s));
-                    if (width == 2) tma_load_2d(sB + s * STAGE_B + STAGE, &tmB, k * BKE, (tile + 1) * BN, full(s));
+        // ================= copy warp: one thread runs the whole loop (its waits are plain polls) =================
+        if (lane == 0) {
+            int it = 0;
+            for (int j = 0; j < my_items; ++j) {
+                int tile, width;
+                item(j, tile, width);
+                for (int k = 0; k < n_k; ++k, ++it) {
+                    const int s = it % NSTG;
+                    const uint32_t ph = (uint32_t)(it / NSTG) & 1u;
+                    if (it >= NSTG && !failed && !mbar_wait_thread(empty(s), ph ^ 1u)) failed = true;
+                    if (!failed) {
+                        mbar_expect_tx(full(s), (1 + width) * STAGE);
+                        tma_load_2d(sA + s * STAGE, &tmA, k * BKE, 0, full(s));
+                        tma_load_2d(sB + s * STAGE_B, &tmB, k * BKE, tile * BN, full(s));
+                        if (width == 2) tma_load_2d(sB + s * STAGE_B + STAGE, &tmB, k * BKE, (tile + 1) * BN, full(s));
+                    }
                 }
-                __syncwarp();
             }
+            if (failed) s_fail = 1;
         }
-        if (failed) s_fail = 1;
+        __syncwarp();
     } else if (warp == 1) {
-        // ================= tensor-core warp: one lane issues every tcgen05.mma =================
-        const uint32_t elect = lane == 0;
+        // ================= tensor-core warp: one thread runs the whole loop =================
+        if (lane == 0) {
+        const uint32_t elect = 1;
         const uint32_t hi = (uint32_t)(make_desc(0, 16) >> 32);
         const uint32_t a_lo = (uint32_t)make_desc(sA, 16), b_lo = (uint32_t)make_desc(sB, 16);
         const uint32_t idesc2 = make_idesc(false, 2 * BN), idesc1 = make_idesc(false, BN);
@@ -134,12 +137,12 @@ lm_head_stats_kernel(const Args a, const __grid_constant__ CUtensorMap tmA, cons
             const uint32_t idesc = width == 2 ? idesc2 : idesc1;
             const int buf = j & 1;
             // the accumulator is free once the epilogue has read the tile that used it two tiles ago
-            if (j >= 2 && !failed && !mbar_wait(acce(buf), (uint32_t)((j - 2) >> 1) & 1u)) failed = true;
+            if (j >= 2 && !failed && !mbar_wait_thread(acce(buf), (uint32_t)((j - 2) >> 1) & 1u)) failed = true;
             tc_fence_after();
             for (int k = 0; k < n_k; ++k, ++it) {
                 const int s = it % NSTG;
                 const uint32_t ph = (uint32_t)(it / NSTG) & 1u;
-                if (!failed && !mbar_wait(full(s), ph)) failed = true;
+                if (!failed && !mbar_wait_thread(full(s), ph)) failed = true;
                 if (!failed) {
                     tc_fence_after();
                     const uint32_t soa = (uint32_t)s * (STAGE >> 4), sob = (uint32_t)s * (STAGE_B >> 4);
@@ -153,6 +156,7 @@ lm_head_stats_kernel(const Args a, const __grid_constant__ CUtensorMap tmA, cons
             }
         }
         if (failed) s_fail = 1;
+        }
         __syncwarp();
     } else {
         // ================= epilogue warps: one row per thread =================
