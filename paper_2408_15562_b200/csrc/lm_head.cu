@@ -302,9 +302,21 @@ lm_head_merge_kernel(const FspadStatsPart *__restrict__ tile_parts, int R, int n
     const float kk = lmh::kLog2e / T;
     float m = -INFINITY, s = 0.f;
     int arg = 0x7fffffff;
-    for (int t = t0 + lane; t < t1; t += 32) {
-        const int4 v = __ldcg(reinterpret_cast<const int4 *>(tile_parts + (size_t)r * n_tiles + t));
-        merge_part(m, s, arg, __int_as_float(v.x), __int_as_float(v.y), v.z, kk);
+    // A lane's partials are requested eight at a time, before any of them is merged: the merge carries a
+    // dependency from one partial to the next, and with one request per step a row of a thousand tiles was
+    // thirty-two trips to L2 one after the other (about 19 us of a 190 us call).
+    constexpr int kAhead = 8;
+    for (int tb = t0 + lane; tb < t1; tb += 32 * kAhead) {
+        int4 v[kAhead];
+#pragma unroll
+        for (int u = 0; u < kAhead; ++u) {
+            const int t = tb + 32 * u;
+            v[u] = make_int4(__float_as_int(-INFINITY), 0, 0x7fffffff, 0);
+            if (t < t1) v[u] = __ldcg(reinterpret_cast<const int4 *>(tile_parts + (size_t)r * n_tiles + t));
+        }
+#pragma unroll
+        for (int u = 0; u < kAhead; ++u)
+            if (tb + 32 * u < t1) merge_part(m, s, arg, __int_as_float(v[u].x), __int_as_float(v[u].y), v[u].z, kk);
     }
     double sd = 0.0;
     {
