@@ -74,7 +74,7 @@ template <> struct Unit<1> {
 };
 
 template <int UNIT>
-__global__ void __launch_bounds__(kThreads, 2)
+__global__ void __launch_bounds__(kThreads, 1024 / kThreads)
 accept_stats_kernel(const float *__restrict__ logits, const float *__restrict__ temperature,
                     int rows_per_seq, const FspadStatsGeom g, FspadStatsPart *__restrict__ parts)
 {

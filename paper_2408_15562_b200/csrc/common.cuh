@@ -13,7 +13,7 @@
 #define FSPAD_MAX_CANDIDATES 1024
 #define FSPAD_MAX_FRONTIER 16      /* frontier nodes per sequence, and top-k per row, of a draft step */
 #define FSPAD_HEAD_DIM 128
-#define FSPAD_STATS_THREADS 512     /* threads per CTA of the vocabulary scan */
+#define FSPAD_STATS_THREADS 256
 
 // Scratch and bookkeeping owned by a context (all device pointers unless noted).
 struct fspad_ctx {
@@ -88,7 +88,7 @@ static inline FspadStatsGeom fspad_stats_geom(int sm_count, int rows, int V, boo
     g.upr = V / g.unit;
     g.slots = slots;
     g.total = (long long)rows * g.upr;
-    long long n = (long long)sm_count * 2;                 // two 512-thread CTAs per SM, one wave
+    long long n = (long long)sm_count * (1024 / FSPAD_STATS_THREADS);   // 1024 threads per SM, one wave
     const long long by_size = (g.total + FSPAD_STATS_THREADS - 1) / FSPAD_STATS_THREADS;   // at least one unit per thread
     if (n > by_size) n = by_size;
     if (n < 1) n = 1;
