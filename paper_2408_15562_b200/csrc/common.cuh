@@ -93,6 +93,13 @@ static inline FspadStatsGeom fspad_stats_geom(int sm_count, int rows, int V, boo
     if (n > by_size) n = by_size;
     if (n < 1) n = 1;
     g.chunk = (g.total + n - 1) / n;
+    // A CTA whose range crosses a row boundary runs its reduction sequence twice and finishes about a
+    // microsecond behind the others.  Where a row divides evenly into a whole number k of pieces such that
+    // rows * k CTAs still fill three quarters of the wave, ranges are cut at the rows instead.
+    if (rows >= 1 && n >= rows) {
+        for (long long k = n / rows; k >= 1 && (long long)rows * k * 4 >= n * 3; --k)
+            if (g.upr % k == 0) { g.chunk = g.upr / k; break; }
+    }
     // a row may be shared by at most `slots` CTAs
     const long long min_chunk = (g.upr + (slots - 2) - 1) / (slots - 2);
     if (g.chunk < min_chunk) g.chunk = min_chunk;
