@@ -20,7 +20,7 @@
 
 namespace {
 
-constexpr int kThreads = FSPAD_STATS_THREADS;   // 512
+constexpr int kThreads = FSPAD_STATS_THREADS;   // 256; small arrays are scanned by CTAs of half that
 constexpr int kDeep = 4;                  // load units per batch per thread (two batches in flight)
 constexpr float kLog2e = 1.4426950408889634f;
 
@@ -73,7 +73,7 @@ template <> struct Unit<1> {
     static __device__ __forceinline__ int first_eq(const T &v, float bm, int j, int a) { return v == bm ? j : a; }
 };
 
-template <int UNIT>
+template <int UNIT, int kThreads>
 __global__ void __launch_bounds__(kThreads, 1024 / kThreads)
 accept_stats_kernel(const float *__restrict__ logits, const float *__restrict__ temperature,
                     int rows_per_seq, const FspadStatsGeom g, FspadStatsPart *__restrict__ parts)
@@ -214,10 +214,17 @@ accept_stats_merge_kernel(const FspadStatsPart *__restrict__ parts, const FspadS
 cudaError_t launch_partials(const float *logits, const float *temperature, int rows_per_seq,
                             const FspadStatsGeom &g, FspadStatsPart *parts, cudaStream_t st, bool pdl = true)
 {
+    if (g.threads == kThreads / 2) {
+        if (g.unit == 4)
+            return fspad_launch_opt(pdl, accept_stats_kernel<4, kThreads / 2>, dim3(g.n_cta), dim3(kThreads / 2), 0, st, 0, logits,
+                                    temperature, rows_per_seq, g, parts);
+        return fspad_launch_opt(pdl, accept_stats_kernel<1, kThreads / 2>, dim3(g.n_cta), dim3(kThreads / 2), 0, st, 0, logits,
+                                temperature, rows_per_seq, g, parts);
+    }
     if (g.unit == 4)
-        return fspad_launch_opt(pdl, accept_stats_kernel<4>, dim3(g.n_cta), dim3(kThreads), 0, st, 0, logits, temperature,
+        return fspad_launch_opt(pdl, accept_stats_kernel<4, kThreads>, dim3(g.n_cta), dim3(kThreads), 0, st, 0, logits, temperature,
                             rows_per_seq, g, parts);
-    return fspad_launch_opt(pdl, accept_stats_kernel<1>, dim3(g.n_cta), dim3(kThreads), 0, st, 0, logits, temperature,
+    return fspad_launch_opt(pdl, accept_stats_kernel<1, kThreads>, dim3(g.n_cta), dim3(kThreads), 0, st, 0, logits, temperature,
                             rows_per_seq, g, parts);
 }
 
@@ -229,7 +236,7 @@ cudaError_t fspad_launch_stats_partials(fspad_ctx *ctx, const float *logits, con
 {
     const bool vec = (V % 4 == 0) && ((reinterpret_cast<uintptr_t>(logits) & 15) == 0);
     if (sms <= 0 || sms > ctx->sm_count) sms = ctx->sm_count;
-    *geom = fspad_stats_geom(sms, rows, V, vec, ctx->stats_slots);
+    *geom = fspad_stats_geom(sms, rows, V, vec, ctx->stats_slots, true);
     ctx->launches++;
     return launch_partials(logits, temperature, rows_per_seq, *geom, ctx->st_part, st, pdl);
 }

@@ -360,6 +360,7 @@ FspadStatsGeom fspad_lm_head_geom(int rows, int V, bool vec, int slots)
     g.upr = V / g.unit;
     g.slots = slots;
     g.total = (long long)rows * g.upr;
+    g.threads = FSPAD_STATS_THREADS;            // no scan kernel runs on this geometry; the walk reads the pieces only
     const int tile_units = lmh::BN / g.unit;
     if (V % lmh::BN == 0) {
         const int n_tiles = V / lmh::BN;
