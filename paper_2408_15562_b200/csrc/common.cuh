@@ -104,8 +104,16 @@ static inline FspadStatsGeom fspad_stats_geom(int sm_count, int rows, int V, boo
     // microsecond behind the others.  Where a row divides evenly into a whole number k of pieces such that
     // rows * k CTAs still fill three quarters of the wave, ranges are cut at the rows instead.
     if (rows >= 1 && n >= rows) {
-        for (long long k = n / rows; k >= 1 && (long long)rows * k * 4 >= n * 3; --k)
-            if (g.upr % k == 0) { g.chunk = g.upr / k; break; }
+        bool cut = false;
+        // The acceptance walk keeps the masses of at most 16 pieces per row for its bonus draw (with more it
+        // sweeps the whole row): with few rows, 16 pieces per row are preferred to a full wave as long as
+        // every SM still gets a CTA.
+        if (n / rows > 16 && (long long)rows * 16 >= sm_count) {
+            for (long long k = 16; k >= 8 && !cut; --k)
+                if (g.upr % k == 0) { g.chunk = g.upr / k; cut = true; }
+        }
+        for (long long k = n / rows; !cut && k >= 1 && (long long)rows * k * 4 >= n * 3; --k)
+            if (g.upr % k == 0) { g.chunk = g.upr / k; cut = true; }
     }
     // a row may be shared by at most `slots` CTAs
     const long long min_chunk = (g.upr + (slots - 2) - 1) / (slots - 2);
