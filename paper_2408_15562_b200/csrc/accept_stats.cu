@@ -6,9 +6,11 @@
 // this kernel produces all of them in one HBM-bound sweep.
 //
 // Layout: logits [rows][V] fp32, viewed as one flat array that is cut into
-// equal contiguous ranges, one per CTA (two 512-thread CTAs per SM, a single
-// wave), so the load is balanced whatever rows and V are.  A range may cross row
-// boundaries; each (row, CTA) piece yields one partial (max, argmax, sum).
+// equal contiguous ranges, one per CTA (1024 threads per SM in a single wave:
+// CTAs of 128 threads for a small array, of 256 otherwise), so the load is
+// balanced whatever rows and V are.  Where the sizes allow, the ranges are cut at
+// the rows; otherwise a range may cross row boundaries and runs the reductions
+// once per row it touches.  Each (row, CTA) piece yields one partial (max, argmax, sum).
 // A thread works in batches of four 128-bit loads, with the next batch already
 // in flight: it takes the maximum of the 16 values in registers, rescales its
 // running sum once and adds the 16 exponentials: no per-element branch.  Partials are merged per
